@@ -1,0 +1,206 @@
+/*
+ * ls.h -- C ABI of the local-update SGD library for one NVIDIA B200 (sm_100a).
+ *
+ * The library runs the data-parallel hot path of periodic-averaging SGD
+ * (PASGD, Section 2 of "Adaptive Communication Strategies to Achieve the Best
+ * Error-Runtime Trade-off in Local-Update SGD") for m model replicas that all
+ * live in one GPU's memory, and the AdaComm communication-period rule
+ * (Section 4.2).  Every arithmetic step runs in CUDA kernels of this library;
+ * there is no CPU fallback.
+ *
+ * Conventions
+ *  - Every function returns an int status: LS_OK (0) or a negative LS_ERR_*.
+ *    Nothing throws or aborts across this boundary.  ls_strerror() names a code.
+ *  - "dev" pointers are CUDA device pointers on the current device, "host"
+ *    pointers are ordinary host memory.  The library allocates no device
+ *    memory: the caller allocates one state block of ls_state_bytes() bytes
+ *    (256-byte aligned) and lends it to the handle until ls_destroy().
+ *  - Kernels are enqueued on the CUDA stream given to ls_create() and the call
+ *    returns without waiting unless stated otherwise.  An asynchronous CUDA
+ *    error surfaces as LS_ERR_CUDA from a later call or from ls_sync().
+ *  - A handle is not thread-safe.
+ *
+ * Model: a fully connected network
+ *      x -> W_L relu( ... relu(W_1 x + b_1) ... ) + b_L
+ *  with dims = (d_in, h_1, ..., d_out).  n_layers == 1 is a linear model
+ *  (softmax regression, or least squares with LS_LOSS_MSE_HALF and d_out == 1).
+ *
+ * Flat parameter layout of one replica (P = ls_param_count() floats): for
+ *  l = 1..L the matrix W_l as [dims[l]][dims[l-1]] row-major, then b_l
+ *  (dims[l] floats) when has_bias.  Momentum buffers use the same layout.
+ *  Inside the state block replica i's vector starts at i * ls_param_stride()
+ *  floats (the stride is P rounded up to a multiple of 64 floats).
+ */
+#ifndef LS_H_
+#define LS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LS_MAX_LAYERS 8
+#define LS_MAX_REPLICAS 64
+#define LS_MAX_BATCH 1024
+#define LS_MAX_OUT 1024          /* largest d_out (width of the loss layer) */
+
+enum {
+  LS_OK = 0,
+  LS_ERR_INVALID_ARG = -1,       /* null pointer, size out of range, bad enum, non-finite number */
+  LS_ERR_BAD_HANDLE = -2,
+  LS_ERR_STATE_SIZE = -3,        /* state block too small or misaligned */
+  LS_ERR_NO_DATASET = -4,        /* ls_bind_dataset() has not been called */
+  LS_ERR_ROW_RANGE = -5,         /* a mini-batch would read past the bound dataset */
+  LS_ERR_CUDA = -6,              /* a CUDA runtime call failed; ls_last_cuda_error() has its code */
+  LS_ERR_UNSUPPORTED = -7,       /* valid request that this build does not implement (e.g. weight decay) */
+  LS_ERR_OVERFLOW = -8           /* a result does not fit its type */
+};
+
+enum { LS_LOSS_SOFTMAX_CE = 0, LS_LOSS_MSE_HALF = 1 };
+enum { LS_GEMM_FP32 = 0, LS_GEMM_BF16 = 1 };
+/* What an averaging step does with the per-replica momentum buffers.
+ * AVERAGE: replaced by their mean like the parameters (makes tau = 1 equal to
+ *          synchronous momentum SGD on the m-fold batch).
+ * KEEP:    left alone (the independent-buffer scheme of Section 5.3).
+ * RESET:   cleared (the local half of the block-momentum scheme, Section 5.3). */
+enum { LS_MOMENTUM_AVERAGE = 0, LS_MOMENTUM_KEEP = 1, LS_MOMENTUM_RESET = 2 };
+
+typedef struct ls_model_spec {
+  int32_t n_layers;                  /* L, 1..LS_MAX_LAYERS */
+  int32_t dims[LS_MAX_LAYERS + 1];   /* dims[0..L] */
+  int32_t loss;                      /* LS_LOSS_* */
+  int32_t has_bias;                  /* 0 or 1 */
+  int32_t gemm_dtype;                /* LS_GEMM_*: input type of the matrix products (accumulation is fp32) */
+  int32_t momentum_mode;             /* LS_MOMENTUM_* */
+  float weight_decay;                /* must be 0 */
+} ls_model_spec;
+
+typedef struct ls_handle ls_handle;
+
+const char* ls_strerror(int code);
+
+/* ---- sizes ------------------------------------------------------------- */
+
+/* P, the number of parameters of one replica.  (x in R^d of Section 2.) */
+int ls_param_count(const ls_model_spec* spec, int64_t* P);
+
+/* Bytes of the caller-allocated state block for m replicas and mini-batches of
+ * `batch` rows: parameters, momentum, bf16 weight copies (bf16 models),
+ * activation / gradient workspace, staging for host batches. */
+int ls_state_bytes(int m, const ls_model_spec* spec, int batch, size_t* bytes);
+
+/* ---- life cycle -------------------------------------------------------- */
+
+/* Create a handle for m replicas (1..LS_MAX_REPLICAS) that train with
+ * learning rate lr (eta of Section 2) and momentum factor `momentum`
+ * (0 <= momentum < 1; 0 means plain SGD and the buffers are never touched).
+ * state_dev: device block of >= ls_state_bytes() bytes, 256-byte aligned; it is
+ * borrowed until ls_destroy().  All parameters and momentum buffers start at
+ * zero (enqueued on `cuda_stream`, a cudaStream_t passed as void*, may be 0).
+ * Creates one auxiliary CUDA stream and a few events; allocates a small pinned
+ * host buffer; no device memory. */
+int ls_create(ls_handle** h, int m, const ls_model_spec* spec, float lr, float momentum, int batch,
+              void* state_dev, size_t state_bytes, void* cuda_stream);
+int ls_destroy(ls_handle* h);
+/* Wait for everything enqueued so far; returns LS_ERR_CUDA if any of it failed. */
+int ls_sync(ls_handle* h);
+int ls_last_cuda_error(const ls_handle* h);
+int ls_set_lr(ls_handle* h, float lr);
+
+/* ---- replica state  (X_k = [x^(1) ... x^(m)] of the proof's notation) --- */
+
+/* All workers start at the same point x_1 (Section 2): copy the P host floats
+ * to every replica, clear every momentum buffer.  Synchronous. */
+int ls_set_params(ls_handle* h, const float* x1_host);
+/* Overwrite / read one replica's parameters and momentum (P host floats each;
+ * either pointer may be NULL to skip it).  Synchronous. */
+int ls_set_state(ls_handle* h, int replica, const float* params_host, const float* momentum_host);
+int ls_get_state(ls_handle* h, int replica, float* params_host, float* momentum_host);
+/* Device views of the packed replicas: base pointers and the stride between
+ * replicas in floats.  The memory belongs to the state block. */
+int ls_state_view(ls_handle* h, float** params_dev, float** momentum_dev, int64_t* stride_floats);
+
+/* ---- data -------------------------------------------------------------- */
+
+/* Bind the training set resident in device memory: x_dev is [n_rows][dims[0]]
+ * row-major, float for LS_GEMM_FP32 and bf16 for LS_GEMM_BF16 (16-byte aligned);
+ * y_dev is int32[n_rows] class labels for LS_LOSS_SOFTMAX_CE (each in
+ * [0, d_out)) or float[n_rows] targets for LS_LOSS_MSE_HALF.  Borrowed: must
+ * stay valid while the handle uses it. */
+int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t n_rows);
+
+/* ---- the hot path ------------------------------------------------------ */
+
+/* tau local updates on every replica, no communication (Section 2, PASGD
+ * update rule, the case k mod tau != 0, applied tau times):
+ *      for s = 0..tau-1, for every replica i independently:
+ *          xi  = dataset rows [row_offset[s*m + i], + batch)
+ *          g   = (1/|xi|) sum_{s in xi} grad f(x^(i); s)      (Section 2)
+ *          v^(i) <- momentum * v^(i) + g ;  x^(i) <- x^(i) - lr * v^(i)
+ * row_offset_host: host int64[tau][m], read before the call returns.
+ * loss_dev: optional device float[tau][m]; entry [s][i] receives the mean loss
+ * of replica i's mini-batch at step s, evaluated before that step's update.
+ * Errors: tau < 1, NULL offsets, a batch outside the dataset. */
+int ls_local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev);
+
+/* Same steps, but the mini-batches come from host memory and the losses go
+ * back to host memory: x_host is [tau][m][batch][dims[0]] (float or bf16 as
+ * for ls_bind_dataset), y_host [tau][m][batch] (int32 or float), loss_host
+ * float[tau][m].  Pinned host memory lets the copies overlap the kernels of
+ * the previous step.  Synchronous: returns when loss_host is filled. */
+int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y_host, float* loss_host);
+
+/* Model averaging (Section 2, PASGD update rule, the case k mod tau = 0;
+ * X <- X J with J = 1 1^T / m): every replica's parameters are replaced by the
+ * mean over replicas; momentum buffers follow spec.momentum_mode.
+ * The mean is defined to the bit: s = x^(0); s = s + x^(j) for j = 1..m-1 in
+ * fp32, then one fp32 division by (float)m.  Afterwards all replicas are
+ * bitwise equal. */
+int ls_average(ls_handle* h);
+
+/* The averaging kernel on a raw buffer: m vectors of P floats, vector j
+ * starting at buf_dev + j*stride floats (stride >= P).  Same arithmetic as
+ * ls_average().  Fast path when buf_dev is 16-byte aligned and stride is a
+ * multiple of 4. */
+int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride, void* cuda_stream);
+
+/* Training loss of one replica on dataset rows [row_offset, +n_rows), the
+ * empirical risk F of Section 2 restricted to those rows; n_rows must be a
+ * positive multiple of `batch`.  Forward pass only.  Synchronous; writes one
+ * host float. */
+int ls_eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_rows, float* F_host);
+
+/* AdaComm basic update rule (Section 4.2):
+ *      tau_l = ceil( sqrt(F_t / F_0) * tau_0 ),   F_inf taken as 0,
+ * evaluated in IEEE double exactly as written, clamped below at 1 (growth
+ * above tau_0 is allowed).  Pure host function.  Returns the new period (>= 1)
+ * or a negative LS_ERR_* (F_0 <= 0, F_t < 0, non-finite input, tau_0 < 1,
+ * result beyond INT32_MAX). */
+int adacomm_next_tau(double F_t, double F_0, int tau_0);
+
+/* Whole training run in native code: K local iterations cut into periods of
+ * tau local steps, each followed by ls_average().  With interval > 0 the
+ * period is re-chosen by adacomm_next_tau() at the first averaging point at or
+ * past each multiple of `interval` iterations, from the loss of replica 0 on
+ * dataset rows [0, probe_rows) (F_0 is that loss at the starting point);
+ * interval == 0 keeps tau fixed.  A period is never cut by an interval
+ * boundary; the last period is cut at K and averaged.
+ * row_offset_host: int64[K][m].  loss_dev: optional device float[K][m].
+ * Outputs (host, optional): period_tau[max_periods] / n_periods list the period
+ * lengths requested; decision_k / decision_F / decision_tau [max_decisions] /
+ * n_decisions log every AdaComm decision; F0_host the initial loss. */
+int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
+           const int64_t* row_offset_host, float* loss_dev,
+           int32_t* period_tau, int64_t max_periods, int64_t* n_periods,
+           int64_t* decision_k, float* decision_F, int32_t* decision_tau, int64_t max_decisions,
+           int64_t* n_decisions, float* F0_host);
+
+/* Number of kernels this handle has launched so far. */
+int ls_launch_count(const ls_handle* h, int64_t* n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LS_H_ */

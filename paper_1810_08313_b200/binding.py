@@ -1,0 +1,305 @@
+"""ctypes binding of libls.so (include/ls.h).
+
+Argument marshalling only: every arithmetic step runs inside the CUDA library.
+torch is used for device memory and streams.  If the library cannot be built
+or loaded this module raises; there is no other implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+LS_MAX_LAYERS = 8
+LS_MAX_REPLICAS = 64
+
+LS_OK = 0
+LS_ERR_INVALID_ARG = -1
+LS_ERR_BAD_HANDLE = -2
+LS_ERR_STATE_SIZE = -3
+LS_ERR_NO_DATASET = -4
+LS_ERR_ROW_RANGE = -5
+LS_ERR_CUDA = -6
+LS_ERR_UNSUPPORTED = -7
+LS_ERR_OVERFLOW = -8
+
+LOSS = {"softmax_ce": 0, "mse_half": 1}
+GEMM = {"fp32": 0, "bf16": 1}
+MOMENTUM_MODE = {"average": 0, "keep": 1, "reset": 2}
+
+
+class ModelSpec(C.Structure):
+    _fields_ = [
+        ("n_layers", C.c_int32),
+        ("dims", C.c_int32 * (LS_MAX_LAYERS + 1)),
+        ("loss", C.c_int32),
+        ("has_bias", C.c_int32),
+        ("gemm_dtype", C.c_int32),
+        ("momentum_mode", C.c_int32),
+        ("weight_decay", C.c_float),
+    ]
+
+
+class LsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_lib().ls_strerror(code).decode()} ({code})")
+
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = _build.build()          # compiles with nvcc when missing or stale; raises on failure
+    lib = C.CDLL(path)
+    vp, i64, f32 = C.c_void_p, C.c_int64, C.c_float
+    P = C.POINTER
+    sig = {
+        "ls_strerror": (C.c_char_p, [C.c_int]),
+        "ls_param_count": (C.c_int, [P(ModelSpec), P(i64)]),
+        "ls_state_bytes": (C.c_int, [C.c_int, P(ModelSpec), C.c_int, P(C.c_size_t)]),
+        "ls_create": (C.c_int, [P(vp), C.c_int, P(ModelSpec), f32, f32, C.c_int, vp, C.c_size_t, vp]),
+        "ls_destroy": (C.c_int, [vp]),
+        "ls_sync": (C.c_int, [vp]),
+        "ls_last_cuda_error": (C.c_int, [vp]),
+        "ls_set_lr": (C.c_int, [vp, f32]),
+        "ls_set_params": (C.c_int, [vp, vp]),
+        "ls_set_state": (C.c_int, [vp, C.c_int, vp, vp]),
+        "ls_get_state": (C.c_int, [vp, C.c_int, vp, vp]),
+        "ls_state_view": (C.c_int, [vp, P(vp), P(vp), P(i64)]),
+        "ls_bind_dataset": (C.c_int, [vp, vp, vp, i64]),
+        "ls_local_steps": (C.c_int, [vp, C.c_int, vp, vp]),
+        "ls_local_steps_host": (C.c_int, [vp, C.c_int, vp, vp, vp]),
+        "ls_average": (C.c_int, [vp]),
+        "ls_average_flat": (C.c_int, [vp, C.c_int, i64, i64, vp]),
+        "ls_eval_loss": (C.c_int, [vp, C.c_int, i64, i64, P(f32)]),
+        "adacomm_next_tau": (C.c_int, [C.c_double, C.c_double, C.c_int]),
+        "ls_run": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, vp, i64, P(i64), vp, vp, vp, i64, P(i64),
+                             P(f32)]),
+        "ls_launch_count": (C.c_int, [vp, P(i64)]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _LIB = lib
+    return lib
+
+
+def library_path() -> str:
+    _lib()
+    return _build.LIB_PATH
+
+
+def _check(code: int, where: str):
+    if code != LS_OK:
+        raise LsError(code, where)
+
+
+def make_spec(dims: Sequence[int], loss: str = "softmax_ce", has_bias: bool = True, gemm_dtype: str = "fp32",
+              momentum_mode: str = "average", weight_decay: float = 0.0) -> ModelSpec:
+    s = ModelSpec()
+    if not (2 <= len(dims) <= LS_MAX_LAYERS + 1):
+        raise ValueError("1..8 layers")
+    s.n_layers = len(dims) - 1
+    for i, d in enumerate(dims):
+        s.dims[i] = int(d)
+    s.loss = LOSS[loss]
+    s.has_bias = int(bool(has_bias))
+    s.gemm_dtype = GEMM[gemm_dtype]
+    s.momentum_mode = MOMENTUM_MODE[momentum_mode]
+    s.weight_decay = float(weight_decay)
+    return s
+
+
+def param_count(spec: ModelSpec) -> int:
+    n = C.c_int64()
+    _check(_lib().ls_param_count(C.byref(spec), C.byref(n)), "ls_param_count")
+    return n.value
+
+
+def state_bytes(m: int, spec: ModelSpec, batch: int) -> int:
+    n = C.c_size_t()
+    _check(_lib().ls_state_bytes(m, C.byref(spec), batch, C.byref(n)), "ls_state_bytes")
+    return n.value
+
+
+def adacomm_next_tau(F_t: float, F_0: float, tau_0: int) -> int:
+    r = _lib().adacomm_next_tau(float(F_t), float(F_0), int(tau_0))
+    if r < 0:
+        raise LsError(r, "adacomm_next_tau")
+    return r
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def average_flat(buf, m: int, P: int, stride: Optional[int] = None, stream=None) -> None:
+    """Average m float32 vectors of P elements held in the CUDA tensor `buf`
+    (vector j starts at element j*stride) in place."""
+    import torch
+    if not (buf.is_cuda and buf.dtype == torch.float32 and buf.is_contiguous()):
+        raise ValueError("buf must be a contiguous float32 CUDA tensor")
+    stride = int(P if stride is None else stride)
+    if buf.numel() < (m - 1) * stride + P:
+        raise ValueError("buf too small")
+    _check(_lib().ls_average_flat(buf.data_ptr(), int(m), int(P), stride, _stream_ptr(stream)), "ls_average_flat")
+
+
+class LocalSGD:
+    """m replicas of a fully connected model on one GPU, trained by local SGD
+    steps and periodic averaging.  Thin wrapper over the ls_* calls."""
+
+    def __init__(self, m: int, dims: Sequence[int], loss: str = "softmax_ce", has_bias: bool = True,
+                 gemm_dtype: str = "fp32", lr: float = 0.05, momentum: float = 0.0, batch: int = 32,
+                 momentum_mode: str = "average", device: str = "cuda:0", stream=None):
+        import torch
+        self._torch = torch
+        self.lib = _lib()
+        self.m, self.batch, self.dims = int(m), int(batch), tuple(int(d) for d in dims)
+        self.gemm_dtype = gemm_dtype
+        self.loss_kind = loss
+        self.spec = make_spec(dims, loss, has_bias, gemm_dtype, momentum_mode)
+        self.P = param_count(self.spec)
+        nbytes = state_bytes(self.m, self.spec, self.batch)
+        self.device = torch.device(device)
+        with torch.cuda.device(self.device):
+            self.state = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.state.data_ptr()
+            self._state_ptr = (base + 255) // 256 * 256
+            self.stream = stream if stream is not None else torch.cuda.current_stream()
+            h = C.c_void_p()
+            _check(self.lib.ls_create(C.byref(h), self.m, C.byref(self.spec), float(lr), float(momentum), self.batch,
+                                      self._state_ptr, nbytes, int(self.stream.cuda_stream)), "ls_create")
+        self.h = h
+        self._x = self._y = None
+
+    # -- life cycle -------------------------------------------------------
+    def close(self):
+        if getattr(self, "h", None) is not None and self.h.value:
+            self.lib.ls_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def sync(self):
+        _check(self.lib.ls_sync(self.h), "ls_sync")
+
+    def set_lr(self, lr: float):
+        _check(self.lib.ls_set_lr(self.h, float(lr)), "ls_set_lr")
+
+    # -- state ------------------------------------------------------------
+    def set_params(self, x1: np.ndarray):
+        a = np.ascontiguousarray(x1, dtype=np.float32)
+        if a.size != self.P:
+            raise ValueError("x1 has the wrong size")
+        _check(self.lib.ls_set_params(self.h, a.ctypes.data), "ls_set_params")
+
+    def set_state(self, replica: int, params: Optional[np.ndarray] = None, momentum: Optional[np.ndarray] = None):
+        p = None if params is None else np.ascontiguousarray(params, dtype=np.float32)
+        v = None if momentum is None else np.ascontiguousarray(momentum, dtype=np.float32)
+        for a in (p, v):
+            if a is not None and a.size != self.P:
+                raise ValueError("wrong size")
+        _check(self.lib.ls_set_state(self.h, int(replica), None if p is None else p.ctypes.data,
+                                     None if v is None else v.ctypes.data), "ls_set_state")
+
+    def get_state(self, replica: int):
+        p = np.empty(self.P, dtype=np.float32)
+        v = np.empty(self.P, dtype=np.float32)
+        _check(self.lib.ls_get_state(self.h, int(replica), p.ctypes.data, v.ctypes.data), "ls_get_state")
+        return p, v
+
+    def get_all(self):
+        ps, vs = zip(*(self.get_state(i) for i in range(self.m)))
+        return np.stack(ps), np.stack(vs)
+
+    def state_view(self):
+        """(params, momentum) as float32 CUDA tensors [m][stride] aliasing the state block."""
+        torch = self._torch
+        pp, vp, st = C.c_void_p(), C.c_void_p(), C.c_int64()
+        _check(self.lib.ls_state_view(self.h, C.byref(pp), C.byref(vp), C.byref(st)), "ls_state_view")
+        base = self.state.data_ptr()
+        out = []
+        for ptr in (pp.value, vp.value):
+            off = ptr - base
+            out.append(self.state[off:off + self.m * st.value * 4].view(torch.float32).view(self.m, st.value))
+        return out[0], out[1]
+
+    # -- data ---------------------------------------------------------------
+    def bind_dataset(self, x, y):
+        torch = self._torch
+        want = torch.bfloat16 if self.gemm_dtype == "bf16" else torch.float32
+        ywant = torch.int32 if self.loss_kind == "softmax_ce" else torch.float32
+        if not (x.is_cuda and x.dtype == want and x.is_contiguous() and x.dim() == 2 and x.shape[1] == self.dims[0]):
+            raise ValueError(f"x must be a contiguous CUDA {want} tensor [n_rows][{self.dims[0]}]")
+        if not (y.is_cuda and y.dtype == ywant and y.is_contiguous() and y.numel() == x.shape[0]):
+            raise ValueError(f"y must be a contiguous CUDA {ywant} tensor [n_rows]")
+        self._x, self._y = x, y
+        _check(self.lib.ls_bind_dataset(self.h, x.data_ptr(), y.data_ptr(), int(x.shape[0])), "ls_bind_dataset")
+
+    # -- hot path -----------------------------------------------------------
+    def local_steps(self, tau: int, row_offsets: np.ndarray, loss_out=None):
+        offs = np.ascontiguousarray(row_offsets, dtype=np.int64)
+        if offs.size != tau * self.m:
+            raise ValueError("row_offsets must be [tau][m]")
+        lp = None
+        if loss_out is not None:
+            torch = self._torch
+            if not (loss_out.is_cuda and loss_out.dtype == torch.float32 and loss_out.is_contiguous()
+                    and loss_out.numel() >= tau * self.m):
+                raise ValueError("loss_out must be a contiguous float32 CUDA tensor [tau][m]")
+            lp = loss_out.data_ptr()
+        _check(self.lib.ls_local_steps(self.h, int(tau), offs.ctypes.data, lp), "ls_local_steps")
+
+    def local_steps_host(self, tau: int, x_host, y_host, loss_host):
+        """x_host [tau][m][batch][d_in], y_host [tau][m][batch], loss_host float32 [tau][m]: CPU torch
+        tensors (pinned for overlap)."""
+        _check(self.lib.ls_local_steps_host(self.h, int(tau), x_host.data_ptr(), y_host.data_ptr(),
+                                            loss_host.data_ptr()), "ls_local_steps_host")
+
+    def average(self):
+        _check(self.lib.ls_average(self.h), "ls_average")
+
+    def eval_loss(self, replica: int, row_offset: int, n_rows: int) -> float:
+        f = C.c_float()
+        _check(self.lib.ls_eval_loss(self.h, int(replica), int(row_offset), int(n_rows), C.byref(f)), "ls_eval_loss")
+        return float(f.value)
+
+    def run(self, K: int, tau_0: int, row_offsets: np.ndarray, interval: int = 0, probe_rows: int = 0, loss_out=None):
+        """K iterations of local steps + averaging in native code; AdaComm when interval > 0."""
+        offs = np.ascontiguousarray(row_offsets, dtype=np.int64)
+        if offs.size != K * self.m:
+            raise ValueError("row_offsets must be [K][m]")
+        max_p = int(K) + 1
+        period_tau = np.zeros(max_p, dtype=np.int32)
+        dk = np.zeros(max_p, dtype=np.int64)
+        dF = np.zeros(max_p, dtype=np.float32)
+        dt = np.zeros(max_p, dtype=np.int32)
+        n_p, n_d, F0 = C.c_int64(), C.c_int64(), C.c_float()
+        lp = None if loss_out is None else loss_out.data_ptr()
+        _check(self.lib.ls_run(self.h, int(K), int(tau_0), int(interval), int(probe_rows), offs.ctypes.data, lp,
+                               period_tau.ctypes.data, max_p, C.byref(n_p), dk.ctypes.data, dF.ctypes.data,
+                               dt.ctypes.data, max_p, C.byref(n_d), C.byref(F0)), "ls_run")
+        n_p, n_d = n_p.value, n_d.value
+        return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
+                "decision_tau": dt[:n_d].tolist(), "F_0": float(F0.value) if interval > 0 else None}
+
+    def launch_count(self) -> int:
+        n = C.c_int64()
+        _check(self.lib.ls_launch_count(self.h, C.byref(n)), "ls_launch_count")
+        return n.value

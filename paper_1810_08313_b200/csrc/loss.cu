@@ -1,0 +1,128 @@
+// Loss layer and small per-layer kernels.
+//
+//   loss_kernel   per-sample loss f(x; s_i), its mini-batch mean (the
+//                 empirical risk of Section 2 restricted to the batch) and the
+//                 gradient of that mean with respect to the network output:
+//                   softmax cross-entropy  dZ = (softmax(z) - onehot(y)) / |xi|
+//                   half squared error     dZ = (z - y) / |xi|
+//   bias_kernel   gb = column sums of dZ; v <- mu v + gb; b <- b - eta v
+//   to_bf16       refresh of the bf16 weight copies
+//
+// All sums run in a fixed order (no floating-point atomics).
+#include "ls_internal.h"
+
+namespace ls {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ void put(float* p, float v) { *p = v; }
+__device__ __forceinline__ void put(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+template <typename TD>
+__global__ void __launch_bounds__(kThreads)
+loss_kernel(const float* __restrict__ logits, const void* __restrict__ y, const int64_t* __restrict__ row_off,
+            TD* __restrict__ dZ, float* __restrict__ loss_out, int B, int C, int kind) {
+  __shared__ float red[kThreads];
+  const int g = blockIdx.x;
+  const float* z = logits + (int64_t)g * B * C;
+  TD* dz = dZ ? dZ + (int64_t)g * B * C : nullptr;
+  const int64_t r0 = row_off[g];
+  const float invB = 1.0f / (float)B;
+  float part = 0.f;
+  for (int b = threadIdx.x; b < B; b += kThreads) {
+    const float* zb = z + (int64_t)b * C;
+    if (kind == LS_LOSS_SOFTMAX_CE) {
+      const int label = static_cast<const int32_t*>(y)[r0 + b];
+      float mx = zb[0];
+      for (int c = 1; c < C; ++c) mx = fmaxf(mx, zb[c]);
+      float sum = 0.f;
+      for (int c = 0; c < C; ++c) sum += expf(zb[c] - mx);
+      const float zy = (label >= 0 && label < C) ? zb[label] : mx;
+      part += (mx + logf(sum)) - zy;
+      if (dz) {
+        const float inv = 1.0f / sum;
+        for (int c = 0; c < C; ++c) {
+          const float p = expf(zb[c] - mx) * inv;
+          put(dz + (int64_t)b * C + c, (p - (c == label ? 1.f : 0.f)) * invB);
+        }
+      }
+    } else {
+      const float t = static_cast<const float*>(y)[r0 + b];
+      const float r = zb[0] - t;
+      part += 0.5f * r * r;
+      if (dz) put(dz + b, r * invB);
+    }
+  }
+  red[threadIdx.x] = part;
+  __syncthreads();
+  for (int s = kThreads / 2; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0 && loss_out) loss_out[g] = red[0] * invB;
+}
+
+template <typename TD>
+__global__ void __launch_bounds__(kThreads)
+bias_kernel(const TD* __restrict__ dZ, float* __restrict__ bias, float* __restrict__ vbias, int64_t gstride, int B,
+            int N, float lr, float mu) {
+  const int g = blockIdx.y;
+  const int j = blockIdx.x * kThreads + threadIdx.x;
+  if (j >= N) return;
+  const TD* d = dZ + (int64_t)g * B * N + j;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) {
+    if constexpr (sizeof(TD) == 2) s += __bfloat162float(d[(int64_t)b * N]);
+    else s += d[(int64_t)b * N];
+  }
+  const int64_t at = (int64_t)g * gstride + j;
+  float step = s;
+  if (mu != 0.f) {
+    step = fmaf(mu, vbias[at], s);
+    vbias[at] = step;
+  }
+  bias[at] = fmaf(-lr, step, bias[at]);
+}
+
+__global__ void __launch_bounds__(kThreads)
+to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t n) {
+  const int64_t step = (int64_t)gridDim.x * kThreads;
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+}  // namespace
+
+int launch_loss(const LossArgs& a, bool dz_bf16, cudaStream_t st, int64_t* launches) {
+  if (launches) ++*launches;
+  if (dz_bf16)
+    loss_kernel<__nv_bfloat16><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<__nv_bfloat16*>(a.dZ),
+                                                              a.loss_out, a.B, a.C, a.loss_kind);
+  else
+    loss_kernel<float><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<float*>(a.dZ), a.loss_out,
+                                                      a.B, a.C, a.loss_kind);
+  return cudaGetLastError();
+}
+
+int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches) {
+  if (launches) ++*launches;
+  dim3 grid((unsigned)((a.N + kThreads - 1) / kThreads), (unsigned)a.groups);
+  if (bf16)
+    bias_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(a.dZ), a.bias, a.vbias,
+                                                          a.gstride, a.B, a.N, a.lr, a.mu);
+  else
+    bias_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(a.dZ), a.bias, a.vbias, a.gstride, a.B, a.N,
+                                                  a.lr, a.mu);
+  return cudaGetLastError();
+}
+
+int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches) {
+  if (n <= 0) return cudaSuccess;
+  if (launches) ++*launches;
+  int64_t gx = (n + kThreads - 1) / kThreads;
+  if (gx > 148 * 16) gx = 148 * 16;
+  to_bf16_kernel<<<(unsigned)gx, kThreads, 0, st>>>(src, dst, n);
+  return cudaGetLastError();
+}
+
+}  // namespace ls

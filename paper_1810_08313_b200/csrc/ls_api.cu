@@ -1,0 +1,541 @@
+// Host side of libls.so: the C ABI declared in include/ls.h, the memory layout
+// of the replicas, and the launch sequence of one local step.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "ls_internal.h"
+
+using namespace ls;
+
+namespace ls {
+
+static inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+static inline size_t round_up_sz(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static int check_spec(const ls_model_spec* s) {
+  if (s == nullptr) return LS_ERR_INVALID_ARG;
+  if (s->n_layers < 1 || s->n_layers > LS_MAX_LAYERS) return LS_ERR_INVALID_ARG;
+  for (int l = 0; l <= s->n_layers; ++l)
+    if (s->dims[l] < 1 || s->dims[l] > (1 << 20)) return LS_ERR_INVALID_ARG;
+  if (s->dims[s->n_layers] > LS_MAX_OUT) return LS_ERR_INVALID_ARG;
+  if (s->loss != LS_LOSS_SOFTMAX_CE && s->loss != LS_LOSS_MSE_HALF) return LS_ERR_INVALID_ARG;
+  if (s->loss == LS_LOSS_MSE_HALF && s->dims[s->n_layers] != 1) return LS_ERR_INVALID_ARG;
+  if (s->has_bias != 0 && s->has_bias != 1) return LS_ERR_INVALID_ARG;
+  if (s->gemm_dtype != LS_GEMM_FP32 && s->gemm_dtype != LS_GEMM_BF16) return LS_ERR_INVALID_ARG;
+  if (s->momentum_mode < LS_MOMENTUM_AVERAGE || s->momentum_mode > LS_MOMENTUM_RESET) return LS_ERR_INVALID_ARG;
+  if (!(s->weight_decay == 0.0f)) return isfinite(s->weight_decay) ? LS_ERR_UNSUPPORTED : LS_ERR_INVALID_ARG;
+  return LS_OK;
+}
+
+int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
+  int rc = check_spec(spec);
+  if (rc != LS_OK) return rc;
+  if (m < 1 || m > LS_MAX_REPLICAS || batch < 1 || batch > LS_MAX_BATCH || out == nullptr) return LS_ERR_INVALID_ARG;
+  Layout lay;
+  lay.L = spec->n_layers;
+  lay.has_bias = spec->has_bias;
+  lay.bf16 = spec->gemm_dtype == LS_GEMM_BF16;
+  lay.m = m;
+  lay.batch = batch;
+  int64_t cur = 0, flat = 0;
+  for (int l = 0; l <= lay.L; ++l) lay.dims[l] = spec->dims[l];
+  for (int l = 0; l < lay.L; ++l) {
+    const int64_t n_out = lay.dims[l + 1], n_in = lay.dims[l];
+    if (n_out > lay.max_width) lay.max_width = (int)n_out;
+    lay.w_off[l] = cur;
+    lay.w_flat[l] = flat;
+    cur = round_up(cur + n_out * n_in, kAlignFloats);
+    flat += n_out * n_in;
+    lay.b_off[l] = cur;
+    lay.b_flat[l] = flat;
+    if (lay.has_bias) {
+      cur = round_up(cur + n_out, kAlignFloats);
+      flat += n_out;
+    }
+  }
+  lay.P = flat;
+  lay.stride = cur;
+  const size_t A = 256;
+  const size_t esz = lay.bf16 ? 2 : 4;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off = round_up_sz(off + bytes, A); return at; };
+  lay.params_off = take((size_t)m * lay.stride * 4);
+  lay.mom_off = take((size_t)m * lay.stride * 4);
+  lay.shadow_off = take(lay.bf16 ? (size_t)m * lay.stride * 2 : 0);
+  for (int l = 1; l < lay.L; ++l) lay.act_off[l] = take((size_t)m * batch * lay.dims[l] * esz);
+  lay.dz_off[0] = take((size_t)m * batch * lay.max_width * esz);
+  lay.dz_off[1] = take((size_t)m * batch * lay.max_width * esz);
+  lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
+  lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
+  lay.evaloff_off = take((size_t)kEvalCap * 8);
+  lay.evalloss_off = take((size_t)kEvalCap * 4);
+  for (int s = 0; s < 2; ++s) {
+    lay.stage_x_off[s] = take((size_t)m * batch * lay.dims[0] * esz);
+    lay.stage_y_off[s] = take((size_t)m * batch * 4);
+  }
+  lay.stage_loss_off = take((size_t)kRowOffCap * m * 4);
+  lay.total = off;
+  *out = lay;
+  return LS_OK;
+}
+
+static inline bool ok_handle(const ls_handle* h) { return h != nullptr && h->magic == kMagic; }
+
+static int cuda_fail(ls_handle* h, int e) {
+  if (h) h->last_cuda = e;
+  return LS_ERR_CUDA;
+}
+#define LS_CUDA(h, expr)                                 \
+  do {                                                   \
+    int _e = (int)(expr);                                \
+    if (_e != (int)cudaSuccess) return cuda_fail(h, _e); \
+  } while (0)
+
+static int refresh_shadow(ls_handle* h) {
+  if (!h->lay.bf16) return LS_OK;
+  LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), (int64_t)h->lay.m * h->lay.stride, h->stream, &h->launches));
+  return LS_OK;
+}
+
+// One forward pass of `groups` mini-batches.  Group g reads rows
+// [row_off[g], +batch) of x/y and uses the weights at w_base + g*w_gstride
+// (w_gstride == 0: every group uses the same replica).
+static int forward(ls_handle* h, const void* x, const void* y, const int64_t* row_off_dev, int groups,
+                   int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
+  const Layout& lay = h->lay;
+  const bool bf = lay.bf16;
+  const float* P = params_of(h) + replica0 * lay.stride;
+  const __nv_bfloat16* S = bf ? shadow_of(h) + replica0 * lay.stride : nullptr;
+  for (int l = 0; l < lay.L; ++l) {
+    FwdArgs a;
+    a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
+    a.row_off = (l == 0) ? row_off_dev : nullptr;
+    a.W = bf ? (const void*)(S + lay.w_off[l]) : (const void*)(P + lay.w_off[l]);
+    a.w_gstride = w_gstride;
+    a.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
+    a.bias_gstride = w_gstride;
+    const bool last = (l == lay.L - 1);
+    a.C = last ? (void*)(h->state + lay.logits_off) : (void*)(h->state + lay.act_off[l + 1]);
+    a.M = lay.batch; a.N = lay.dims[l + 1]; a.K = lay.dims[l]; a.groups = groups;
+    a.relu = last ? 0 : 1;
+    LS_CUDA(h, launch_fwd(a, bf, bf, bf && !last, h->stream, &h->launches));
+  }
+  LossArgs la;
+  la.logits = reinterpret_cast<const float*>(h->state + lay.logits_off);
+  la.y = y; la.row_off = row_off_dev;
+  la.dZ = want_dz ? (void*)(h->state + lay.dz_off[0]) : nullptr;
+  la.loss_out = loss_out;
+  la.B = lay.batch; la.C = lay.dims[lay.L]; la.groups = groups; la.loss_kind = h->spec.loss;
+  LS_CUDA(h, launch_loss(la, bf, h->stream, &h->launches));
+  return LS_OK;
+}
+
+// One local update of all m replicas (forward, backward, fused SGD-momentum).
+static int local_step(ls_handle* h, const void* x, const void* y, const int64_t* row_off_dev, float* loss_out) {
+  const Layout& lay = h->lay;
+  const bool bf = lay.bf16;
+  int rc = forward(h, x, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
+  if (rc != LS_OK) return rc;
+  int cur = 0;
+  for (int l = lay.L - 1; l >= 0; --l) {
+    void* dZ = h->state + lay.dz_off[cur];
+    if (l > 0) {
+      // the data gradient reads W_l before the update below overwrites it
+      DxArgs d;
+      d.dZ = dZ;
+      d.W = bf ? (const void*)(shadow_of(h) + lay.w_off[l]) : (const void*)(params_of(h) + lay.w_off[l]);
+      d.w_gstride = lay.stride;
+      d.act = h->state + lay.act_off[l];
+      d.C = h->state + lay.dz_off[cur ^ 1];
+      d.M = lay.batch; d.N = lay.dims[l]; d.K = lay.dims[l + 1]; d.groups = lay.m;
+      LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
+    }
+    DwArgs w;
+    w.dZ = dZ;
+    w.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
+    w.row_off = (l == 0) ? row_off_dev : nullptr;
+    w.W = params_of(h) + lay.w_off[l];
+    w.V = mom_of(h) + lay.w_off[l];
+    w.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
+    w.w_gstride = lay.stride;
+    w.M = lay.dims[l + 1]; w.N = lay.dims[l]; w.B = lay.batch; w.groups = lay.m;
+    w.lr = h->lr; w.mu = h->mu;
+    LS_CUDA(h, launch_dw(w, bf, h->stream, &h->launches));
+    if (lay.has_bias) {
+      BiasArgs b;
+      b.dZ = dZ;
+      b.bias = params_of(h) + lay.b_off[l];
+      b.vbias = mom_of(h) + lay.b_off[l];
+      b.gstride = lay.stride;
+      b.B = lay.batch; b.N = lay.dims[l + 1]; b.groups = lay.m;
+      b.lr = h->lr; b.mu = h->mu;
+      LS_CUDA(h, launch_bias(b, bf, h->stream, &h->launches));
+    }
+    cur ^= 1;
+  }
+  return LS_OK;
+}
+
+static int average(ls_handle* h) {
+  const Layout& lay = h->lay;
+  const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
+  const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
+  LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
+                            lay.bf16 ? shadow_of(h) : nullptr, h->stream, &h->launches));
+  if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
+    LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  return LS_OK;
+}
+
+static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_rows, float* F_host) {
+  const Layout& lay = h->lay;
+  if (h->x_dev == nullptr) return LS_ERR_NO_DATASET;
+  if (replica < 0 || replica >= lay.m || F_host == nullptr || n_rows < lay.batch || n_rows % lay.batch != 0)
+    return LS_ERR_INVALID_ARG;
+  if (row_offset < 0 || row_offset + n_rows > h->n_rows) return LS_ERR_ROW_RANGE;
+  const int64_t chunks = n_rows / lay.batch;
+  if (chunks > kEvalCap) return LS_ERR_INVALID_ARG;
+  std::vector<int64_t> offs((size_t)chunks);
+  for (int64_t c = 0; c < chunks; ++c) offs[(size_t)c] = row_offset + c * lay.batch;
+  int64_t* off_dev = reinterpret_cast<int64_t*>(h->state + lay.evaloff_off);
+  float* loss_dev = reinterpret_cast<float*>(h->state + lay.evalloss_off);
+  LS_CUDA(h, cudaMemcpyAsync(off_dev, offs.data(), (size_t)chunks * 8, cudaMemcpyHostToDevice, h->stream));
+  for (int64_t c0 = 0; c0 < chunks; c0 += lay.m) {
+    const int groups = (int)((chunks - c0 < lay.m) ? chunks - c0 : lay.m);
+    int rc = forward(h, h->x_dev, h->y_dev, off_dev + c0, groups, replica, 0, false, loss_dev + c0);
+    if (rc != LS_OK) return rc;
+  }
+  LS_CUDA(h, cudaMemcpyAsync(h->pinned, loss_dev, (size_t)chunks * 4, cudaMemcpyDeviceToHost, h->stream));
+  LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  double s = 0.0;
+  for (int64_t c = 0; c < chunks; ++c) s += (double)h->pinned[c];
+  *F_host = (float)(s / (double)chunks);
+  return LS_OK;
+}
+
+static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev) {
+  const Layout& lay = h->lay;
+  if (tau < 1 || row_offset_host == nullptr) return LS_ERR_INVALID_ARG;
+  if (h->x_dev == nullptr) return LS_ERR_NO_DATASET;
+  for (int64_t i = 0; i < (int64_t)tau * lay.m; ++i)
+    if (row_offset_host[i] < 0 || row_offset_host[i] + lay.batch > h->n_rows) return LS_ERR_ROW_RANGE;
+  int64_t* off_dev = reinterpret_cast<int64_t*>(h->state + lay.rowoff_off);
+  for (int s0 = 0; s0 < tau; s0 += kRowOffCap) {
+    const int n = (tau - s0 < kRowOffCap) ? tau - s0 : kRowOffCap;
+    LS_CUDA(h, cudaMemcpyAsync(off_dev, row_offset_host + (int64_t)s0 * lay.m, (size_t)n * lay.m * 8,
+                               cudaMemcpyHostToDevice, h->stream));
+    for (int s = 0; s < n; ++s) {
+      int rc = local_step(h, h->x_dev, h->y_dev, off_dev + (int64_t)s * lay.m,
+                          loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr);
+      if (rc != LS_OK) return rc;
+    }
+  }
+  return LS_OK;
+}
+
+}  // namespace ls
+
+// ---------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------
+
+extern "C" {
+
+const char* ls_strerror(int code) {
+  switch (code) {
+    case LS_OK: return "ok";
+    case LS_ERR_INVALID_ARG: return "invalid argument";
+    case LS_ERR_BAD_HANDLE: return "bad handle";
+    case LS_ERR_STATE_SIZE: return "state block too small or misaligned";
+    case LS_ERR_NO_DATASET: return "no dataset bound";
+    case LS_ERR_ROW_RANGE: return "mini-batch rows outside the dataset";
+    case LS_ERR_CUDA: return "CUDA error";
+    case LS_ERR_UNSUPPORTED: return "not supported";
+    case LS_ERR_OVERFLOW: return "result does not fit";
+    default: return "unknown error";
+  }
+}
+
+int ls_param_count(const ls_model_spec* spec, int64_t* P) {
+  int rc = check_spec(spec);
+  if (rc != LS_OK) return rc;
+  if (P == nullptr) return LS_ERR_INVALID_ARG;
+  int64_t n = 0;
+  for (int l = 0; l < spec->n_layers; ++l)
+    n += (int64_t)spec->dims[l + 1] * spec->dims[l] + (spec->has_bias ? spec->dims[l + 1] : 0);
+  *P = n;
+  return LS_OK;
+}
+
+int ls_state_bytes(int m, const ls_model_spec* spec, int batch, size_t* bytes) {
+  if (bytes == nullptr) return LS_ERR_INVALID_ARG;
+  Layout lay;
+  int rc = make_layout(m, spec, batch, &lay);
+  if (rc != LS_OK) return rc;
+  *bytes = lay.total;
+  return LS_OK;
+}
+
+int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float momentum, int batch, void* state_dev,
+              size_t state_bytes, void* cuda_stream) {
+  if (out == nullptr) return LS_ERR_INVALID_ARG;
+  *out = nullptr;
+  Layout lay;
+  int rc = make_layout(m, spec, batch, &lay);
+  if (rc != LS_OK) return rc;
+  if (!isfinite(lr) || !isfinite(momentum) || momentum < 0.f || momentum >= 1.f) return LS_ERR_INVALID_ARG;
+  if (state_dev == nullptr || reinterpret_cast<uintptr_t>(state_dev) % 256 != 0 || state_bytes < lay.total)
+    return LS_ERR_STATE_SIZE;
+  ls_handle* h = new (std::nothrow) ls_handle();
+  if (h == nullptr) return LS_ERR_INVALID_ARG;
+  memset(h, 0, sizeof(*h));
+  h->magic = kMagic;
+  h->lay = lay;
+  h->spec = *spec;
+  h->lr = lr;
+  h->mu = momentum;
+  h->state = static_cast<char*>(state_dev);
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  int e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
+  for (int s = 0; s < 2 && e == cudaSuccess; ++s) {
+    e = cudaEventCreateWithFlags(&h->ev_copied[s], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_consumed[s], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&h->pinned), (size_t)kEvalCap * 4);
+  // parameters, momentum, workspace start at zero; the staging row offsets are g*batch
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->state, 0, lay.total, h->stream);
+  if (e != cudaSuccess) {
+    ls_destroy(h);
+    return LS_ERR_CUDA;
+  }
+  *out = h;
+  return LS_OK;
+}
+
+int ls_destroy(ls_handle* h) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  cudaStreamSynchronize(h->stream);
+  if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
+  for (int s = 0; s < 2; ++s) {
+    if (h->ev_copied[s]) cudaEventDestroy(h->ev_copied[s]);
+    if (h->ev_consumed[s]) cudaEventDestroy(h->ev_consumed[s]);
+  }
+  if (h->pinned) cudaFreeHost(h->pinned);
+  h->magic = 0;
+  delete h;
+  return LS_OK;
+}
+
+int ls_sync(ls_handle* h) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  LS_CUDA(h, cudaGetLastError());
+  return LS_OK;
+}
+
+int ls_last_cuda_error(const ls_handle* h) { return ok_handle(h) ? h->last_cuda : LS_ERR_BAD_HANDLE; }
+
+int ls_set_lr(ls_handle* h, float lr) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (!isfinite(lr)) return LS_ERR_INVALID_ARG;
+  h->lr = lr;
+  return LS_OK;
+}
+
+// copy one replica between the flat interface layout (host) and the padded device layout
+static int copy_replica(ls_handle* h, float* dev_base, float* host, bool to_dev) {
+  const Layout& lay = h->lay;
+  for (int l = 0; l < lay.L; ++l) {
+    const size_t wn = (size_t)lay.dims[l + 1] * lay.dims[l] * 4, bn = (size_t)lay.dims[l + 1] * 4;
+    if (to_dev) {
+      LS_CUDA(h, cudaMemcpyAsync(dev_base + lay.w_off[l], host + lay.w_flat[l], wn, cudaMemcpyHostToDevice, h->stream));
+      if (lay.has_bias)
+        LS_CUDA(h, cudaMemcpyAsync(dev_base + lay.b_off[l], host + lay.b_flat[l], bn, cudaMemcpyHostToDevice, h->stream));
+    } else {
+      LS_CUDA(h, cudaMemcpyAsync(host + lay.w_flat[l], dev_base + lay.w_off[l], wn, cudaMemcpyDeviceToHost, h->stream));
+      if (lay.has_bias)
+        LS_CUDA(h, cudaMemcpyAsync(host + lay.b_flat[l], dev_base + lay.b_off[l], bn, cudaMemcpyDeviceToHost, h->stream));
+    }
+  }
+  return LS_OK;
+}
+
+int ls_set_params(ls_handle* h, const float* x1_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (x1_host == nullptr) return LS_ERR_INVALID_ARG;
+  const Layout& lay = h->lay;
+  int rc = copy_replica(h, params_of(h), const_cast<float*>(x1_host), true);
+  if (rc != LS_OK) return rc;
+  for (int i = 1; i < lay.m; ++i)
+    LS_CUDA(h, cudaMemcpyAsync(params_of(h) + (int64_t)i * lay.stride, params_of(h), (size_t)lay.stride * 4,
+                               cudaMemcpyDeviceToDevice, h->stream));
+  LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  rc = refresh_shadow(h);
+  if (rc != LS_OK) return rc;
+  return ls_sync(h);
+}
+
+int ls_set_state(ls_handle* h, int replica, const float* params_host, const float* momentum_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (replica < 0 || replica >= h->lay.m) return LS_ERR_INVALID_ARG;
+  int rc = LS_OK;
+  if (params_host)
+    rc = copy_replica(h, params_of(h) + (int64_t)replica * h->lay.stride, const_cast<float*>(params_host), true);
+  if (rc == LS_OK && momentum_host)
+    rc = copy_replica(h, mom_of(h) + (int64_t)replica * h->lay.stride, const_cast<float*>(momentum_host), true);
+  if (rc == LS_OK && params_host) rc = refresh_shadow(h);
+  if (rc != LS_OK) return rc;
+  return ls_sync(h);
+}
+
+int ls_get_state(ls_handle* h, int replica, float* params_host, float* momentum_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (replica < 0 || replica >= h->lay.m) return LS_ERR_INVALID_ARG;
+  int rc = LS_OK;
+  if (params_host) rc = copy_replica(h, params_of(h) + (int64_t)replica * h->lay.stride, params_host, false);
+  if (rc == LS_OK && momentum_host)
+    rc = copy_replica(h, mom_of(h) + (int64_t)replica * h->lay.stride, momentum_host, false);
+  if (rc != LS_OK) return rc;
+  return ls_sync(h);
+}
+
+int ls_state_view(ls_handle* h, float** params_dev, float** momentum_dev, int64_t* stride_floats) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (params_dev) *params_dev = params_of(h);
+  if (momentum_dev) *momentum_dev = mom_of(h);
+  if (stride_floats) *stride_floats = h->lay.stride;
+  return LS_OK;
+}
+
+int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t n_rows) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (x_dev == nullptr || y_dev == nullptr || n_rows < h->lay.batch) return LS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(x_dev) % 16 != 0 || reinterpret_cast<uintptr_t>(y_dev) % 4 != 0)
+    return LS_ERR_INVALID_ARG;
+  h->x_dev = x_dev;
+  h->y_dev = y_dev;
+  h->n_rows = n_rows;
+  return LS_OK;
+}
+
+int ls_local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  return local_steps(h, tau, row_offset_host, loss_dev);
+}
+
+int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y_host, float* loss_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (tau < 1 || x_host == nullptr || y_host == nullptr || loss_host == nullptr) return LS_ERR_INVALID_ARG;
+  const Layout& lay = h->lay;
+  const size_t esz = lay.bf16 ? 2 : 4;
+  const size_t xb = (size_t)lay.m * lay.batch * lay.dims[0] * esz, yb = (size_t)lay.m * lay.batch * 4;
+  // group g of a staged step reads rows [g*batch, +batch) of the staging buffer
+  int64_t* stage_off = reinterpret_cast<int64_t*>(h->state + lay.evaloff_off);
+  {
+    int64_t offs[LS_MAX_REPLICAS];
+    for (int g = 0; g < lay.m; ++g) offs[g] = (int64_t)g * lay.batch;
+    LS_CUDA(h, cudaMemcpyAsync(stage_off, offs, (size_t)lay.m * 8, cudaMemcpyHostToDevice, h->stream));
+    LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  }
+  float* loss_stage = reinterpret_cast<float*>(h->state + lay.stage_loss_off);
+  bool used[2] = {false, false};
+  for (int s0 = 0; s0 < tau; s0 += kRowOffCap) {
+    const int n = (tau - s0 < kRowOffCap) ? tau - s0 : kRowOffCap;
+    for (int s = 0; s < n; ++s) {
+      const int slot = (s0 + s) & 1;
+      void* xs = h->state + lay.stage_x_off[slot];
+      void* ys = h->state + lay.stage_y_off[slot];
+      if (used[slot]) LS_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed[slot], 0));
+      LS_CUDA(h, cudaMemcpyAsync(xs, static_cast<const char*>(x_host) + (size_t)(s0 + s) * xb, xb,
+                                 cudaMemcpyHostToDevice, h->copy_stream));
+      LS_CUDA(h, cudaMemcpyAsync(ys, static_cast<const char*>(y_host) + (size_t)(s0 + s) * yb, yb,
+                                 cudaMemcpyHostToDevice, h->copy_stream));
+      LS_CUDA(h, cudaEventRecord(h->ev_copied[slot], h->copy_stream));
+      LS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_copied[slot], 0));
+      int rc = local_step(h, xs, ys, stage_off, loss_stage + (int64_t)s * lay.m);
+      if (rc != LS_OK) return rc;
+      LS_CUDA(h, cudaEventRecord(h->ev_consumed[slot], h->stream));
+      used[slot] = true;
+    }
+    LS_CUDA(h, cudaMemcpyAsync(loss_host + (int64_t)s0 * lay.m, loss_stage, (size_t)n * lay.m * 4,
+                               cudaMemcpyDeviceToHost, h->stream));
+    LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  }
+  return LS_OK;
+}
+
+int ls_average(ls_handle* h) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  return average(h);
+}
+
+int ls_eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_rows, float* F_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  return eval_loss(h, replica, row_offset, n_rows, F_host);
+}
+
+int adacomm_next_tau(double F_t, double F_0, int tau_0) {
+  if (!isfinite(F_t) || !isfinite(F_0) || !(F_0 > 0.0) || F_t < 0.0 || tau_0 < 1) return LS_ERR_INVALID_ARG;
+  const double ratio = F_t / F_0;
+  const double t = sqrt(ratio) * (double)tau_0;
+  double n = ceil(t);
+  if (n < 1.0) n = 1.0;
+  if (!(n <= 2147483647.0)) return LS_ERR_OVERFLOW;
+  return (int)n;
+}
+
+int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
+           float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
+           float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions, float* F0_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (K < 1 || tau_0 < 1 || interval < 0 || row_offset_host == nullptr) return LS_ERR_INVALID_ARG;
+  const Layout& lay = h->lay;
+  float F_0 = 0.f;
+  if (interval > 0) {
+    int rc = eval_loss(h, 0, 0, probe_rows, &F_0);
+    if (rc != LS_OK) return rc;
+    if (F0_host) *F0_host = F_0;
+  }
+  int64_t k = 0, np = 0, nd = 0, next_interval = 1;
+  int tau = tau_0;
+  while (k < K) {
+    const int steps = (int)((K - k < tau) ? K - k : tau);
+    if (period_tau && np < max_periods) period_tau[np] = tau;
+    ++np;
+    int rc = local_steps(h, steps, row_offset_host + k * lay.m, loss_dev ? loss_dev + k * lay.m : nullptr);
+    if (rc != LS_OK) return rc;
+    k += steps;
+    rc = average(h);
+    if (rc != LS_OK) return rc;
+    if (interval > 0 && k >= next_interval * (int64_t)interval) {
+      float F_t = 0.f;
+      rc = eval_loss(h, 0, 0, probe_rows, &F_t);
+      if (rc != LS_OK) return rc;
+      const int t = adacomm_next_tau((double)F_t, (double)F_0, tau_0);
+      if (t < 0) return t;
+      tau = t;
+      if (nd < max_decisions) {
+        if (decision_k) decision_k[nd] = k;
+        if (decision_F) decision_F[nd] = F_t;
+        if (decision_tau) decision_tau[nd] = t;
+      }
+      ++nd;
+      next_interval = k / interval + 1;
+    }
+  }
+  if (n_periods) *n_periods = np;
+  if (n_decisions) *n_decisions = nd;
+  return LS_OK;
+}
+
+int ls_launch_count(const ls_handle* h, int64_t* n) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (n == nullptr) return LS_ERR_INVALID_ARG;
+  *n = h->launches;
+  return LS_OK;
+}
+
+}  // extern "C"

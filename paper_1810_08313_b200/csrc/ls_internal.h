@@ -1,0 +1,146 @@
+// Internal declarations shared by the translation units of libls.so.
+// Nothing here is part of the C ABI (see include/ls.h for that).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "ls.h"
+
+namespace ls {
+
+constexpr int kRowOffCap = 512;        // local steps per offsets upload
+constexpr int kEvalCap = 8192;         // mini-batch chunks per ls_eval_loss call
+constexpr int64_t kAlignFloats = 64;   // every tensor and every replica starts on a 256-byte boundary
+
+// Where everything lives.  Offsets inside one replica are in elements (the
+// same for the fp32 master copy, the momentum buffer and the bf16 copy);
+// offsets inside the state block are in bytes.
+struct Layout {
+  int L = 0;
+  int dims[LS_MAX_LAYERS + 1] = {0};
+  int has_bias = 0;
+  int bf16 = 0;
+  int m = 0;
+  int batch = 0;
+  int max_width = 0;                   // max(dims[1..L])
+  int64_t P = 0;                       // interface parameter count
+  int64_t stride = 0;                  // elements between replicas (padded)
+  int64_t w_off[LS_MAX_LAYERS] = {0};  // padded offsets inside a replica
+  int64_t b_off[LS_MAX_LAYERS] = {0};
+  int64_t w_flat[LS_MAX_LAYERS] = {0}; // offsets in the flat interface layout
+  int64_t b_flat[LS_MAX_LAYERS] = {0};
+  size_t params_off = 0, mom_off = 0, shadow_off = 0;
+  size_t act_off[LS_MAX_LAYERS + 1] = {0};   // post-ReLU activations of layers 1..L-1
+  size_t dz_off[2] = {0, 0};                 // ping-pong gradient buffers [m][batch][max_width]
+  size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
+  size_t rowoff_off = 0;                     // int64 [kRowOffCap][m]
+  size_t evaloff_off = 0;                    // int64 [m]  (two slots)
+  size_t evalloss_off = 0;                   // float [kEvalCap]
+  size_t stage_x_off[2] = {0, 0};            // [m][batch][dims[0]] input staging for host batches
+  size_t stage_y_off[2] = {0, 0};            // [m][batch] labels / targets
+  size_t stage_loss_off = 0;                 // float [kRowOffCap][m]
+  size_t total = 0;
+};
+
+int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out);
+
+}  // namespace ls
+
+struct ls_handle {
+  uint32_t magic;
+  ls::Layout lay;
+  ls_model_spec spec;
+  float lr, mu;
+  char* state;
+  cudaStream_t stream;
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copied[2], ev_consumed[2];
+  const void* x_dev;
+  const void* y_dev;
+  int64_t n_rows;
+  int last_cuda;
+  int64_t launches;
+  float* pinned;          // small pinned host scratch (eval losses)
+};
+
+namespace ls {
+
+constexpr uint32_t kMagic = 0x4c53474du;
+
+inline float* params_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.params_off); }
+inline float* mom_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.mom_off); }
+inline __nv_bfloat16* shadow_of(const ls_handle* h) {
+  return reinterpret_cast<__nv_bfloat16*>(h->state + h->lay.shadow_off);
+}
+
+// ---- averaging (average.cu) ---------------------------------------------
+// n_buf buffers of m vectors each; buffer b starts at base + b*buf_stride floats,
+// vector j of it at + j*stride.  shadow (optional) receives the bf16 rounding of
+// the mean of buffer 0 with the same strides.  Returns a cudaError_t.
+int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
+                   __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches);
+
+// ---- fp32-accumulate CUDA-core grouped GEMMs (gemm_simt.cu) ---------------
+struct FwdArgs {           // Z = A W^T + b, optional ReLU
+  const void* A;           // [groups][M][K] (or dataset rows through row_off)
+  const int64_t* row_off;  // device, per group first row of A; null: group g starts at g*M
+  const void* W;           // weight matrix of group 0, [N][K]
+  int64_t w_gstride;       // elements between groups' weights (0: shared)
+  const float* bias;       // fp32 master bias of group 0 or null
+  int64_t bias_gstride;
+  void* C;                 // [groups][M][N]
+  int M, N, K, groups;
+  int relu;
+};
+struct DxArgs {            // dZ_prev = (dZ W) * 1[act > 0]
+  const void* dZ;          // [groups][M][K]
+  const void* W;           // [K][N]
+  int64_t w_gstride;
+  const void* act;         // [groups][M][N] post-ReLU activation of the previous layer
+  void* C;                 // [groups][M][N]
+  int M, N, K, groups;
+};
+struct DwArgs {            // G = dZ^T A ; v = mu v + G ; W -= lr v ; optional bf16 copy
+  const void* dZ;          // [groups][B][M]
+  const void* A;           // [groups][B][N] (or dataset rows through row_off)
+  const int64_t* row_off;
+  float* W;                // fp32 master [M][N] of group 0
+  float* V;                // momentum, same layout (unused when mu == 0)
+  __nv_bfloat16* Wb;       // bf16 copy or null
+  int64_t w_gstride;
+  int M, N, B, groups;
+  float lr, mu;
+};
+int launch_fwd(const FwdArgs& a, bool a_bf16, bool w_bf16, bool c_bf16, cudaStream_t st, int64_t* launches);
+int launch_dx(const DxArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
+int launch_dw(const DwArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
+
+// ---- loss, dZ_L, bias update (loss.cu) ------------------------------------
+struct LossArgs {
+  const float* logits;     // [groups][B][C]
+  const void* y;           // int32 labels or float targets of the bound rows
+  const int64_t* row_off;  // device, per group first row in y
+  void* dZ;                // [groups][B][C] or null (forward only)
+  float* loss_out;         // [groups] or null
+  int B, C, groups;
+  int loss_kind;
+};
+int launch_loss(const LossArgs& a, bool dz_bf16, cudaStream_t st, int64_t* launches);
+
+struct BiasArgs {          // gb = colsum(dZ); v = mu v + gb; b -= lr v
+  const void* dZ;          // [groups][B][N]
+  float* bias;
+  float* vbias;
+  int64_t gstride;
+  int B, N, groups;
+  float lr, mu;
+};
+int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
+
+// fp32 -> bf16 copy of n elements (refresh of the weight copies)
+int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);
+
+}  // namespace ls

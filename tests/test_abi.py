@@ -1,0 +1,78 @@
+"""The C-ABI library builds, loads and exports every symbol include/ls.h declares.
+(No compute calls: this runs without a GPU.)"""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if not fn.endswith(".h"):
+            continue
+        src = open(os.path.join(ROOT, "include", fn)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        for m in re.finditer(r"^\s*(?:const\s+)?[A-Za-z_][\w\s\*]*?\b(\w+)\s*\([^;{]*\)\s*;", src, flags=re.M):
+            names.add(m.group(1))
+    return names
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    from paper_1810_08313_b200 import build
+    path = build.build()
+    assert os.path.exists(path)
+    lib = ctypes.CDLL(path)
+    names = _declared_functions()
+    assert {"ls_create", "ls_local_steps", "ls_average", "adacomm_next_tau", "ls_average_flat"} <= names
+    for n in sorted(names):
+        assert hasattr(lib, n), n
+
+
+def test_pure_host_entry_points():
+    from paper_1810_08313_b200 import binding
+    # controller: identical decisions to the hand table (Section 4.2 basic rule)
+    rows = []
+    for line in open(os.path.join(ROOT, "tests", "golden", "adacomm_table.txt")):
+        line = line.split("#")[0].strip()
+        if line:
+            a = line.split()
+            rows.append((float(a[0]), float(a[1]), int(a[2]), int(a[3])))
+    for F_t, F_0, tau_0, want in rows:
+        assert binding.adacomm_next_tau(F_t, F_0, tau_0) == want
+    lib = binding._lib()
+    for bad in [(1.0, 0.0, 20), (1.0, -1.0, 20), (-0.5, 1.0, 20), (float("nan"), 1.0, 20), (1.0, float("inf"), 20),
+                (1.0, 1.0, 0)]:
+        assert lib.adacomm_next_tau(*bad) == binding.LS_ERR_INVALID_ARG
+    assert lib.adacomm_next_tau(1e300, 1e-300, 2 ** 30) == binding.LS_ERR_OVERFLOW
+    # sizes
+    spec = binding.make_spec((3072, 512, 512, 10))
+    assert binding.param_count(spec) == 1_841_162
+    assert binding.param_count(binding.make_spec((3072, 2048, 2048, 2048, 10))) == 14_706_698
+    assert binding.param_count(binding.make_spec((784, 10))) == 7_850
+    assert binding.param_count(binding.make_spec((4096, 1), "mse_half", False)) == 4_096
+    assert binding.state_bytes(8, spec, 128) > 2 * 8 * 1_841_162 * 4
+    bad = binding.make_spec((16, 8))
+    bad.n_layers = 0
+    n = ctypes.c_int64()
+    assert lib.ls_param_count(ctypes.byref(bad), ctypes.byref(n)) == binding.LS_ERR_INVALID_ARG
+    wd = binding.make_spec((16, 8), weight_decay=5e-4)
+    assert lib.ls_param_count(ctypes.byref(wd), ctypes.byref(n)) == binding.LS_ERR_UNSUPPORTED
+    assert lib.ls_destroy(None) == binding.LS_ERR_BAD_HANDLE
+    assert lib.ls_average(None) == binding.LS_ERR_BAD_HANDLE
+    assert binding.LsError(binding.LS_ERR_ROW_RANGE, "x").code == binding.LS_ERR_ROW_RANGE
+
+
+def test_controller_agrees_with_oracle_on_a_dense_sweep():
+    from oracle import localsgd_oracle as orc
+    from paper_1810_08313_b200 import binding
+    import numpy as np
+    rng = np.random.default_rng(0)
+    for _ in range(5000):
+        F_0 = float(rng.uniform(0.01, 5.0)); F_t = float(rng.uniform(0.0, 6.0)); tau_0 = int(rng.integers(1, 200))
+        assert binding.adacomm_next_tau(F_t, F_0, tau_0) == orc.adacomm_next_tau(F_t, F_0, tau_0)
+    # float32 losses widened to double, as the run loop does
+    for _ in range(2000):
+        F_0 = float(np.float32(rng.uniform(0.01, 5.0))); F_t = float(np.float32(rng.uniform(0.0, 6.0)))
+        assert binding.adacomm_next_tau(F_t, F_0, 20) == orc.adacomm_next_tau(F_t, F_0, 20)

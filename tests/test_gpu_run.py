@@ -1,0 +1,184 @@
+"""Whole PASGD runs on the GPU vs the oracle (Section 2 PASGD update rule,
+Section 4.2 basic update rule)."""
+import numpy as np
+import pytest
+
+from oracle import localsgd_oracle as orc
+from paper_1810_08313_b200 import workloads as wl
+from tests.helpers import f32, max_rel_err_per_tensor, small_problem, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _bitwise_equal_replicas(eng):
+    p, v = eng.state_view()
+    return bool((p[0:1] == p).all()) and bool((v[0:1] == v).all())
+
+
+def test_softmax_regression_config_every_step():
+    """784-dim softmax regression, m = 4, B = 32, tau = 10, 100 iterations, lr 0.05, zero start:
+    free-running, parameters compared with the oracle after every period, losses at every step."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    w = wl.WORKLOADS["c1_softmax"]
+    X, y = wl.make_dataset(w, n_rows=8192)
+    spec = orc.ModelSpec(w.dims, w.loss, w.has_bias)
+    x1 = wl.initial_point(w)
+    offs = wl.batch_row_offsets(w.seed, w.n_iters, w.m, X.shape[0], w.batch)
+    snaps = {}
+
+    def hook(k, xs, vs, averaged):
+        if averaged:
+            snaps[k] = xs.copy()
+
+    ref = orc.run_pasgd(spec, x1, X, y, offs, w.batch, f32(w.lr), 0.0, 10, state_hook=hook)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(w.m, w.dims, w.loss, w.has_bias, "fp32", lr=w.lr, momentum=0.0, batch=w.batch)
+    eng.bind_dataset(xd, yd)
+    eng.set_params(x1)
+    loss_dev = torch.zeros((w.n_iters, w.m), dtype=torch.float32, device="cuda")
+    for k0 in range(0, w.n_iters, 10):
+        eng.local_steps(10, offs[k0:k0 + 10], loss_dev[k0:k0 + 10])
+        eng.average()
+        eng.sync()
+        assert _bitwise_equal_replicas(eng)
+        gx, _ = eng.get_all()
+        for i in range(w.m):
+            assert max_rel_err_per_tensor(gx[i], snaps[k0 + 10][i], w.dims, w.has_bias) <= 1e-5
+    got = loss_dev.cpu().numpy()
+    assert np.max(np.abs(got - ref.loss) / ref.loss) <= 1e-5
+    assert got[-1].mean() < got[0].mean()          # it learns
+    eng.close()
+
+
+@pytest.mark.parametrize("mode", ["average", "keep", "reset"])
+def test_native_run_matches_oracle_over_three_periods(mode):
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, tau, K = (96, 64, 48, 10), 4, 32, 5, 15
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 21)
+    offs = wl.batch_row_offsets(2, K, m, 1024, B)
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(0.9), tau, momentum_mode=mode)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B, momentum_mode=mode)
+    eng.bind_dataset(xd, yd)
+    eng.set_params(x1)
+    loss_dev = torch.zeros((K, m), dtype=torch.float32, device="cuda")
+    out = eng.run(K, tau, offs, loss_out=loss_dev)
+    eng.sync()
+    assert out["taus"] == ref.taus == [5, 5, 5]
+    gx, gv = eng.get_all()
+    for i in range(m):
+        assert max_rel_err_per_tensor(gx[i], ref.params[i], dims, True) <= 1e-4     # 15 free-running steps
+        if mode == "reset":
+            assert np.all(gv[i] == 0)
+        else:
+            assert max_rel_err_per_tensor(gv[i], ref.momentum[i], dims, True) <= 1e-3
+    got = loss_dev.cpu().numpy()
+    assert np.max(np.abs(got - ref.loss) / ref.loss) <= 1e-4
+    p, v = eng.state_view()
+    assert bool((p[0:1] == p).all())
+    assert bool((v[0:1] == v).all()) == (mode != "keep")
+    eng.close()
+
+
+def test_tau1_equals_large_batch_sgd_on_gpu():
+    """tau = 1 with m replicas equals one replica trained on the concatenated m*B batch
+    (fully synchronous SGD, Section 2 special case), both run on the GPU."""
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, K = (64, 48, 10), 4, 16, 8
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 4)
+    blocks = np.random.default_rng(0).integers(0, 1024 // (m * B), K) * (m * B)
+    offs_m = np.stack([blocks + i * B for i in range(m)], axis=1).astype(np.int64)   # m adjacent blocks
+    xd, yd = to_device(X, y)
+    a = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B); a.bind_dataset(xd, yd); a.set_params(x1)
+    a.run(K, 1, offs_m)
+    b = LocalSGD(1, dims, lr=0.05, momentum=0.9, batch=m * B); b.bind_dataset(xd, yd); b.set_params(x1)
+    b.run(K, 1, blocks.reshape(K, 1).astype(np.int64))
+    pa, _ = a.get_state(0); pb, _ = b.get_state(0)
+    assert max_rel_err_per_tensor(pa, pb, dims, True) <= 1e-5
+    a.close(); b.close()
+
+
+def test_m1_equals_oracle_plain_sgd():
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, B, K = (64, 48, 10), 16, 6
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 512, 6)
+    offs = wl.batch_row_offsets(3, K, 1, 512, B)
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(0.9), 4)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(1, dims, lr=0.05, momentum=0.9, batch=B); eng.bind_dataset(xd, yd); eng.set_params(x1)
+    eng.run(K, 4, offs)
+    p, v = eng.get_state(0)
+    assert max_rel_err_per_tensor(p, ref.params[0], dims, True) <= 1e-5
+    eng.close()
+
+
+def test_eval_loss_and_adacomm_run():
+    """AdaComm run: the decisions logged by the native loop are recomputed bit-exactly by the
+    oracle's rule from the logged losses; the losses themselves match the oracle's."""
+    from paper_1810_08313_b200 import binding
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, K, tau0, I, probe = (96, 64, 10), 4, 32, 60, 8, 10, 256
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 2048, 33)
+    offs = wl.batch_row_offsets(9, K, m, 2048, B)
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), 0.0, tau0, adacomm_interval=I, probe_rows=probe)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=0.0, batch=B); eng.bind_dataset(xd, yd); eng.set_params(x1)
+    F0 = eng.eval_loss(0, 0, probe)
+    assert abs(F0 - ref.F_0) / ref.F_0 <= 1e-5
+    assert abs(eng.eval_loss(0, 512, 64) - orc.batch_loss(spec, x1, X[512:576], y[512:576])) <= 1e-5 * ref.F_0
+    out = eng.run(K, tau0, offs, interval=I, probe_rows=probe)
+    # bit-exact tau schedule from the GPU's own logged loss trace
+    want_taus = orc.tau_schedule_from_trace(out["F_0"], tau0, [float(F) for F in out["decision_F"]])
+    assert out["decision_tau"] == want_taus
+    assert [binding.adacomm_next_tau(float(F), out["F_0"], tau0) for F in out["decision_F"]] == want_taus
+    # and the run follows the oracle's: same decision points, losses within fp32 tolerance, same periods
+    assert out["decision_k"] == [k for k, _, _ in ref.F_trace]
+    for F, (_, Fr, _) in zip(out["decision_F"], ref.F_trace):
+        assert abs(float(F) - Fr) / Fr <= 1e-4
+    assert out["taus"] == ref.taus
+    eng.close()
+
+
+def test_host_batches_match_resident_dataset():
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, tau = (64, 48, 10), 3, 16, 5
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 512, 8)
+    offs = wl.batch_row_offsets(4, tau, m, 512, B)
+    xd, yd = to_device(X, y)
+    a = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B); a.bind_dataset(xd, yd); a.set_params(x1)
+    la = torch.zeros((tau, m), device="cuda")
+    a.local_steps(tau, offs, la); a.sync()
+    xh = torch.empty((tau, m, B, dims[0]), dtype=torch.float32).pin_memory()
+    yh = torch.empty((tau, m, B), dtype=torch.int32).pin_memory()
+    for s in range(tau):
+        for i in range(m):
+            r0 = int(offs[s, i])
+            xh[s, i] = torch.from_numpy(X[r0:r0 + B]); yh[s, i] = torch.from_numpy(y[r0:r0 + B])
+    lh = torch.zeros((tau, m), dtype=torch.float32).pin_memory()
+    b = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B); b.set_params(x1)
+    b.local_steps_host(tau, xh, yh, lh)
+    pa, va = a.get_all(); pb, vb = b.get_all()
+    assert np.array_equal(pa, pb) and np.array_equal(va, vb)
+    assert np.array_equal(la.cpu().numpy(), lh.numpy())
+    a.close(); b.close()
+
+
+def test_least_squares_config_short():
+    """Least squares 4096-dim, m = 32, B = 64, tau = 50, lr 1e-4: two periods vs the oracle."""
+    from paper_1810_08313_b200.binding import LocalSGD
+    w = wl.WORKLOADS["c4_lsq"]
+    X, y = wl.make_dataset(w)
+    spec = orc.ModelSpec(w.dims, w.loss, w.has_bias)
+    K = 100
+    offs = wl.batch_row_offsets(w.seed, K, w.m, w.n_rows, w.batch)
+    ref = orc.run_pasgd(spec, wl.initial_point(w), X, y, offs, w.batch, f32(w.lr), 0.0, 50)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(w.m, w.dims, w.loss, w.has_bias, "fp32", lr=w.lr, momentum=0.0, batch=w.batch)
+    eng.bind_dataset(xd, yd); eng.set_params(wl.initial_point(w))
+    eng.run(K, 50, offs)
+    p, _ = eng.get_state(0)
+    assert max_rel_err_per_tensor(p, ref.params[0], w.dims, w.has_bias) <= 1e-5
+    eng.close()

@@ -1,0 +1,127 @@
+"""Local-step kernels vs the oracle on identical injected state
+(Section 2: mini-batch SGD update; PASGD update rule)."""
+import numpy as np
+import pytest
+
+from oracle import localsgd_oracle as orc
+from paper_1810_08313_b200 import workloads as wl
+from tests.helpers import f32, max_rel_err_per_tensor, small_problem, to_device
+
+pytestmark = pytest.mark.gpu
+
+FP32_TOL = 1e-5     # max|a-b| / max|b| per tensor, fp32 paths
+
+
+def _oracle_steps(spec, xs, vs, X, y, offs, B, lr, mu):
+    """tau teacher-forced local steps from the given fp32 state; returns new state and losses."""
+    xs = xs.copy(); vs = vs.copy()
+    tau, m = offs.shape
+    losses = np.zeros((tau, m))
+    for s in range(tau):
+        for i in range(m):
+            r0 = int(offs[s, i])
+            loss, g = orc.loss_and_grad(spec, xs[i], X[r0:r0 + B], y[r0:r0 + B])
+            losses[s, i] = loss
+            xn, vn = orc.sgd_momentum_step(xs[i], vs[i], g, lr, mu)
+            xs[i] = xn.astype(np.float32); vs[i] = vn.astype(np.float32)
+    return xs, vs, losses
+
+
+CASES = [
+    # dims, loss, bias, m, B, mu
+    ((784, 10), "softmax_ce", True, 4, 32, 0.0),                 # softmax regression shape
+    ((100, 70, 50, 10), "softmax_ce", True, 3, 37, 0.9),         # ragged everything
+    ((3072, 512, 512, 10), "softmax_ce", True, 2, 128, 0.9),     # the fp32 MLP's layer shapes
+    ((130, 65, 10), "softmax_ce", False, 5, 64, 0.5),            # no bias
+    ((4096, 1), "mse_half", False, 4, 64, 0.0),                  # least squares
+    ((50, 33, 1), "mse_half", True, 2, 16, 0.9),
+]
+
+
+@pytest.mark.parametrize("dims,loss,bias,m,B,mu", CASES)
+def test_one_step_and_one_period_teacher_forced(dims, loss, bias, m, B, mu):
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    lr = 1e-4 if loss == "mse_half" and len(dims) == 2 else 0.05
+    spec, X, y, x1 = small_problem(dims, loss, bias, n_rows=2048, seed=11)
+    xd, yd = to_device(X, y)
+    rng = np.random.default_rng(3)
+    # distinct, non-trivial state per replica
+    xs = np.stack([x1 + 0.01 * rng.standard_normal(x1.size).astype(np.float32) for _ in range(m)]).astype(np.float32)
+    vs = (0.01 * rng.standard_normal((m, x1.size))).astype(np.float32) if mu > 0 else np.zeros((m, x1.size), np.float32)
+    tau = 4
+    offs = wl.batch_row_offsets(5, tau, m, X.shape[0], B)
+    eng = LocalSGD(m, dims, loss, bias, "fp32", lr=lr, momentum=mu, batch=B)
+    eng.bind_dataset(xd, yd)
+    loss_dev = torch.zeros((tau, m), dtype=torch.float32, device="cuda")
+    for steps in (1, tau):
+        for i in range(m):
+            eng.set_state(i, xs[i], vs[i])
+        eng.local_steps(steps, offs[:steps], loss_dev)
+        eng.sync()
+        gx, gv = eng.get_all()
+        wx, wv, wl_ = _oracle_steps(spec, xs, vs, X, y, offs[:steps], B, f32(lr), f32(mu))
+        for i in range(m):
+            assert max_rel_err_per_tensor(gx[i], wx[i], dims, bias) <= FP32_TOL
+            if mu > 0:
+                assert max_rel_err_per_tensor(gv[i], wv[i], dims, bias) <= FP32_TOL
+        got_loss = loss_dev.cpu().numpy()[:steps]
+        assert np.max(np.abs(got_loss - wl_) / np.maximum(np.abs(wl_), 1e-30)) <= FP32_TOL
+    eng.close()
+
+
+def test_momentum_zero_never_touches_the_buffers():
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims = (64, 32, 10)
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 512, 2)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(2, dims, lr=0.05, momentum=0.0, batch=16)
+    eng.bind_dataset(xd, yd)
+    v = np.full(x1.size, 7.0, np.float32)
+    for i in range(2):
+        eng.set_state(i, x1, v)
+    eng.local_steps(3, wl.batch_row_offsets(1, 3, 2, 512, 16))
+    eng.average()
+    eng.sync()
+    _, gv = eng.get_all()
+    assert np.all(gv == 7.0)
+    eng.close()
+
+
+def test_error_codes():
+    import torch
+    from paper_1810_08313_b200 import binding
+    from paper_1810_08313_b200.binding import LocalSGD, LsError
+    dims = (16, 8, 4)
+    eng = LocalSGD(2, dims, lr=0.05, momentum=0.0, batch=8)
+    offs = np.zeros((1, 2), np.int64)
+    with pytest.raises(LsError) as e:
+        eng.local_steps(1, offs)
+    assert e.value.code == binding.LS_ERR_NO_DATASET
+    X = torch.zeros((32, 16), device="cuda"); y = torch.zeros(32, dtype=torch.int32, device="cuda")
+    eng.bind_dataset(X, y)
+    with pytest.raises(LsError) as e:
+        eng.local_steps(1, np.array([[0, 25]], np.int64))       # 25 + 8 > 32
+    assert e.value.code == binding.LS_ERR_ROW_RANGE
+    with pytest.raises(LsError) as e:
+        eng.local_steps(1, np.array([[-1, 0]], np.int64))
+    assert e.value.code == binding.LS_ERR_ROW_RANGE
+    assert eng.lib.ls_local_steps(eng.h, 0, offs.ctypes.data, None) == binding.LS_ERR_INVALID_ARG
+    assert eng.lib.ls_local_steps(eng.h, 1, None, None) == binding.LS_ERR_INVALID_ARG
+    with pytest.raises(LsError):
+        eng.eval_loss(0, 0, 12)           # not a multiple of the batch
+    with pytest.raises(LsError):
+        eng.eval_loss(2, 0, 8)            # replica out of range
+    eng.local_steps(1, offs)              # still usable after the errors
+    eng.sync()
+    eng.close()
+    with pytest.raises(LsError):
+        LocalSGD(0, dims)
+    with pytest.raises(LsError):
+        LocalSGD(65, dims)
+    with pytest.raises(LsError):
+        LocalSGD(2, dims, momentum=1.0)
+    with pytest.raises(LsError):
+        LocalSGD(2, dims, lr=float("nan"))
+    with pytest.raises(LsError):
+        LocalSGD(2, (16, 8, 2), loss="mse_half")

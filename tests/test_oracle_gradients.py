@@ -65,7 +65,7 @@ def _torch_mlp_loss(dims, bias, x_flat, X, y, loss):
     else:
         out = 0.5 * torch.nn.functional.mse_loss(a[:, 0], torch.tensor(y, dtype=torch.float64))
     out.backward()
-    return float(out), x.grad.numpy()
+    return float(out.detach()), x.grad.numpy()
 
 
 @pytest.mark.parametrize("dims,loss,bias", [
