@@ -1,0 +1,469 @@
+#!/usr/bin/env python
+"""Benchmark of the local-update SGD hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--tau T]
+
+One timed "step" is one communication period of the whole path on the
+workload's m replicas: tau local SGD(-momentum) iterations on every replica
+(forward, loss, backward, fused update), one model-averaging step, one
+evaluation of the synchronized model's training loss on the probe block and
+one AdaComm decision.  The metric is replica-steps/s = m * tau * K / time.
+
+Prints ONE JSON line (rank 0).  With --gpus N > 1 (launched by torchrun) every
+rank runs an independent copy of the job (the path keeps all replicas of one
+job on one GPU and has no cross-GPU step), time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1810_08313_b200 import workloads as wl  # noqa: E402
+
+METRIC = "replica-steps/s (m-replica local SGD); model-avg HBM GB/s vs ~8 TB/s peak"
+UNIT = "replica-steps/s"
+FALLBACK_HBM_GBS = 6650.0
+PROBE_ROWS = 4096
+
+
+# --------------------------------------------------------------------------
+# helpers with no GPU dependency (covered by CPU tests)
+# --------------------------------------------------------------------------
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops", 0.0)),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", 0.0)), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+                "source": "fallback"}
+
+
+def probe_rows_for(w: wl.Workload) -> int:
+    n = min(PROBE_ROWS, w.n_rows)
+    return max(w.batch, n // w.batch * w.batch)
+
+
+def layer_shapes(w: wl.Workload):
+    return [(w.dims[l + 1], w.dims[l]) for l in range(len(w.dims) - 1)]
+
+
+def flops_per_replica_step(w: wl.Workload) -> float:
+    """forward + weight gradient for every layer, data gradient for all but the first."""
+    f = 0.0
+    for l, (n_out, n_in) in enumerate(layer_shapes(w)):
+        f += 2.0 * w.batch * n_out * n_in * (2 if l == 0 else 3)
+    return f
+
+
+def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
+    """Algorithmic bytes of one weight-gradient + update launch for layer `layer` (all m replicas):
+    read and write W (and v when momentum is on), read the two GEMM operands, write the bf16 copy."""
+    n_out, n_in = layer_shapes(w)[layer]
+    esz = 2 if w.gemm_dtype == "bf16" else 4
+    per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if w.gemm_dtype == "bf16" else 0)
+    return float(w.m) * (per_param * n_out * n_in + esz * w.batch * (n_out + n_in))
+
+
+def gemm_flops_per_launch(w: wl.Workload, layer: int) -> float:
+    n_out, n_in = layer_shapes(w)[layer]
+    return 2.0 * w.m * w.batch * n_out * n_in
+
+
+def fp32_alu_peak_tflops(sm_mhz: float, sms: int = 148) -> float:
+    """128 fp32 lanes per SM, one FMA (2 flops) per lane per clock."""
+    return sms * 128 * 2 * sm_mhz * 1e6 / 1e12
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float):
+    """(max ms over ranks, total units) with torch.distributed when initialised."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, units_local
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        return parse_clock_csv(open(self.path).read())
+
+
+def parse_clock_csv(text: str):
+    sm, mx, reasons = [], [], set()
+    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    for line in text.strip().splitlines():
+        a = [x.strip() for x in line.split(",")]
+        if len(a) < 7:
+            continue
+        try:
+            sm.append(float(a[0])); mx.append(float(a[1]))
+        except ValueError:
+            continue
+        for name, val in zip(names, a[3:7]):
+            if val.lower().startswith("active"):
+                reasons.add(name)
+    if not sm:
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+            "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------
+# the oracle arm (CPU): --impl reference and the cpu_baseline leg
+# --------------------------------------------------------------------------
+
+def oracle_replica_steps_per_s(w: wl.Workload, X, y, x1, tau: int, budget_s: float, max_iters: int):
+    """Times the CPU oracle, as it stands, on whole iterations (all m replicas) of the workload plus
+    the averaging step every tau iterations.  Returns (replica-steps/s, iterations, seconds)."""
+    from oracle import localsgd_oracle as orc
+    spec = orc.ModelSpec(w.dims, w.loss, w.has_bias)
+    lr, mu = float(np.float32(w.lr)), float(np.float32(w.momentum))
+    iters = 0
+    t0 = time.perf_counter()
+    offs_all = wl.batch_row_offsets(w.seed + 1, max_iters, w.m, X.shape[0], w.batch)
+    xs = np.repeat(x1[None], w.m, axis=0).astype(np.float32)
+    vs = np.zeros_like(xs)
+    t0 = time.perf_counter()
+    while iters < max_iters:
+        for i in range(w.m):
+            r0 = int(offs_all[iters, i])
+            _, g = orc.loss_and_grad(spec, xs[i], X[r0:r0 + w.batch], y[r0:r0 + w.batch])
+            xn, vn = orc.sgd_momentum_step(xs[i], vs[i], g, lr, mu)
+            xs[i] = xn.astype(np.float32); vs[i] = vn.astype(np.float32)
+        iters += 1
+        if iters % tau == 0:
+            orc.average_replicas(xs)
+            if mu != 0:
+                orc.average_replicas(vs)
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return w.m * iters / dt, iters, dt
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, w: wl.Workload):
+    """The oracle timed on the host cores: each step is one whole iteration (m replica-steps)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_rows = min(w.n_rows, 8192)
+    X, y = wl.make_dataset(w, n_rows=n_rows)
+    x1 = wl.initial_point(w)
+    from oracle import localsgd_oracle as orc
+    spec = orc.ModelSpec(w.dims, w.loss, w.has_bias)
+    lr, mu = float(np.float32(w.lr)), float(np.float32(w.momentum))
+    tau = args.tau
+    xs = np.repeat(x1[None], w.m, axis=0).astype(np.float32)
+    vs = np.zeros_like(xs)
+    total = args.warmup + args.steps
+    offs = wl.batch_row_offsets(w.seed + 1, total, w.m, n_rows, w.batch)
+
+    def one_iter(k):
+        for i in range(w.m):
+            r0 = int(offs[k, i])
+            _, g = orc.loss_and_grad(spec, xs[i], X[r0:r0 + w.batch], y[r0:r0 + w.batch])
+            xn, vn = orc.sgd_momentum_step(xs[i], vs[i], g, lr, mu)
+            xs[i] = xn.astype(np.float32); vs[i] = vn.astype(np.float32)
+        if (k + 1) % tau == 0:
+            orc.average_replicas(xs)
+            if mu != 0:
+                orc.average_replicas(vs)
+
+    for k in range(args.warmup):
+        one_iter(k)
+    t0 = time.perf_counter()
+    for k in range(args.warmup, total):
+        one_iter(k)
+    dt = time.perf_counter() - t0
+    value = w.m * args.steps / dt
+    cores = cpu_threads()
+    sample = f"{args.steps} whole iterations (m={w.m} replica-steps each, averaging every {tau}) of {w.name} on {n_rows} rows"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "dims": list(w.dims), "m": w.m, "batch": w.batch, "tau": tau,
+                   "step": "one iteration of all m replicas on the CPU oracle"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------
+
+def run_ours(args, w: wl.Workload):
+    import torch
+    import torch.distributed as dist
+    from paper_1810_08313_b200.binding import LocalSGD, adacomm_next_tau, average_flat
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl")
+    peaks = load_peaks()
+    tau, K, W = args.tau, args.steps, args.warmup
+    m, B = w.m, w.batch
+
+    # ---- synthetic inputs, resident in HBM before the timed region ----------
+    X, y = wl.make_dataset(w)
+    x1 = wl.initial_point(w)
+    xd = torch.from_numpy(X).cuda()
+    if w.gemm_dtype == "bf16":
+        xd = xd.to(torch.bfloat16)
+    yd = torch.from_numpy(y).cuda()
+    eng = LocalSGD(m, w.dims, w.loss, w.has_bias, w.gemm_dtype, lr=w.lr, momentum=w.momentum, batch=B,
+                   device=f"cuda:{local_rank}")
+    eng.bind_dataset(xd, yd)
+    eng.set_params(x1)
+    probe = probe_rows_for(w)
+    total_periods = W + K
+    offs = wl.batch_row_offsets(w.seed + 100 + rank, total_periods * tau, m, w.n_rows, B)
+    loss_dev = torch.zeros((tau, m), dtype=torch.float32, device="cuda")
+    F_0 = eng.eval_loss(0, 0, probe)
+
+    def period(p):
+        eng.local_steps(tau, offs[p * tau:(p + 1) * tau], loss_dev)
+        eng.average()
+        F_t = eng.eval_loss(0, 0, probe)
+        return F_t, adacomm_next_tau(F_t, F_0, tau)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up, with every kernel class timed to find the dominant one ----
+    eng.profile_begin()
+    for p in range(W):
+        period(p)
+    shares_raw = eng.profile_end()
+    tot = sum(v[0] for v in shares_raw.values()) or 1.0
+    shares = {f"{c}{l}": round(v[0] / tot, 4) for (c, l), v in sorted(shares_raw.items(), key=lambda kv: -kv[1][0])}
+    dom = max(shares_raw.items(), key=lambda kv: kv[1][0])[0] if shares_raw else ("dw", 0)
+
+    # ---- timed region ---------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    eng.profile_begin([dom[0]], dom[1])
+    launches0 = eng.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    F_t, next_tau = 0.0, tau
+    for p in range(W, W + K):
+        F_t, next_tau = period(p)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_local = e0.elapsed_time(e1)
+    launches = eng.launch_count() - launches0
+    dom_ms, dom_n = eng.profile_end().get(dom, (0.0, 0))
+    ms, units = aggregate_over_ranks(ms_local, float(m * tau * K))
+    value = units / (ms * 1e-3)
+
+    # ---- roofline of the dominant kernel ---------------------------------------
+    roofline = None
+    if dom_n:
+        dur_s = dom_ms * 1e-3 / dom_n
+        cls, layer = dom
+        if cls in ("dw",) and w.gemm_dtype == "bf16":
+            by = update_bytes_per_launch(w, layer)
+            ach = by / dur_s / 1e9
+            roofline = {"kernel": f"{cls} layer {layer}", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                        "peak_source": f"of {peaks['source']}", "ms_per_launch": dur_s * 1e3}
+        elif cls == "avg":
+            nbuf = 2 if w.momentum != 0 else 1
+            by = 8.0 * m * wl.n_params(w.dims, w.has_bias) * nbuf
+            ach = by / dur_s / 1e9
+            roofline = {"kernel": "averaging", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                        "peak_source": f"of {peaks['source']}", "ms_per_launch": dur_s * 1e3}
+        elif cls in ("fwd", "dx", "dw"):
+            fl = gemm_flops_per_launch(w, layer)
+            if cls == "dx":
+                n_out, n_in = layer_shapes(w)[layer]
+                fl = 2.0 * m * B * n_out * n_in
+            ach = fl / dur_s / 1e12
+            mhz = clocks.get("sm_mhz") or 1965.0
+            if w.gemm_dtype == "bf16":
+                peak, src, bound = peaks["bf16_tflops_sustained"], f"of {peaks['source']} (sustained bf16)", "tensor"
+            else:
+                peak, src, bound = fp32_alu_peak_tflops(mhz), f"derived: 148 SMs x 128 lanes x 2 x {mhz:.0f} MHz", "alu"
+            roofline = {"kernel": f"{cls} layer {layer}", "bound": bound, "achieved": ach, "peak": peak,
+                        "unit": "TFLOP/s", "frac": ach / peak, "traffic": None, "peak_source": src,
+                        "ms_per_launch": dur_s * 1e3}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.gemm_dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "dims": list(w.dims), "m": m, "batch": B, "tau": tau,
+                   "momentum": w.momentum, "lr": w.lr, "dataset_rows": w.n_rows,
+                   "step": "one period: tau local iterations x m replicas + averaging + probe loss + AdaComm decision",
+                   "l2": "inputs larger than L2: mini-batches are drawn at random from a %.0f MB resident dataset"
+                         % (xd.numel() * xd.element_size() / 1e6),
+                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks, "gpu_launches": int(launches), "kernel_time_shares": shares,
+        "last_probe_loss": F_t, "next_tau": next_tau,
+    }
+    if roofline:
+        line["roofline"] = roofline
+
+    if rank == 0 and world == 1 and not args.kernel_only:
+        # ---- end to end: mini-batches from pinned host memory, losses back to the host -------
+        e_steps = max(1, min(K, 3))
+        xh = torch.empty((tau, m, B, w.dims[0]), dtype=xd.dtype).pin_memory()
+        yh = torch.empty((tau, m, B), dtype=yd.dtype).pin_memory()
+        lh = torch.zeros((tau, m), dtype=torch.float32).pin_memory()
+        o = offs[:tau]
+        for s in range(tau):
+            for i in range(m):
+                r0 = int(o[s, i])
+                xh[s, i].copy_(xd[r0:r0 + B].cpu()); yh[s, i].copy_(yd[r0:r0 + B].cpu())
+        def e2e_period():
+            eng.local_steps_host(tau, xh, yh, lh)
+            eng.average()
+            F = eng.eval_loss(0, 0, probe)
+            return adacomm_next_tau(F, F_0, tau)
+        e2e_period()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            e2e_period()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        line["e2e"] = {"value": m * tau * e_steps / dt, "unit": UNIT,
+                       "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * yh.element_size()),
+                       "d2h_bytes_per_step": int(lh.numel() * 4 + 4),
+                       "note": "per period; batches copied from pinned host memory inside the timed region"}
+
+        # ---- averaging bandwidth on the model-sized flat vectors (params + momentum) ----------
+        avg = {}
+        for P in (14_706_698, 23_500_000):
+            buf = torch.rand((2 * 16, P), device="cuda", dtype=torch.float32) * 2 - 1
+            for mm in (4, 8, 16):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                for _ in range(3):
+                    average_flat(buf[:mm].view(-1), mm, P); average_flat(buf[16:16 + mm].view(-1), mm, P)
+                ev[0].record()
+                reps = 10
+                for _ in range(reps):
+                    average_flat(buf[:mm].view(-1), mm, P); average_flat(buf[16:16 + mm].view(-1), mm, P)
+                ev[1].record()
+                torch.cuda.synchronize()
+                gbs = 2 * 8.0 * mm * P * reps / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9
+                avg[f"P{P}_m{mm}"] = {"GB/s": round(gbs, 1), "frac_measured_peak": round(gbs / peaks["hbm_gbs"], 4),
+                                      "frac_8TBs": round(gbs / 8000.0, 4)}
+            del buf
+        line["averaging_gbs"] = avg
+
+        # ---- the CPU oracle on the host cores, bounded sample -----------------------------------
+        if not args.no_cpu_baseline:
+            v, iters, dt = oracle_replica_steps_per_s(w, X[:8192], y[:8192], x1, tau, budget_s=args.cpu_budget,
+                                                      max_iters=10 * tau)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": f"{iters} whole iterations (m={m} replica-steps each) in {dt:.1f} s on "
+                                              f"the first 8192 rows"}
+    eng.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_mlp_fp32", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--tau", type=int, default=20)
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only the device-timed region (for profiler runs): no e2e, averaging sweep or CPU baseline")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

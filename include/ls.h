@@ -197,6 +197,19 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
            int64_t* decision_k, float* decision_F, int32_t* decision_tau, int64_t max_decisions,
            int64_t* n_decisions, float* F0_host);
 
+/* Per-kernel device timing.  Between ls_profile_begin() and ls_profile_end()
+ * every launch of a kernel class selected by class_mask (bit c = class c; for
+ * the per-layer classes only layer `layer`, 0-based, or all layers when
+ * layer < 0) is bracketed by a pair of CUDA events on the handle's stream.
+ * ls_profile_end() waits for the stream and adds up, per class and layer, the
+ * elapsed milliseconds and the number of launches into
+ * ms[LS_K_CLASSES * LS_MAX_LAYERS] and launches[...] (index class*LS_MAX_LAYERS
+ * + layer; LS_K_LOSS and LS_K_AVG use layer 0).  At most 16384 launches are
+ * recorded per profile; later ones are run but not timed. */
+enum { LS_K_FWD = 0, LS_K_LOSS = 1, LS_K_DX = 2, LS_K_DW = 3, LS_K_BIAS = 4, LS_K_AVG = 5, LS_K_CLASSES = 6 };
+int ls_profile_begin(ls_handle* h, uint32_t class_mask, int layer);
+int ls_profile_end(ls_handle* h, double* ms, int64_t* launches);
+
 /* Number of kernels this handle has launched so far. */
 int ls_launch_count(const ls_handle* h, int64_t* n);
 

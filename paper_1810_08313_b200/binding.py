@@ -30,6 +30,7 @@ LS_ERR_OVERFLOW = -8
 LOSS = {"softmax_ce": 0, "mse_half": 1}
 GEMM = {"fp32": 0, "bf16": 1}
 MOMENTUM_MODE = {"average": 0, "keep": 1, "reset": 2}
+KERNEL_CLASSES = ("fwd", "loss", "dx", "dw", "bias", "avg")
 
 
 class ModelSpec(C.Structure):
@@ -84,6 +85,8 @@ def _lib():
         "ls_run": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, vp, i64, P(i64), vp, vp, vp, i64, P(i64),
                              P(f32)]),
         "ls_launch_count": (C.c_int, [vp, P(i64)]),
+        "ls_profile_begin": (C.c_int, [vp, C.c_uint32, C.c_int]),
+        "ls_profile_end": (C.c_int, [vp, P(C.c_double), P(i64)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -298,6 +301,25 @@ class LocalSGD:
         n_p, n_d = n_p.value, n_d.value
         return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
                 "decision_tau": dt[:n_d].tolist(), "F_0": float(F0.value) if interval > 0 else None}
+
+    def profile_begin(self, classes: Sequence[str] = KERNEL_CLASSES, layer: int = -1):
+        mask = 0
+        for c in classes:
+            mask |= 1 << KERNEL_CLASSES.index(c)
+        _check(self.lib.ls_profile_begin(self.h, mask, int(layer)), "ls_profile_begin")
+
+    def profile_end(self):
+        """{(class, layer): (total ms, launches)} for what ran since profile_begin()."""
+        n = len(KERNEL_CLASSES) * LS_MAX_LAYERS
+        ms = (C.c_double * n)()
+        cnt = (C.c_int64 * n)()
+        _check(self.lib.ls_profile_end(self.h, ms, cnt), "ls_profile_end")
+        out = {}
+        for ci, cname in enumerate(KERNEL_CLASSES):
+            for l in range(LS_MAX_LAYERS):
+                if cnt[ci * LS_MAX_LAYERS + l]:
+                    out[(cname, l)] = (ms[ci * LS_MAX_LAYERS + l], cnt[ci * LS_MAX_LAYERS + l])
+        return out
 
     def launch_count(self) -> int:
         n = C.c_int64()

@@ -94,6 +94,25 @@ static int cuda_fail(ls_handle* h, int e) {
     if (_e != (int)cudaSuccess) return cuda_fail(h, _e); \
   } while (0)
 
+constexpr int kProfCap = 16384;
+
+// Brackets one launch with a pair of events when its class/layer is being profiled.
+struct ProfScope {
+  ls_handle* h;
+  int rec;
+  ProfScope(ls_handle* h_, int cls, int layer) : h(h_), rec(-1) {
+    if (!(h->prof_mask & (1u << cls))) return;
+    if (h->prof_layer >= 0 && layer != h->prof_layer && cls != LS_K_LOSS && cls != LS_K_AVG) return;
+    if (h->prof_used >= h->prof_cap) return;
+    rec = h->prof_used++;
+    h->prof_tag[rec] = (int16_t)(cls * LS_MAX_LAYERS + layer);
+    cudaEventRecord(h->prof_ev[2 * rec], h->stream);
+  }
+  ~ProfScope() {
+    if (rec >= 0) cudaEventRecord(h->prof_ev[2 * rec + 1], h->stream);
+  }
+};
+
 static int refresh_shadow(ls_handle* h) {
   if (!h->lay.bf16) return LS_OK;
   LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), (int64_t)h->lay.m * h->lay.stride, h->stream, &h->launches));
@@ -121,6 +140,7 @@ static int forward(ls_handle* h, const void* x, const void* y, const int64_t* ro
     a.C = last ? (void*)(h->state + lay.logits_off) : (void*)(h->state + lay.act_off[l + 1]);
     a.M = lay.batch; a.N = lay.dims[l + 1]; a.K = lay.dims[l]; a.groups = groups;
     a.relu = last ? 0 : 1;
+    ProfScope ps(h, LS_K_FWD, l);
     LS_CUDA(h, launch_fwd(a, bf, bf, bf && !last, h->stream, &h->launches));
   }
   LossArgs la;
@@ -129,6 +149,7 @@ static int forward(ls_handle* h, const void* x, const void* y, const int64_t* ro
   la.dZ = want_dz ? (void*)(h->state + lay.dz_off[0]) : nullptr;
   la.loss_out = loss_out;
   la.B = lay.batch; la.C = lay.dims[lay.L]; la.groups = groups; la.loss_kind = h->spec.loss;
+  ProfScope ps(h, LS_K_LOSS, 0);
   LS_CUDA(h, launch_loss(la, bf, h->stream, &h->launches));
   return LS_OK;
 }
@@ -151,6 +172,7 @@ static int local_step(ls_handle* h, const void* x, const void* y, const int64_t*
       d.act = h->state + lay.act_off[l];
       d.C = h->state + lay.dz_off[cur ^ 1];
       d.M = lay.batch; d.N = lay.dims[l]; d.K = lay.dims[l + 1]; d.groups = lay.m;
+      ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
     }
     DwArgs w;
@@ -163,7 +185,10 @@ static int local_step(ls_handle* h, const void* x, const void* y, const int64_t*
     w.w_gstride = lay.stride;
     w.M = lay.dims[l + 1]; w.N = lay.dims[l]; w.B = lay.batch; w.groups = lay.m;
     w.lr = h->lr; w.mu = h->mu;
-    LS_CUDA(h, launch_dw(w, bf, h->stream, &h->launches));
+    {
+      ProfScope ps(h, LS_K_DW, l);
+      LS_CUDA(h, launch_dw(w, bf, h->stream, &h->launches));
+    }
     if (lay.has_bias) {
       BiasArgs b;
       b.dZ = dZ;
@@ -172,6 +197,7 @@ static int local_step(ls_handle* h, const void* x, const void* y, const int64_t*
       b.gstride = lay.stride;
       b.B = lay.batch; b.N = lay.dims[l + 1]; b.groups = lay.m;
       b.lr = h->lr; b.mu = h->mu;
+      ProfScope ps(h, LS_K_BIAS, l);
       LS_CUDA(h, launch_bias(b, bf, h->stream, &h->launches));
     }
     cur ^= 1;
@@ -183,8 +209,11 @@ static int average(ls_handle* h) {
   const Layout& lay = h->lay;
   const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
   const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
-  LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                            lay.bf16 ? shadow_of(h) : nullptr, h->stream, &h->launches));
+  {
+    ProfScope ps(h, LS_K_AVG, 0);
+    LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
+                              lay.bf16 ? shadow_of(h) : nullptr, h->stream, &h->launches));
+  }
   if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
   return LS_OK;
@@ -324,6 +353,11 @@ int ls_destroy(ls_handle* h) {
     if (h->ev_consumed[s]) cudaEventDestroy(h->ev_consumed[s]);
   }
   if (h->pinned) cudaFreeHost(h->pinned);
+  if (h->prof_ev) {
+    for (int i = 0; i < 2 * h->prof_cap; ++i) cudaEventDestroy(h->prof_ev[i]);
+    delete[] h->prof_ev;
+    delete[] h->prof_tag;
+  }
   h->magic = 0;
   delete h;
   return LS_OK;
@@ -528,6 +562,41 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
   }
   if (n_periods) *n_periods = np;
   if (n_decisions) *n_decisions = nd;
+  return LS_OK;
+}
+
+int ls_profile_begin(ls_handle* h, uint32_t class_mask, int layer) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (layer >= LS_MAX_LAYERS || class_mask >= (1u << LS_K_CLASSES)) return LS_ERR_INVALID_ARG;
+  if (h->prof_ev == nullptr) {
+    h->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfCap];
+    h->prof_tag = new (std::nothrow) int16_t[kProfCap];
+    if (h->prof_ev == nullptr || h->prof_tag == nullptr) return LS_ERR_INVALID_ARG;
+    h->prof_cap = 0;
+    for (int i = 0; i < 2 * kProfCap; ++i) {
+      LS_CUDA(h, cudaEventCreate(&h->prof_ev[i]));
+      if (i & 1) h->prof_cap = (i + 1) / 2;
+    }
+  }
+  h->prof_used = 0;
+  h->prof_layer = layer;
+  h->prof_mask = class_mask;
+  return LS_OK;
+}
+
+int ls_profile_end(ls_handle* h, double* ms, int64_t* launches) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (ms == nullptr || launches == nullptr) return LS_ERR_INVALID_ARG;
+  h->prof_mask = 0;
+  LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  for (int i = 0; i < LS_K_CLASSES * LS_MAX_LAYERS; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (int r = 0; r < h->prof_used; ++r) {
+    float t = 0.f;
+    LS_CUDA(h, cudaEventElapsedTime(&t, h->prof_ev[2 * r], h->prof_ev[2 * r + 1]));
+    ms[h->prof_tag[r]] += (double)t;
+    launches[h->prof_tag[r]] += 1;
+  }
+  h->prof_used = 0;
   return LS_OK;
 }
 

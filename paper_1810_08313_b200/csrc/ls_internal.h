@@ -64,6 +64,13 @@ struct ls_handle {
   int last_cuda;
   int64_t launches;
   float* pinned;          // small pinned host scratch (eval losses)
+  // per-kernel timing (ls_profile_begin / ls_profile_end)
+  uint32_t prof_mask;
+  int prof_layer;
+  int prof_used;
+  int prof_cap;
+  cudaEvent_t* prof_ev;   // 2 events per record
+  int16_t* prof_tag;      // class * LS_MAX_LAYERS + layer per record
 };
 
 namespace ls {
