@@ -77,6 +77,7 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
     lay.stage_y_off[s] = take((size_t)m * batch * 4);
   }
   lay.stage_loss_off = take((size_t)kRowOffCap * m * 4);
+  lay.err_off = take(256);
   lay.total = off;
   *out = lay;
   return LS_OK;
@@ -122,13 +123,30 @@ static int refresh_shadow(ls_handle* h) {
 // One forward pass of `groups` mini-batches.  Group g reads rows
 // [row_off[g], +batch) of x/y and uses the weights at w_base + g*w_gstride
 // (w_gstride == 0: every group uses the same replica).
-static int forward(ls_handle* h, const void* x, const void* y, const int64_t* row_off_dev, int groups,
-                   int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
+static inline int* err_flag_of(const ls_handle* h) { return reinterpret_cast<int*>(h->state + h->lay.err_off); }
+
+static int forward(ls_handle* h, const void* x, const CUtensorMap* xmap, const void* y, const int64_t* row_off_dev,
+                   int groups, int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
   const float* P = params_of(h) + replica0 * lay.stride;
   const __nv_bfloat16* S = bf ? shadow_of(h) + replica0 * lay.stride : nullptr;
   for (int l = 0; l < lay.L; ++l) {
+    if (bf && l < lay.L - 1 && tc_shape_ok(lay.batch, lay.dims[l + 1], lay.dims[l])) {
+      TcFwdArgs t;
+      t.mapA = (l == 0) ? xmap : &h->maps.act[l];
+      t.mapW = &h->maps.w[l];
+      t.row_off = (l == 0) ? row_off_dev : nullptr;
+      t.w_z0 = (int)replica0; t.w_zstep = w_gstride != 0 ? 1 : 0;
+      t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
+      t.bias_gstride = w_gstride;
+      t.C = h->state + lay.act_off[l + 1];
+      t.M = lay.batch; t.N = lay.dims[l + 1]; t.K = lay.dims[l]; t.groups = groups; t.relu = 1;
+      t.err_flag = err_flag_of(h);
+      ProfScope ps(h, LS_K_FWD, l);
+      LS_CUDA(h, launch_tc_fwd(t, h->stream, &h->launches));
+      continue;
+    }
     FwdArgs a;
     a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
     a.row_off = (l == 0) ? row_off_dev : nullptr;
@@ -155,16 +173,27 @@ static int forward(ls_handle* h, const void* x, const void* y, const int64_t* ro
 }
 
 // One local update of all m replicas (forward, backward, fused SGD-momentum).
-static int local_step(ls_handle* h, const void* x, const void* y, const int64_t* row_off_dev, float* loss_out) {
+static int local_step(ls_handle* h, const void* x, const CUtensorMap* xmap, const void* y, const int64_t* row_off_dev,
+                      float* loss_out) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
-  int rc = forward(h, x, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
+  int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
   if (rc != LS_OK) return rc;
   int cur = 0;
   for (int l = lay.L - 1; l >= 0; --l) {
     void* dZ = h->state + lay.dz_off[cur];
-    if (l > 0) {
+    if (l > 0 && bf && tc_shape_ok(lay.batch, lay.dims[l], lay.dims[l + 1])) {
       // the data gradient reads W_l before the update below overwrites it
+      TcDxArgs t;
+      t.mapDz = &h->maps.dz[l];
+      t.mapW = &h->maps.w[l];
+      t.act = h->state + lay.act_off[l];
+      t.C = h->state + lay.dz_off[cur ^ 1];
+      t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
+      t.err_flag = err_flag_of(h);
+      ProfScope ps(h, LS_K_DX, l);
+      LS_CUDA(h, launch_tc_dx(t, h->stream, &h->launches));
+    } else if (l > 0) {
       DxArgs d;
       d.dZ = dZ;
       d.W = bf ? (const void*)(shadow_of(h) + lay.w_off[l]) : (const void*)(params_of(h) + lay.w_off[l]);
@@ -175,6 +204,21 @@ static int local_step(ls_handle* h, const void* x, const void* y, const int64_t*
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
     }
+    if (bf && tc_shape_ok(lay.dims[l + 1], lay.dims[l], lay.batch)) {
+      TcDwArgs t;
+      t.mapDz = &h->maps.dz[l];
+      t.mapA = (l == 0) ? xmap : &h->maps.act[l];
+      t.row_off = (l == 0) ? row_off_dev : nullptr;
+      t.W = params_of(h) + lay.w_off[l];
+      t.V = mom_of(h) + lay.w_off[l];
+      t.Wb = shadow_of(h) + lay.w_off[l];
+      t.w_gstride = lay.stride;
+      t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
+      t.lr = h->lr; t.mu = h->mu;
+      t.err_flag = err_flag_of(h);
+      ProfScope ps(h, LS_K_DW, l);
+      LS_CUDA(h, launch_tc_dw(t, h->stream, &h->launches));
+    } else {
     DwArgs w;
     w.dZ = dZ;
     w.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
@@ -188,6 +232,7 @@ static int local_step(ls_handle* h, const void* x, const void* y, const int64_t*
     {
       ProfScope ps(h, LS_K_DW, l);
       LS_CUDA(h, launch_dw(w, bf, h->stream, &h->launches));
+    }
     }
     if (lay.has_bias) {
       BiasArgs b;
@@ -234,7 +279,7 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
   LS_CUDA(h, cudaMemcpyAsync(off_dev, offs.data(), (size_t)chunks * 8, cudaMemcpyHostToDevice, h->stream));
   for (int64_t c0 = 0; c0 < chunks; c0 += lay.m) {
     const int groups = (int)((chunks - c0 < lay.m) ? chunks - c0 : lay.m);
-    int rc = forward(h, h->x_dev, h->y_dev, off_dev + c0, groups, replica, 0, false, loss_dev + c0);
+    int rc = forward(h, h->x_dev, &h->maps.x_data, h->y_dev, off_dev + c0, groups, replica, 0, false, loss_dev + c0);
     if (rc != LS_OK) return rc;
   }
   LS_CUDA(h, cudaMemcpyAsync(h->pinned, loss_dev, (size_t)chunks * 4, cudaMemcpyDeviceToHost, h->stream));
@@ -257,7 +302,7 @@ static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, fl
     LS_CUDA(h, cudaMemcpyAsync(off_dev, row_offset_host + (int64_t)s0 * lay.m, (size_t)n * lay.m * 8,
                                cudaMemcpyHostToDevice, h->stream));
     for (int s = 0; s < n; ++s) {
-      int rc = local_step(h, h->x_dev, h->y_dev, off_dev + (int64_t)s * lay.m,
+      int rc = local_step(h, h->x_dev, &h->maps.x_data, h->y_dev, off_dev + (int64_t)s * lay.m,
                           loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr);
       if (rc != LS_OK) return rc;
     }
@@ -284,6 +329,7 @@ const char* ls_strerror(int code) {
     case LS_ERR_CUDA: return "CUDA error";
     case LS_ERR_UNSUPPORTED: return "not supported";
     case LS_ERR_OVERFLOW: return "result does not fit";
+    case LS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
     default: return "unknown error";
   }
 }
@@ -336,7 +382,25 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&h->pinned), (size_t)kEvalCap * 4);
   // parameters, momentum, workspace start at zero; the staging row offsets are g*batch
   if (e == cudaSuccess) e = cudaMemsetAsync(h->state, 0, lay.total, h->stream);
+  if (e == cudaSuccess && lay.bf16) {
+    // TMA descriptors (every bf16 tensor start is 256-byte aligned; rows must be 16-byte multiples)
+    // A tensor gets a descriptor when its rows are 16-byte multiples; the tensor-core kernels are
+    // only chosen for shapes (multiples of 64) whose tensors all satisfy this.
+    const int64_t rows = (int64_t)m * batch;
+    for (int l = 0; l < lay.L && e == cudaSuccess; ++l) {
+      if (lay.dims[l] % 8 == 0) {
+        e = tc_make_map_3d(&h->maps.w[l], shadow_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride);
+        if (e == cudaSuccess && l >= 1)
+          e = tc_make_map_2d(&h->maps.act[l], h->state + lay.act_off[l], rows, lay.dims[l]);
+      }
+      if (e == cudaSuccess && lay.dims[l + 1] % 8 == 0)
+        e = tc_make_map_2d(&h->maps.dz[l], h->state + lay.dz_off[(lay.L - 1 - l) & 1], rows, lay.dims[l + 1]);
+    }
+    for (int s = 0; s < 2 && e == cudaSuccess && lay.dims[0] % 8 == 0; ++s)
+      e = tc_make_map_2d(&h->maps.x_stage[s], h->state + lay.stage_x_off[s], rows, lay.dims[0]);
+  }
   if (e != cudaSuccess) {
+    h->last_cuda = e;
     ls_destroy(h);
     return LS_ERR_CUDA;
   }
@@ -367,6 +431,9 @@ int ls_sync(ls_handle* h) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   LS_CUDA(h, cudaStreamSynchronize(h->stream));
   LS_CUDA(h, cudaGetLastError());
+  int flag = 0;
+  LS_CUDA(h, cudaMemcpy(&flag, err_flag_of(h), sizeof(int), cudaMemcpyDeviceToHost));
+  if (flag != 0) return LS_ERR_DEVICE_TIMEOUT;
   return LS_OK;
 }
 
@@ -449,6 +516,8 @@ int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t 
   if (x_dev == nullptr || y_dev == nullptr || n_rows < h->lay.batch) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(x_dev) % 16 != 0 || reinterpret_cast<uintptr_t>(y_dev) % 4 != 0)
     return LS_ERR_INVALID_ARG;
+  if (h->lay.bf16 && h->lay.dims[0] % 8 == 0)
+    LS_CUDA(h, tc_make_map_2d(&h->maps.x_data, x_dev, n_rows, h->lay.dims[0]));
   h->x_dev = x_dev;
   h->y_dev = y_dev;
   h->n_rows = n_rows;
@@ -489,7 +558,7 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
                                  cudaMemcpyHostToDevice, h->copy_stream));
       LS_CUDA(h, cudaEventRecord(h->ev_copied[slot], h->copy_stream));
       LS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_copied[slot], 0));
-      int rc = local_step(h, xs, ys, stage_off, loss_stage + (int64_t)s * lay.m);
+      int rc = local_step(h, xs, &h->maps.x_stage[slot], ys, stage_off, loss_stage + (int64_t)s * lay.m);
       if (rc != LS_OK) return rc;
       LS_CUDA(h, cudaEventRecord(h->ev_consumed[slot], h->stream));
       used[slot] = true;

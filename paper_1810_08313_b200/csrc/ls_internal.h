@@ -2,6 +2,7 @@
 // Nothing here is part of the C ABI (see include/ls.h for that).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -42,6 +43,7 @@ struct Layout {
   size_t stage_x_off[2] = {0, 0};            // [m][batch][dims[0]] input staging for host batches
   size_t stage_y_off[2] = {0, 0};            // [m][batch] labels / targets
   size_t stage_loss_off = 0;                 // float [kRowOffCap][m]
+  size_t err_off = 0;                        // int: device-side error flag (bounded waits that ran out)
   size_t total = 0;
 };
 
@@ -49,7 +51,17 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out);
 
 }  // namespace ls
 
+// TMA descriptors of the bf16 tensors the tensor-core kernels read (built once per handle).
+struct alignas(64) TcMaps {
+  CUtensorMap w[LS_MAX_LAYERS];      // bf16 weight copies, 3-D [replica][out][in]
+  CUtensorMap act[LS_MAX_LAYERS];    // input activations of layer l >= 1, 2-D [m*batch][dims[l]]
+  CUtensorMap dz[LS_MAX_LAYERS];     // dZ_l, 2-D [m*batch][dims[l+1]]
+  CUtensorMap x_data;                // bound dataset, 2-D [n_rows][dims[0]]
+  CUtensorMap x_stage[2];            // staging buffers of host batches
+};
+
 struct ls_handle {
+  TcMaps maps;
   uint32_t magic;
   ls::Layout lay;
   ls_model_spec spec;
@@ -146,6 +158,40 @@ struct BiasArgs {          // gb = colsum(dZ); v = mu v + gb; b -= lr v
   float lr, mu;
 };
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
+
+// ---- tcgen05 grouped GEMMs, bf16 operands (gemm_tc.cu) ----------------------
+int tc_make_map_2d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols);
+int tc_make_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups, int64_t gstride);
+bool tc_shape_ok(int M, int N, int K);   // output rows, output columns, contraction length
+struct TcFwdArgs {
+  const CUtensorMap* mapA;   // [rows][K] input (dataset rows through row_off, else group g at row g*M)
+  const CUtensorMap* mapW;   // 3-D weight copies
+  const int64_t* row_off;
+  int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
+  const float* bias; int64_t bias_gstride;
+  void* C;                   // bf16 [groups][M][N]
+  int M, N, K, groups, relu;
+  int* err_flag;
+};
+struct TcDxArgs {
+  const CUtensorMap* mapDz;  // dZ_l [groups*M][K]
+  const CUtensorMap* mapW;
+  const void* act; void* C;  // bf16 [groups][M][N]
+  int M, N, K, groups;
+  int* err_flag;
+};
+struct TcDwArgs {
+  const CUtensorMap* mapDz;  // dZ_l [groups*B][M]
+  const CUtensorMap* mapA;   // layer input [rows][N]
+  const int64_t* row_off;
+  float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride;
+  int M, N, B, groups;
+  float lr, mu;
+  int* err_flag;
+};
+int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);
+int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches);
+int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches);
 
 // fp32 -> bf16 copy of n elements (refresh of the weight copies)
 int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);

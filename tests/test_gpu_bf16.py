@@ -67,3 +67,52 @@ def test_eval_loss_bf16():
     want = orc.batch_loss(spec, x1, X[:512], y[:512])
     assert abs(F - want) / want <= BF16_LOSS_TOL
     eng.close()
+
+
+def _one_step_gradients(dims, m, B, seed=29):
+    """Momentum buffers after one step from v = 0 (they equal the stochastic gradient) vs the oracle's gradient."""
+    from paper_1810_08313_b200.binding import LocalSGD
+    import torch
+    from tests.helpers import tensor_slices
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, seed, bf16=True)
+    offs = wl.batch_row_offsets(7, 1, m, 1024, B)
+    rng = np.random.default_rng(1)
+    xs = np.stack([x1 + 0.01 * rng.standard_normal(x1.size).astype(np.float32) for _ in range(m)])
+    xd, yd = to_device(X, y, bf16=True)
+    eng = LocalSGD(m, dims, gemm_dtype="bf16", lr=0.05, momentum=0.9, batch=B)
+    eng.bind_dataset(xd, yd)
+    for i in range(m):
+        eng.set_state(i, xs[i], np.zeros_like(xs[i]))
+    ld = torch.zeros((1, m), device="cuda")
+    eng.local_steps(1, offs, ld)
+    eng.sync()
+    _, gv = eng.get_all()
+    eng.close()
+    out = []
+    for i in range(m):
+        r0 = int(offs[0, i])
+        loss, g = orc.loss_and_grad(spec, xs[i], X[r0:r0 + B], y[r0:r0 + B])
+        assert abs(float(ld[0, i]) - loss) / loss < 5e-3
+        for name, s in tensor_slices(dims, True):
+            want = g[s]; got = gv[i][s].astype(np.float64)
+            err = np.max(np.abs(got - want)) / np.max(np.abs(want))
+            cos = float(got @ want / (np.linalg.norm(got) * np.linalg.norm(want)))
+            out.append((i, name, err, cos))
+    return out
+
+
+def test_tensor_core_update_kernel_tight():
+    """One linear layer 256 -> 128 classes, B = 128: the weight gradient runs on the tensor-core update
+    kernel with nothing but bf16 rounding of dZ between it and the oracle, so a tight bound holds.
+    (A wrong tile, operand orientation or replica index is off by O(1).)"""
+    for i, name, err, cos in _one_step_gradients((256, 128), 3, 128):
+        assert err < 1e-2 and cos > 0.99995, (i, name, err, cos)
+
+
+@pytest.mark.parametrize("dims,m,B", [((256, 256, 128, 10), 2, 128), ((384, 256, 256, 256, 10), 3, 256),
+                                      ((256, 128, 128), 2, 128)])
+def test_single_step_gradients_through_relu(dims, m, B):
+    """All three tensor-core kernels in one step.  bf16 rounding flips a few ReLU masks, which moves single
+    entries by O(10 %) of the largest one; the direction of every tensor's gradient is what is checked."""
+    for i, name, err, cos in _one_step_gradients(dims, m, B):
+        assert cos > 0.995 and err < 0.5, (i, name, err, cos)
