@@ -56,9 +56,10 @@ struct Params {
 template <int BN, int STAGES, int EPI>
 struct Smem {
   static constexpr int kStageBytes = BM * KB_BYTES + BN * KB_BYTES;
-  static constexpr int kStagingBytes = (EPI == EPI_DW) ? 4 * 32 * kStageLd * 4 : 0;
+  // the update epilogue stages its 32x32 blocks in stage 0, which is free once the accumulator is complete
   static constexpr int kBarBytes = (2 * STAGES + 1) * 8 + 16;
-  static constexpr int kTotal = 1024 + STAGES * kStageBytes + kStagingBytes + kBarBytes;
+  static constexpr int kTotal = 1024 + STAGES * kStageBytes + kBarBytes;
+  static_assert(4 * 32 * kStageLd * 4 <= kStageBytes, "staging must fit in one stage");
 };
 
 __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, const Operand& op, int g,
@@ -92,7 +93,7 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* p, const float* v) {
 }
 
 template <int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, (Smem<BN, STAGES, EPI>::kTotal <= 113 * 1024) ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
   using L = Smem<BN, STAGES, EPI>;
   constexpr int ELEMS = KB_BYTES / 2;          // bf16 elements per 128-byte row = K elements per stage
@@ -102,8 +103,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  float* staging = reinterpret_cast<float*>(smem + STAGES * L::kStageBytes);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * L::kStageBytes + L::kStagingBytes);
+  float* staging = reinterpret_cast<float*>(smem);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * L::kStageBytes);
   uint64_t* empty = full + STAGES;
   uint64_t* accum = empty + STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
@@ -220,41 +221,39 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             __uint_as_float(r[4 * i + 3]));
           __syncwarp();
           const int cc = (lane & 7) * 4;
+          // all 16 row-segment loads of this block are issued before the first use
+          float4 w4[8], v4[8];
+          const int64_t at0 = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + (lane >> 3)) * p.N + col + cc;
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            float4 w4[4], v4[4];
+          for (int it = 0; it < 8; ++it) {
+            const int64_t at = at0 + (int64_t)(it * 4) * p.N;
+            w4[it] = *reinterpret_cast<const float4*>(p.W + at);
+            if (p.mu != 0.f) v4[it] = *reinterpret_cast<const float4*>(p.V + at);
+          }
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int rr = (half * 4 + it) * 4 + (lane >> 3);
-              const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + rr) * p.N + col + cc;
-              w4[it] = *reinterpret_cast<const float4*>(p.W + at);
-              if (p.mu != 0.f) v4[it] = *reinterpret_cast<const float4*>(p.V + at);
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3);
+            const int64_t at = at0 + (int64_t)(it * 4) * p.N;
+            const float4 gacc = *reinterpret_cast<const float4*>(&st[rr * kStageLd + cc]);
+            float gs[4] = {gacc.x, gacc.y, gacc.z, gacc.w};
+            float ws[4] = {w4[it].x, w4[it].y, w4[it].z, w4[it].w};
+            float vs[4] = {0.f, 0.f, 0.f, 0.f};
+            if (p.mu != 0.f) { vs[0] = v4[it].x; vs[1] = v4[it].y; vs[2] = v4[it].z; vs[3] = v4[it].w; }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float step = (p.mu != 0.f) ? fmaf(p.mu, vs[e], gs[e]) : gs[e];
+              vs[e] = step;
+              ws[e] = fmaf(-p.lr, step, ws[e]);
             }
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int rr = (half * 4 + it) * 4 + (lane >> 3);
-              const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + rr) * p.N + col + cc;
-              const float4 gacc = *reinterpret_cast<const float4*>(&st[rr * kStageLd + cc]);
-              float gs[4] = {gacc.x, gacc.y, gacc.z, gacc.w};
-              float ws[4] = {w4[it].x, w4[it].y, w4[it].z, w4[it].w};
-              float vs[4] = {0.f, 0.f, 0.f, 0.f};
-              if (p.mu != 0.f) { vs[0] = v4[it].x; vs[1] = v4[it].y; vs[2] = v4[it].z; vs[3] = v4[it].w; }
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float step = (p.mu != 0.f) ? fmaf(p.mu, vs[e], gs[e]) : gs[e];
-                vs[e] = step;
-                ws[e] = fmaf(-p.lr, step, ws[e]);
-              }
-              *reinterpret_cast<float4*>(p.W + at) = make_float4(ws[0], ws[1], ws[2], ws[3]);
-              if (p.mu != 0.f) *reinterpret_cast<float4*>(p.V + at) = make_float4(vs[0], vs[1], vs[2], vs[3]);
-              if (p.Wb != nullptr) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
-                __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
-                uint2 u;
-                u.x = *reinterpret_cast<uint32_t*>(&lo);
-                u.y = *reinterpret_cast<uint32_t*>(&hi);
-                *reinterpret_cast<uint2*>(p.Wb + at) = u;
-              }
+            *reinterpret_cast<float4*>(p.W + at) = make_float4(ws[0], ws[1], ws[2], ws[3]);
+            if (p.mu != 0.f) *reinterpret_cast<float4*>(p.V + at) = make_float4(vs[0], vs[1], vs[2], vs[3]);
+            if (p.Wb != nullptr) {
+              __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
+              __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
+              uint2 u;
+              u.x = *reinterpret_cast<uint32_t*>(&lo);
+              u.y = *reinterpret_cast<uint32_t*>(&hi);
+              *reinterpret_cast<uint2*>(p.Wb + at) = u;
             }
           }
           __syncwarp();
@@ -367,7 +366,7 @@ int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches) {
   p.W = a.W; p.V = a.V; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.lr = a.lr; p.mu = a.mu;
   p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  return launch_one<128, true, true, EPI_DW, 4>(*a.mapDz, *a.mapA, p, a.groups, st);
+  return launch_one<128, true, true, EPI_DW, 3>(*a.mapDz, *a.mapA, p, a.groups, st);
 }
 
 }  // namespace ls
