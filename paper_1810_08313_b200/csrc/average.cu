@@ -23,6 +23,7 @@ __device__ __forceinline__ float4 add4(float4 a, float4 b) {
 __device__ __forceinline__ float4 div4(float4 a, float d) {
   return make_float4(__fdiv_rn(a.x, d), __fdiv_rn(a.y, d), __fdiv_rn(a.z, d), __fdiv_rn(a.w, d));
 }
+__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, float4 v) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
   __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
@@ -37,10 +38,11 @@ __device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, float4 v) {
 template <int M>
 __global__ void __launch_bounds__(kThreads)
 average_vec4_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
-                    __nv_bfloat16* __restrict__ shadow) {
+                    __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
   const int m = M > 0 ? M : m_rt;
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
   const bool do_shadow = (shadow != nullptr) && blockIdx.y == 0;
+  const bool do_lo = (lo != nullptr) && blockIdx.y == 0;
   const float mf = (float)m;
   const int64_t step = (int64_t)gridDim.x * kThreads;
   for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += step) {
@@ -73,6 +75,10 @@ average_vec4_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int6
     if (do_shadow) {
       for (int j = 0; j < m; ++j) store_bf16x4(shadow + (int64_t)j * stride + i * 4, mean);
     }
+    if (do_lo) {
+      const float4 l4 = make_float4(tf32_lo(mean.x), tf32_lo(mean.y), tf32_lo(mean.z), tf32_lo(mean.w));
+      for (int j = 0; j < m; ++j) *reinterpret_cast<float4*>(lo + (int64_t)j * stride + i * 4) = l4;
+    }
   }
 }
 
@@ -80,7 +86,7 @@ average_vec4_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int6
 // 16-byte aligned.  Same arithmetic, one element per thread.
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
-                      __nv_bfloat16* __restrict__ shadow) {
+                      __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
   const bool do_shadow = (shadow != nullptr) && blockIdx.y == 0;
   const float mf = (float)m;
@@ -92,6 +98,8 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
     for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
     if (do_shadow)
       for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + i] = __float2bfloat16_rn(mean);
+    if (lo != nullptr && blockIdx.y == 0)
+      for (int j = 0; j < m; ++j) lo[(int64_t)j * stride + i] = tf32_lo(mean);
   }
 }
 
@@ -107,17 +115,18 @@ int num_sms() {
 
 template <int M>
 void launch_vec4(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
-                 __nv_bfloat16* shadow) {
-  average_vec4_kernel<M><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow);
+                 __nv_bfloat16* shadow, float* lo) {
+  average_vec4_kernel<M><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo);
 }
 
 }  // namespace
 
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches) {
+                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches) {
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
   const bool aligned = (reinterpret_cast<uintptr_t>(base) % 16 == 0) && (stride % 4 == 0) && (buf_stride % 4 == 0) &&
-                       (shadow == nullptr || reinterpret_cast<uintptr_t>(shadow) % 8 == 0);
+                       (shadow == nullptr || reinterpret_cast<uintptr_t>(shadow) % 8 == 0) &&
+                       (lo == nullptr || reinterpret_cast<uintptr_t>(lo) % 16 == 0);
   const int64_t n_vec = aligned ? n / 4 : 0;
   const int sms = num_sms();
   if (n_vec > 0) {
@@ -128,11 +137,11 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     if (want < gx) gx = want;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
     switch (m) {
-      case 2: launch_vec4<2>(grid, st, base, buf_stride, m, n_vec, stride, shadow); break;
-      case 4: launch_vec4<4>(grid, st, base, buf_stride, m, n_vec, stride, shadow); break;
-      case 8: launch_vec4<8>(grid, st, base, buf_stride, m, n_vec, stride, shadow); break;
-      case 16: launch_vec4<16>(grid, st, base, buf_stride, m, n_vec, stride, shadow); break;
-      default: launch_vec4<0>(grid, st, base, buf_stride, m, n_vec, stride, shadow); break;
+      case 2: launch_vec4<2>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
+      case 4: launch_vec4<4>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
+      case 8: launch_vec4<8>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
+      case 16: launch_vec4<16>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
+      default: launch_vec4<0>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
     }
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
@@ -144,7 +153,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     int64_t gx = (rem + kThreads - 1) / kThreads;
     if (gx > (int64_t)sms * 8) gx = (int64_t)sms * 8;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow);
+    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, lo);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -157,6 +166,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
 extern "C" int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride, void* cuda_stream) {
   if (buf_dev == nullptr || m < 1 || P < 0 || stride < P) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(buf_dev) % 4 != 0) return LS_ERR_INVALID_ARG;
-  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr);
+  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
+                             nullptr);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

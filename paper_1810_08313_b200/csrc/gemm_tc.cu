@@ -5,10 +5,21 @@
 //   warp 0      TMA producer: cp.async.bulk.tensor tiles (128-byte swizzle) into a ring of stages
 //   warp 1      allocates tensor memory, issues tcgen05.mma (one elected thread), accumulator in TMEM
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (warp w owns TMEM lanes 32*(w%4)..+31) and apply
-//                 forward   Z = A W^T + b, relu, store as bf16            (evaluating f, Section 2)
-//                 backward  dZ_prev = (dZ W) * 1[act > 0], store as bf16
-//                 update    G = dZ^T A; v <- mu v + G; W <- W - eta v; refresh the bf16 copy of W
-//                           (Section 2 mini-batch SGD update, Section 5.3 momentum); G never leaves the SM
+//                 forward   Z = A W^T + b, relu                            (evaluating f, Section 2)
+//                 backward  dZ_prev = (dZ W) * 1[act > 0]
+//                 update    G = dZ^T A; v <- mu v + G; W <- W - eta v      (Section 2 mini-batch SGD
+//                           update, Section 5.3 momentum); G never leaves the SM
+//
+// Two operand formats:
+//   bf16   one tcgen05.mma kind::f16 per 16 elements of K; outputs rounded to bf16.
+//   fp32   every fp32 operand x is used as the pair (hi, lo): hi is x itself, of which the tensor
+//          core reads the upper 19 bits (tf32), lo = x - tf32(x) lives in a second array that the
+//          producing kernel wrote next to x.  Three kind::tf32 MMAs per 8 elements of K
+//          (lo*hi + hi*lo + hi*hi) give products accurate to about 2^-21, accumulated in fp32.
+//          The tensor core's fp32 accumulation truncates, which biases a long sum; the forward and
+//          backward kernels therefore restart the TMEM accumulator every kChunkStages stages (two
+//          accumulators, double-buffered) and the epilogue warps add the partial sums in registers
+//          with round-to-nearest while the next chunk is being multiplied.
 //
 // Operands are read in place whatever their orientation: a K-major operand
 // ([rows][K], K contiguous) and an MN-major operand ([K][rows], rows contiguous)
@@ -27,10 +38,9 @@ using namespace ptx;
 
 constexpr int BM = 128;            // rows of the output tile = TMEM lanes
 constexpr int KB_BYTES = 128;      // bytes of K per stage row (one swizzle row)
-constexpr int CHUNK_ROWS = 64;     // rows per TMA box
-constexpr int CHUNK_BYTES = CHUNK_ROWS * KB_BYTES;   // 8 KB per TMA box
 constexpr int kThreads = 192;
 constexpr int kStageLd = 36;       // floats per staged row (32 + 4 padding) in the update epilogue
+constexpr int kChunkStages = 4;    // fp32 forward/backward: stages per TMEM accumulation chunk (48 MMAs)
 
 enum { EPI_FWD = 0, EPI_DX = 1, EPI_DW = 2 };
 
@@ -42,43 +52,45 @@ struct Operand {
 };
 
 struct Params {
-  Operand a, b;
+  Operand a, b, a_lo, b_lo;
   int M, N, K;               // per group, in elements
   // forward
   const float* bias; int64_t bias_gstride; int relu;
-  // forward / backward output, backward mask
-  void* C; const void* act;
+  // forward / backward output (+ its lo part in fp32 mode), backward mask
+  void* C; float* Clo; const void* act;
   // update
-  float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride; float lr, mu;
+  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride; float lr, mu;
   int* err_flag;
 };
 
-template <int BN, int STAGES, int EPI>
+template <bool TF32, int BN, int STAGES>
 struct Smem {
-  static constexpr int kStageBytes = BM * KB_BYTES + BN * KB_BYTES;
+  static constexpr int kTiles = TF32 ? 2 : 1;      // hi and lo copies of each operand tile
+  static constexpr int kABytes = BM * KB_BYTES;
+  static constexpr int kBBytes = BN * KB_BYTES;
+  static constexpr int kStageBytes = kTiles * (kABytes + kBBytes);
   // the update epilogue stages its 32x32 blocks in stage 0, which is free once the accumulator is complete
-  static constexpr int kBarBytes = (2 * STAGES + 1) * 8 + 16;
+  static constexpr int kBarBytes = (2 * STAGES + 4) * 8 + 16;
   static constexpr int kTotal = 1024 + STAGES * kStageBytes + kBarBytes;
   static_assert(4 * 32 * kStageLd * 4 <= kStageBytes, "staging must fit in one stage");
+  static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
 
+// Bring one operand tile of `tile_extent` MN-rows x ELEMS K-elements into shared memory as boxes of
+// 128 bytes x ELEMS rows.  K-major: box rows are MN-rows, inner coordinate k0.  MN-major: box rows are
+// K-rows, inner coordinate is the tile start; chunks of ELEMS MN-elements follow each other.
+template <int ELEMS>
 __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, const Operand& op, int g,
-                                           bool mn_major, int tile0, int tile_extent, int k0, int elems_per_row) {
-  // K-major: boxes of 64 rows, inner coordinate k0.  MN-major: boxes of 64 K-rows, inner coordinate = tile start.
+                                           bool mn_major, int tile0, int tile_extent, int k0) {
+  constexpr int kChunkBytes = ELEMS * KB_BYTES;
   const int row_base = op.rank3 ? 0 : (int)(op.row_off ? op.row_off[g] : (int64_t)g * op.rows_per_group);
   const int z = op.z0 + g * op.z_step;
-  if (!mn_major) {
-    for (int r = 0; r < tile_extent / CHUNK_ROWS; ++r) {
-      char* d = static_cast<char*>(dst) + r * CHUNK_BYTES;
-      if (op.rank3) tma_load_3d(d, tm, bar, k0, tile0 + r * CHUNK_ROWS, z);
-      else tma_load_2d(d, tm, bar, k0, row_base + tile0 + r * CHUNK_ROWS);
-    }
-  } else {
-    for (int c = 0; c < tile_extent / elems_per_row; ++c) {
-      char* d = static_cast<char*>(dst) + c * CHUNK_BYTES;
-      if (op.rank3) tma_load_3d(d, tm, bar, tile0 + c * elems_per_row, k0, z);
-      else tma_load_2d(d, tm, bar, tile0 + c * elems_per_row, row_base + k0);
-    }
+  for (int c = 0; c < tile_extent / ELEMS; ++c) {
+    char* d = static_cast<char*>(dst) + c * kChunkBytes;
+    const int x = mn_major ? tile0 + c * ELEMS : k0;
+    const int y = mn_major ? k0 : tile0 + c * ELEMS;
+    if (op.rank3) tma_load_3d(d, tm, bar, x, y, z);
+    else tma_load_2d(d, tm, bar, x, row_base + y);
   }
 }
 
@@ -92,13 +104,41 @@ __device__ __forceinline__ void store_bf16x8(__nv_bfloat16* p, const float* v) {
   *reinterpret_cast<uint4*>(p) = u;
 }
 
-template <int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
-__global__ void __launch_bounds__(kThreads, (Smem<BN, STAGES, EPI>::kTotal <= 113 * 1024) ? 2 : 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
-  using L = Smem<BN, STAGES, EPI>;
-  constexpr int ELEMS = KB_BYTES / 2;          // bf16 elements per 128-byte row = K elements per stage
-  constexpr int MMA_K = 16;                    // K of one tcgen05.mma, bf16
-  constexpr uint32_t IDESC = make_idesc(1u /*bf16*/, A_MN, B_MN, BM, BN);
+// The part of x that a tf32 read keeps (upper 19 bits) and the remainder.
+__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ float tf32_lo(float x) { return x - tf32_hi(x); }
+
+// Store 32 consecutive outputs of one row: bf16, or fp32 plus the lo parts.
+template <bool TF32>
+__device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, const float (&o)[32]) {
+  if (TF32) {
+    float4* c4 = reinterpret_cast<float4*>(static_cast<float*>(C) + at);
+    float4* l4 = reinterpret_cast<float4*>(Clo + at);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      c4[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+      l4[i] = make_float4(tf32_lo(o[4 * i]), tf32_lo(o[4 * i + 1]), tf32_lo(o[4 * i + 2]), tf32_lo(o[4 * i + 3]));
+    }
+  } else {
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(C) + at;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) store_bf16x8(out + i * 8, o + i * 8);
+  }
+}
+
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
+__global__ void __launch_bounds__(kThreads, (Smem<TF32, BN, STAGES>::kTotal <= 113 * 1024) ? 2 : 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo, const Params p) {
+  using L = Smem<TF32, BN, STAGES>;
+  constexpr int EB = TF32 ? 4 : 2;             // bytes per operand element
+  constexpr int ELEMS = KB_BYTES / EB;         // K elements per stage
+  constexpr int MMA_K = 32 / EB;               // K of one tcgen05.mma (32 bytes)
+  constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
+  constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, A_MN, B_MN, BM, BN);
+  constexpr bool CHUNKED = TF32 && EPI != EPI_DW;
+  constexpr int CS = kChunkStages;
+  constexpr uint32_t TMEM_COLS = CHUNKED ? 2 * BN : BN;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -106,8 +146,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   float* staging = reinterpret_cast<float*>(smem);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * L::kStageBytes);
   uint64_t* empty = full + STAGES;
-  uint64_t* accum = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  uint64_t* acc_full = empty + STAGES;      // [2] accumulator (chunk) complete
+  uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the 4 epilogue warps
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.z;
@@ -116,13 +157,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(accum, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    if (TF32) { prefetch_tmap(&tmAlo); prefetch_tmap(&tmBlo); }
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -137,48 +179,110 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { atomicExch(p.err_flag, 1); break; }
         mbar_expect_tx(&full[s], L::kStageBytes);
         uint8_t* sa = stage_base + s * L::kStageBytes;
-        uint8_t* sb = sa + BM * KB_BYTES;
-        issue_tile(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM, kb * ELEMS, ELEMS);
-        issue_tile(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, kb * ELEMS, ELEMS);
+        uint8_t* sb = sa + L::kABytes;
+        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM, kb * ELEMS);
+        issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, kb * ELEMS);
+        if (TF32) {
+          uint8_t* sal = sb + L::kBBytes;
+          uint8_t* sbl = sal + L::kABytes;
+          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM, kb * ELEMS);
+          issue_tile<ELEMS>(sbl, &tmBlo, &full[s], p.b_lo, g, B_MN, n0, BN, kb * ELEMS);
+        }
       }
     }
   } else if (warp == 1) {
     if (elect_one()) {
-      bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
+      for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
-        if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { atomicExch(p.err_flag, 2); ok = false; break; }
+        const int chunk = CHUNKED ? kb / CS : 0;
+        const uint32_t d_tmem = tmem_base + (uint32_t)((chunk & 1) * BN);
+        const bool chunk_start = CHUNKED ? (kb % CS == 0) : (kb == 0);
+        if (CHUNKED && chunk_start && chunk >= 2 && !mbar_wait(&acc_empty[chunk & 1], ((chunk >> 1) - 1) & 1)) {
+          atomicExch(p.err_flag, 4);
+          break;
+        }
+        if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { atomicExch(p.err_flag, 2); break; }
         tc_fence_after_sync();
         const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
-        const uint32_t b_addr = a_addr + BM * KB_BYTES;
+        const uint32_t b_addr = a_addr + L::kABytes;
+        const uint32_t alo_addr = b_addr + L::kBBytes;
+        const uint32_t blo_addr = alo_addr + L::kABytes;
 #pragma unroll
         for (int k = 0; k < ELEMS / MMA_K; ++k) {
-          // K-major: the next 16 elements of K are 32 bytes further along each swizzled row.
-          // MN-major: they are the next 16 K-rows (16 x 128 bytes); chunks of 64 rows-of-MN follow every 8 KB.
-          const uint64_t da = A_MN ? make_smem_desc(a_addr + k * MMA_K * KB_BYTES, CHUNK_BYTES, 1024)
-                                   : make_smem_desc(a_addr + k * MMA_K * 2, 16, 1024);
-          const uint64_t db = B_MN ? make_smem_desc(b_addr + k * MMA_K * KB_BYTES, CHUNK_BYTES, 1024)
-                                   : make_smem_desc(b_addr + k * MMA_K * 2, 16, 1024);
-          mma_bf16(tmem_base, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+          // K-major: the next MMA_K elements of K are 32 bytes further along each swizzled row.
+          // MN-major: they are the next MMA_K K-rows of 128 bytes; chunks of MN follow every CHUNK_BYTES.
+          const uint32_t a_adv = A_MN ? k * MMA_K * KB_BYTES : k * 32;
+          const uint32_t b_adv = B_MN ? k * MMA_K * KB_BYTES : k * 32;
+          // An MN-major operand of 32-bit elements must use the 128-byte swizzle with 32-byte units,
+          // whose period is 4 K-rows (512 bytes); everything else uses 16-byte units, period 8 rows.
+          const uint32_t a_lbo = A_MN ? CHUNK_BYTES : 16, b_lbo = B_MN ? CHUNK_BYTES : 16;
+          const uint32_t a_sw = (TF32 && A_MN) ? kSwizzle128B_32B : kSwizzle128B;
+          const uint32_t b_sw = (TF32 && B_MN) ? kSwizzle128B_32B : kSwizzle128B;
+          const uint32_t a_sbo = (TF32 && A_MN) ? 512 : 1024, b_sbo = (TF32 && B_MN) ? 512 : 1024;
+          const uint64_t da = make_smem_desc(a_addr + a_adv, a_lbo, a_sbo, a_sw);
+          const uint64_t db = make_smem_desc(b_addr + b_adv, b_lbo, b_sbo, b_sw);
+          if (TF32) {
+            const uint64_t dal = make_smem_desc(alo_addr + a_adv, a_lbo, a_sbo, a_sw);
+            const uint64_t dbl = make_smem_desc(blo_addr + b_adv, b_lbo, b_sbo, b_sw);
+            mma_tf32(d_tmem, dal, db, IDESC, (chunk_start && k == 0) ? 0u : 1u);
+            mma_tf32(d_tmem, da, dbl, IDESC, 1u);
+            mma_tf32(d_tmem, da, db, IDESC, 1u);
+          } else {
+            mma_bf16(d_tmem, da, db, IDESC, (chunk_start && k == 0) ? 0u : 1u);
+          }
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+        if (CHUNKED ? (kb % CS == CS - 1 || kb == num_kb - 1) : (kb == num_kb - 1))
+          mma_commit(&acc_full[chunk & 1]);     // this accumulator is complete
       }
-      mma_commit(accum);           // accumulator complete
     }
   } else {
     // ---- epilogue warps ---------------------------------------------------------
     const int q = warp & 3;
     const int row = m0 + q * 32 + lane;        // output row this thread owns
-    bool ok = mbar_wait(accum, 0);
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    float sum[CHUNKED ? BN : 1];
+    bool ok = true;
+    if (CHUNKED) {
+      // add the partial accumulators in registers (this thread owns one output row) as they complete
+#pragma unroll
+      for (int i = 0; i < BN; ++i) sum[i] = 0.f;
+      const int num_chunks = (num_kb + CS - 1) / CS;
+      for (int ch = 0; ch < num_chunks && ok; ++ch) {
+        const int buf = ch & 1;
+        ok = mbar_wait(&acc_full[buf], (ch >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(taddr + buf * BN + c * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sum[c * 32 + i] += __uint_as_float(r[i]);
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      }
+    } else {
+      ok = mbar_wait(&acc_full[0], 0);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after_sync();
+    }
     if (!ok && lane == 0) atomicExch(p.err_flag, 3);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after_sync();
     if (ok) {
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
-        tmem_ld_32x32(taddr + c * 32, r);
-        tmem_ld_wait();
+        if (CHUNKED) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[c * 32 + i]);
+        } else {
+          tmem_ld_32x32(taddr + c * 32, r);
+          tmem_ld_wait();
+        }
         const int col = n0 + c * 32;
         if (EPI == EPI_FWD) {
           float o[32];
@@ -189,28 +293,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (bias) v += __ldg(bias + i);
             o[i] = (p.relu && !(v > 0.f)) ? 0.f : v;
           }
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.C) + ((int64_t)g * p.M + row) * p.N + col;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) store_bf16x8(out + i * 8, o + i * 8);
+          store_row32<TF32>(p.C, p.Clo, ((int64_t)g * p.M + row) * p.N + col, o);
         } else if (EPI == EPI_DX) {
           const int64_t at = ((int64_t)g * p.M + row) * p.N + col;
-          const uint4* a4 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) + at);
           float o[32];
+          if (TF32) {
+            const float4* a4 = reinterpret_cast<const float4*>(static_cast<const float*>(p.act) + at);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint4 u = a4[i];
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+            for (int i = 0; i < 8; ++i) {
+              const float4 a = a4[i];
+              o[4 * i] = a.x > 0.f ? __uint_as_float(r[4 * i]) : 0.f;
+              o[4 * i + 1] = a.y > 0.f ? __uint_as_float(r[4 * i + 1]) : 0.f;
+              o[4 * i + 2] = a.z > 0.f ? __uint_as_float(r[4 * i + 2]) : 0.f;
+              o[4 * i + 3] = a.w > 0.f ? __uint_as_float(r[4 * i + 3]) : 0.f;
+            }
+          } else {
+            const uint4* a4 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) + at);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              // a bf16 is positive iff it is non-zero with the sign bit clear
-              const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
-              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2]) : 0.f;
-              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2 + 1]) : 0.f;
+            for (int i = 0; i < 4; ++i) {
+              const uint4 u = a4[i];
+              const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                // a bf16 is positive iff it is non-zero with the sign bit clear
+                const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
+                o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2]) : 0.f;
+                o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2 + 1]) : 0.f;
+              }
             }
           }
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.C) + at;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) store_bf16x8(out + i * 8, o + i * 8);
+          store_row32<TF32>(p.C, p.Clo, at, o);
         } else {
           // transpose the 32x32 block through shared memory so that global accesses run along rows
           float* st = staging + (warp - 2) * 32 * kStageLd;
@@ -247,7 +359,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             *reinterpret_cast<float4*>(p.W + at) = make_float4(ws[0], ws[1], ws[2], ws[3]);
             if (p.mu != 0.f) *reinterpret_cast<float4*>(p.V + at) = make_float4(vs[0], vs[1], vs[2], vs[3]);
-            if (p.Wb != nullptr) {
+            if (TF32) {
+              *reinterpret_cast<float4*>(p.Wlo + at) =
+                  make_float4(tf32_lo(ws[0]), tf32_lo(ws[1]), tf32_lo(ws[2]), tf32_lo(ws[3]));
+            } else if (p.Wb != nullptr) {
               __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
               __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
               uint2 u;
@@ -266,7 +381,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     __syncwarp();
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, BN);
+    tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
@@ -288,10 +403,10 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
-int launch_one(const CUtensorMap& a, const CUtensorMap& b, const Params& p, int groups, cudaStream_t st) {
-  using L = Smem<BN, STAGES, EPI>;
-  auto kern = tc_gemm_kernel<BN, A_MN, B_MN, EPI, STAGES>;
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
+int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
+  using L = Smem<TF32, BN, STAGES>;
+  auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
@@ -299,74 +414,98 @@ int launch_one(const CUtensorMap& a, const CUtensorMap& b, const Params& p, int 
     configured = true;
   }
   dim3 grid((unsigned)(p.N / BN), (unsigned)(p.M / BM), (unsigned)groups);
-  kern<<<grid, kThreads, L::kTotal, st>>>(a, b, p);
+  const CUtensorMap* alo = TF32 ? mp.a_lo : mp.a;
+  const CUtensorMap* blo = TF32 ? mp.b_lo : mp.b;
+  kern<<<grid, kThreads, L::kTotal, st>>>(*mp.a, *mp.b, *alo, *blo, p);
   return cudaGetLastError();
 }
 
+int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, int rank, int64_t rows, int64_t cols,
+             int64_t groups, int64_t gstride) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t eb = fp32 ? 4 : 2;
+  const cuuint32_t elems = (cuuint32_t)(KB_BYTES / eb);
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * eb, (cuuint64_t)gstride * eb};
+  cuuint32_t box[3] = {elems, elems, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+                  const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  (fp32 && mn32) ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+inline int few_tiles(int M, int N, int groups, int bn) { return (M / BM) * (N / bn) * groups; }
+
 }  // namespace
 
-// 2-D map over a row-major bf16 matrix [rows][cols], box 64 x 64, 128-byte swizzle.
-int tc_make_map_2d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return cudaErrorNotSupported;
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {64, 64};
-  cuuint32_t es[2] = {1, 1};
-  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+// 2-D map over a row-major matrix [rows][cols] of bf16 or fp32; box = 128 bytes x (64 | 32) rows, 128-byte
+// swizzle.  mn32: the fp32 tensor will be read as an MN-major operand (swizzle in 32-byte units).
+int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols) {
+  return make_map(out, base, fp32, mn32, 2, rows, cols, 1, 0);
+}
+// 3-D map over `groups` row-major matrices [rows][cols] that start every gstride elements.
+int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
+                   int64_t groups, int64_t gstride) {
+  return make_map(out, base, fp32, mn32, 3, rows, cols, groups, gstride);
 }
 
-// 3-D map over `groups` row-major bf16 matrices [rows][cols] that start every gstride elements.
-int tc_make_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups, int64_t gstride) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return cudaErrorNotSupported;
-  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
-  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)gstride * 2};
-  cuuint32_t box[3] = {64, 64, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+// M output rows, N output columns, K contraction length of one group.
+bool tc_shape_ok(bool fp32, int M, int N, int K) {
+  if (M <= 0 || N <= 0 || K <= 0 || M % BM != 0) return false;
+  return fp32 ? (N % 64 == 0 && K % 32 == 0) : (N % 128 == 0 && K % 64 == 0);
 }
-
-bool tc_shape_ok(int M, int N, int K) { return M % BM == 0 && N % 128 == 0 && K % 64 == 0 && M > 0 && N > 0 && K > 0; }
 
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
   p.a = Operand{a.row_off, a.M, 0, 0, 0};
-  p.b = Operand{nullptr, 0, a.w_z0, a.w_zstep, 1};
+  p.a_lo = Operand{nullptr, a.M, 0, 0, 0};
+  p.b = p.b_lo = Operand{nullptr, 0, a.w_z0, a.w_zstep, 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.bias = a.bias; p.bias_gstride = a.bias_gstride; p.relu = a.relu;
-  p.C = a.C; p.err_flag = a.err_flag;
+  p.C = a.C; p.Clo = a.Clo; p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  if (a.N % 256 == 0) return launch_one<256, false, false, EPI_FWD, 4>(*a.mapA, *a.mapW, p, a.groups, st);
-  return launch_one<128, false, false, EPI_FWD, 4>(*a.mapA, *a.mapW, p, a.groups, st);
+  if (a.fp32) {
+    if (a.N % 128 == 0 && few_tiles(a.M, a.N, a.groups, 128) >= 148)
+      return launch_one<true, 128, false, false, EPI_FWD, 3>(a.maps, p, a.groups, st);
+    return launch_one<true, 64, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
+  }
+  if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
+  return launch_one<false, 128, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
 }
 
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
-  p.a = Operand{nullptr, a.M, 0, 0, 0};
-  p.b = Operand{nullptr, 0, 0, 1, 1};
+  p.a = p.a_lo = Operand{nullptr, a.M, 0, 0, 0};
+  p.b = p.b_lo = Operand{nullptr, 0, 0, 1, 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
-  p.C = a.C; p.act = a.act; p.err_flag = a.err_flag;
+  p.C = a.C; p.Clo = a.Clo; p.act = a.act; p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  if (a.N % 256 == 0) return launch_one<256, false, true, EPI_DX, 4>(*a.mapDz, *a.mapW, p, a.groups, st);
-  return launch_one<128, false, true, EPI_DX, 4>(*a.mapDz, *a.mapW, p, a.groups, st);
+  if (a.fp32) {
+    if (a.N % 128 == 0 && few_tiles(a.M, a.N, a.groups, 128) >= 148)
+      return launch_one<true, 128, false, true, EPI_DX, 3>(a.maps, p, a.groups, st);
+    return launch_one<true, 64, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
+  }
+  if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
+  return launch_one<false, 128, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
 }
 
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
-  p.a = Operand{nullptr, a.B, 0, 0, 0};
+  p.a = p.a_lo = Operand{nullptr, a.B, 0, 0, 0};
   p.b = Operand{a.row_off, a.B, 0, 0, 0};
+  p.b_lo = Operand{nullptr, a.B, 0, 0, 0};
   p.M = a.M; p.N = a.N; p.K = a.B;
-  p.W = a.W; p.V = a.V; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.lr = a.lr; p.mu = a.mu;
+  p.W = a.W; p.V = a.V; p.Wb = a.Wb; p.Wlo = a.Wlo; p.w_gstride = a.w_gstride; p.lr = a.lr; p.mu = a.mu;
   p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  return launch_one<128, true, true, EPI_DW, 3>(*a.mapDz, *a.mapA, p, a.groups, st);
+  if (a.fp32) {
+    if (a.N % 128 == 0) return launch_one<true, 128, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
+    return launch_one<true, 64, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
+  }
+  return launch_one<false, 128, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
 }
 
 }  // namespace ls

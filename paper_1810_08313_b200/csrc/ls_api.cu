@@ -64,10 +64,16 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   auto take = [&](size_t bytes) { size_t at = off; off = round_up_sz(off + bytes, A); return at; };
   lay.params_off = take((size_t)m * lay.stride * 4);
   lay.mom_off = take((size_t)m * lay.stride * 4);
-  lay.shadow_off = take(lay.bf16 ? (size_t)m * lay.stride * 2 : 0);
-  for (int l = 1; l < lay.L; ++l) lay.act_off[l] = take((size_t)m * batch * lay.dims[l] * esz);
-  lay.dz_off[0] = take((size_t)m * batch * lay.max_width * esz);
-  lay.dz_off[1] = take((size_t)m * batch * lay.max_width * esz);
+  lay.shadow_off = take((size_t)m * lay.stride * (lay.bf16 ? 2 : 4));
+  for (int l = 1; l < lay.L; ++l) {
+    lay.act_off[l] = take((size_t)m * batch * lay.dims[l] * esz);
+    if (!lay.bf16) lay.actlo_off[l] = take((size_t)m * batch * lay.dims[l] * 4);
+  }
+  for (int s = 0; s < 2; ++s) {
+    lay.dz_off[s] = take((size_t)m * batch * lay.max_width * esz);
+    if (!lay.bf16) lay.dzlo_off[s] = take((size_t)m * batch * lay.max_width * 4);
+  }
+  if (!lay.bf16) lay.xlo_off = take((size_t)m * batch * lay.dims[0] * 4);
   lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
   lay.evaloff_off = take((size_t)kEvalCap * 8);
@@ -114,10 +120,21 @@ struct ProfScope {
   }
 };
 
+// Refresh the operand copies of the weights (bf16 rounding, or the lo twin of fp32 models).
 static int refresh_shadow(ls_handle* h) {
-  if (!h->lay.bf16) return LS_OK;
-  LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), (int64_t)h->lay.m * h->lay.stride, h->stream, &h->launches));
+  const int64_t n = (int64_t)h->lay.m * h->lay.stride;
+  if (h->lay.bf16) LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), n, h->stream, &h->launches));
+  else LS_CUDA(h, launch_split_lo(params_of(h), wlo_of(h), n, h->stream, &h->launches));
   return LS_OK;
+}
+
+static inline float* lo_at(const ls_handle* h, size_t off) {
+  return h->lay.bf16 ? nullptr : reinterpret_cast<float*>(h->state + off);
+}
+// fp32 models: does any tensor-core kernel read the mini-batch rows (layer 1 forward or update)?
+static inline bool needs_x_lo(const Layout& lay) {
+  return !lay.bf16 && ((lay.L > 1 && tc_shape_ok(true, lay.batch, lay.dims[1], lay.dims[0])) ||
+                       tc_shape_ok(true, lay.dims[1], lay.dims[0], lay.batch));
 }
 
 // One forward pass of `groups` mini-batches.  Group g reads rows
@@ -125,17 +142,27 @@ static int refresh_shadow(ls_handle* h) {
 // (w_gstride == 0: every group uses the same replica).
 static inline int* err_flag_of(const ls_handle* h) { return reinterpret_cast<int*>(h->state + h->lay.err_off); }
 
-static int forward(ls_handle* h, const void* x, const CUtensorMap* xmap, const void* y, const int64_t* row_off_dev,
+// x maps: [0] for K-major reads, [1] for MN-major reads of the mini-batch rows
+struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; };
+
+static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
                    int groups, int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
   const float* P = params_of(h) + replica0 * lay.stride;
   const __nv_bfloat16* S = bf ? shadow_of(h) + replica0 * lay.stride : nullptr;
+  if (needs_x_lo(lay))
+    LS_CUDA(h, launch_gather_lo(static_cast<const float*>(x), row_off_dev, lo_at(h, lay.xlo_off), groups, lay.batch,
+                                lay.dims[0], h->stream, &h->launches));
   for (int l = 0; l < lay.L; ++l) {
-    if (bf && l < lay.L - 1 && tc_shape_ok(lay.batch, lay.dims[l + 1], lay.dims[l])) {
+    if (l < lay.L - 1 && tc_shape_ok(!bf, lay.batch, lay.dims[l + 1], lay.dims[l])) {
       TcFwdArgs t;
-      t.mapA = (l == 0) ? xmap : &h->maps.act[l];
-      t.mapW = &h->maps.w[l];
+      t.fp32 = !bf;
+      t.maps.a = (l == 0) ? xmap.k : &h->maps.act[l];
+      t.maps.a_lo = (l == 0) ? &h->maps.x_lo : &h->maps.act_lo[l];
+      t.maps.b = &h->maps.w[l];
+      t.maps.b_lo = &h->maps.w_lo[l];
+      t.Clo = lo_at(h, lay.actlo_off[l + 1]);
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.w_z0 = (int)replica0; t.w_zstep = w_gstride != 0 ? 1 : 0;
       t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
@@ -156,6 +183,7 @@ static int forward(ls_handle* h, const void* x, const CUtensorMap* xmap, const v
     a.bias_gstride = w_gstride;
     const bool last = (l == lay.L - 1);
     a.C = last ? (void*)(h->state + lay.logits_off) : (void*)(h->state + lay.act_off[l + 1]);
+    a.Clo = last ? nullptr : lo_at(h, lay.actlo_off[l + 1]);
     a.M = lay.batch; a.N = lay.dims[l + 1]; a.K = lay.dims[l]; a.groups = groups;
     a.relu = last ? 0 : 1;
     ProfScope ps(h, LS_K_FWD, l);
@@ -165,6 +193,7 @@ static int forward(ls_handle* h, const void* x, const CUtensorMap* xmap, const v
   la.logits = reinterpret_cast<const float*>(h->state + lay.logits_off);
   la.y = y; la.row_off = row_off_dev;
   la.dZ = want_dz ? (void*)(h->state + lay.dz_off[0]) : nullptr;
+  la.dZlo = want_dz ? lo_at(h, lay.dzlo_off[0]) : nullptr;
   la.loss_out = loss_out;
   la.B = lay.batch; la.C = lay.dims[lay.L]; la.groups = groups; la.loss_kind = h->spec.loss;
   ProfScope ps(h, LS_K_LOSS, 0);
@@ -173,22 +202,27 @@ static int forward(ls_handle* h, const void* x, const CUtensorMap* xmap, const v
 }
 
 // One local update of all m replicas (forward, backward, fused SGD-momentum).
-static int local_step(ls_handle* h, const void* x, const CUtensorMap* xmap, const void* y, const int64_t* row_off_dev,
+static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
                       float* loss_out) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
+  const TcMaps& mn = bf ? h->maps : h->maps_mn;     // descriptors for MN-major reads
   int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
   if (rc != LS_OK) return rc;
   int cur = 0;
   for (int l = lay.L - 1; l >= 0; --l) {
     void* dZ = h->state + lay.dz_off[cur];
-    if (l > 0 && bf && tc_shape_ok(lay.batch, lay.dims[l], lay.dims[l + 1])) {
+    if (l > 0 && tc_shape_ok(!bf, lay.batch, lay.dims[l], lay.dims[l + 1])) {
       // the data gradient reads W_l before the update below overwrites it
       TcDxArgs t;
-      t.mapDz = &h->maps.dz[l];
-      t.mapW = &h->maps.w[l];
+      t.fp32 = !bf;
+      t.maps.a = &h->maps.dz[l];
+      t.maps.a_lo = &h->maps.dz_lo[l];
+      t.maps.b = &mn.w[l];
+      t.maps.b_lo = &mn.w_lo[l];
       t.act = h->state + lay.act_off[l];
       t.C = h->state + lay.dz_off[cur ^ 1];
+      t.Clo = lo_at(h, lay.dzlo_off[cur ^ 1]);
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
       t.err_flag = err_flag_of(h);
       ProfScope ps(h, LS_K_DX, l);
@@ -200,18 +234,23 @@ static int local_step(ls_handle* h, const void* x, const CUtensorMap* xmap, cons
       d.w_gstride = lay.stride;
       d.act = h->state + lay.act_off[l];
       d.C = h->state + lay.dz_off[cur ^ 1];
+      d.Clo = lo_at(h, lay.dzlo_off[cur ^ 1]);
       d.M = lay.batch; d.N = lay.dims[l]; d.K = lay.dims[l + 1]; d.groups = lay.m;
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
     }
-    if (bf && tc_shape_ok(lay.dims[l + 1], lay.dims[l], lay.batch)) {
+    if (tc_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
       TcDwArgs t;
-      t.mapDz = &h->maps.dz[l];
-      t.mapA = (l == 0) ? xmap : &h->maps.act[l];
+      t.fp32 = !bf;
+      t.maps.a = &mn.dz[l];
+      t.maps.a_lo = &mn.dz_lo[l];
+      t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
+      t.maps.b_lo = (l == 0) ? &mn.x_lo : &mn.act_lo[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.W = params_of(h) + lay.w_off[l];
       t.V = mom_of(h) + lay.w_off[l];
-      t.Wb = shadow_of(h) + lay.w_off[l];
+      t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
+      t.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
       t.w_gstride = lay.stride;
       t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
       t.lr = h->lr; t.mu = h->mu;
@@ -226,6 +265,7 @@ static int local_step(ls_handle* h, const void* x, const CUtensorMap* xmap, cons
     w.W = params_of(h) + lay.w_off[l];
     w.V = mom_of(h) + lay.w_off[l];
     w.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
+    w.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
     w.w_gstride = lay.stride;
     w.M = lay.dims[l + 1]; w.N = lay.dims[l]; w.B = lay.batch; w.groups = lay.m;
     w.lr = h->lr; w.mu = h->mu;
@@ -257,7 +297,7 @@ static int average(ls_handle* h) {
   {
     ProfScope ps(h, LS_K_AVG, 0);
     LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                              lay.bf16 ? shadow_of(h) : nullptr, h->stream, &h->launches));
+                              shadow_of(h), wlo_of(h), h->stream, &h->launches));
   }
   if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
@@ -279,7 +319,8 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
   LS_CUDA(h, cudaMemcpyAsync(off_dev, offs.data(), (size_t)chunks * 8, cudaMemcpyHostToDevice, h->stream));
   for (int64_t c0 = 0; c0 < chunks; c0 += lay.m) {
     const int groups = (int)((chunks - c0 < lay.m) ? chunks - c0 : lay.m);
-    int rc = forward(h, h->x_dev, &h->maps.x_data, h->y_dev, off_dev + c0, groups, replica, 0, false, loss_dev + c0);
+    int rc = forward(h, h->x_dev, XMaps{&h->maps.x_data, &h->maps_mn.x_data}, h->y_dev, off_dev + c0, groups, replica, 0,
+                     false, loss_dev + c0);
     if (rc != LS_OK) return rc;
   }
   LS_CUDA(h, cudaMemcpyAsync(h->pinned, loss_dev, (size_t)chunks * 4, cudaMemcpyDeviceToHost, h->stream));
@@ -302,7 +343,8 @@ static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, fl
     LS_CUDA(h, cudaMemcpyAsync(off_dev, row_offset_host + (int64_t)s0 * lay.m, (size_t)n * lay.m * 8,
                                cudaMemcpyHostToDevice, h->stream));
     for (int s = 0; s < n; ++s) {
-      int rc = local_step(h, h->x_dev, &h->maps.x_data, h->y_dev, off_dev + (int64_t)s * lay.m,
+      const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
+      int rc = local_step(h, h->x_dev, XMaps{&h->maps.x_data, &mnm.x_data}, h->y_dev, off_dev + (int64_t)s * lay.m,
                           loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr);
       if (rc != LS_OK) return rc;
     }
@@ -382,22 +424,38 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&h->pinned), (size_t)kEvalCap * 4);
   // parameters, momentum, workspace start at zero; the staging row offsets are g*batch
   if (e == cudaSuccess) e = cudaMemsetAsync(h->state, 0, lay.total, h->stream);
-  if (e == cudaSuccess && lay.bf16) {
-    // TMA descriptors (every bf16 tensor start is 256-byte aligned; rows must be 16-byte multiples)
-    // A tensor gets a descriptor when its rows are 16-byte multiples; the tensor-core kernels are
-    // only chosen for shapes (multiples of 64) whose tensors all satisfy this.
+  if (e == cudaSuccess) {
+    // A tensor gets a TMA descriptor when its rows are 16-byte multiples; the tensor-core kernels are
+    // only chosen for shapes (multiples of 32 / 64) whose tensors all satisfy this.
+    const bool f = !lay.bf16;
+    const int q = f ? 4 : 8;                       // elements per 16 bytes
     const int64_t rows = (int64_t)m * batch;
-    for (int l = 0; l < lay.L && e == cudaSuccess; ++l) {
-      if (lay.dims[l] % 8 == 0) {
-        e = tc_make_map_3d(&h->maps.w[l], shadow_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride);
-        if (e == cudaSuccess && l >= 1)
-          e = tc_make_map_2d(&h->maps.act[l], h->state + lay.act_off[l], rows, lay.dims[l]);
+    auto ok = [&](int e2) { if (e == cudaSuccess) e = e2; };
+    for (int v = 0; v < (f ? 2 : 1); ++v) {        // v = 1: the MN-major descriptors of an fp32 model
+      TcMaps& mp = v ? h->maps_mn : h->maps;
+      const bool mn = v != 0;
+      for (int l = 0; l < lay.L; ++l) {
+        if (lay.dims[l] % q == 0) {
+          const void* wsrc = f ? (const void*)(params_of(h) + lay.w_off[l]) : (const void*)(shadow_of(h) + lay.w_off[l]);
+          ok(tc_make_map_3d(&mp.w[l], wsrc, f, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+          if (f) ok(tc_make_map_3d(&mp.w_lo[l], wlo_of(h) + lay.w_off[l], true, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+          if (l >= 1) {
+            ok(tc_make_map_2d(&mp.act[l], h->state + lay.act_off[l], f, mn, rows, lay.dims[l]));
+            if (f) ok(tc_make_map_2d(&mp.act_lo[l], h->state + lay.actlo_off[l], true, mn, rows, lay.dims[l]));
+          }
+        }
+        if (lay.dims[l + 1] % q == 0) {
+          const int buf = (lay.L - 1 - l) & 1;
+          ok(tc_make_map_2d(&mp.dz[l], h->state + lay.dz_off[buf], f, mn, rows, lay.dims[l + 1]));
+          if (f) ok(tc_make_map_2d(&mp.dz_lo[l], h->state + lay.dzlo_off[buf], true, mn, rows, lay.dims[l + 1]));
+        }
       }
-      if (e == cudaSuccess && lay.dims[l + 1] % 8 == 0)
-        e = tc_make_map_2d(&h->maps.dz[l], h->state + lay.dz_off[(lay.L - 1 - l) & 1], rows, lay.dims[l + 1]);
+      if (lay.dims[0] % q == 0) {
+        for (int s = 0; s < 2; ++s)
+          ok(tc_make_map_2d(&mp.x_stage[s], h->state + lay.stage_x_off[s], f, mn, rows, lay.dims[0]));
+        if (f) ok(tc_make_map_2d(&mp.x_lo, h->state + lay.xlo_off, true, mn, rows, lay.dims[0]));
+      }
     }
-    for (int s = 0; s < 2 && e == cudaSuccess && lay.dims[0] % 8 == 0; ++s)
-      e = tc_make_map_2d(&h->maps.x_stage[s], h->state + lay.stage_x_off[s], rows, lay.dims[0]);
   }
   if (e != cudaSuccess) {
     h->last_cuda = e;
@@ -516,8 +574,10 @@ int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t 
   if (x_dev == nullptr || y_dev == nullptr || n_rows < h->lay.batch) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(x_dev) % 16 != 0 || reinterpret_cast<uintptr_t>(y_dev) % 4 != 0)
     return LS_ERR_INVALID_ARG;
-  if (h->lay.bf16 && h->lay.dims[0] % 8 == 0)
-    LS_CUDA(h, tc_make_map_2d(&h->maps.x_data, x_dev, n_rows, h->lay.dims[0]));
+  if (h->lay.dims[0] % (h->lay.bf16 ? 8 : 4) == 0) {
+    LS_CUDA(h, tc_make_map_2d(&h->maps.x_data, x_dev, !h->lay.bf16, false, n_rows, h->lay.dims[0]));
+    if (!h->lay.bf16) LS_CUDA(h, tc_make_map_2d(&h->maps_mn.x_data, x_dev, true, true, n_rows, h->lay.dims[0]));
+  }
   h->x_dev = x_dev;
   h->y_dev = y_dev;
   h->n_rows = n_rows;
@@ -558,7 +618,9 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
                                  cudaMemcpyHostToDevice, h->copy_stream));
       LS_CUDA(h, cudaEventRecord(h->ev_copied[slot], h->copy_stream));
       LS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_copied[slot], 0));
-      int rc = local_step(h, xs, &h->maps.x_stage[slot], ys, stage_off, loss_stage + (int64_t)s * lay.m);
+      const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
+      int rc = local_step(h, xs, XMaps{&h->maps.x_stage[slot], &mnm.x_stage[slot]}, ys, stage_off,
+                          loss_stage + (int64_t)s * lay.m);
       if (rc != LS_OK) return rc;
       LS_CUDA(h, cudaEventRecord(h->ev_consumed[slot], h->stream));
       used[slot] = true;

@@ -17,8 +17,13 @@ constexpr int kEvalCap = 8192;         // mini-batch chunks per ls_eval_loss cal
 constexpr int64_t kAlignFloats = 64;   // every tensor and every replica starts on a 256-byte boundary
 
 // Where everything lives.  Offsets inside one replica are in elements (the
-// same for the fp32 master copy, the momentum buffer and the bf16 copy);
+// same for the fp32 master copy, the momentum buffer and the operand copy);
 // offsets inside the state block are in bytes.
+//
+// Operand copies.  bf16 models keep a bf16 rounding of the weights.  fp32 models keep, for every
+// tensor that can be a matrix-product operand (weights, layer inputs, dZ, the gathered mini-batch),
+// a "lo" twin holding x - tf32(x): the tensor-core kernels read x as its tf32 upper part and add
+// the lo products (see gemm_tc.cu).  Whoever writes such a tensor writes its twin.
 struct Layout {
   int L = 0;
   int dims[LS_MAX_LAYERS + 1] = {0};
@@ -33,12 +38,16 @@ struct Layout {
   int64_t b_off[LS_MAX_LAYERS] = {0};
   int64_t w_flat[LS_MAX_LAYERS] = {0}; // offsets in the flat interface layout
   int64_t b_flat[LS_MAX_LAYERS] = {0};
-  size_t params_off = 0, mom_off = 0, shadow_off = 0;
-  size_t act_off[LS_MAX_LAYERS + 1] = {0};   // post-ReLU activations of layers 1..L-1
+  size_t params_off = 0, mom_off = 0;
+  size_t shadow_off = 0;                     // bf16 [m][stride] (bf16 models) or float lo twin [m][stride] (fp32)
+  size_t act_off[LS_MAX_LAYERS + 1] = {0};   // post-ReLU activations = inputs of layers 1..L-1
+  size_t actlo_off[LS_MAX_LAYERS + 1] = {0}; // their lo twins (fp32 models)
   size_t dz_off[2] = {0, 0};                 // ping-pong gradient buffers [m][batch][max_width]
+  size_t dzlo_off[2] = {0, 0};
+  size_t xlo_off = 0;                        // lo twin of the current mini-batches [m][batch][dims[0]] (fp32 models)
   size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
   size_t rowoff_off = 0;                     // int64 [kRowOffCap][m]
-  size_t evaloff_off = 0;                    // int64 [m]  (two slots)
+  size_t evaloff_off = 0;                    // int64 [kEvalCap]
   size_t evalloss_off = 0;                   // float [kEvalCap]
   size_t stage_x_off[2] = {0, 0};            // [m][batch][dims[0]] input staging for host batches
   size_t stage_y_off[2] = {0, 0};            // [m][batch] labels / targets
@@ -51,17 +60,20 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out);
 
 }  // namespace ls
 
-// TMA descriptors of the bf16 tensors the tensor-core kernels read (built once per handle).
+// TMA descriptors of the tensors the tensor-core kernels read (built once per handle).
+// The *_lo maps are used by fp32 models only.
 struct alignas(64) TcMaps {
-  CUtensorMap w[LS_MAX_LAYERS];      // bf16 weight copies, 3-D [replica][out][in]
-  CUtensorMap act[LS_MAX_LAYERS];    // input activations of layer l >= 1, 2-D [m*batch][dims[l]]
-  CUtensorMap dz[LS_MAX_LAYERS];     // dZ_l, 2-D [m*batch][dims[l+1]]
-  CUtensorMap x_data;                // bound dataset, 2-D [n_rows][dims[0]]
-  CUtensorMap x_stage[2];            // staging buffers of host batches
+  CUtensorMap w[LS_MAX_LAYERS], w_lo[LS_MAX_LAYERS];      // weights as operands, 3-D [replica][out][in]
+  CUtensorMap act[LS_MAX_LAYERS], act_lo[LS_MAX_LAYERS];  // input of layer l >= 1, 2-D [m*batch][dims[l]]
+  CUtensorMap dz[LS_MAX_LAYERS], dz_lo[LS_MAX_LAYERS];    // dZ_l, 2-D [m*batch][dims[l+1]]
+  CUtensorMap x_data;                                     // bound dataset, 2-D [n_rows][dims[0]]
+  CUtensorMap x_stage[2];                                 // staging buffers of host batches
+  CUtensorMap x_lo;                                       // lo twin of the current mini-batches
 };
 
 struct ls_handle {
-  TcMaps maps;
+  TcMaps maps;       // for K-major reads (and every read of a bf16 tensor)
+  TcMaps maps_mn;    // fp32 models: the same tensors for MN-major reads (swizzle in 32-byte units)
   uint32_t magic;
   ls::Layout lay;
   ls_model_spec spec;
@@ -92,15 +104,18 @@ constexpr uint32_t kMagic = 0x4c53474du;
 inline float* params_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.params_off); }
 inline float* mom_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.mom_off); }
 inline __nv_bfloat16* shadow_of(const ls_handle* h) {
-  return reinterpret_cast<__nv_bfloat16*>(h->state + h->lay.shadow_off);
+  return h->lay.bf16 ? reinterpret_cast<__nv_bfloat16*>(h->state + h->lay.shadow_off) : nullptr;
+}
+inline float* wlo_of(const ls_handle* h) {
+  return h->lay.bf16 ? nullptr : reinterpret_cast<float*>(h->state + h->lay.shadow_off);
 }
 
 // ---- averaging (average.cu) ---------------------------------------------
 // n_buf buffers of m vectors each; buffer b starts at base + b*buf_stride floats,
-// vector j of it at + j*stride.  shadow (optional) receives the bf16 rounding of
-// the mean of buffer 0 with the same strides.  Returns a cudaError_t.
+// vector j of it at + j*stride.  shadow / lo (optional, same strides) receive the
+// bf16 rounding / the tf32 remainder of the mean of buffer 0.  Returns a cudaError_t.
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches);
+                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches);
 
 // ---- fp32-accumulate CUDA-core grouped GEMMs (gemm_simt.cu) ---------------
 struct FwdArgs {           // Z = A W^T + b, optional ReLU
@@ -111,6 +126,7 @@ struct FwdArgs {           // Z = A W^T + b, optional ReLU
   const float* bias;       // fp32 master bias of group 0 or null
   int64_t bias_gstride;
   void* C;                 // [groups][M][N]
+  float* Clo;              // lo twin of C (fp32 outputs) or null
   int M, N, K, groups;
   int relu;
 };
@@ -120,15 +136,17 @@ struct DxArgs {            // dZ_prev = (dZ W) * 1[act > 0]
   int64_t w_gstride;
   const void* act;         // [groups][M][N] post-ReLU activation of the previous layer
   void* C;                 // [groups][M][N]
+  float* Clo;
   int M, N, K, groups;
 };
-struct DwArgs {            // G = dZ^T A ; v = mu v + G ; W -= lr v ; optional bf16 copy
+struct DwArgs {            // G = dZ^T A ; v = mu v + G ; W -= lr v ; operand copy of W
   const void* dZ;          // [groups][B][M]
   const void* A;           // [groups][B][N] (or dataset rows through row_off)
   const int64_t* row_off;
   float* W;                // fp32 master [M][N] of group 0
   float* V;                // momentum, same layout (unused when mu == 0)
   __nv_bfloat16* Wb;       // bf16 copy or null
+  float* Wlo;              // lo twin or null
   int64_t w_gstride;
   int M, N, B, groups;
   float lr, mu;
@@ -143,6 +161,7 @@ struct LossArgs {
   const void* y;           // int32 labels or float targets of the bound rows
   const int64_t* row_off;  // device, per group first row in y
   void* dZ;                // [groups][B][C] or null (forward only)
+  float* dZlo;             // lo twin (fp32 dZ) or null
   float* loss_out;         // [groups] or null
   int B, C, groups;
   int loss_kind;
@@ -159,32 +178,44 @@ struct BiasArgs {          // gb = colsum(dZ); v = mu v + gb; b -= lr v
 };
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
 
-// ---- tcgen05 grouped GEMMs, bf16 operands (gemm_tc.cu) ----------------------
-int tc_make_map_2d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols);
-int tc_make_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups, int64_t gstride);
-bool tc_shape_ok(int M, int N, int K);   // output rows, output columns, contraction length
+// fp32 -> bf16 copy of n elements (refresh of the weight copies)
+int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);
+// dst = src - tf32(src) for n elements (refresh of the lo twins)
+int launch_split_lo(const float* src, float* dst, int64_t n, cudaStream_t st, int64_t* launches);
+// lo twin of the mini-batches: dst[g][b][:] = lo(X[row_off[g] + b][:]) for g < groups, b < B
+int launch_gather_lo(const float* X, const int64_t* row_off, float* dst, int groups, int B, int d, cudaStream_t st,
+                     int64_t* launches);
+
+// ---- tcgen05 grouped GEMMs (gemm_tc.cu) -------------------------------------
+int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols);
+int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
+                   int64_t groups, int64_t gstride);
+bool tc_shape_ok(bool fp32, int M, int N, int K);   // output rows, output columns, contraction length
+struct TcOperandMaps {
+  const CUtensorMap *a, *b, *a_lo, *b_lo;   // lo maps: fp32 only
+};
 struct TcFwdArgs {
-  const CUtensorMap* mapA;   // [rows][K] input (dataset rows through row_off, else group g at row g*M)
-  const CUtensorMap* mapW;   // 3-D weight copies
+  TcOperandMaps maps;        // a: [rows][K] input (dataset rows through row_off, else group g at row g*M); b: weights
+  bool fp32;
   const int64_t* row_off;
   int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
   const float* bias; int64_t bias_gstride;
-  void* C;                   // bf16 [groups][M][N]
+  void* C; float* Clo;       // [groups][M][N] bf16, or fp32 + lo twin
   int M, N, K, groups, relu;
   int* err_flag;
 };
 struct TcDxArgs {
-  const CUtensorMap* mapDz;  // dZ_l [groups*M][K]
-  const CUtensorMap* mapW;
-  const void* act; void* C;  // bf16 [groups][M][N]
+  TcOperandMaps maps;        // a: dZ_l [groups*M][K]; b: weights
+  bool fp32;
+  const void* act; void* C; float* Clo;
   int M, N, K, groups;
   int* err_flag;
 };
 struct TcDwArgs {
-  const CUtensorMap* mapDz;  // dZ_l [groups*B][M]
-  const CUtensorMap* mapA;   // layer input [rows][N]
+  TcOperandMaps maps;        // a: dZ_l [groups*B][M]; b: layer input [rows][N]
+  bool fp32;
   const int64_t* row_off;
-  float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride;
+  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride;
   int M, N, B, groups;
   float lr, mu;
   int* err_flag;
@@ -192,8 +223,5 @@ struct TcDwArgs {
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches);
-
-// fp32 -> bf16 copy of n elements (refresh of the weight copies)
-int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);
 
 }  // namespace ls

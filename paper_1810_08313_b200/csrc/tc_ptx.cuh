@@ -108,16 +108,18 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 
 // ---- MMA ---------------------------------------------------------------------------
-// Shared-memory matrix descriptor, 128-byte swizzle, for tiles whose rows are 128 bytes:
+// Shared-memory matrix descriptor for tiles whose rows are 128 bytes:
 //   bits  0-13 start address >> 4, 16-29 leading byte offset >> 4, 32-45 stride byte offset >> 4,
-//   46-47 version (1 on sm_100), 61-63 swizzle mode (2 = 128 B).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+//   46-47 version (1 on sm_100), 61-63 swizzle mode (2 = 128 B in 16-byte units, 1 = 128 B in 32-byte units).
+constexpr uint32_t kSwizzle128B = 2, kSwizzle128B_32B = 1;
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint32_t swizzle = kSwizzle128B) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
   d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
+  d |= (uint64_t)swizzle << 61;
   return d;
 }
 // Instruction descriptor for kind::f16 / kind::tf32 with fp32 accumulation:
