@@ -239,7 +239,25 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
     }
-    if (tc_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
+    if (tc_update_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
+      TcUpdateArgs t;
+      t.fp32 = !bf;
+      t.maps.a = &mn.dz[l];
+      t.maps.a_lo = &mn.dz_lo[l];
+      t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
+      t.maps.b_lo = (l == 0) ? &mn.x_lo : &mn.act_lo[l];
+      t.mapW = &h->maps.wf[l];
+      t.mapV = &h->maps.vf[l];
+      t.row_off = (l == 0) ? row_off_dev : nullptr;
+      t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
+      t.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
+      t.w_gstride = lay.stride;
+      t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
+      t.lr = h->lr; t.mu = h->mu;
+      t.err_flag = err_flag_of(h);
+      ProfScope ps(h, LS_K_DW, l);
+      LS_CUDA(h, launch_tc_update(t, h->stream, &h->launches));
+    } else if (tc_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
       TcDwArgs t;
       t.fp32 = !bf;
       t.maps.a = &mn.dz[l];
@@ -449,6 +467,13 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
           ok(tc_make_map_2d(&mp.dz[l], h->state + lay.dz_off[buf], f, mn, rows, lay.dims[l + 1]));
           if (f) ok(tc_make_map_2d(&mp.dz_lo[l], h->state + lay.dzlo_off[buf], true, mn, rows, lay.dims[l + 1]));
         }
+      }
+      if (!mn) {
+        for (int l = 0; l < lay.L; ++l)
+          if (lay.dims[l] % 4 == 0) {
+            ok(tc_make_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], true, false, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+            ok(tc_make_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], true, false, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+          }
       }
       if (lay.dims[0] % q == 0) {
         for (int s = 0; s < 2; ++s)

@@ -69,6 +69,7 @@ struct alignas(64) TcMaps {
   CUtensorMap x_data;                                     // bound dataset, 2-D [n_rows][dims[0]]
   CUtensorMap x_stage[2];                                 // staging buffers of host batches
   CUtensorMap x_lo;                                       // lo twin of the current mini-batches
+  CUtensorMap wf[LS_MAX_LAYERS], vf[LS_MAX_LAYERS];       // fp32 master weights / momentum, 32 x 32 blocks
 };
 
 struct ls_handle {
@@ -220,6 +221,20 @@ struct TcDwArgs {
   float lr, mu;
   int* err_flag;
 };
+// persistent streaming update kernel (update_tc.cu)
+struct TcUpdateArgs {
+  TcOperandMaps maps;        // a: dZ_l [groups*B][M]; b: layer input [rows][N]   (MN-major reads)
+  const CUtensorMap* mapW;   // fp32 master weights [replica][M][N], 32 x 32 blocks
+  const CUtensorMap* mapV;   // momentum, same shape
+  bool fp32;
+  const int64_t* row_off;
+  __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride;
+  int M, N, B, groups;
+  float lr, mu;
+  int* err_flag;
+};
+bool tc_update_shape_ok(bool fp32, int M, int N, int B);
+int launch_tc_update(const TcUpdateArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches);

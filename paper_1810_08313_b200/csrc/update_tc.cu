@@ -1,0 +1,341 @@
+// Weight gradient + SGD-momentum update as one persistent, warp-specialised
+// streaming kernel (Section 2 mini-batch SGD update; Section 5.3 momentum):
+//
+//     G = dZ^T A  (per replica, 128 x 128 tiles on tcgen05, accumulator in TMEM)
+//     v <- mu v + G ;  W <- W - eta v ;  refresh the operand copy of W
+//
+// The gradient never leaves the SM.  The kernel is bound by the read-modify-write
+// of W and v (16 bytes per parameter with momentum, plus the operand copy), so it
+// is built as a stream: one CTA per SM walks over output tiles, and
+//
+//   warp 0      TMA producer of the dZ / A operand tiles (ring of stages)
+//   warp 1      tcgen05.mma issuer; two TMEM accumulators, so the products of tile t+1
+//               overlap the update of tile t
+//   warps 4-7   update warps.  Each owns 32 rows of the tile and a private ring of
+//               shared-memory slots: TMA loads bring its 32 x 32 blocks of W and v in
+//               (issued up to a whole tile ahead), the warp adds the TMEM gradient in
+//               place, and TMA stores write the blocks back.  Loads and stores are
+//               asynchronous bulk copies, so tens of KB per SM are always in flight.
+//
+// Every mbarrier wait is bounded (see tc_ptx.cuh); a wait that runs out sets
+// *err_flag and the CTA drains its copies, frees its tensor memory and returns.
+#include "ls_internal.h"
+#include "tc_ptx.cuh"
+
+namespace ls {
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128, BN = 128;
+constexpr int KB_BYTES = 128;
+constexpr int kThreads = 256;
+constexpr int kSlotBytes = 8192;       // one 32 x 32 fp32 block of W (4 KB) and of v (4 KB)
+
+struct UParams {
+  int M, N, K, groups;                 // per replica: out features, in features, batch
+  const int64_t* b_row_off;            // layer input = dataset rows: first row of replica g, else null
+  int rows_per_group;                  // = batch
+  float lr, mu;
+  __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
+  float* Wlo;                          // lo twin of W (fp32 models) or null
+  int64_t w_gstride;                   // elements between replicas
+  int* err_flag;
+};
+
+template <bool TF32, int STAGES, int R>
+struct USmem {
+  static constexpr int kTiles = TF32 ? 2 : 1;
+  static constexpr int kStageBytes = kTiles * (BM + BN) * KB_BYTES;
+  static constexpr int kRingBytes = 4 * R * kSlotBytes;
+  static constexpr int kBars = 2 * STAGES + 4 + 4 * R;
+  static constexpr int kTotal = 1024 + STAGES * kStageBytes + kRingBytes + kBars * 8 + 16;
+  static_assert(kTotal <= 227 * 1024, "shared memory budget");
+};
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(m)),
+               "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
+template <int ELEMS>
+__device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, int tile0, int extent,
+                                              int row0) {
+  // MN-major operand: boxes of 128 bytes (ELEMS MN-elements) x ELEMS K-rows, one per chunk of MN
+  for (int c = 0; c < extent / ELEMS; ++c)
+    tma_load_2d(static_cast<char*>(dst) + c * ELEMS * KB_BYTES, tm, bar, tile0 + c * ELEMS, row0);
+}
+
+template <bool TF32, int STAGES, int R>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo,
+                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmV, const UParams p) {
+  using L = USmem<TF32, STAGES, R>;
+  constexpr int EB = TF32 ? 4 : 2;
+  constexpr int ELEMS = KB_BYTES / EB;          // K elements per stage
+  constexpr int MMA_K = 32 / EB;
+  constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
+  constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN);
+  constexpr uint32_t SW = TF32 ? kSwizzle128B_32B : kSwizzle128B;
+  constexpr uint32_t SBO = TF32 ? 512 : 1024;
+  constexpr int kABytes = BM * KB_BYTES, kBBytes = BN * KB_BYTES;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem;
+  uint8_t* ring_base = smem + STAGES * L::kStageBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(ring_base + L::kRingBytes);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;       // [2]
+  uint64_t* tmem_empty = tmem_full + 2;       // [2]
+  uint64_t* wv_full = tmem_empty + 2;         // [4][R]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wv_full + 4 * R);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tiles = p.M / BM, n_tiles = p.N / BN;
+  const int tiles_per_group = m_tiles * n_tiles;
+  const int total_tiles = tiles_per_group * p.groups;
+  const int num_kb = p.K / ELEMS;
+  const bool has_v = p.mu != 0.f;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
+    for (int i = 0; i < 4 * R; ++i) mbar_init(&wv_full[i], 1);
+    fence_mbar_init();
+    prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmW); prefetch_tmap(&tmV);
+    if (TF32) { prefetch_tmap(&tmAlo); prefetch_tmap(&tmBlo); }
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 2 * BN);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---- operand producer ---------------------------------------------------------
+    if (elect_one()) {
+      int it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int g = t / tiles_per_group, rem = t % tiles_per_group;
+        const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+        const int a_row = g * p.rows_per_group;
+        const int b_row = p.b_row_off ? (int)p.b_row_off[g] : a_row;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1)) { atomicExch(p.err_flag, 11); ok = false; break; }
+          mbar_expect_tx(&full[s], L::kStageBytes);
+          uint8_t* sa = stage_base + s * L::kStageBytes;
+          uint8_t* sb = sa + kABytes;
+          issue_mn_tile<ELEMS>(sa, &tmA, &full[s], m0, BM, a_row + kb * ELEMS);
+          issue_mn_tile<ELEMS>(sb, &tmB, &full[s], n0, BN, b_row + kb * ELEMS);
+          if (TF32) {
+            issue_mn_tile<ELEMS>(sb + kBBytes, &tmAlo, &full[s], m0, BM, a_row + kb * ELEMS);
+            issue_mn_tile<ELEMS>(sb + kBBytes + kABytes, &tmBlo, &full[s], n0, BN, a_row + kb * ELEMS);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer -----------------------------------------------------------------
+    if (elect_one()) {
+      int it = 0, n = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++n) {
+        const int buf = n & 1;
+        if (!mbar_wait(&tmem_empty[buf], ((n >> 1) & 1) ^ 1)) { atomicExch(p.err_flag, 12); break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&full[s], (it / STAGES) & 1)) { atomicExch(p.err_flag, 13); ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < ELEMS / MMA_K; ++k) {
+            const uint32_t adv = k * MMA_K * KB_BYTES;      // next MMA_K K-rows
+            const uint64_t da = make_smem_desc(a_addr + adv, CHUNK_BYTES, SBO, SW);
+            const uint64_t db = make_smem_desc(b_addr + adv, CHUNK_BYTES, SBO, SW);
+            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+            if (TF32) {
+              const uint64_t dal = make_smem_desc(b_addr + kBBytes + adv, CHUNK_BYTES, SBO, SW);
+              const uint64_t dbl = make_smem_desc(b_addr + kBBytes + kABytes + adv, CHUNK_BYTES, SBO, SW);
+              mma_tf32(d_tmem, dal, db, IDESC, acc);
+              mma_tf32(d_tmem, da, dbl, IDESC, 1u);
+              mma_tf32(d_tmem, da, db, IDESC, 1u);
+            } else {
+              mma_bf16(d_tmem, da, db, IDESC, acc);
+            }
+          }
+          mma_commit(&empty[s]);
+        }
+        if (ok) mma_commit(&tmem_full[buf]);
+      }
+    }
+  } else if (warp >= 4) {
+    // ---- update warps -----------------------------------------------------------------
+    const int q = warp & 3;
+    uint8_t* my_ring = ring_base + q * R * kSlotBytes;
+    uint64_t* my_full = wv_full + q * R;
+    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int my_chunks = my_tiles * (BN / 32);
+
+    // chunk j of this CTA: tile ordinal j / 4, column block j % 4; rows q*32.. of the tile
+    auto load_chunk = [&](int j) {
+      if (j >= my_chunks) return;
+      const int t = blockIdx.x + (j >> 2) * gridDim.x;
+      const int g = t / tiles_per_group, rem = t % tiles_per_group;
+      const int y = (rem / n_tiles) * BM + q * 32, x = (rem % n_tiles) * BN + (j & 3) * 32;
+      uint8_t* slot = my_ring + (j % R) * kSlotBytes;
+      mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
+      tma_load_3d(slot, &tmW, &my_full[j % R], x, y, g);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &tmV, &my_full[j % R], x, y, g);
+    };
+    if (lane == 0)
+      for (int j = 0; j < R; ++j) load_chunk(j);
+
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    bool ok = true;
+    int j = 0;
+    for (int n = 0; n < my_tiles && ok; ++n) {
+      const int t = blockIdx.x + n * gridDim.x;
+      const int g = t / tiles_per_group, rem = t % tiles_per_group;
+      const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+      const int buf = n & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (n >> 1) & 1));
+      if (!ok) { if (lane == 0) atomicExch(p.err_flag, 14); break; }
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c, ++j) {
+        uint8_t* slot = my_ring + (j % R) * kSlotBytes;
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + buf * BN + c * 32, r);
+        ok = __all_sync(0xffffffffu, mbar_wait(&my_full[j % R], (j / R) & 1));
+        tmem_ld_wait();
+        if (c == BN / 32 - 1) {
+          // the accumulator has been read: hand the TMEM buffer back to the MMA warp
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+        }
+        if (!ok) { if (lane == 0) atomicExch(p.err_flag, 15); break; }
+        // this thread's row of the 32 x 32 block; 16-byte pieces are XOR-swizzled by the row (128-byte swizzle)
+        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * p.N + n0 + c * 32;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+          float4 w = *reinterpret_cast<float4*>(slot + off);
+          float ws[4] = {w.x, w.y, w.z, w.w};
+          float vs[4] = {0.f, 0.f, 0.f, 0.f};
+          if (has_v) {
+            const float4 v = *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off);
+            vs[0] = v.x; vs[1] = v.y; vs[2] = v.z; vs[3] = v.w;
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float gr = __uint_as_float(r[jj * 4 + e]);
+            const float step = has_v ? fmaf(p.mu, vs[e], gr) : gr;
+            vs[e] = step;
+            ws[e] = fmaf(-p.lr, step, ws[e]);
+          }
+          *reinterpret_cast<float4*>(slot + off) = make_float4(ws[0], ws[1], ws[2], ws[3]);
+          if (has_v) *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) = make_float4(vs[0], vs[1], vs[2], vs[3]);
+          if (TF32) {
+            *reinterpret_cast<float4*>(p.Wlo + at + jj * 4) =
+                make_float4(tf32_lo(ws[0]), tf32_lo(ws[1]), tf32_lo(ws[2]), tf32_lo(ws[3]));
+          } else if (p.Wb != nullptr) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
+            uint2 u;
+            u.x = *reinterpret_cast<uint32_t*>(&lo);
+            u.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(p.Wb + at + jj * 4) = u;
+          }
+        }
+        // make the in-place update visible to the bulk-copy engine, then write the blocks back
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int y = m0 + q * 32, x = n0 + c * 32;
+          tma_store_3d(&tmW, slot, x, y, g);
+          if (has_v) tma_store_3d(&tmV, slot + kSlotBytes / 2, x, y, g);
+          bulk_commit();
+          // the slot used one chunk ago is free once its store has read shared memory: refill it
+          bulk_wait_read<1>();
+          if (j >= 1) load_chunk(j - 1 + R);
+        }
+        __syncwarp();
+      }
+    }
+    if (lane == 0) bulk_wait_all();
+    tc_fence_before_sync();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+int num_sms() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
+template <bool TF32, int STAGES, int R>
+int launch_update(const TcUpdateArgs& a, cudaStream_t st) {
+  using L = USmem<TF32, STAGES, R>;
+  auto kern = tc_update_kernel<TF32, STAGES, R>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  UParams p{};
+  p.M = a.M; p.N = a.N; p.K = a.B; p.groups = a.groups;
+  p.b_row_off = a.row_off; p.rows_per_group = a.B;
+  p.lr = a.lr; p.mu = a.mu; p.Wb = a.Wb; p.Wlo = a.Wlo; p.w_gstride = a.w_gstride; p.err_flag = a.err_flag;
+  const int total = (a.M / BM) * (a.N / BN) * a.groups;
+  const int grid = total < num_sms() ? total : num_sms();
+  const CUtensorMap* alo = TF32 ? a.maps.a_lo : a.maps.a;
+  const CUtensorMap* blo = TF32 ? a.maps.b_lo : a.maps.b;
+  kern<<<grid, kThreads, L::kTotal, st>>>(*a.maps.a, *a.maps.b, *alo, *blo, *a.mapW, *a.mapV, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
+  return M > 0 && N > 0 && B > 0 && M % BM == 0 && N % BN == 0 && B % (fp32 ? 32 : 64) == 0;
+}
+
+int launch_tc_update(const TcUpdateArgs& a, cudaStream_t st, int64_t* launches) {
+  if (launches) ++*launches;
+  if (a.fp32) return launch_update<true, 2, 3>(a, st);
+  return launch_update<false, 3, 4>(a, st);
+}
+
+}  // namespace ls
