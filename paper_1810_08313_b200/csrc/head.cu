@@ -1,0 +1,304 @@
+// The output layer when it is narrow (at most 16 outputs: the 10-class loss layer, or the
+// single output of least squares).  Such a layer cannot fill a tensor-core tile, and as five
+// generic launches (product, loss, two gradients, bias) it is all overhead, so it is two kernels:
+//
+//   head_fwd_kernel   z = A W^T + b, per-sample loss f(x; s_i), the mini-batch mean of it (the
+//                     empirical risk of Section 2 restricted to the batch) and dZ = d(mean loss)/dz.
+//                     Rows are spread over CTAs; the last CTA of a replica to finish adds the row
+//                     losses in row order, so the mean does not depend on scheduling.
+//   head_bwd_kernel   one pass over the layer input A for both gradients:
+//                       dZ_prev = (dZ W) * 1[A > 0]          (skipped for a one-layer model)
+//                       G = dZ^T A ; v <- mu v + G ; W <- W - eta v ; same for the bias
+//                     (Section 2 mini-batch SGD update, Section 5.3 momentum).
+//
+// All sums run in a fixed order; W is read from the fp32 master copy.
+#include "ls_internal.h"
+
+namespace ls {
+namespace {
+
+constexpr int CMAX = 16;
+constexpr int kThreads = 256;
+constexpr int kRowsPerCta = 4;         // head_fwd: rows per CTA (the 8 warps split K)
+constexpr int kColsPerCta = 32;        // head_bwd: 32 columns x 8 row slices
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ void put(float* p, float v) { *p = v; }
+__device__ __forceinline__ void put(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ void load4(const float* p, float (&r)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&r)[4]) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x);
+  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+  r[0] = __low2float(a); r[1] = __high2float(a); r[2] = __low2float(b); r[3] = __high2float(b);
+}
+
+// One CTA = kRowsPerCta (4) mini-batch rows of one replica.  The 8 warps split K; partial dot products are
+// combined lane-wise by a butterfly and warp-wise through shared memory in warp order.
+template <typename TA>
+__global__ void __launch_bounds__(kThreads)
+head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ W,
+                int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
+                const int64_t* __restrict__ y_row_off, float* __restrict__ dZ, float* __restrict__ row_loss,
+                float* __restrict__ loss_out, unsigned int* __restrict__ counters, int B, int C, int K, int kind,
+                int vec_ok) {
+  __shared__ float part[8][kRowsPerCta * CMAX];
+  __shared__ float zs[kRowsPerCta][CMAX];
+  __shared__ unsigned int is_last;
+  __shared__ float red[kThreads];
+  const int g = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
+  const float* Wg = W + (int64_t)g * w_gstride;
+  const int b0 = blockIdx.x * kRowsPerCta;
+  const int kchunk = (((K + 7) / 8) + 3) / 4 * 4;
+  const int kw0 = warp * kchunk, kw1 = min(K, kw0 + kchunk);
+
+  float acc[kRowsPerCta][CMAX];
+#pragma unroll
+  for (int r = 0; r < kRowsPerCta; ++r)
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c) acc[r][c] = 0.f;
+  if (vec_ok) {
+    for (int k = kw0 + lane * 4; k < kw1; k += 128) {
+      float a[kRowsPerCta][4];
+#pragma unroll
+      for (int r = 0; r < kRowsPerCta; ++r) {
+        if (b0 + r < B) load4(Ag + (int64_t)(b0 + r) * K + k, a[r]);
+        else a[r][0] = a[r][1] = a[r][2] = a[r][3] = 0.f;
+      }
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c)
+        if (c < C) {
+          float w[4];
+          load4(Wg + (int64_t)c * K + k, w);
+#pragma unroll
+          for (int r = 0; r < kRowsPerCta; ++r)
+            acc[r][c] = fmaf(a[r][3], w[3], fmaf(a[r][2], w[2], fmaf(a[r][1], w[1], fmaf(a[r][0], w[0], acc[r][c]))));
+        }
+    }
+  } else {
+    for (int k = kw0 + lane; k < kw1; k += 32) {
+      float a[kRowsPerCta];
+#pragma unroll
+      for (int r = 0; r < kRowsPerCta; ++r) a[r] = (b0 + r < B) ? to_f(Ag[(int64_t)(b0 + r) * K + k]) : 0.f;
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c)
+        if (c < C) {
+          const float w = Wg[(int64_t)c * K + k];
+#pragma unroll
+          for (int r = 0; r < kRowsPerCta; ++r) acc[r][c] = fmaf(a[r], w, acc[r][c]);
+        }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kRowsPerCta; ++r)
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c)
+      if (c < C) {
+        float v = acc[r][c];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) part[warp][r * CMAX + c] = v;
+      }
+  __syncthreads();
+  if (threadIdx.x < kRowsPerCta * CMAX) {
+    const int r = threadIdx.x / CMAX, c = threadIdx.x % CMAX;
+    float s = 0.f;
+    if (c < C) {
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
+      if (bias) s += bias[(int64_t)g * w_gstride + c];
+    }
+    zs[r][c] = s;
+  }
+  __syncthreads();
+  const float invB = 1.0f / (float)B;
+  if (warp < kRowsPerCta && b0 + warp < B) {
+    // warp r finishes row r: lane c holds class c
+    const int b = b0 + warp;
+    const int64_t y0 = y_row_off[g];
+    const float z = (lane < C) ? zs[warp][lane] : -INFINITY;
+    float loss, d;
+    if (kind == LS_LOSS_SOFTMAX_CE) {
+      const int label = static_cast<const int32_t*>(y)[y0 + b];
+      float mx = z;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float e = (lane < C) ? expf(z - mx) : 0.f;
+      float sum = e;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float zy = __shfl_sync(0xffffffffu, z, (label >= 0 && label < C) ? label : 0);
+      loss = (mx + logf(sum)) - ((label >= 0 && label < C) ? zy : mx);
+      d = (e / sum - (lane == label ? 1.f : 0.f)) * invB;
+    } else {
+      const float res = zs[warp][0] - static_cast<const float*>(y)[y0 + b];
+      loss = 0.5f * res * res;
+      d = res * invB;
+    }
+    if (lane == 0) row_loss[(int64_t)g * B + b] = loss;
+    if (dZ != nullptr && lane < C) dZ[((int64_t)g * B + b) * C + lane] = d;
+  }
+  // the last CTA of this replica adds the row losses in row order
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicInc(&counters[g], gridDim.x - 1) == gridDim.x - 1) ? 1u : 0u;
+  __syncthreads();
+  if (is_last && loss_out != nullptr) {
+    __threadfence();
+    float p = 0.f;
+    for (int b = threadIdx.x; b < B; b += kThreads) p += __ldcg(&row_loss[(int64_t)g * B + b]);
+    red[threadIdx.x] = p;
+    __syncthreads();
+    for (int s = kThreads / 2; s > 0; s >>= 1) {
+      if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) loss_out[g] = red[0] * invB;
+  }
+}
+
+template <typename TA>
+__global__ void __launch_bounds__(kThreads)
+head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
+                float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb, float* __restrict__ Wlo,
+                float* __restrict__ bias, float* __restrict__ vbias, int64_t w_gstride, TA* __restrict__ dPrev,
+                float* __restrict__ dPrevLo, int B, int C, int K, float lr, float mu) {
+  extern __shared__ float sm[];
+  float* dz = sm;                                   // [B][C]
+  float* part = sm + (size_t)B * C;                 // [8][CMAX][kColsPerCta]
+  const int g = blockIdx.y;
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int k = blockIdx.x * kColsPerCta + cx;
+  const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
+  for (int i = threadIdx.x; i < B * C; i += kThreads) dz[i] = dZ[(int64_t)g * B * C + i];
+  __syncthreads();
+
+  float wreg[CMAX], gw[CMAX];
+#pragma unroll
+  for (int c = 0; c < CMAX; ++c) {
+    wreg[c] = (c < C && k < K) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k] : 0.f;
+    gw[c] = 0.f;
+  }
+  if (k < K) {
+    for (int bb = ry; bb < B; bb += 64) {
+      // eight rows per trip so that eight loads of A are in flight
+      float av[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) av[u] = (bb + 8 * u < B) ? to_f(Ag[(int64_t)(bb + 8 * u) * K + k]) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int b = bb + 8 * u;
+        if (b >= B) break;
+        const float a = av[u];
+        float da = 0.f;
+#pragma unroll
+        for (int c = 0; c < CMAX; ++c)
+          if (c < C) {
+            const float d = dz[b * C + c];
+            gw[c] = fmaf(d, a, gw[c]);
+            da = fmaf(d, wreg[c], da);
+          }
+        if (dPrev != nullptr) {
+          const float o = a > 0.f ? da : 0.f;
+          const int64_t at = ((int64_t)g * B + b) * K + k;
+          put(dPrev + at, o);
+          if (dPrevLo != nullptr) dPrevLo[at] = tf32_lo(o);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < CMAX; ++c) part[(ry * CMAX + c) * kColsPerCta + cx] = gw[c];
+  __syncthreads();
+  if (ry == 0 && k < K) {
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c)
+      if (c < C) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) s += part[(r * CMAX + c) * kColsPerCta + cx];
+        const int64_t at = (int64_t)g * w_gstride + (int64_t)c * K + k;
+        float step = s;
+        if (mu != 0.f) {
+          step = fmaf(mu, V[at], s);
+          V[at] = step;
+        }
+        const float w = fmaf(-lr, step, wreg[c]);
+        W[at] = w;
+        if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
+        if (Wlo != nullptr) Wlo[at] = tf32_lo(w);
+      }
+  }
+  if (blockIdx.x == 0 && bias != nullptr && threadIdx.x < C) {
+    const int c = threadIdx.x;
+    float s = 0.f;
+    for (int b = 0; b < B; ++b) s += dz[b * C + c];
+    const int64_t at = (int64_t)g * w_gstride + c;
+    float step = s;
+    if (mu != 0.f) {
+      step = fmaf(mu, vbias[at], s);
+      vbias[at] = step;
+    }
+    bias[at] = fmaf(-lr, step, bias[at]);
+  }
+}
+
+}  // namespace
+
+bool head_shape_ok(int B, int C) { return C >= 1 && C <= CMAX && B >= 1 && (size_t)B * C * 4 <= 64 * 1024; }
+
+int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
+  if (launches) ++*launches;
+  dim3 grid((unsigned)((a.B + kRowsPerCta - 1) / kRowsPerCta), (unsigned)a.groups);
+  const int vec_ok = (a.K % 4 == 0) && (reinterpret_cast<uintptr_t>(a.A) % 16 == 0) &&
+                     (reinterpret_cast<uintptr_t>(a.W) % 16 == 0) && (a.w_gstride % 4 == 0);
+  if (a_bf16)
+    head_fwd_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W,
+                                                             a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss,
+                                                             a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
+  else
+    head_fwd_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.W, a.w_gstride,
+                                                      a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out,
+                                                      a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
+  return cudaGetLastError();
+}
+
+int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
+  if (launches) ++*launches;
+  dim3 grid((unsigned)((a.K + kColsPerCta - 1) / kColsPerCta), (unsigned)a.groups);
+  const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * kColsPerCta) * sizeof(float);
+  if (a_bf16) {
+    auto kern = head_bwd_kernel<__nv_bfloat16>;
+    static bool configured = false;
+    if (!configured) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+      if (e != cudaSuccess) return e;
+      configured = true;
+    }
+    kern<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo,
+                                       a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev), nullptr, a.B,
+                                       a.C, a.K, a.lr, a.mu);
+  } else {
+    auto kern = head_bwd_kernel<float>;
+    static bool configured = false;
+    if (!configured) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+      if (e != cudaSuccess) return e;
+      configured = true;
+    }
+    kern<<<grid, kThreads, smem, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo, a.bias,
+                                       a.vbias, a.w_gstride, static_cast<float*>(a.dPrev), a.dPrevLo, a.B, a.C, a.K,
+                                       a.lr, a.mu);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace ls

@@ -72,15 +72,26 @@ template <typename TD>
 __global__ void __launch_bounds__(kThreads)
 bias_kernel(const TD* __restrict__ dZ, float* __restrict__ bias, float* __restrict__ vbias, int64_t gstride, int B,
             int N, float lr, float mu) {
+  // 32 columns x 8 row slices per block: each thread adds every 8th row, then the 8 partial sums of a
+  // column are added in slice order
+  __shared__ float part[8][32];
   const int g = blockIdx.y;
-  const int j = blockIdx.x * kThreads + threadIdx.x;
-  if (j >= N) return;
-  const TD* d = dZ + (int64_t)g * B * N + j;
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int j = blockIdx.x * 32 + cx;
   float s = 0.f;
-  for (int b = 0; b < B; ++b) {
-    if constexpr (sizeof(TD) == 2) s += __bfloat162float(d[(int64_t)b * N]);
-    else s += d[(int64_t)b * N];
+  if (j < N) {
+    const TD* d = dZ + (int64_t)g * B * N + j;
+    for (int b = ry; b < B; b += 8) {
+      if constexpr (sizeof(TD) == 2) s += __bfloat162float(d[(int64_t)b * N]);
+      else s += d[(int64_t)b * N];
+    }
   }
+  part[ry][cx] = s;
+  __syncthreads();
+  if (ry != 0 || j >= N) return;
+  s = 0.f;
+#pragma unroll
+  for (int r = 0; r < 8; ++r) s += part[r][cx];
   const int64_t at = (int64_t)g * gstride + j;
   float step = s;
   if (mu != 0.f) {
@@ -149,7 +160,7 @@ int launch_loss(const LossArgs& a, bool dz_bf16, cudaStream_t st, int64_t* launc
 
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
-  dim3 grid((unsigned)((a.N + kThreads - 1) / kThreads), (unsigned)a.groups);
+  dim3 grid((unsigned)((a.N + 31) / 32), (unsigned)a.groups);
   if (bf16)
     bias_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(a.dZ), a.bias, a.vbias,
                                                           a.gstride, a.B, a.N, a.lr, a.mu);

@@ -75,6 +75,9 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   }
   if (!lay.bf16) lay.xlo_off = take((size_t)m * batch * lay.dims[0] * 4);
   lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
+  lay.dzl_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
+  lay.rowloss_off = take((size_t)m * batch * 4);
+  lay.headcnt_off = take((size_t)LS_MAX_REPLICAS * 4);
   lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
   lay.evaloff_off = take((size_t)kEvalCap * 8);
   lay.evalloss_off = take((size_t)kEvalCap * 4);
@@ -155,6 +158,23 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
     LS_CUDA(h, launch_gather_lo(static_cast<const float*>(x), row_off_dev, lo_at(h, lay.xlo_off), groups, lay.batch,
                                 lay.dims[0], h->stream, &h->launches));
   for (int l = 0; l < lay.L; ++l) {
+    if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
+      // narrow output layer: product, loss and dZ in one kernel
+      HeadFwdArgs a;
+      a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
+      a.a_row_off = (l == 0) ? row_off_dev : nullptr;
+      a.W = P + lay.w_off[l]; a.w_gstride = w_gstride;
+      a.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
+      a.y = y; a.y_row_off = row_off_dev;
+      a.dZ = want_dz ? reinterpret_cast<float*>(h->state + lay.dzl_off) : nullptr;
+      a.row_loss = reinterpret_cast<float*>(h->state + lay.rowloss_off);
+      a.loss_out = loss_out;
+      a.counters = reinterpret_cast<unsigned int*>(h->state + lay.headcnt_off);
+      a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = groups; a.loss_kind = h->spec.loss;
+      ProfScope ps(h, LS_K_FWD, l);
+      LS_CUDA(h, launch_head_fwd(a, bf, h->stream, &h->launches));
+      return LS_OK;
+    }
     if (l < lay.L - 1 && tc_shape_ok(!bf, lay.batch, lay.dims[l + 1], lay.dims[l])) {
       TcFwdArgs t;
       t.fp32 = !bf;
@@ -212,6 +232,27 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   int cur = 0;
   for (int l = lay.L - 1; l >= 0; --l) {
     void* dZ = h->state + lay.dz_off[cur];
+    if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
+      // narrow output layer: both gradients, the update and the bias in one pass over its input
+      HeadBwdArgs a;
+      a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
+      a.a_row_off = (l == 0) ? row_off_dev : nullptr;
+      a.dZ = reinterpret_cast<const float*>(h->state + lay.dzl_off);
+      a.W = params_of(h) + lay.w_off[l]; a.V = mom_of(h) + lay.w_off[l];
+      a.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
+      a.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
+      a.bias = lay.has_bias ? params_of(h) + lay.b_off[l] : nullptr;
+      a.vbias = mom_of(h) + lay.b_off[l];
+      a.w_gstride = lay.stride;
+      a.dPrev = (l > 0) ? (void*)(h->state + lay.dz_off[cur ^ 1]) : nullptr;
+      a.dPrevLo = (l > 0) ? lo_at(h, lay.dzlo_off[cur ^ 1]) : nullptr;
+      a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = lay.m;
+      a.lr = h->lr; a.mu = h->mu;
+      ProfScope ps(h, LS_K_DW, l);
+      LS_CUDA(h, launch_head_bwd(a, bf, h->stream, &h->launches));
+      cur ^= 1;
+      continue;
+    }
     if (l > 0 && tc_shape_ok(!bf, lay.batch, lay.dims[l], lay.dims[l + 1])) {
       // the data gradient reads W_l before the update below overwrites it
       TcDxArgs t;

@@ -46,6 +46,9 @@ struct Layout {
   size_t dzlo_off[2] = {0, 0};
   size_t xlo_off = 0;                        // lo twin of the current mini-batches [m][batch][dims[0]] (fp32 models)
   size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
+  size_t dzl_off = 0;                        // fp32 dZ of a narrow output layer [m][batch][dims[L]]
+  size_t rowloss_off = 0;                    // per-sample losses [m][batch]
+  size_t headcnt_off = 0;                    // per-replica CTA counters of the output-layer kernel
   size_t rowoff_off = 0;                     // int64 [kRowOffCap][m]
   size_t evaloff_off = 0;                    // int64 [kEvalCap]
   size_t evalloss_off = 0;                   // float [kEvalCap]
@@ -178,6 +181,27 @@ struct BiasArgs {          // gb = colsum(dZ); v = mu v + gb; b -= lr v
   float lr, mu;
 };
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
+
+// ---- narrow output layer (head.cu) ---------------------------------------------
+struct HeadFwdArgs {
+  const void* A; const int64_t* a_row_off;   // layer input [groups][B][K] (or dataset rows)
+  const float* W; int64_t w_gstride; const float* bias;
+  const void* y; const int64_t* y_row_off;
+  float* dZ;                                 // [groups][B][C] or null (forward only)
+  float* row_loss; float* loss_out; unsigned int* counters;
+  int B, C, K, groups, loss_kind;
+};
+struct HeadBwdArgs {
+  const void* A; const int64_t* a_row_off;
+  const float* dZ;
+  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; float* bias; float* vbias; int64_t w_gstride;
+  void* dPrev; float* dPrevLo;               // dZ of the layer below [groups][B][K] (+ lo twin) or null
+  int B, C, K, groups;
+  float lr, mu;
+};
+bool head_shape_ok(int B, int C);
+int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches);
+int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches);
 
 // fp32 -> bf16 copy of n elements (refresh of the weight copies)
 int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);
