@@ -56,7 +56,8 @@ enum {
   LS_ERR_CUDA = -6,              /* a CUDA runtime call failed; ls_last_cuda_error() has its code */
   LS_ERR_UNSUPPORTED = -7,       /* valid request that this build does not implement (e.g. weight decay) */
   LS_ERR_OVERFLOW = -8,          /* a result does not fit its type */
-  LS_ERR_DEVICE_TIMEOUT = -9     /* a bounded wait inside a kernel ran out; results of that launch are invalid */
+  LS_ERR_DEVICE_TIMEOUT = -9,    /* a bounded wait inside a kernel ran out; results of that launch are invalid */
+  LS_ERR_TOO_LARGE = -10         /* a size exceeds a fixed capacity of the entry point */
 };
 
 enum { LS_LOSS_SOFTMAX_CE = 0, LS_LOSS_MSE_HALF = 1 };
@@ -197,6 +198,36 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
            int32_t* period_tau, int64_t max_periods, int64_t* n_periods,
            int64_t* decision_k, float* decision_F, int32_t* decision_tau, int64_t max_decisions,
            int64_t* n_decisions, float* F0_host);
+
+/* Mean loss of a linear model on device-resident rows, for callers that must not allocate.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Some callers cannot obtain device memory when they need a loss value: code that runs inside a
+ * memory pool owned by somebody else, a monitoring hook that fires when the device is nearly
+ * full, a plugin that is forbidden to call cudaMalloc, code that must not disturb an allocator's
+ * fragmentation state.  ls_eval_loss() needs the caller to have allocated a whole state block,
+ * because the output-layer kernel keeps per-row losses, CTA counters and chunk offsets in
+ * scratch memory.  Here that scratch is a fixed array inside the library image (about 260 KB of
+ * every GPU that loads the library, held until the process exits), and the call allocates
+ * nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ * Computes, for chunk c = 0 .. n_rows/chunk_rows - 1 of chunk_rows consecutive rows, the mean
+ * loss of z = W x + b on those rows and writes it to chunk_loss_dev[c] (the caller's own device
+ * buffer).  W_dev is float [d_out][d_in], bias_dev float [d_out] or NULL, x_dev float
+ * [n_rows][d_in] (16-byte aligned for the fast path), y_dev int32 labels (LS_LOSS_SOFTMAX_CE) or
+ * float targets (LS_LOSS_MSE_HALF, d_out == 1).  Same kernel and arithmetic as ls_eval_loss() on a
+ * one-layer fp32 model with mini-batch chunk_rows.  Enqueued on cuda_stream; returns at once.
+ *
+ * Limits: d_out <= 16, at most 256 chunks and 65 536 rows per call, chunk_rows <= LS_MAX_BATCH;
+ * beyond them the call returns LS_ERR_TOO_LARGE and does nothing.
+ * The first call on each device looks up the scratch array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one scratch array: it keeps the previous call's contents (the
+ * entry point re-clears what must start at zero), and two calls whose kernels overlap on the GPU
+ * (different streams) race on it -- serialise them. */
+int ls_linear_loss_static(const float* W_dev, const float* bias_dev, const float* x_dev, const void* y_dev,
+                          int64_t n_rows, int d_in, int d_out, int loss, int chunk_rows, float* chunk_loss_dev,
+                          void* cuda_stream);
 
 /* Per-kernel device timing.  Between ls_profile_begin() and ls_profile_end()
  * every launch of a kernel class selected by class_mask (bit c = class c; for

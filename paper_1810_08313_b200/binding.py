@@ -26,6 +26,8 @@ LS_ERR_ROW_RANGE = -5
 LS_ERR_CUDA = -6
 LS_ERR_UNSUPPORTED = -7
 LS_ERR_OVERFLOW = -8
+LS_ERR_DEVICE_TIMEOUT = -9
+LS_ERR_TOO_LARGE = -10
 
 LOSS = {"softmax_ce": 0, "mse_half": 1}
 GEMM = {"fp32": 0, "bf16": 1}
@@ -85,6 +87,7 @@ def _lib():
         "ls_run": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, vp, i64, P(i64), vp, vp, vp, i64, P(i64),
                              P(f32)]),
         "ls_launch_count": (C.c_int, [vp, P(i64)]),
+        "ls_linear_loss_static": (C.c_int, [vp, vp, vp, vp, i64, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]),
         "ls_profile_begin": (C.c_int, [vp, C.c_uint32, C.c_int]),
         "ls_profile_end": (C.c_int, [vp, P(C.c_double), P(i64)]),
     }
@@ -157,6 +160,17 @@ def average_flat(buf, m: int, P: int, stride: Optional[int] = None, stream=None)
     if buf.numel() < (m - 1) * stride + P:
         raise ValueError("buf too small")
     _check(_lib().ls_average_flat(buf.data_ptr(), int(m), int(P), stride, _stream_ptr(stream)), "ls_average_flat")
+
+
+def linear_loss_static(W, bias, x, y, chunk_rows: int, chunk_loss, loss: str = "softmax_ce", stream=None) -> None:
+    """Per-chunk mean loss of z = W x + b on the rows of x, computed by the library without allocating
+    any memory (its scratch is a fixed array inside the library).  W [d_out][d_in], bias [d_out] or None,
+    x [n_rows][d_in] float32, y int32 labels / float32 targets, chunk_loss float32 [n_rows // chunk_rows]:
+    all CUDA tensors owned by the caller.  Calls that overlap on the GPU must be serialised."""
+    _check(_lib().ls_linear_loss_static(W.data_ptr(), None if bias is None else bias.data_ptr(), x.data_ptr(),
+                                        y.data_ptr(), int(x.shape[0]), int(x.shape[1]), int(W.shape[0]), LOSS[loss],
+                                        int(chunk_rows), chunk_loss.data_ptr(), _stream_ptr(stream)),
+           "ls_linear_loss_static")
 
 
 class LocalSGD:

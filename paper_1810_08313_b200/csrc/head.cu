@@ -302,3 +302,62 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
 }
 
 }  // namespace ls
+
+// ---------------------------------------------------------------------------
+// ls_linear_loss_static: the output-layer kernel for callers that cannot allocate.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxChunks = 256;       // chunks (groups) per call
+constexpr int kStaticMaxRows = 65536;       // rows per call
+// Scratch of the kernel: CTA counters, per-chunk first rows, per-row losses.  It lives in the
+// library image, so every GPU that loads the library holds these ~260 KB until the process exits.
+struct StaticScratch {
+  unsigned int counters[kStaticMaxChunks];
+  long long row_off[kStaticMaxChunks];
+  float row_loss[kStaticMaxRows];
+};
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+// Device address of the scratch, looked up once per device (index = CUDA device ordinal).
+static StaticScratch* g_scratch_addr[64] = {nullptr};
+
+}  // namespace
+
+extern "C" int ls_linear_loss_static(const float* W_dev, const float* bias_dev, const float* x_dev, const void* y_dev,
+                                     int64_t n_rows, int d_in, int d_out, int loss, int chunk_rows,
+                                     float* chunk_loss_dev, void* cuda_stream) {
+  using namespace ls;
+  if (W_dev == nullptr || x_dev == nullptr || y_dev == nullptr || chunk_loss_dev == nullptr) return LS_ERR_INVALID_ARG;
+  if (d_in < 1 || d_out < 1 || chunk_rows < 1 || n_rows < chunk_rows || n_rows % chunk_rows != 0)
+    return LS_ERR_INVALID_ARG;
+  if (loss != LS_LOSS_SOFTMAX_CE && loss != LS_LOSS_MSE_HALF) return LS_ERR_INVALID_ARG;
+  if (loss == LS_LOSS_MSE_HALF && d_out != 1) return LS_ERR_INVALID_ARG;
+  const int64_t chunks = n_rows / chunk_rows;
+  if (d_out > CMAX || chunks > kStaticMaxChunks || n_rows > kStaticMaxRows || chunk_rows > LS_MAX_BATCH)
+    return LS_ERR_TOO_LARGE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LS_ERR_CUDA;
+  if (g_scratch_addr[dev] == nullptr) {
+    // In host code the array's name is only a handle: ask the runtime for its address on this device.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return LS_ERR_CUDA;
+    g_scratch_addr[dev] = static_cast<StaticScratch*>(p);
+  }
+  StaticScratch* sc = g_scratch_addr[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // the counters must start at zero; the first row of every chunk is chunk * chunk_rows
+  if (cudaMemsetAsync(sc->counters, 0, sizeof(sc->counters), st) != cudaSuccess) return LS_ERR_CUDA;
+  long long offs[kStaticMaxChunks];
+  for (int64_t c = 0; c < chunks; ++c) offs[c] = c * (long long)chunk_rows;
+  if (cudaMemcpyAsync(sc->row_off, offs, (size_t)chunks * sizeof(long long), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return LS_ERR_CUDA;
+  HeadFwdArgs a;
+  a.A = x_dev; a.a_row_off = reinterpret_cast<const int64_t*>(sc->row_off);
+  a.W = W_dev; a.w_gstride = 0; a.bias = bias_dev;
+  a.y = y_dev; a.y_row_off = reinterpret_cast<const int64_t*>(sc->row_off);
+  a.dZ = nullptr;
+  a.row_loss = sc->row_loss; a.loss_out = chunk_loss_dev; a.counters = sc->counters;
+  a.B = chunk_rows; a.C = d_out; a.K = d_in; a.groups = (int)chunks; a.loss_kind = loss;
+  return launch_head_fwd(a, false, st, nullptr) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}

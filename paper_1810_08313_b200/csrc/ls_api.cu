@@ -431,6 +431,7 @@ const char* ls_strerror(int code) {
     case LS_ERR_UNSUPPORTED: return "not supported";
     case LS_ERR_OVERFLOW: return "result does not fit";
     case LS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case LS_ERR_TOO_LARGE: return "size beyond the fixed capacity of this entry point";
     default: return "unknown error";
   }
 }
