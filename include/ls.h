@@ -164,8 +164,9 @@ int ls_average(ls_handle* h);
 
 /* The averaging kernel on a raw buffer: m vectors of P floats, vector j
  * starting at buf_dev + j*stride floats (stride >= P).  Same arithmetic as
- * ls_average().  Fast path when buf_dev is 16-byte aligned and stride is a
- * multiple of 4. */
+ * ls_average().  Fastest when buf_dev is 32-byte aligned and stride is a
+ * multiple of 8 floats (256-bit accesses); 16-byte alignment and a stride
+ * multiple of 4 give 128-bit accesses; anything else runs element by element. */
 int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride, void* cuda_stream);
 
 /* Training loss of one replica on dataset rows [row_offset, +n_rows), the

@@ -1,13 +1,17 @@
 // Model averaging: X <- X J, J = 1 1^T / m (Section 2, PASGD update rule, the
 // case k mod tau = 0; operator J of the convergence proof's notation).
 //
-// Bandwidth-bound streaming kernel.  Every thread owns one 16-byte column
-// slice: it issues the m independent 128-bit loads of that slice (one per
-// replica) before using any of them, adds them in replica order in fp32,
-// divides once by (float)m and stores the mean back to all m replicas.
-// Algorithmic traffic is 8*m bytes per parameter: each element is read once
-// and written once.  No shared memory, no inter-thread communication: the
-// reduction order is fixed by construction, so the result is bit-reproducible.
+// Bandwidth-bound streaming kernel.  Every thread owns one 32-byte column slice
+// (eight floats; sixteen bytes when the buffers are only 16-byte aligned): it
+// issues the m independent 256-bit loads of that slice, one per replica, before
+// using any of them, adds them in replica order in fp32, divides once by
+// (float)m and stores the mean back to all m replicas.  One slice per thread
+// and a grid that covers the vector exactly: measured on B200 this streams
+// faster than a persistent grid-stride loop (the hardware scheduler keeps more
+// independent loads in flight than a loop that reuses its registers).
+// Algorithmic traffic is 8*m bytes per parameter: each element is read once and
+// written once.  No shared memory, no inter-thread communication: the reduction
+// order is fixed by construction, so the result is bit-reproducible.
 #include "ls_internal.h"
 
 namespace ls {
@@ -16,142 +20,159 @@ namespace {
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b) {
-  // plain IEEE adds; no multiply nearby, so nothing can be contracted into an FMA
-  return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
-}
-__device__ __forceinline__ float4 div4(float4 a, float d) {
-  return make_float4(__fdiv_rn(a.x, d), __fdiv_rn(a.y, d), __fdiv_rn(a.z, d), __fdiv_rn(a.w, d));
-}
+template <int W> struct Vec;
+template <> struct Vec<4> {
+  float v[4];
+  __device__ __forceinline__ void load(const float* p) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  __device__ __forceinline__ void store(float* p) const {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+};
+template <> struct Vec<8> {
+  float v[8];
+  __device__ __forceinline__ void load(const float* p) {
+    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+  }
+  __device__ __forceinline__ void store(float* p) const {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+                 "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
+  }
+};
+
 __device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
-__device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, float4 v) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
-  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
-  uint2 u;
-  u.x = *reinterpret_cast<uint32_t*>(&lo);
-  u.y = *reinterpret_cast<uint32_t*>(&hi);
-  *reinterpret_cast<uint2*>(p) = u;
+
+template <int W>
+__device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&v)[W]) {
+  uint32_t u[W / 2];
+#pragma unroll
+  for (int e = 0; e < W / 2; ++e) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+    u[e] = *reinterpret_cast<uint32_t*>(&t);
+  }
+  if constexpr (W == 8) *reinterpret_cast<uint4*>(p) = make_uint4(u[0], u[1], u[2], u[3]);
+  else *reinterpret_cast<uint2*>(p) = make_uint2(u[0], u[1]);
 }
 
-// M > 0: replica count known at compile time (loads fully unrolled, all in flight).
-// M == 0: any m, processed in chunks of 8 loads, still in replica order.
-template <int M>
+// M > 0: replica count known at compile time (all m loads in flight at once).
+// M == 0: any m, processed in chunks of 8 replicas, still in replica order.
+// W: floats per thread (8 or 4).  Plain IEEE adds and one IEEE division: there is no
+// multiply nearby, so nothing can be contracted into an FMA.
+template <int M, int W>
 __global__ void __launch_bounds__(kThreads)
-average_vec4_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
-                    __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
+average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
+               __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
+  const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (i >= n_vec) return;
   const int m = M > 0 ? M : m_rt;
-  float* buf = base + (int64_t)blockIdx.y * buf_stride;
-  const bool do_shadow = (shadow != nullptr) && blockIdx.y == 0;
-  const bool do_lo = (lo != nullptr) && blockIdx.y == 0;
+  float* p = base + (int64_t)blockIdx.y * buf_stride + i * W;
   const float mf = (float)m;
-  const int64_t step = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += step) {
-    float4* p = reinterpret_cast<float4*>(buf) + i;
-    const int64_t s4 = stride / 4;
-    float4 mean;
-    if (M > 0) {
-      float4 v[M > 0 ? M : 1];
+  Vec<W> s;
+  if (M > 0) {
+    Vec<W> v[M > 0 ? M : 1];
 #pragma unroll
-      for (int j = 0; j < M; ++j) v[j] = __ldcs(p + j * s4);
-      float4 s = v[0];
+    for (int j = 0; j < M; ++j) v[j].load(p + (int64_t)j * stride);
+    s = v[0];
 #pragma unroll
-      for (int j = 1; j < M; ++j) s = add4(s, v[j]);
-      mean = div4(s, mf);
-    } else {
-      float4 s = __ldcs(p);
-      for (int j0 = 1; j0 < m; j0 += 8) {
-        float4 v[8];
+    for (int j = 1; j < M; ++j)
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (j0 + j < m) v[j] = __ldcs(p + (int64_t)(j0 + j) * s4);
+      for (int e = 0; e < W; ++e) s.v[e] = __fadd_rn(s.v[e], v[j].v[e]);
+  } else {
+    s.load(p);
+    for (int j0 = 1; j0 < m; j0 += 8) {
+      Vec<W> v[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (j0 + j < m) s = add4(s, v[j]);
-      }
-      mean = div4(s, mf);
+      for (int j = 0; j < 8; ++j)
+        if (j0 + j < m) v[j].load(p + (int64_t)(j0 + j) * stride);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (j0 + j < m)
+#pragma unroll
+          for (int e = 0; e < W; ++e) s.v[e] = __fadd_rn(s.v[e], v[j].v[e]);
     }
+  }
+#pragma unroll
+  for (int e = 0; e < W; ++e) s.v[e] = __fdiv_rn(s.v[e], mf);
 #pragma unroll 4
-    for (int j = 0; j < m; ++j) p[(int64_t)j * s4] = mean;
-    if (do_shadow) {
-      for (int j = 0; j < m; ++j) store_bf16x4(shadow + (int64_t)j * stride + i * 4, mean);
-    }
-    if (do_lo) {
-      const float4 l4 = make_float4(tf32_lo(mean.x), tf32_lo(mean.y), tf32_lo(mean.z), tf32_lo(mean.w));
-      for (int j = 0; j < m; ++j) *reinterpret_cast<float4*>(lo + (int64_t)j * stride + i * 4) = l4;
+  for (int j = 0; j < m; ++j) s.store(p + (int64_t)j * stride);
+  if (blockIdx.y == 0) {
+    if (shadow != nullptr)
+      for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + i * W, s.v);
+    if (lo != nullptr) {
+      Vec<W> l;
+#pragma unroll
+      for (int e = 0; e < W; ++e) l.v[e] = tf32_lo(s.v[e]);
+      for (int j = 0; j < m; ++j) l.store(lo + (int64_t)j * stride + i * W);
     }
   }
 }
 
-// Scalar path: the ragged tail (n mod 4 elements) and buffers that are not
+// Scalar path: the ragged tail (n mod W elements) and buffers that are not
 // 16-byte aligned.  Same arithmetic, one element per thread.
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
                       __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
-  const bool do_shadow = (shadow != nullptr) && blockIdx.y == 0;
   const float mf = (float)m;
-  const int64_t step = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = first + (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) {
-    float s = buf[i];
-    for (int j = 1; j < m; ++j) s = __fadd_rn(s, buf[(int64_t)j * stride + i]);
-    const float mean = __fdiv_rn(s, mf);
-    for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
-    if (do_shadow)
+  const int64_t i = first + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (i >= n) return;
+  float s = buf[i];
+  for (int j = 1; j < m; ++j) s = __fadd_rn(s, buf[(int64_t)j * stride + i]);
+  const float mean = __fdiv_rn(s, mf);
+  for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
+  if (blockIdx.y == 0) {
+    if (shadow != nullptr)
       for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + i] = __float2bfloat16_rn(mean);
-    if (lo != nullptr && blockIdx.y == 0)
+    if (lo != nullptr)
       for (int j = 0; j < m; ++j) lo[(int64_t)j * stride + i] = tf32_lo(mean);
   }
 }
 
-int num_sms() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+template <int W>
+void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
+                __nv_bfloat16* shadow, float* lo) {
+  switch (m) {
+    case 2: average_kernel<2, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
+    case 4: average_kernel<4, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
+    case 8: average_kernel<8, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
+    case 16: average_kernel<16, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
+    default: average_kernel<0, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
   }
-  return sms;
 }
 
-template <int M>
-void launch_vec4(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
-                 __nv_bfloat16* shadow, float* lo) {
-  average_vec4_kernel<M><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo);
-}
+inline bool aligned_to(const void* p, size_t a) { return p == nullptr || reinterpret_cast<uintptr_t>(p) % a == 0; }
 
 }  // namespace
 
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
                    __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches) {
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
-  const bool aligned = (reinterpret_cast<uintptr_t>(base) % 16 == 0) && (stride % 4 == 0) && (buf_stride % 4 == 0) &&
-                       (shadow == nullptr || reinterpret_cast<uintptr_t>(shadow) % 8 == 0) &&
-                       (lo == nullptr || reinterpret_cast<uintptr_t>(lo) % 16 == 0);
-  const int64_t n_vec = aligned ? n / 4 : 0;
-  const int sms = num_sms();
+  // widest slice the addresses allow: 8 floats (32-byte aligned), 4 floats (16-byte), else scalar
+  int W = 0;
+  if (aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 && aligned_to(shadow, 16) && aligned_to(lo, 32))
+    W = 8;
+  else if (aligned_to(base, 16) && stride % 4 == 0 && buf_stride % 4 == 0 && aligned_to(shadow, 8) && aligned_to(lo, 16))
+    W = 4;
+  const int64_t n_vec = W ? n / W : 0;
   if (n_vec > 0) {
-    // whole multiples of the SM count; each thread keeps m 16-byte loads in flight
-    int per_sm = m <= 8 ? 8 : 4;
-    int64_t want = (n_vec + kThreads - 1) / kThreads;
-    int64_t gx = (int64_t)sms * per_sm;
-    if (want < gx) gx = want;
+    const int64_t gx = (n_vec + kThreads - 1) / kThreads;
+    if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    switch (m) {
-      case 2: launch_vec4<2>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
-      case 4: launch_vec4<4>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
-      case 8: launch_vec4<8>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
-      case 16: launch_vec4<16>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
-      default: launch_vec4<0>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo); break;
-    }
+    if (W == 8) launch_vec<8>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo);
+    else launch_vec<4>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  const int64_t first = n_vec * 4;
+  const int64_t first = n_vec * W;
   if (first < n) {
-    int64_t rem = n - first;
-    int64_t gx = (rem + kThreads - 1) / kThreads;
-    if (gx > (int64_t)sms * 8) gx = (int64_t)sms * 8;
+    const int64_t gx = (n - first + kThreads - 1) / kThreads;
+    if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
     average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, lo);
     if (launches) ++*launches;
