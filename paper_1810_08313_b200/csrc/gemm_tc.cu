@@ -20,6 +20,10 @@
 //          backward kernels therefore restart the TMEM accumulator every kChunkStages stages (two
 //          accumulators, double-buffered) and the epilogue warps add the partial sums in registers
 //          with round-to-nearest while the next chunk is being multiplied.
+//          When a layer has too few output tiles to occupy the GPU (small batch x width), K is split
+//          over a thread-block cluster of 2 or 4 CTAs: every CTA sums its K slice as above, the
+//          partial rows are exchanged through distributed shared memory and added in rank order by
+//          the rank-0 CTA, which then runs the epilogue.  No atomics, so the result is reproducible.
 //
 // Operands are read in place whatever their orientation: a K-major operand
 // ([rows][K], K contiguous) and an MN-major operand ([K][rows], rows contiguous)
@@ -82,13 +86,16 @@ struct Smem {
 template <int ELEMS>
 __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, const Operand& op, int g,
                                            bool mn_major, int tile0, int tile_extent, int k0) {
-  constexpr int kChunkBytes = ELEMS * KB_BYTES;
+  // rows per box: a K-major box always holds 64 MN-rows, an MN-major box holds ELEMS K-rows
+  const int box_rows = mn_major ? ELEMS : 64;
+  const int kChunkBytes = box_rows * KB_BYTES;
   const int row_base = op.rank3 ? 0 : (int)(op.row_off ? op.row_off[g] : (int64_t)g * op.rows_per_group);
   const int z = op.z0 + g * op.z_step;
-  for (int c = 0; c < tile_extent / ELEMS; ++c) {
+  const int n_boxes = mn_major ? tile_extent / ELEMS : tile_extent / 64;
+  for (int c = 0; c < n_boxes; ++c) {
     char* d = static_cast<char*>(dst) + c * kChunkBytes;
     const int x = mn_major ? tile0 + c * ELEMS : k0;
-    const int y = mn_major ? k0 : tile0 + c * ELEMS;
+    const int y = mn_major ? k0 : tile0 + c * 64;
     if (op.rank3) tma_load_3d(d, tm, bar, x, y, z);
     else tma_load_2d(d, tm, bar, x, row_base + y);
   }
@@ -126,7 +133,7 @@ __device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, con
   }
 }
 
-template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT>
 __global__ void __launch_bounds__(kThreads, (Smem<TF32, BN, STAGES>::kTotal <= 113 * 1024) ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo, const Params p) {
@@ -139,6 +146,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr bool CHUNKED = TF32 && EPI != EPI_DW;
   constexpr int CS = kChunkStages;
   constexpr uint32_t TMEM_COLS = CHUNKED ? 2 * BN : BN;
+  static_assert(SPLIT == 1 || CHUNKED, "split-K needs the register-resident partial sums");
+  static_assert(SPLIT == 1 || BN * BM * 4 <= STAGES * Smem<TF32, BN, STAGES>::kStageBytes, "exchange buffer");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -152,8 +161,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.z;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int num_kb = p.K / ELEMS;
+  const int m0 = blockIdx.y * BM, n0 = (int)(blockIdx.x / SPLIT) * BN;
+  const int rank = SPLIT > 1 ? (int)cluster_ctarank() : 0;     // which K slice this CTA sums
+  const int num_kb = p.K / ELEMS / SPLIT;
+  const int kb0 = rank * num_kb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -172,6 +183,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
+  // epilogue-warp state (warps 2-5): this thread owns output row `row`
+  const int q = warp & 3;
+  const int row = m0 + q * 32 + lane;
+  const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+  float sum[CHUNKED ? BN : 1];
+  bool ok = true;
+
   if (warp == 0) {
     if (elect_one()) {
       for (int kb = 0; kb < num_kb; ++kb) {
@@ -180,13 +198,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         mbar_expect_tx(&full[s], L::kStageBytes);
         uint8_t* sa = stage_base + s * L::kStageBytes;
         uint8_t* sb = sa + L::kABytes;
-        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM, kb * ELEMS);
-        issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, kb * ELEMS);
+        const int k0 = (kb0 + kb) * ELEMS;
+        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM, k0);
+        issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, k0);
         if (TF32) {
           uint8_t* sal = sb + L::kBBytes;
           uint8_t* sbl = sal + L::kABytes;
-          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM, kb * ELEMS);
-          issue_tile<ELEMS>(sbl, &tmBlo, &full[s], p.b_lo, g, B_MN, n0, BN, kb * ELEMS);
+          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM, k0);
+          issue_tile<ELEMS>(sbl, &tmBlo, &full[s], p.b_lo, g, B_MN, n0, BN, k0);
         }
       }
     }
@@ -237,12 +256,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    // ---- epilogue warps ---------------------------------------------------------
-    const int q = warp & 3;
-    const int row = m0 + q * 32 + lane;        // output row this thread owns
-    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-    float sum[CHUNKED ? BN : 1];
-    bool ok = true;
+    // ---- epilogue warps: collect the accumulator(s) ------------------------------
     if (CHUNKED) {
       // add the partial accumulators in registers (this thread owns one output row) as they complete
 #pragma unroll
@@ -272,7 +286,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after_sync();
     }
     if (!ok && lane == 0) atomicExch(p.err_flag, 3);
-    if (ok) {
+    if (SPLIT > 1 && rank != 0 && ok) {
+      // every load of this CTA has been consumed and every MMA has completed: the stage buffers are
+      // free, and hold this CTA's partial rows for rank 0 ([column][row], so lanes are conflict-free)
+      float* xbuf = reinterpret_cast<float*>(smem);
+#pragma unroll
+      for (int i = 0; i < (CHUNKED ? BN : 1); ++i) xbuf[i * BM + q * 32 + lane] = sum[i];
+    }
+  }
+  if (SPLIT > 1) {
+    cluster_sync_all();
+    if (warp >= 2 && rank == 0 && ok) {
+      const uint32_t mine = smem_u32(reinterpret_cast<float*>(smem) + q * 32 + lane);
+      for (int r = 1; r < SPLIT; ++r) {
+        const uint32_t remote = map_to_rank(mine, (uint32_t)r);
+#pragma unroll
+        for (int i = 0; i < (CHUNKED ? BN : 1); ++i) sum[i] += ld_cluster_f32(remote + (uint32_t)(i * BM * 4));
+      }
+    }
+    cluster_sync_all();      // the other CTAs stay alive until rank 0 has read their rows
+  }
+  if (warp >= 2) {
+    if (ok && (SPLIT == 1 || rank == 0)) {
 #pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
@@ -403,32 +438,69 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES>
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT = 1>
 int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
   using L = Smem<TF32, BN, STAGES>;
-  auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES>;
+  auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES, SPLIT>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((unsigned)(p.N / BN), (unsigned)(p.M / BM), (unsigned)groups);
+  dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / BM), (unsigned)groups);
   const CUtensorMap* alo = TF32 ? mp.a_lo : mp.a;
   const CUtensorMap* blo = TF32 ? mp.b_lo : mp.b;
-  kern<<<grid, kThreads, L::kTotal, st>>>(*mp.a, *mp.b, *alo, *blo, p);
-  return cudaGetLastError();
+  if (SPLIT == 1) {
+    kern<<<grid, kThreads, L::kTotal, st>>>(*mp.a, *mp.b, *alo, *blo, p);
+    return cudaGetLastError();
+  }
+  // the SPLIT CTAs that share an output tile form one cluster along x
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = L::kTotal;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = SPLIT;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, *mp.a, *mp.b, *alo, *blo, p);
 }
 
-int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, int rank, int64_t rows, int64_t cols,
-             int64_t groups, int64_t gstride) {
+// fp32 forward / backward: tile width and K split.  128-wide tiles when N allows; K is split over a
+// cluster while that keeps the grid within one wave of SMs and every slice keeps whole stages.
+template <bool A_MN, bool B_MN, int EPI>
+int launch_fp32(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
+  const int bn = (p.N % 128 == 0) ? 128 : 64;
+  const int tiles = (p.M / BM) * (p.N / bn) * groups;
+  const int num_kb = p.K / 32;
+  int split = 1;
+  while (split < 4 && tiles * split * 2 <= 148 && num_kb % (split * 2) == 0 && num_kb / (split * 2) >= 8) split *= 2;
+  if (bn == 128) {
+    if (split == 4) return launch_one<true, 128, A_MN, B_MN, EPI, 3, 4>(mp, p, groups, st);
+    if (split == 2) return launch_one<true, 128, A_MN, B_MN, EPI, 3, 2>(mp, p, groups, st);
+    return launch_one<true, 128, A_MN, B_MN, EPI, 3, 1>(mp, p, groups, st);
+  }
+  if (split == 4) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 4>(mp, p, groups, st);
+  if (split == 2) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 2>(mp, p, groups, st);
+  return launch_one<true, 64, A_MN, B_MN, EPI, 4, 1>(mp, p, groups, st);
+}
+
+int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, bool block32, int rank, int64_t rows,
+             int64_t cols, int64_t groups, int64_t gstride) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
   const cuuint64_t eb = fp32 ? 4 : 2;
   const cuuint32_t elems = (cuuint32_t)(KB_BYTES / eb);
   cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)groups};
   cuuint64_t strides[2] = {(cuuint64_t)cols * eb, (cuuint64_t)gstride * eb};
-  cuuint32_t box[3] = {elems, elems, 1};
+  // K-major reads take boxes of 64 rows; MN-major reads (and the 32 x 32 blocks of the update kernel) of
+  // fp32 tensors take 32 rows.  For bf16 both are 64.
+  cuuint32_t box[3] = {elems, (fp32 && !mn32 && !block32) ? 64u : elems, 1};
   cuuint32_t es[3] = {1, 1, 1};
   CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
                   const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -437,19 +509,22 @@ int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, int rank,
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-inline int few_tiles(int M, int N, int groups, int bn) { return (M / BM) * (N / bn) * groups; }
-
 }  // namespace
 
 // 2-D map over a row-major matrix [rows][cols] of bf16 or fp32; box = 128 bytes x (64 | 32) rows, 128-byte
 // swizzle.  mn32: the fp32 tensor will be read as an MN-major operand (swizzle in 32-byte units).
 int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols) {
-  return make_map(out, base, fp32, mn32, 2, rows, cols, 1, 0);
+  return make_map(out, base, fp32, mn32, false, 2, rows, cols, 1, 0);
 }
 // 3-D map over `groups` row-major matrices [rows][cols] that start every gstride elements.
 int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
                    int64_t groups, int64_t gstride) {
-  return make_map(out, base, fp32, mn32, 3, rows, cols, groups, gstride);
+  return make_map(out, base, fp32, mn32, false, 3, rows, cols, groups, gstride);
+}
+// 3-D map over fp32 matrices read and written in 32 x 32 blocks (128-byte swizzle, 16-byte units).
+int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups,
+                         int64_t gstride) {
+  return make_map(out, base, true, false, true, 3, rows, cols, groups, gstride);
 }
 
 // M output rows, N output columns, K contraction length of one group.
@@ -467,11 +542,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   p.bias = a.bias; p.bias_gstride = a.bias_gstride; p.relu = a.relu;
   p.C = a.C; p.Clo = a.Clo; p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  if (a.fp32) {
-    if (a.N % 128 == 0 && few_tiles(a.M, a.N, a.groups, 128) >= 148)
-      return launch_one<true, 128, false, false, EPI_FWD, 3>(a.maps, p, a.groups, st);
-    return launch_one<true, 64, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
-  }
+  if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
 }
@@ -483,11 +554,7 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.C = a.C; p.Clo = a.Clo; p.act = a.act; p.err_flag = a.err_flag;
   if (launches) ++*launches;
-  if (a.fp32) {
-    if (a.N % 128 == 0 && few_tiles(a.M, a.N, a.groups, 128) >= 148)
-      return launch_one<true, 128, false, true, EPI_DX, 3>(a.maps, p, a.groups, st);
-    return launch_one<true, 64, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
-  }
+  if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
 }

@@ -513,8 +513,8 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
       if (!mn) {
         for (int l = 0; l < lay.L; ++l)
           if (lay.dims[l] % 4 == 0) {
-            ok(tc_make_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], true, false, lay.dims[l + 1], lay.dims[l], m, lay.stride));
-            ok(tc_make_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], true, false, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+            ok(tc_make_block_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
+            ok(tc_make_block_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
           }
       }
       if (lay.dims[0] % q == 0) {

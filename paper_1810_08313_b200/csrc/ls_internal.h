@@ -215,6 +215,8 @@ int launch_gather_lo(const float* X, const int64_t* row_off, float* dst, int gro
 int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols);
 int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
                    int64_t groups, int64_t gstride);
+int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups,
+                         int64_t gstride);
 bool tc_shape_ok(bool fp32, int M, int N, int K);   // output rows, output columns, contraction length
 struct TcOperandMaps {
   const CUtensorMap *a, *b, *a_lo, *b_lo;   // lo maps: fp32 only
