@@ -20,7 +20,7 @@ namespace {
 constexpr int CMAX = 16;
 constexpr int kThreads = 256;
 constexpr int kRowsPerCta = 4;         // head_fwd: rows per CTA (the 8 warps split K)
-constexpr int kColsPerCta = 32;        // head_bwd: 32 columns x 8 row slices
+constexpr int kColsPerCta = 64;        // head_bwd: 32 lanes x 2 columns, 8 row slices
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -42,7 +42,7 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&r)[4]) {
 // One CTA = kRowsPerCta (4) mini-batch rows of one replica.  The 8 warps split K; partial dot products are
 // combined lane-wise by a butterfly and warp-wise through shared memory in warp order.
 template <typename TA>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ W,
                 int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
                 const int64_t* __restrict__ y_row_off, float* __restrict__ dZ, float* __restrict__ row_loss,
@@ -165,77 +165,113 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   }
 }
 
+__device__ __forceinline__ void load2(const float* p, float (&r)[2]) {
+  const float2 v = *reinterpret_cast<const float2*>(p);
+  r[0] = v.x; r[1] = v.y;
+}
+__device__ __forceinline__ void load2(const __nv_bfloat16* p, float (&r)[2]) {
+  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(p);
+  r[0] = __low2float(v); r[1] = __high2float(v);
+}
+__device__ __forceinline__ void store2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16* p, float a, float b) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b);
+}
+
+// One CTA = kColsPerCta (64) columns of the layer input of one replica: 32 lanes x 2 adjacent columns,
+// 8 warps = 8 interleaved row slices.  pair_ok: K is even and the pointers are aligned for 2-element accesses.
 template <typename TA>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
                 float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb, float* __restrict__ Wlo,
                 float* __restrict__ bias, float* __restrict__ vbias, int64_t w_gstride, TA* __restrict__ dPrev,
-                float* __restrict__ dPrevLo, int B, int C, int K, float lr, float mu) {
+                float* __restrict__ dPrevLo, int B, int C, int K, float lr, float mu, int pair_ok) {
   extern __shared__ float sm[];
   float* dz = sm;                                   // [B][C]
   float* part = sm + (size_t)B * C;                 // [8][CMAX][kColsPerCta]
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int k = blockIdx.x * kColsPerCta + cx;
+  const int k = blockIdx.x * kColsPerCta + cx * 2;  // this thread's columns k, k + 1
   const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
+  const bool in0 = k < K, in1 = k + 1 < K;
+
+  float wreg[CMAX][2], gw[CMAX][2];
+#pragma unroll
+  for (int c = 0; c < CMAX; ++c) {
+    wreg[c][0] = (c < C && in0) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k] : 0.f;
+    wreg[c][1] = (c < C && in1) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k + 1] : 0.f;
+    gw[c][0] = gw[c][1] = 0.f;
+  }
   for (int i = threadIdx.x; i < B * C; i += kThreads) dz[i] = dZ[(int64_t)g * B * C + i];
   __syncthreads();
 
-  float wreg[CMAX], gw[CMAX];
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    wreg[c] = (c < C && k < K) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k] : 0.f;
-    gw[c] = 0.f;
-  }
-  if (k < K) {
+  if (in0) {
     for (int bb = ry; bb < B; bb += 64) {
       // eight rows per trip so that eight loads of A are in flight
-      float av[8];
+      float av[8][2];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) av[u] = (bb + 8 * u < B) ? to_f(Ag[(int64_t)(bb + 8 * u) * K + k]) : 0.f;
+      for (int u = 0; u < 8; ++u) {
+        av[u][0] = av[u][1] = 0.f;
+        if (bb + 8 * u < B) {
+          const TA* src = Ag + (int64_t)(bb + 8 * u) * K + k;
+          if (pair_ok) load2(src, av[u]);
+          else { av[u][0] = to_f(src[0]); if (in1) av[u][1] = to_f(src[1]); }
+        }
+      }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int b = bb + 8 * u;
         if (b >= B) break;
-        const float a = av[u];
-        float da = 0.f;
+        float da0 = 0.f, da1 = 0.f;
 #pragma unroll
         for (int c = 0; c < CMAX; ++c)
           if (c < C) {
             const float d = dz[b * C + c];
-            gw[c] = fmaf(d, a, gw[c]);
-            da = fmaf(d, wreg[c], da);
+            gw[c][0] = fmaf(d, av[u][0], gw[c][0]);
+            gw[c][1] = fmaf(d, av[u][1], gw[c][1]);
+            da0 = fmaf(d, wreg[c][0], da0);
+            da1 = fmaf(d, wreg[c][1], da1);
           }
         if (dPrev != nullptr) {
-          const float o = a > 0.f ? da : 0.f;
+          const float o0 = av[u][0] > 0.f ? da0 : 0.f, o1 = av[u][1] > 0.f ? da1 : 0.f;
           const int64_t at = ((int64_t)g * B + b) * K + k;
-          put(dPrev + at, o);
-          if (dPrevLo != nullptr) dPrevLo[at] = tf32_lo(o);
+          if (pair_ok) {
+            store2(dPrev + at, o0, o1);
+            if (dPrevLo != nullptr) store2(dPrevLo + at, tf32_lo(o0), tf32_lo(o1));
+          } else {
+            put(dPrev + at, o0);
+            if (in1) put(dPrev + at + 1, o1);
+            if (dPrevLo != nullptr) { dPrevLo[at] = tf32_lo(o0); if (in1) dPrevLo[at + 1] = tf32_lo(o1); }
+          }
         }
       }
     }
   }
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c) part[(ry * CMAX + c) * kColsPerCta + cx] = gw[c];
+  for (int c = 0; c < CMAX; ++c) {
+    part[(ry * CMAX + c) * kColsPerCta + cx * 2] = gw[c][0];
+    part[(ry * CMAX + c) * kColsPerCta + cx * 2 + 1] = gw[c][1];
+  }
   __syncthreads();
-  if (ry == 0 && k < K) {
+  // 8 warps x 64 columns: thread t < 64 * C finishes column t % 64 of output row t / 64 ... done by all
+  // threads in a strided loop so that the V / W accesses are coalesced along k
+  for (int t = threadIdx.x; t < C * kColsPerCta; t += kThreads) {
+    const int c = t / kColsPerCta, col = t % kColsPerCta;
+    const int kk = blockIdx.x * kColsPerCta + col;
+    if (kk >= K) continue;
+    float s = 0.f;
 #pragma unroll
-    for (int c = 0; c < CMAX; ++c)
-      if (c < C) {
-        float s = 0.f;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) s += part[(r * CMAX + c) * kColsPerCta + cx];
-        const int64_t at = (int64_t)g * w_gstride + (int64_t)c * K + k;
-        float step = s;
-        if (mu != 0.f) {
-          step = fmaf(mu, V[at], s);
-          V[at] = step;
-        }
-        const float w = fmaf(-lr, step, wreg[c]);
-        W[at] = w;
-        if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
-        if (Wlo != nullptr) Wlo[at] = tf32_lo(w);
-      }
+    for (int r = 0; r < 8; ++r) s += part[(r * CMAX + c) * kColsPerCta + col];
+    const int64_t at = (int64_t)g * w_gstride + (int64_t)c * K + kk;
+    float step = s;
+    if (mu != 0.f) {
+      step = fmaf(mu, V[at], s);
+      V[at] = step;
+    }
+    const float w = fmaf(-lr, step, W[at]);
+    W[at] = w;
+    if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
+    if (Wlo != nullptr) Wlo[at] = tf32_lo(w);
   }
   if (blockIdx.x == 0 && bias != nullptr && threadIdx.x < C) {
     const int c = threadIdx.x;
@@ -275,6 +311,10 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   if (launches) ++*launches;
   dim3 grid((unsigned)((a.K + kColsPerCta - 1) / kColsPerCta), (unsigned)a.groups);
   const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * kColsPerCta) * sizeof(float);
+  const size_t esz = a_bf16 ? 2 : 4;
+  const int pair_ok = (a.K % 2 == 0) && reinterpret_cast<uintptr_t>(a.A) % (2 * esz) == 0 &&
+                      (a.dPrev == nullptr || reinterpret_cast<uintptr_t>(a.dPrev) % (2 * esz) == 0) &&
+                      (a.dPrevLo == nullptr || reinterpret_cast<uintptr_t>(a.dPrevLo) % 8 == 0);
   if (a_bf16) {
     auto kern = head_bwd_kernel<__nv_bfloat16>;
     static bool configured = false;
@@ -285,7 +325,7 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
     }
     kern<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo,
                                        a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev), nullptr, a.B,
-                                       a.C, a.K, a.lr, a.mu);
+                                       a.C, a.K, a.lr, a.mu, pair_ok);
   } else {
     auto kern = head_bwd_kernel<float>;
     static bool configured = false;
@@ -296,7 +336,7 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
     }
     kern<<<grid, kThreads, smem, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo, a.bias,
                                        a.vbias, a.w_gstride, static_cast<float*>(a.dPrev), a.dPrevLo, a.B, a.C, a.K,
-                                       a.lr, a.mu);
+                                       a.lr, a.mu, pair_ok);
   }
   return cudaGetLastError();
 }
