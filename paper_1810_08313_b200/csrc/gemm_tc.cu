@@ -67,10 +67,10 @@ struct Params {
   int* err_flag;
 };
 
-template <bool TF32, int BN, int STAGES>
+template <bool TF32, int BN, int STAGES, int MT = 1>
 struct Smem {
   static constexpr int kTiles = TF32 ? 2 : 1;      // hi and lo copies of each operand tile
-  static constexpr int kABytes = BM * KB_BYTES;
+  static constexpr int kABytes = MT * BM * KB_BYTES;   // MT row blocks of 128 share one B tile
   static constexpr int kBBytes = BN * KB_BYTES;
   static constexpr int kStageBytes = kTiles * (kABytes + kBBytes);
   // the update epilogue stages its 32x32 blocks in stage 0, which is free once the accumulator is complete
@@ -133,11 +133,13 @@ __device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, con
   }
 }
 
-template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT>
-__global__ void __launch_bounds__(kThreads, (Smem<TF32, BN, STAGES>::kTotal <= 113 * 1024) ? 2 : 1)
+// MT = 2: the CTA computes two 128-row blocks (a 256 x BN tile) from one B tile in shared memory, with two
+// TMEM accumulators: a third less operand traffic from L2 per flop, which is what bounds these kernels.
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT, int MT>
+__global__ void __launch_bounds__(kThreads, (Smem<TF32, BN, STAGES, MT>::kTotal <= 113 * 1024) ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo, const Params p) {
-  using L = Smem<TF32, BN, STAGES>;
+  using L = Smem<TF32, BN, STAGES, MT>;
   constexpr int EB = TF32 ? 4 : 2;             // bytes per operand element
   constexpr int ELEMS = KB_BYTES / EB;         // K elements per stage
   constexpr int MMA_K = 32 / EB;               // K of one tcgen05.mma (32 bytes)
@@ -145,9 +147,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, A_MN, B_MN, BM, BN);
   constexpr bool CHUNKED = TF32 && EPI != EPI_DW;
   constexpr int CS = kChunkStages;
-  constexpr uint32_t TMEM_COLS = CHUNKED ? 2 * BN : BN;
+  constexpr uint32_t TMEM_COLS = CHUNKED ? 2 * BN : MT * BN;
+  static_assert(MT == 1 || (!CHUNKED && !A_MN && EPI != EPI_DW && MT * BN <= 512), "two row blocks: bf16 forward/backward");
   static_assert(SPLIT == 1 || CHUNKED, "split-K needs the register-resident partial sums");
-  static_assert(SPLIT == 1 || BN * BM * 4 <= STAGES * Smem<TF32, BN, STAGES>::kStageBytes, "exchange buffer");
+  static_assert(SPLIT == 1 || BN * BM * 4 <= STAGES * L::kStageBytes, "exchange buffer");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -161,7 +164,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.z;
-  const int m0 = blockIdx.y * BM, n0 = (int)(blockIdx.x / SPLIT) * BN;
+  const int m0 = blockIdx.y * BM * MT, n0 = (int)(blockIdx.x / SPLIT) * BN;
   const int rank = SPLIT > 1 ? (int)cluster_ctarank() : 0;     // which K slice this CTA sums
   const int num_kb = p.K / ELEMS / SPLIT;
   const int kb0 = rank * num_kb;
@@ -185,7 +188,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   // epilogue-warp state (warps 2-5): this thread owns output row `row`
   const int q = warp & 3;
-  const int row = m0 + q * 32 + lane;
+  const int row0 = m0 + q * 32 + lane;
   const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
   float sum[CHUNKED ? BN : 1];
   bool ok = true;
@@ -199,12 +202,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t* sa = stage_base + s * L::kStageBytes;
         uint8_t* sb = sa + L::kABytes;
         const int k0 = (kb0 + kb) * ELEMS;
-        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM, k0);
+        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM * MT, k0);
         issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, k0);
         if (TF32) {
           uint8_t* sal = sb + L::kBBytes;
           uint8_t* sbl = sal + L::kABytes;
-          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM, k0);
+          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM * MT, k0);
           issue_tile<ELEMS>(sbl, &tmBlo, &full[s], p.b_lo, g, B_MN, n0, BN, k0);
         }
       }
@@ -248,6 +251,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mma_tf32(d_tmem, da, db, IDESC, 1u);
           } else {
             mma_bf16(d_tmem, da, db, IDESC, (chunk_start && k == 0) ? 0u : 1u);
+            if (MT == 2) {
+              // second row block: same B tile, A rows 128..255 (16 KB further in the stage)
+              const uint64_t da2 = make_smem_desc(a_addr + BM * KB_BYTES + a_adv, a_lbo, a_sbo, a_sw);
+              mma_bf16(d_tmem + BN, da2, db, IDESC, (chunk_start && k == 0) ? 0u : 1u);
+            }
           }
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
@@ -309,13 +317,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp >= 2) {
     if (ok && (SPLIT == 1 || rank == 0)) {
 #pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc32 = 0; cc32 < MT * (BN / 32); ++cc32) {
+        const int mt = cc32 / (BN / 32), c = cc32 % (BN / 32);
+        const int row = row0 + mt * BM;          // output row this thread owns in row block mt
         uint32_t r[32];
         if (CHUNKED) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum[c * 32 + i]);
         } else {
-          tmem_ld_32x32(taddr + c * 32, r);
+          tmem_ld_32x32(taddr + mt * BN + c * 32, r);
           tmem_ld_wait();
         }
         const int col = n0 + c * 32;
@@ -438,17 +448,17 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT = 1>
+template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT = 1, int MT = 1>
 int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
-  using L = Smem<TF32, BN, STAGES>;
-  auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES, SPLIT>;
+  using L = Smem<TF32, BN, STAGES, MT>;
+  auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES, SPLIT, MT>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / BM), (unsigned)groups);
+  dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / (BM * MT)), (unsigned)groups);
   const CUtensorMap* alo = TF32 ? mp.a_lo : mp.a;
   const CUtensorMap* blo = TF32 ? mp.b_lo : mp.b;
   if (SPLIT == 1) {
@@ -543,6 +553,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   p.C = a.C; p.Clo = a.Clo; p.err_flag = a.err_flag;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
+  if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
 }
@@ -555,6 +566,7 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   p.C = a.C; p.Clo = a.Clo; p.act = a.act; p.err_flag = a.err_flag;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
+  if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
 }
