@@ -66,6 +66,12 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// one 32-byte (whole sector) store; p must be 32-byte aligned
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
 __device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
 template <int ELEMS>
@@ -237,6 +243,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!ok) { if (lane == 0) atomicExch(p.err_flag, 15); break; }
         // this thread's row of the 32 x 32 block; 16-byte pieces are XOR-swizzled by the row (128-byte swizzle)
         const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * p.N + n0 + c * 32;
+        uint32_t cp[8];
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
           const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
@@ -256,16 +263,17 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
           *reinterpret_cast<float4*>(slot + off) = make_float4(ws[0], ws[1], ws[2], ws[3]);
           if (has_v) *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) = make_float4(vs[0], vs[1], vs[2], vs[3]);
+          // operand copy of the new weights, collected so that it leaves in whole 32-byte sectors
           if (TF32) {
-            *reinterpret_cast<float4*>(p.Wlo + at + jj * 4) =
-                make_float4(tf32_lo(ws[0]), tf32_lo(ws[1]), tf32_lo(ws[2]), tf32_lo(ws[3]));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cp[(jj & 1) * 4 + e] = __float_as_uint(tf32_lo(ws[e]));
+            if (jj & 1) st_global_v8(p.Wlo + at + (jj - 1) * 4, cp);
           } else if (p.Wb != nullptr) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
             __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
-            uint2 u;
-            u.x = *reinterpret_cast<uint32_t*>(&lo);
-            u.y = *reinterpret_cast<uint32_t*>(&hi);
-            *reinterpret_cast<uint2*>(p.Wb + at + jj * 4) = u;
+            cp[(jj & 3) * 2] = *reinterpret_cast<uint32_t*>(&lo);
+            cp[(jj & 3) * 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
+            if ((jj & 3) == 3) st_global_v8(p.Wb + at + (jj - 3) * 4, cp);
           }
         }
         // make the in-place update visible to the bulk-copy engine, then write the blocks back
