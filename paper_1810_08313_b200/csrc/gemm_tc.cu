@@ -101,35 +101,45 @@ __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uin
   }
 }
 
-__device__ __forceinline__ void store_bf16x8(__nv_bfloat16* p, const float* v) {
-  uint4 u;
-  __nv_bfloat162 t;
-  t = __floats2bfloat162_rn(v[0], v[1]); u.x = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(v[2], v[3]); u.y = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(v[4], v[5]); u.z = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(v[6], v[7]); u.w = *reinterpret_cast<uint32_t*>(&t);
-  *reinterpret_cast<uint4*>(p) = u;
-}
-
 // The part of x that a tf32 read keeps (upper 19 bits) and the remainder.
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ float tf32_lo(float x) { return x - tf32_hi(x); }
 
-// Store 32 consecutive outputs of one row: bf16, or fp32 plus the lo parts.
+// one 32-byte (whole sector) store; p must be 32-byte aligned
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
+// Store 32 consecutive outputs of one row (bf16, or fp32 plus the lo parts) in whole 32-byte sectors.
 template <bool TF32>
 __device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, const float (&o)[32]) {
   if (TF32) {
-    float4* c4 = reinterpret_cast<float4*>(static_cast<float*>(C) + at);
-    float4* l4 = reinterpret_cast<float4*>(Clo + at);
+    float* c = static_cast<float*>(C) + at;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      c4[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-      l4[i] = make_float4(tf32_lo(o[4 * i]), tf32_lo(o[4 * i + 1]), tf32_lo(o[4 * i + 2]), tf32_lo(o[4 * i + 3]));
+    for (int i = 0; i < 4; ++i) {
+      uint32_t hi[8], lo[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        hi[e] = __float_as_uint(o[8 * i + e]);
+        lo[e] = __float_as_uint(tf32_lo(o[8 * i + e]));
+      }
+      st_global_v8(c + 8 * i, hi);
+      st_global_v8(Clo + at + 8 * i, lo);
     }
   } else {
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(C) + at;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) store_bf16x8(out + i * 8, o + i * 8);
+    for (int i = 0; i < 2; ++i) {
+      uint32_t u[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        __nv_bfloat162 t = __floats2bfloat162_rn(o[16 * i + 2 * e], o[16 * i + 2 * e + 1]);
+        u[e] = *reinterpret_cast<uint32_t*>(&t);
+      }
+      st_global_v8(out + 16 * i, u);
+    }
   }
 }
 
