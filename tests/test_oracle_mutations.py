@@ -1,0 +1,123 @@
+"""The pins must catch plausible mistakes: each test plants one in the oracle (on the CPU, by
+monkeypatching) and checks that a pin from the other test files then fails."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import localsgd_oracle as orc
+from tests import test_oracle_adacomm as pins_tau
+from tests import test_oracle_average as pins_avg
+from tests import test_oracle_gradients as pins_grad
+from tests import test_oracle_pasgd as pins_loop
+
+
+def _fails(fn, *args):
+    try:
+        fn(*args)
+    except AssertionError:
+        return True
+    except Exception:
+        return True          # a crash is also a detected mistake
+    return False
+
+
+def test_pins_pass_on_the_unmodified_oracle():
+    pins_grad.test_gradient_matches_central_differences((5, 4, 3), orc.LOSS_SOFTMAX_CE, True)
+    pins_loop.test_m1_is_plain_sgd(0.9)
+    pins_avg.test_brute_force_scalar_fp32_chain(4)
+    pins_tau.test_hand_table()
+
+
+def test_dropped_batch_normalisation_is_caught(monkeypatch):
+    real = orc.loss_and_grad
+    monkeypatch.setattr(orc, "loss_and_grad", lambda s, x, X, y: (real(s, x, X, y)[0], real(s, x, X, y)[1] * X.shape[0]))
+    assert _fails(pins_grad.test_gradient_matches_central_differences, (5, 4, 3), orc.LOSS_SOFTMAX_CE, True)
+    assert _fails(pins_loop.test_m1_is_plain_sgd, 0.0)
+
+
+def test_wrong_sign_in_a_layer_gradient_is_caught(monkeypatch):
+    real = orc.loss_and_grad
+
+    def flipped(spec, x, X, y):
+        loss, g = real(spec, x, X, y)
+        g = g.copy()
+        n0 = spec.dims[1] * spec.dims[0]
+        g[:n0] = -g[:n0]                       # first-layer weight gradient with the wrong sign
+        return loss, g
+
+    monkeypatch.setattr(orc, "loss_and_grad", flipped)
+    assert _fails(pins_grad.test_gradient_matches_central_differences, (5, 4, 3), orc.LOSS_SOFTMAX_CE, True)
+    assert _fails(pins_grad.test_matches_torch_autograd, (12, 9, 7, 5), orc.LOSS_SOFTMAX_CE, True)
+
+
+def test_momentum_mistakes_are_caught(monkeypatch):
+    # dampened momentum: v = mu v + (1 - mu) g
+    monkeypatch.setattr(orc, "sgd_momentum_step",
+                        lambda x, v, g, lr, mu: (np.asarray(x, np.float64) - lr * (mu * np.asarray(v, np.float64) + (1 - mu) * g),
+                                                 mu * np.asarray(v, np.float64) + (1 - mu) * g))
+    assert _fails(pins_loop.test_m1_is_plain_sgd, 0.9)
+    assert _fails(pins_loop.test_tau1_is_synchronous_sgd_on_the_m_fold_batch, 0.9)
+
+
+def test_learning_rate_inside_the_buffer_is_caught_only_by_a_changing_rate(monkeypatch):
+    # v = mu v + lr g; x -= v is identical at constant lr: the pins cannot (and need not) tell them apart
+    monkeypatch.setattr(orc, "sgd_momentum_step",
+                        lambda x, v, g, lr, mu: (np.asarray(x, np.float64) - (mu * np.asarray(v, np.float64) * lr + lr * g),
+                                                 mu * np.asarray(v, np.float64) + g))
+    pins_loop.test_m1_is_plain_sgd(0.9)
+
+
+def test_averaging_mistakes_are_caught(monkeypatch):
+    def wrong_divisor(X):
+        s = X[0].copy()
+        for j in range(1, X.shape[0]):
+            s = s + X[j]
+        X[:] = (s / np.float32(max(1, X.shape[0] - 1)))[None, :]
+    monkeypatch.setattr(orc, "average_replicas", wrong_divisor)
+    assert _fails(pins_avg.test_brute_force_scalar_fp32_chain, 4)
+    assert _fails(pins_avg.test_within_rounding_bound_of_exact_rational_mean, 4)
+    assert _fails(pins_loop.test_tau1_is_synchronous_sgd_on_the_m_fold_batch, 0.0)
+
+    def reversed_order(X):
+        s = X[-1].copy()
+        for j in range(X.shape[0] - 2, -1, -1):
+            s = s + X[j]
+        X[:] = (s / np.float32(X.shape[0]))[None, :]
+    monkeypatch.setattr(orc, "average_replicas", reversed_order)
+    assert _fails(pins_avg.test_order_matters_and_is_index_order)
+
+    def double_precision_sum(X):
+        X[:] = X.astype(np.float64).mean(axis=0).astype(np.float32)[None, :]
+    monkeypatch.setattr(orc, "average_replicas", double_precision_sum)
+    assert _fails(pins_avg.test_order_matters_and_is_index_order)
+
+    def forgets_last_replica(X):
+        s = X[0].copy()
+        for j in range(1, X.shape[0] - 1):
+            s = s + X[j]
+        X[:] = (s / np.float32(X.shape[0]))[None, :]
+    monkeypatch.setattr(orc, "average_replicas", forgets_last_replica)
+    assert _fails(pins_avg.test_within_rounding_bound_of_exact_rational_mean, 8)
+
+
+def test_averaging_before_the_update_is_caught(monkeypatch):
+    # a loop that averages every tau steps but one step early / late changes the averaging points
+    real = orc.run_pasgd
+
+    def off_by_one(spec, x1, X, y, offs, batch, lr, mu, tau, **kw):
+        return real(spec, x1, X, y, offs, batch, lr, mu, tau + 1, **kw)
+    monkeypatch.setattr(orc, "run_pasgd", off_by_one)
+    assert _fails(pins_loop.test_replicas_identical_after_every_average_and_differ_inside)
+    assert _fails(pins_loop.test_tau1_is_synchronous_sgd_on_the_m_fold_batch, 0.0)
+
+
+def test_controller_mistakes_are_caught(monkeypatch):
+    monkeypatch.setattr(orc, "adacomm_next_tau", lambda F_t, F_0, tau_0: max(1, math.ceil(F_t / F_0 * tau_0)))   # no sqrt
+    assert _fails(pins_tau.test_hand_table)
+    monkeypatch.setattr(orc, "adacomm_next_tau", lambda F_t, F_0, tau_0: max(1, int(round(math.sqrt(F_t / F_0) * tau_0))))
+    assert _fails(pins_tau.test_hand_table)          # round instead of ceil
+    monkeypatch.setattr(orc, "adacomm_next_tau", lambda F_t, F_0, tau_0: max(1, math.floor(math.sqrt(F_t / F_0) * tau_0)))
+    assert _fails(pins_tau.test_result_is_the_smallest_integer_not_below)
+    monkeypatch.setattr(orc, "adacomm_next_tau", lambda F_t, F_0, tau_0: math.ceil(math.sqrt(F_t / F_0) * tau_0))   # no clamp
+    assert _fails(pins_tau.test_hand_table)
