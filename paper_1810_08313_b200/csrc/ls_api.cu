@@ -76,7 +76,7 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   if (!lay.bf16) lay.xlo_off = take((size_t)m * batch * lay.dims[0] * 4);
   lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.dzl_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
-  lay.rowloss_off = take((size_t)m * batch * 4);
+  lay.rowloss_off = take((size_t)LS_MAX_REPLICAS * batch * 4);
   lay.headcnt_off = take((size_t)LS_MAX_REPLICAS * 4);
   lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
   lay.evaloff_off = take((size_t)kEvalCap * 8);
@@ -376,8 +376,11 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
   int64_t* off_dev = reinterpret_cast<int64_t*>(h->state + lay.evaloff_off);
   float* loss_dev = reinterpret_cast<float*>(h->state + lay.evalloss_off);
   LS_CUDA(h, cudaMemcpyAsync(off_dev, offs.data(), (size_t)chunks * 8, cudaMemcpyHostToDevice, h->stream));
-  for (int64_t c0 = 0; c0 < chunks; c0 += lay.m) {
-    const int groups = (int)((chunks - c0 < lay.m) ? chunks - c0 : lay.m);
+  // a wave holds as many chunks as the workspace has room for: m per wave in general (activation
+  // buffers), LS_MAX_REPLICAS for a one-layer model, which needs only per-row losses and counters
+  const int cap = (lay.L == 1 && head_shape_ok(lay.batch, lay.dims[1])) ? LS_MAX_REPLICAS : lay.m;
+  for (int64_t c0 = 0; c0 < chunks; c0 += cap) {
+    const int groups = (int)((chunks - c0 < cap) ? chunks - c0 : cap);
     int rc = forward(h, h->x_dev, XMaps{&h->maps.x_data, &h->maps_mn.x_data}, h->y_dev, off_dev + c0, groups, replica, 0,
                      false, loss_dev + c0);
     if (rc != LS_OK) return rc;

@@ -47,7 +47,7 @@ struct Layout {
   size_t xlo_off = 0;                        // lo twin of the current mini-batches [m][batch][dims[0]] (fp32 models)
   size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
   size_t dzl_off = 0;                        // fp32 dZ of a narrow output layer [m][batch][dims[L]]
-  size_t rowloss_off = 0;                    // per-sample losses [m][batch]
+  size_t rowloss_off = 0;                    // per-sample losses [LS_MAX_REPLICAS][batch]
   size_t headcnt_off = 0;                    // per-replica CTA counters of the output-layer kernel
   size_t rowoff_off = 0;                     // int64 [kRowOffCap][m]
   size_t evaloff_off = 0;                    // int64 [kEvalCap]
