@@ -183,6 +183,36 @@ int ls_eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_rows, 
  * result beyond INT32_MAX). */
 int adacomm_next_tau(double F_t, double F_0, int tau_0);
 
+/* AdaComm with the refinements of Section 4.3:
+ *   candidate (Section 4.3.2, learning-rate coupling)   c = ceil( sqrt( (lr_0/lr_l) * F_t/F_0 ) * tau_0 ), >= 1
+ *   faster decay when training saturates (Section 4.3.1, slack s):
+ *        tau_l = c  if c + slack < tau_prev,  else ceil(gamma * tau_prev), >= 1
+ *   lr_changed != 0 (first decision after the learning rate changed): c is returned as it is, so the period
+ *   may grow when the rate drops.
+ * Pure host function, IEEE double.  Returns the period or a negative LS_ERR_* (non-finite input, F_0 <= 0,
+ * F_t < 0, tau_0 < 1, tau_prev < 1, gamma outside (0, 1], slack < 0, a learning rate <= 0). */
+int adacomm_next_tau_refined(double F_t, double F_0, int tau_0, int tau_prev, double gamma, int slack, double lr_0,
+                             double lr_l, int lr_changed);
+
+/* Options of ls_run_refined(). */
+typedef struct ls_adacomm_opts {
+  double gamma;              /* decay factor of Section 4.3.1, in (0, 1]; the paper uses 1/2 */
+  int32_t slack;             /* slack variable s of Section 4.3.1, >= 0 */
+  int32_t n_decay;           /* number of scheduled learning-rate decays */
+  const int64_t* decay_at;   /* host, ascending: iteration counts at which a decay is scheduled */
+  double decay_factor;       /* lr <- lr * decay_factor (the paper divides by 10) */
+} ls_adacomm_opts;
+
+/* ls_run() with the refined rules: the period is chosen by adacomm_next_tau_refined(), and a scheduled
+ * learning-rate decay is applied at the first decision point at or past its iteration at which the period in
+ * force is 1 (Section 4.3.2: let the period decay to 1 first); one decay per decision.  interval must be >= 1.
+ * The handle's learning rate is changed by the decays (read it back with ls_get_lr()). */
+int ls_run_refined(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
+                   const int64_t* row_offset_host, float* loss_dev, const ls_adacomm_opts* opts, int32_t* period_tau,
+                   int64_t max_periods, int64_t* n_periods, int64_t* decision_k, float* decision_F,
+                   int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions, float* F0_host);
+int ls_get_lr(const ls_handle* h, float* lr);
+
 /* Whole training run in native code: K local iterations cut into periods of
  * tau local steps, each followed by ls_average().  With interval > 0 the
  * period is re-chosen by adacomm_next_tau() at the first averaging point at or

@@ -219,6 +219,37 @@ def adacomm_next_tau(F_t: float, F_0: float, tau_0: int) -> int:
     return int(n)
 
 
+def adacomm_next_tau_refined(F_t: float, F_0: float, tau_0: int, tau_prev: int, gamma: float = 0.5,
+                             slack: int = 0, lr_0: float = 1.0, lr_l: float = 1.0, lr_changed: bool = False) -> int:
+    """The refinements of Section 4.3.
+
+    Candidate (Section 4.3.2, the lr-coupled strategy):
+        c = ceil( sqrt( (lr_0 / lr_l) * (F_t / F_0) ) * tau_0 ),  at least 1.
+    Faster decay when training saturates (Section 4.3.1, with the slack variable s):
+        tau_l = c                        if c + s < tau_{l-1}
+                gamma * tau_{l-1}        otherwise.
+    Readings taken where the paper is silent: gamma * tau_{l-1} is rounded up and kept at least 1;
+    the two rules are combined by using c as the candidate of the first; at the first decision after
+    the learning rate changed, c is taken as it is (the saturation test compares periods chosen under
+    the same learning rate, and Section 4.3.2 wants the period to grow when the rate drops).
+    """
+    F_t, F_0, gamma, lr_0, lr_l = float(F_t), float(F_0), float(gamma), float(lr_0), float(lr_l)
+    if not all(math.isfinite(v) for v in (F_t, F_0, gamma, lr_0, lr_l)):
+        raise ValueError("adacomm_next_tau_refined: invalid input")
+    if F_0 <= 0.0 or F_t < 0.0 or int(tau_0) < 1 or int(tau_prev) < 1 or not (0.0 < gamma <= 1.0) or int(slack) < 0 \
+            or lr_0 <= 0.0 or lr_l <= 0.0:
+        raise ValueError("adacomm_next_tau_refined: invalid input")
+    c = math.ceil(math.sqrt((lr_0 / lr_l) * (F_t / F_0)) * float(int(tau_0)))
+    if c < 1:
+        c = 1
+    if c > 2**31 - 1:
+        raise ValueError("adacomm_next_tau_refined: result does not fit an int")
+    if lr_changed or c + int(slack) < int(tau_prev):
+        return int(c)
+    n = math.ceil(gamma * float(int(tau_prev)))
+    return int(max(1, n))
+
+
 # --------------------------------------------------------------------------
 # PASGD loop  (Section 2, PASGD update rule; Section 4 for the interval scheme)
 # --------------------------------------------------------------------------
@@ -238,7 +269,7 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
               batch: int, lr: float, mu: float, tau: int,
               momentum_mode: str = MOMENTUM_AVERAGE,
               adacomm_interval: Optional[int] = None, probe_rows: int = 0,
-              state_hook=None) -> PasgdResult:
+              state_hook=None, refined: Optional[dict] = None) -> PasgdResult:
     """m workers start at the same x_1; each takes local mini-batch steps on its
     own batches; after every tau-th local step (counting from the start of the
     current period) the updated models are replaced by their mean.
@@ -259,6 +290,11 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
         dataset rows is evaluated and tau for the following periods is
         adacomm_next_tau(F_t, F_0, tau_0), where tau_0 = `tau` and F_0 is the
         same loss at x_1.  A period is never cut by an interval boundary.
+      * refined = {"gamma", "slack", "decay_at": [iterations], "decay_factor"} switches the decision
+        to adacomm_next_tau_refined (Section 4.3).  A learning-rate decay scheduled for iteration d
+        is applied at the first decision point with k >= d at which the period in force is 1
+        (Section 4.3.2: first let the period decay to 1, then decay the rate); one decay per
+        decision; the learning rate is kept in float32 as the worker state is.
     """
     K, m = row_offsets.shape
     P = spec.n_params
@@ -272,6 +308,9 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
     tau_0 = int(tau)
     cur_tau = int(tau)
     next_interval = 1
+    lr_0 = lr
+    pending = sorted(int(d) for d in refined.get("decay_at", [])) if refined is not None else []
+    lr_trace: List[Tuple[int, float]] = []
     if adacomm_interval is not None:
         F_0 = batch_loss(spec, xs[0], X[:probe_rows], y[:probe_rows])
     k = 0
@@ -301,10 +340,24 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
             state_hook(k, xs, vs, True)
         if adacomm_interval is not None and k >= next_interval * adacomm_interval:
             F_t = batch_loss(spec, xs[0], X[:probe_rows], y[:probe_rows])
+            if refined is not None:
+                changed = False
+                if pending and pending[0] <= k and cur_tau == 1:
+                    pending.pop(0)
+                    lr = float(np.float32(lr * float(refined.get("decay_factor", 0.1))))
+                    changed = True
+                    lr_trace.append((k, lr))
+                cur_tau = adacomm_next_tau_refined(F_t, F_0, tau_0, cur_tau, refined.get("gamma", 0.5),
+                                                   refined.get("slack", 0), lr_0, lr, changed)
+                F_trace.append((k, F_t, cur_tau))
+                next_interval = k // adacomm_interval + 1
+                continue
             cur_tau = adacomm_next_tau(F_t, F_0, tau_0)
             F_trace.append((k, F_t, cur_tau))
             next_interval = k // adacomm_interval + 1
-    return PasgdResult(xs, vs, losses, taus, avg_points, F_trace, F_0)
+    res = PasgdResult(xs, vs, losses, taus, avg_points, F_trace, F_0)
+    res.lr_trace = lr_trace
+    return res
 
 
 def tau_schedule_from_trace(F_0: float, tau_0: int, F_values: Sequence[float]) -> List[int]:

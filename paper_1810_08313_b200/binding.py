@@ -35,6 +35,11 @@ MOMENTUM_MODE = {"average": 0, "keep": 1, "reset": 2}
 KERNEL_CLASSES = ("fwd", "loss", "dx", "dw", "bias", "avg")
 
 
+class AdacommOpts(C.Structure):
+    _fields_ = [("gamma", C.c_double), ("slack", C.c_int32), ("n_decay", C.c_int32), ("decay_at", C.c_void_p),
+                ("decay_factor", C.c_double)]
+
+
 class ModelSpec(C.Structure):
     _fields_ = [
         ("n_layers", C.c_int32),
@@ -87,6 +92,11 @@ def _lib():
         "ls_run": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, vp, i64, P(i64), vp, vp, vp, i64, P(i64),
                              P(f32)]),
         "ls_launch_count": (C.c_int, [vp, P(i64)]),
+        "adacomm_next_tau_refined": (C.c_int, [C.c_double, C.c_double, C.c_int, C.c_int, C.c_double, C.c_int,
+                                               C.c_double, C.c_double, C.c_int]),
+        "ls_run_refined": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, P(AdacommOpts), vp, i64, P(i64), vp, vp,
+                                     vp, i64, P(i64), P(f32)]),
+        "ls_get_lr": (C.c_int, [vp, P(f32)]),
         "ls_linear_loss_static": (C.c_int, [vp, vp, vp, vp, i64, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]),
         "ls_profile_begin": (C.c_int, [vp, C.c_uint32, C.c_int]),
         "ls_profile_end": (C.c_int, [vp, P(C.c_double), P(i64)]),
@@ -141,6 +151,15 @@ def adacomm_next_tau(F_t: float, F_0: float, tau_0: int) -> int:
     r = _lib().adacomm_next_tau(float(F_t), float(F_0), int(tau_0))
     if r < 0:
         raise LsError(r, "adacomm_next_tau")
+    return r
+
+
+def adacomm_next_tau_refined(F_t: float, F_0: float, tau_0: int, tau_prev: int, gamma: float = 0.5, slack: int = 0,
+                             lr_0: float = 1.0, lr_l: float = 1.0, lr_changed: bool = False) -> int:
+    r = _lib().adacomm_next_tau_refined(float(F_t), float(F_0), int(tau_0), int(tau_prev), float(gamma), int(slack),
+                                        float(lr_0), float(lr_l), int(bool(lr_changed)))
+    if r < 0:
+        raise LsError(r, "adacomm_next_tau_refined")
     return r
 
 
@@ -334,6 +353,33 @@ class LocalSGD:
                 if cnt[ci * LS_MAX_LAYERS + l]:
                     out[(cname, l)] = (ms[ci * LS_MAX_LAYERS + l], cnt[ci * LS_MAX_LAYERS + l])
         return out
+
+    def run_refined(self, K: int, tau_0: int, row_offsets: np.ndarray, interval: int, probe_rows: int,
+                    gamma: float = 0.5, slack: int = 0, decay_at: Sequence[int] = (), decay_factor: float = 0.1,
+                    loss_out=None):
+        """ls_run_refined: AdaComm with the saturation decay and the learning-rate coupling (Section 4.3)."""
+        offs = np.ascontiguousarray(row_offsets, dtype=np.int64)
+        if offs.size != K * self.m:
+            raise ValueError("row_offsets must be [K][m]")
+        dec = np.ascontiguousarray(decay_at, dtype=np.int64)
+        opts = AdacommOpts(float(gamma), int(slack), int(dec.size), dec.ctypes.data if dec.size else None,
+                           float(decay_factor))
+        max_p = int(K) + 1
+        period_tau = np.zeros(max_p, dtype=np.int32)
+        dk = np.zeros(max_p, dtype=np.int64)
+        dF = np.zeros(max_p, dtype=np.float32)
+        dt = np.zeros(max_p, dtype=np.int32)
+        n_p, n_d, F0 = C.c_int64(), C.c_int64(), C.c_float()
+        lp = None if loss_out is None else loss_out.data_ptr()
+        _check(self.lib.ls_run_refined(self.h, int(K), int(tau_0), int(interval), int(probe_rows), offs.ctypes.data, lp,
+                                       C.byref(opts), period_tau.ctypes.data, max_p, C.byref(n_p), dk.ctypes.data,
+                                       dF.ctypes.data, dt.ctypes.data, max_p, C.byref(n_d), C.byref(F0)),
+               "ls_run_refined")
+        lr = C.c_float()
+        _check(self.lib.ls_get_lr(self.h, C.byref(lr)), "ls_get_lr")
+        n_p, n_d = n_p.value, n_d.value
+        return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
+                "decision_tau": dt[:n_d].tolist(), "F_0": float(F0.value), "lr": float(lr.value)}
 
     def launch_count(self) -> int:
         n = C.c_int64()

@@ -722,12 +722,59 @@ int adacomm_next_tau(double F_t, double F_0, int tau_0) {
   return (int)n;
 }
 
+int adacomm_next_tau_refined(double F_t, double F_0, int tau_0, int tau_prev, double gamma, int slack, double lr_0,
+                             double lr_l, int lr_changed) {
+  if (!isfinite(F_t) || !isfinite(F_0) || !isfinite(gamma) || !isfinite(lr_0) || !isfinite(lr_l)) return LS_ERR_INVALID_ARG;
+  if (!(F_0 > 0.0) || F_t < 0.0 || tau_0 < 1 || tau_prev < 1 || !(gamma > 0.0 && gamma <= 1.0) || slack < 0 ||
+      !(lr_0 > 0.0) || !(lr_l > 0.0))
+    return LS_ERR_INVALID_ARG;
+  const double scaled = (lr_0 / lr_l) * (F_t / F_0);
+  double c = ceil(sqrt(scaled) * (double)tau_0);
+  if (c < 1.0) c = 1.0;
+  if (!(c <= 2147483647.0)) return LS_ERR_OVERFLOW;
+  if (lr_changed || c + (double)slack < (double)tau_prev) return (int)c;
+  double n = ceil(gamma * (double)tau_prev);
+  if (n < 1.0) n = 1.0;
+  return (int)n;
+}
+
+static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
+                    float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
+                    float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions,
+                    float* F0_host, const ls_adacomm_opts* opts);
+
 int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
            float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
            float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions, float* F0_host) {
+  return run_loop(h, K, tau_0, interval, probe_rows, row_offset_host, loss_dev, period_tau, max_periods, n_periods,
+                  decision_k, decision_F, decision_tau, max_decisions, n_decisions, F0_host, nullptr);
+}
+
+int ls_run_refined(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
+                   const int64_t* row_offset_host, float* loss_dev, const ls_adacomm_opts* opts, int32_t* period_tau,
+                   int64_t max_periods, int64_t* n_periods, int64_t* decision_k, float* decision_F,
+                   int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions, float* F0_host) {
+  if (opts == nullptr || interval < 1) return LS_ERR_INVALID_ARG;
+  if (!isfinite(opts->gamma) || !(opts->gamma > 0.0 && opts->gamma <= 1.0) || opts->slack < 0 || opts->n_decay < 0 ||
+      (opts->n_decay > 0 && (opts->decay_at == nullptr || !isfinite(opts->decay_factor) || !(opts->decay_factor > 0.0))))
+    return LS_ERR_INVALID_ARG;
+  for (int i = 1; i < opts->n_decay; ++i)
+    if (opts->decay_at[i] < opts->decay_at[i - 1]) return LS_ERR_INVALID_ARG;
+  return run_loop(h, K, tau_0, interval, probe_rows, row_offset_host, loss_dev, period_tau, max_periods, n_periods,
+                  decision_k, decision_F, decision_tau, max_decisions, n_decisions, F0_host, opts);
+}
+
+}  // extern "C"
+
+static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
+                    float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
+                    float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions,
+                    float* F0_host, const ls_adacomm_opts* opts) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   if (K < 1 || tau_0 < 1 || interval < 0 || row_offset_host == nullptr) return LS_ERR_INVALID_ARG;
   const Layout& lay = h->lay;
+  const double lr_0 = (double)h->lr;
+  int next_decay = 0;
   float F_0 = 0.f;
   if (interval > 0) {
     int rc = eval_loss(h, 0, 0, probe_rows, &F_0);
@@ -749,7 +796,20 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
       float F_t = 0.f;
       rc = eval_loss(h, 0, 0, probe_rows, &F_t);
       if (rc != LS_OK) return rc;
-      const int t = adacomm_next_tau((double)F_t, (double)F_0, tau_0);
+      int t;
+      if (opts != nullptr) {
+        // Section 4.3: a scheduled learning-rate decay waits until the period in force is 1
+        int changed = 0;
+        if (next_decay < opts->n_decay && opts->decay_at[next_decay] <= k && tau == 1) {
+          ++next_decay;
+          h->lr = (float)((double)h->lr * opts->decay_factor);
+          changed = 1;
+        }
+        t = adacomm_next_tau_refined((double)F_t, (double)F_0, tau_0, tau, opts->gamma, opts->slack, lr_0, (double)h->lr,
+                                     changed);
+      } else {
+        t = adacomm_next_tau((double)F_t, (double)F_0, tau_0);
+      }
       if (t < 0) return t;
       tau = t;
       if (nd < max_decisions) {
@@ -763,6 +823,15 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
   }
   if (n_periods) *n_periods = np;
   if (n_decisions) *n_decisions = nd;
+  return LS_OK;
+}
+
+extern "C" {
+
+int ls_get_lr(const ls_handle* h, float* lr) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (lr == nullptr) return LS_ERR_INVALID_ARG;
+  *lr = h->lr;
   return LS_OK;
 }
 

@@ -76,3 +76,28 @@ def test_controller_agrees_with_oracle_on_a_dense_sweep():
     for _ in range(2000):
         F_0 = float(np.float32(rng.uniform(0.01, 5.0))); F_t = float(np.float32(rng.uniform(0.0, 6.0)))
         assert binding.adacomm_next_tau(F_t, F_0, 20) == orc.adacomm_next_tau(F_t, F_0, 20)
+
+
+def test_refined_controller_agrees_with_hand_table_and_oracle():
+    """Section 4.3 refinements: the library's rule equals the hand table and the oracle's on a dense sweep."""
+    import numpy as np
+    from oracle import localsgd_oracle as orc
+    from paper_1810_08313_b200 import binding
+    for line in open(os.path.join(ROOT, "tests", "golden", "adacomm_refined_table.txt")):
+        a = line.split("#")[0].split()
+        if len(a) == 10:
+            got = binding.adacomm_next_tau_refined(float(a[0]), float(a[1]), int(a[2]), int(a[3]), float(a[4]), int(a[5]),
+                                                   float(a[6]), float(a[7]), bool(int(a[8])))
+            assert got == int(a[9]), a
+    rng = np.random.default_rng(1)
+    for _ in range(5000):
+        args = (float(np.float32(rng.uniform(0, 4))), float(np.float32(rng.uniform(0.05, 4))), int(rng.integers(1, 100)),
+                int(rng.integers(1, 100)), float(rng.choice([0.25, 0.5, 0.9, 1.0])), int(rng.integers(0, 5)),
+                float(np.float32(0.2)), float(np.float32(0.2) * np.float32(rng.choice([1.0, 0.1, 0.01]))),
+                bool(rng.integers(0, 2)))
+        assert binding.adacomm_next_tau_refined(*args) == orc.adacomm_next_tau_refined(*args)
+    lib = binding._lib()
+    assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 20, 0.0, 0, 0.1, 0.1, 0) == binding.LS_ERR_INVALID_ARG
+    assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 0, 0.5, 0, 0.1, 0.1, 0) == binding.LS_ERR_INVALID_ARG
+    assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 20, 0.5, -1, 0.1, 0.1, 0) == binding.LS_ERR_INVALID_ARG
+    assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 20, 0.5, 0, 0.1, 0.0, 0) == binding.LS_ERR_INVALID_ARG

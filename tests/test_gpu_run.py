@@ -182,3 +182,36 @@ def test_least_squares_config_short():
     p, _ = eng.get_state(0)
     assert max_rel_err_per_tensor(p, ref.params[0], w.dims, w.has_bias) <= 1e-5
     eng.close()
+
+
+def test_refined_adacomm_run_with_deferred_lr_decay():
+    """Section 4.3: saturation decay (gamma = 1/2), lr-coupled candidate, lr decay deferred until tau = 1.
+    The native loop's decisions, learning rate and period list equal the oracle's."""
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, K, tau0, I, probe = (96, 64, 10), 4, 32, 120, 8, 10, 256
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 2048, 35)
+    offs = wl.batch_row_offsets(11, K, m, 2048, B)
+    refined = {"gamma": 0.5, "slack": 0, "decay_at": [30, 60], "decay_factor": 0.1}
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), 0.0, tau0, adacomm_interval=I, probe_rows=probe,
+                        refined=refined)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=0.0, batch=B); eng.bind_dataset(xd, yd); eng.set_params(x1)
+    out = eng.run_refined(K, tau0, offs, I, probe, gamma=0.5, slack=0, decay_at=[30, 60], decay_factor=0.1)
+    assert out["decision_k"] == [k for k, _, _ in ref.F_trace]
+    assert out["decision_tau"] == [t for _, _, t in ref.F_trace]
+    assert out["taus"] == ref.taus
+    for F, (_, Fr, _) in zip(out["decision_F"], ref.F_trace):
+        assert abs(float(F) - Fr) / Fr <= 1e-4
+    # the period reached 1, so at least one scheduled decay was applied, and only at decisions with tau == 1
+    assert len(ref.lr_trace) >= 1 and 1 in out["decision_tau"]
+    assert abs(out["lr"] - ref.lr_trace[-1][1]) <= 1e-12 * max(1.0, ref.lr_trace[-1][1]) or out["lr"] == f32(ref.lr_trace[-1][1])
+    # the decisions recomputed from the GPU's own logged losses are bit-exact
+    lr0, lr, prev, pending = f32(0.05), f32(0.05), tau0, [30, 60]
+    for k, F, t in zip(out["decision_k"], out["decision_F"], out["decision_tau"]):
+        changed = False
+        if pending and pending[0] <= k and prev == 1:
+            pending.pop(0); lr = float(np.float32(lr * 0.1)); changed = True
+        want = orc.adacomm_next_tau_refined(float(F), out["F_0"], tau0, prev, 0.5, 0, lr0, lr, changed)
+        assert t == want
+        prev = t
+    eng.close()

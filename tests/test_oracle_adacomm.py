@@ -59,3 +59,60 @@ def test_invalid_inputs_raise(args):
 def test_schedule_from_trace():
     F = [2.0, 1.0, 0.5, 0.125, 0.02]
     assert orc.tau_schedule_from_trace(2.0, 20, F) == [20, 15, 10, 5, 2]
+
+
+# ---- refinements of Section 4.3 -------------------------------------------------------------------
+
+GOLDEN_REFINED = os.path.join(os.path.dirname(__file__), "golden", "adacomm_refined_table.txt")
+
+
+def _refined_rows():
+    rows = []
+    with open(GOLDEN_REFINED) as f:
+        for line in f:
+            a = line.split("#")[0].split()
+            if len(a) == 10:
+                rows.append((float(a[0]), float(a[1]), int(a[2]), int(a[3]), float(a[4]), int(a[5]), float(a[6]),
+                             float(a[7]), bool(int(a[8])), int(a[9])))
+    return rows
+
+
+def test_refined_hand_table():
+    rows = _refined_rows()
+    assert len(rows) >= 10
+    for *args, want in rows:
+        assert orc.adacomm_next_tau_refined(*args) == want, args
+
+
+def test_refined_rule_properties():
+    import numpy as np
+    rng = np.random.default_rng(0)
+    for _ in range(2000):
+        F_0 = float(rng.uniform(0.1, 3)); F_t = float(rng.uniform(0, 3)); tau_0 = int(rng.integers(1, 64))
+        prev = int(rng.integers(1, 64)); gamma = float(rng.choice([0.25, 0.5, 0.75, 1.0])); s = int(rng.integers(0, 4))
+        t = orc.adacomm_next_tau_refined(F_t, F_0, tau_0, prev, gamma, s)
+        basic = orc.adacomm_next_tau(F_t, F_0, tau_0)
+        assert t >= 1
+        # with equal learning rates the candidate is the basic rule's value
+        if basic + s < prev:
+            assert t == basic
+        else:
+            assert t == max(1, math.ceil(gamma * prev)) and t <= prev        # never grows without an lr change
+    # a sequence of saturated decisions halves the period down to 1 and stays there
+    t, seq = 20, []
+    for _ in range(7):
+        t = orc.adacomm_next_tau_refined(5.0, 1.0, 20, t, 0.5, 0)
+        seq.append(t)
+    assert seq == [10, 5, 3, 2, 1, 1, 1]
+    # the lr-coupled candidate scales with sqrt(lr_0 / lr_l), not with its 3/2 power
+    assert orc.adacomm_next_tau_refined(1.0, 1.0, 10, 1000, 0.5, 0, 1.0, 0.25, True) == 20
+    assert orc.adacomm_next_tau_refined(1.0, 1.0, 10, 1000, 0.5, 0, 1.0, 0.0625, True) == 40
+
+
+@pytest.mark.parametrize("kw", [dict(gamma=0.0), dict(gamma=1.5), dict(slack=-1), dict(lr_l=0.0), dict(tau_prev=0),
+                                dict(lr_0=float("nan"))])
+def test_refined_invalid_inputs(kw):
+    args = dict(F_t=1.0, F_0=1.0, tau_0=20, tau_prev=20, gamma=0.5, slack=0, lr_0=0.1, lr_l=0.1)
+    args.update(kw)
+    with pytest.raises(ValueError):
+        orc.adacomm_next_tau_refined(**args)

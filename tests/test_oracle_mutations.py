@@ -121,3 +121,26 @@ def test_controller_mistakes_are_caught(monkeypatch):
     assert _fails(pins_tau.test_result_is_the_smallest_integer_not_below)
     monkeypatch.setattr(orc, "adacomm_next_tau", lambda F_t, F_0, tau_0: math.ceil(math.sqrt(F_t / F_0) * tau_0))   # no clamp
     assert _fails(pins_tau.test_hand_table)
+
+
+def test_refined_controller_mistakes_are_caught(monkeypatch):
+    real = orc.adacomm_next_tau_refined
+
+    def cube_power(F_t, F_0, tau_0, tau_prev, gamma=0.5, slack=0, lr_0=1.0, lr_l=1.0, lr_changed=False):
+        # the (lr_0/lr_l)^{3/2} form that Section 4.3.2 reports as diverging
+        return real(F_t * (lr_0 / lr_l) ** 2, F_0, tau_0, tau_prev, gamma, slack, lr_0, lr_l, lr_changed)
+    monkeypatch.setattr(orc, "adacomm_next_tau_refined", cube_power)
+    assert _fails(pins_tau.test_refined_hand_table)
+    assert _fails(pins_tau.test_refined_rule_properties)
+
+    def not_strict(F_t, F_0, tau_0, tau_prev, gamma=0.5, slack=0, lr_0=1.0, lr_l=1.0, lr_changed=False):
+        c = orc.adacomm_next_tau(F_t * lr_0 / lr_l, F_0, tau_0)
+        return c if (lr_changed or c + slack <= tau_prev) else max(1, math.ceil(gamma * tau_prev))   # <= instead of <
+    monkeypatch.setattr(orc, "adacomm_next_tau_refined", not_strict)
+    assert _fails(pins_tau.test_refined_hand_table)
+
+    def floor_gamma(F_t, F_0, tau_0, tau_prev, gamma=0.5, slack=0, lr_0=1.0, lr_l=1.0, lr_changed=False):
+        c = orc.adacomm_next_tau(F_t * lr_0 / lr_l, F_0, tau_0)
+        return c if (lr_changed or c + slack < tau_prev) else max(1, math.floor(gamma * tau_prev))
+    monkeypatch.setattr(orc, "adacomm_next_tau_refined", floor_gamma)
+    assert _fails(pins_tau.test_refined_hand_table)
