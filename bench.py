@@ -342,7 +342,7 @@ def run_reference(args, w: wl.Workload):
 def run_ours(args, w: wl.Workload):
     import torch
     import torch.distributed as dist
-    from paper_1810_08313_b200.binding import LocalSGD, adacomm_next_tau, average_flat
+    from paper_1810_08313_b200.binding import LocalSGD, adacomm_next_tau, average_flat, block_average_flat
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -483,6 +483,28 @@ def run_ours(args, w: wl.Workload):
                 gbs = 2 * 8.0 * mm * P * reps / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9
                 avg[f"P{P}_m{mm}"] = {"GB/s": round(gbs, 1), "frac_measured_peak": round(gbs / peaks["hbm_gbs"], 4),
                                       "frac_8TBs": round(gbs / 8000.0, 4)}
+            # the same pass with block momentum (Section 5.3): + period-start model and global buffer,
+            # 8m + 16 bytes per parameter
+            if P < 10 ** 8:
+                anc = torch.zeros(2, stride, device="cuda", dtype=torch.float32)
+                ub = torch.zeros(2, stride, device="cuda", dtype=torch.float32)
+                for mm in (4, 16):
+                    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                    def both():
+                        block_average_flat(buf[:mm].view(-1), anc[0], ub[0], mm, P, 0.05, 0.3, stride)
+                        block_average_flat(buf[16:16 + mm].view(-1), anc[1], ub[1], mm, P, 0.05, 0.3, stride)
+                    for _ in range(3):
+                        both()
+                    ev[0].record()
+                    for _ in range(10):
+                        both()
+                    ev[1].record()
+                    torch.cuda.synchronize()
+                    gbs = 2 * (8.0 * mm + 16.0) * P * 10 / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9
+                    avg[f"block_P{P}_m{mm}"] = {"GB/s": round(gbs, 1),
+                                                "frac_measured_peak": round(gbs / peaks["hbm_gbs"], 4),
+                                                "frac_8TBs": round(gbs / 8000.0, 4)}
+                del anc, ub
             del buf
         line["averaging_gbs"] = avg
 

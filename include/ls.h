@@ -66,8 +66,15 @@ enum { LS_GEMM_FP32 = 0, LS_GEMM_BF16 = 1 };
  * AVERAGE: replaced by their mean like the parameters (makes tau = 1 equal to
  *          synchronous momentum SGD on the m-fold batch).
  * KEEP:    left alone (the independent-buffer scheme of Section 5.3).
- * RESET:   cleared (the local half of the block-momentum scheme, Section 5.3). */
-enum { LS_MOMENTUM_AVERAGE = 0, LS_MOMENTUM_KEEP = 1, LS_MOMENTUM_RESET = 2 };
+ * RESET:   cleared (the local half of the block-momentum scheme, Section 5.3).
+ * BLOCK:   block momentum (Section 5.3): local buffers cleared, and the averaging step
+ *          applies a global momentum buffer u to the period's accumulated step:
+ *            u_j = beta_glob u_{j-1} + G_j,   x_{(j+1)tau+1} = x_{j tau+1} - eta u_j,
+ *          with x_{j tau+1} the synchronized model the period started from and
+ *          G_j = (x_{j tau+1} - mean_i x^(i)) / eta the averaged displacement in gradient units
+ *          (the sum of the averaged gradients when the local steps are plain SGD).
+ *          beta_glob is spec.block_momentum; see ls_average for the exact arithmetic. */
+enum { LS_MOMENTUM_AVERAGE = 0, LS_MOMENTUM_KEEP = 1, LS_MOMENTUM_RESET = 2, LS_MOMENTUM_BLOCK = 3 };
 
 typedef struct ls_model_spec {
   int32_t n_layers;                  /* L, 1..LS_MAX_LAYERS */
@@ -77,6 +84,7 @@ typedef struct ls_model_spec {
   int32_t gemm_dtype;                /* LS_GEMM_*: input type of the matrix products (accumulation is fp32) */
   int32_t momentum_mode;             /* LS_MOMENTUM_* */
   float weight_decay;                /* must be 0 */
+  float block_momentum;              /* beta_glob of Section 5.3, 0 <= beta < 1; read only in LS_MOMENTUM_BLOCK */
 } ls_model_spec;
 
 typedef struct ls_handle ls_handle;
@@ -159,8 +167,26 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
  * mean over replicas; momentum buffers follow spec.momentum_mode.
  * The mean is defined to the bit: s = x^(0); s = s + x^(j) for j = 1..m-1 in
  * fp32, then one fp32 division by (float)m.  Afterwards all replicas are
- * bitwise equal. */
+ * bitwise equal.
+ * LS_MOMENTUM_BLOCK: with `mean` as above, a the model the period started from
+ * and u the global buffer (both kept in the state block, a = x_1 and u = 0 after
+ * ls_set_params), in fp32 with every operation rounded on its own:
+ *   d = a - mean;  G = d / lr;  u' = beta*u + G;  x' = a - lr*u'
+ * x' replaces every replica's parameters and a, u' replaces u, the local
+ * momentum buffers are cleared.  lr is the rate in force when ls_average runs. */
 int ls_average(ls_handle* h);
+
+/* Block-momentum state of a LS_MOMENTUM_BLOCK handle in the flat interface layout
+ * (P floats each): the period-start model and the global buffer.  Either pointer
+ * may be NULL.  Host memory; synchronous.  LS_ERR_UNSUPPORTED in other modes. */
+int ls_set_block_state(ls_handle* h, const float* anchor_host, const float* u_host);
+int ls_get_block_state(ls_handle* h, float* anchor_host, float* u_host);
+
+/* The block-momentum averaging kernel on raw buffers: buf_dev as for
+ * ls_average_flat, anchor_dev and u_dev vectors of P floats (device), lr > 0,
+ * beta >= 0.  Same arithmetic as ls_average in LS_MOMENTUM_BLOCK. */
+int ls_block_average_flat(float* buf_dev, float* anchor_dev, float* u_dev, int m, int64_t P, int64_t stride,
+                          float lr, float beta, void* cuda_stream);
 
 /* The averaging kernel on a raw buffer: m vectors of P floats, vector j
  * starting at buf_dev + j*stride floats (stride >= P).  Same arithmetic as

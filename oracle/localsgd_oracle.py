@@ -40,6 +40,7 @@ LOSS_MSE_HALF = "mse_half"
 MOMENTUM_AVERAGE = "average"   # buffers are averaged with the parameters
 MOMENTUM_KEEP = "keep"         # each worker keeps its own buffer (the paper's "naive" scheme)
 MOMENTUM_RESET = "reset"       # buffers cleared at every period start (local half of block momentum)
+MOMENTUM_BLOCK = "block"       # block momentum: reset local buffers + a global momentum on the period's step
 
 
 @dataclass(frozen=True)
@@ -195,6 +196,37 @@ def average_replicas(X: np.ndarray) -> None:
     X[:] = mean[None, :]
 
 
+def block_momentum_average(X: np.ndarray, anchor: np.ndarray, u: np.ndarray, lr: float, beta: float) -> None:
+    """Averaging step with block momentum (Section 5.3):
+        u_j = beta_glob * u_{j-1} + G_j ;   x_{(j+1)tau+1} = x_{j tau+1} - eta_j * u_j
+    where x_{j tau+1} is the synchronized model the period started from (`anchor`) and G_j is the
+    accumulated step of the period in gradient units.  Reading: G_j = (anchor - mean_i x^(i)) / eta, the
+    averaged displacement divided by the learning rate; this equals the paper's sum of averaged
+    gradients exactly when the local steps are plain SGD, and is the accumulated "big step" between
+    two synchronized models otherwise.
+    Specified to the bit in fp32, every operation rounded separately (no fused multiply-add):
+        mean as in average_replicas;  d = anchor - mean;  G = d / eta;  t = beta * u;  u' = t + G;
+        s = eta * u';  x' = anchor - s.   X rows, anchor <- x';  u <- u'.   In place.
+    """
+    if X.dtype != np.float32 or anchor.dtype != np.float32 or u.dtype != np.float32:
+        raise TypeError("block_momentum_average is specified on float32 state")
+    m = X.shape[0]
+    s = X[0].copy()
+    for j in range(1, m):
+        s = s + X[j]
+    mean = s / np.float32(m)
+    eta, b = np.float32(lr), np.float32(beta)
+    d = anchor - mean
+    G = d / eta
+    t = b * u
+    u_new = t + G
+    step = eta * u_new
+    x_new = anchor - step
+    X[:] = x_new[None, :]
+    anchor[:] = x_new
+    u[:] = u_new
+
+
 # --------------------------------------------------------------------------
 # AdaComm  (Section 4.2, basic update rule)
 # --------------------------------------------------------------------------
@@ -269,7 +301,7 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
               batch: int, lr: float, mu: float, tau: int,
               momentum_mode: str = MOMENTUM_AVERAGE,
               adacomm_interval: Optional[int] = None, probe_rows: int = 0,
-              state_hook=None, refined: Optional[dict] = None) -> PasgdResult:
+              state_hook=None, refined: Optional[dict] = None, block_beta: float = 0.0) -> PasgdResult:
     """m workers start at the same x_1; each takes local mini-batch steps on its
     own batches; after every tau-th local step (counting from the start of the
     current period) the updated models are replaced by their mean.
@@ -290,6 +322,8 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
         dataset rows is evaluated and tau for the following periods is
         adacomm_next_tau(F_t, F_0, tau_0), where tau_0 = `tau` and F_0 is the
         same loss at x_1.  A period is never cut by an interval boundary.
+      * momentum_mode "block" (Section 5.3): the averaging step is block_momentum_average with factor
+        `block_beta` on the model the period started from, and the local buffers restart from zero.
       * refined = {"gamma", "slack", "decay_at": [iterations], "decay_factor"} switches the decision
         to adacomm_next_tau_refined (Section 4.3).  A learning-rate decay scheduled for iteration d
         is applied at the first decision point with k >= d at which the period in force is 1
@@ -300,6 +334,8 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
     P = spec.n_params
     xs = np.repeat(np.asarray(x1, dtype=np.float32)[None, :], m, axis=0).copy()
     vs = np.zeros((m, P), dtype=np.float32)
+    anchor = np.asarray(x1, dtype=np.float32).copy()       # synchronized model at the period start
+    u_glob = np.zeros(P, dtype=np.float32)                  # global block-momentum buffer
     losses = np.zeros((K, m), dtype=np.float64)
     taus: List[int] = []
     avg_points: List[int] = []
@@ -328,13 +364,18 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
             k += 1
             if state_hook is not None:
                 state_hook(k, xs, vs, False)
-        average_replicas(xs)
-        if momentum_mode == MOMENTUM_AVERAGE:
-            average_replicas(vs)
-        elif momentum_mode == MOMENTUM_RESET:
+        if momentum_mode == MOMENTUM_BLOCK:
+            # Section 5.3: global momentum on the period's accumulated step, local buffers restart
+            block_momentum_average(xs, anchor, u_glob, lr, block_beta)
             vs[:] = 0
-        elif momentum_mode != MOMENTUM_KEEP:
-            raise ValueError(momentum_mode)
+        else:
+            average_replicas(xs)
+            if momentum_mode == MOMENTUM_AVERAGE:
+                average_replicas(vs)
+            elif momentum_mode == MOMENTUM_RESET:
+                vs[:] = 0
+            elif momentum_mode != MOMENTUM_KEEP:
+                raise ValueError(momentum_mode)
         avg_points.append(k)
         if state_hook is not None:
             state_hook(k, xs, vs, True)
@@ -357,6 +398,7 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
             next_interval = k // adacomm_interval + 1
     res = PasgdResult(xs, vs, losses, taus, avg_points, F_trace, F_0)
     res.lr_trace = lr_trace
+    res.block_u = u_glob
     return res
 
 

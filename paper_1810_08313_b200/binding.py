@@ -31,7 +31,7 @@ LS_ERR_TOO_LARGE = -10
 
 LOSS = {"softmax_ce": 0, "mse_half": 1}
 GEMM = {"fp32": 0, "bf16": 1}
-MOMENTUM_MODE = {"average": 0, "keep": 1, "reset": 2}
+MOMENTUM_MODE = {"average": 0, "keep": 1, "reset": 2, "block": 3}
 KERNEL_CLASSES = ("fwd", "loss", "dx", "dw", "bias", "avg")
 
 
@@ -49,6 +49,7 @@ class ModelSpec(C.Structure):
         ("gemm_dtype", C.c_int32),
         ("momentum_mode", C.c_int32),
         ("weight_decay", C.c_float),
+        ("block_momentum", C.c_float),
     ]
 
 
@@ -87,6 +88,9 @@ def _lib():
         "ls_local_steps_host": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "ls_average": (C.c_int, [vp]),
         "ls_average_flat": (C.c_int, [vp, C.c_int, i64, i64, vp]),
+        "ls_block_average_flat": (C.c_int, [vp, vp, vp, C.c_int, i64, i64, C.c_float, C.c_float, vp]),
+        "ls_set_block_state": (C.c_int, [vp, vp, vp]),
+        "ls_get_block_state": (C.c_int, [vp, vp, vp]),
         "ls_eval_loss": (C.c_int, [vp, C.c_int, i64, i64, P(f32)]),
         "adacomm_next_tau": (C.c_int, [C.c_double, C.c_double, C.c_int]),
         "ls_run": (C.c_int, [vp, i64, C.c_int, C.c_int, i64, vp, vp, vp, i64, P(i64), vp, vp, vp, i64, P(i64),
@@ -120,7 +124,7 @@ def _check(code: int, where: str):
 
 
 def make_spec(dims: Sequence[int], loss: str = "softmax_ce", has_bias: bool = True, gemm_dtype: str = "fp32",
-              momentum_mode: str = "average", weight_decay: float = 0.0) -> ModelSpec:
+              momentum_mode: str = "average", weight_decay: float = 0.0, block_momentum: float = 0.0) -> ModelSpec:
     s = ModelSpec()
     if not (2 <= len(dims) <= LS_MAX_LAYERS + 1):
         raise ValueError("1..8 layers")
@@ -132,6 +136,7 @@ def make_spec(dims: Sequence[int], loss: str = "softmax_ce", has_bias: bool = Tr
     s.gemm_dtype = GEMM[gemm_dtype]
     s.momentum_mode = MOMENTUM_MODE[momentum_mode]
     s.weight_decay = float(weight_decay)
+    s.block_momentum = float(block_momentum)
     return s
 
 
@@ -181,6 +186,21 @@ def average_flat(buf, m: int, P: int, stride: Optional[int] = None, stream=None)
     _check(_lib().ls_average_flat(buf.data_ptr(), int(m), int(P), stride, _stream_ptr(stream)), "ls_average_flat")
 
 
+def block_average_flat(buf, anchor, u, m: int, P: int, lr: float, beta: float, stride: Optional[int] = None,
+                       stream=None) -> None:
+    """Block-momentum averaging step (Section 5.3) on raw CUDA tensors: buf as for average_flat, anchor and u
+    float32 vectors of P elements (the period-start model and the global buffer), all updated in place."""
+    import torch
+    for t in (buf, anchor, u):
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise ValueError("contiguous float32 CUDA tensors expected")
+    stride = int(P if stride is None else stride)
+    if buf.numel() < (m - 1) * stride + P or anchor.numel() < P or u.numel() < P:
+        raise ValueError("buffer too small")
+    _check(_lib().ls_block_average_flat(buf.data_ptr(), anchor.data_ptr(), u.data_ptr(), int(m), int(P), stride,
+                                        float(lr), float(beta), _stream_ptr(stream)), "ls_block_average_flat")
+
+
 def linear_loss_static(W, bias, x, y, chunk_rows: int, chunk_loss, loss: str = "softmax_ce", stream=None) -> None:
     """Per-chunk mean loss of z = W x + b on the rows of x, computed by the library without allocating
     any memory (its scratch is a fixed array inside the library).  W [d_out][d_in], bias [d_out] or None,
@@ -198,14 +218,14 @@ class LocalSGD:
 
     def __init__(self, m: int, dims: Sequence[int], loss: str = "softmax_ce", has_bias: bool = True,
                  gemm_dtype: str = "fp32", lr: float = 0.05, momentum: float = 0.0, batch: int = 32,
-                 momentum_mode: str = "average", device: str = "cuda:0", stream=None):
+                 momentum_mode: str = "average", device: str = "cuda:0", stream=None, block_momentum: float = 0.0):
         import torch
         self._torch = torch
         self.lib = _lib()
         self.m, self.batch, self.dims = int(m), int(batch), tuple(int(d) for d in dims)
         self.gemm_dtype = gemm_dtype
         self.loss_kind = loss
-        self.spec = make_spec(dims, loss, has_bias, gemm_dtype, momentum_mode)
+        self.spec = make_spec(dims, loss, has_bias, gemm_dtype, momentum_mode, block_momentum=block_momentum)
         self.P = param_count(self.spec)
         nbytes = state_bytes(self.m, self.spec, self.batch)
         self.device = torch.device(device)
@@ -253,6 +273,21 @@ class LocalSGD:
                 raise ValueError("wrong size")
         _check(self.lib.ls_set_state(self.h, int(replica), None if p is None else p.ctypes.data,
                                      None if v is None else v.ctypes.data), "ls_set_state")
+
+    def set_block_state(self, anchor: Optional[np.ndarray] = None, u: Optional[np.ndarray] = None):
+        a = None if anchor is None else np.ascontiguousarray(anchor, dtype=np.float32)
+        b = None if u is None else np.ascontiguousarray(u, dtype=np.float32)
+        for t in (a, b):
+            if t is not None and t.size != self.P:
+                raise ValueError("wrong size")
+        _check(self.lib.ls_set_block_state(self.h, None if a is None else a.ctypes.data,
+                                           None if b is None else b.ctypes.data), "ls_set_block_state")
+
+    def get_block_state(self):
+        a = np.empty(self.P, dtype=np.float32)
+        b = np.empty(self.P, dtype=np.float32)
+        _check(self.lib.ls_get_block_state(self.h, a.ctypes.data, b.ctypes.data), "ls_get_block_state")
+        return a, b
 
     def get_state(self, replica: int):
         p = np.empty(self.P, dtype=np.float32)

@@ -12,6 +12,12 @@
 // Algorithmic traffic is 8*m bytes per parameter: each element is read once and
 // written once.  No shared memory, no inter-thread communication: the reduction
 // order is fixed by construction, so the result is bit-reproducible.
+//
+// Block momentum (Section 5.3) is the same pass with two more streams: the model
+// the period started from (anchor) and the global buffer u.  With mean the average
+// above, d = anchor - mean, G = d / eta, u' = beta*u + G, x' = anchor - eta*u', every
+// operation rounded separately; x' goes to all replicas and the anchor, u' to u.
+// Traffic grows from 8m to 8m + 16 bytes per parameter.
 #include "ls_internal.h"
 
 namespace ls {
@@ -63,16 +69,21 @@ __device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&v)[W]
 // M == 0: any m, processed in chunks of 8 replicas, still in replica order.
 // W: floats per thread (8 or 4).  Plain IEEE adds and one IEEE division: there is no
 // multiply nearby, so nothing can be contracted into an FMA.
-template <int M, int W>
+// BM: block momentum; bm.anchor / bm.u are single vectors laid out like one replica.
+template <int M, int W, bool BM>
 __global__ void __launch_bounds__(kThreads)
 average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
-               __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
+               __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo, BlockMomentum bm) {
   const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (i >= n_vec) return;
   const int m = M > 0 ? M : m_rt;
   float* p = base + (int64_t)blockIdx.y * buf_stride + i * W;
   const float mf = (float)m;
-  Vec<W> s;
+  Vec<W> s, anc, ug;
+  if constexpr (BM) {
+    anc.load(bm.anchor + i * W);
+    ug.load(bm.u + i * W);
+  }
   if (M > 0) {
     Vec<W> v[M > 0 ? M : 1];
 #pragma unroll
@@ -98,6 +109,18 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
   }
 #pragma unroll
   for (int e = 0; e < W; ++e) s.v[e] = __fdiv_rn(s.v[e], mf);
+  if constexpr (BM) {
+#pragma unroll
+    for (int e = 0; e < W; ++e) {
+      const float d = __fsub_rn(anc.v[e], s.v[e]);
+      const float G = __fdiv_rn(d, bm.lr);
+      const float un = __fadd_rn(__fmul_rn(bm.beta, ug.v[e]), G);
+      ug.v[e] = un;
+      s.v[e] = __fsub_rn(anc.v[e], __fmul_rn(bm.lr, un));
+    }
+    ug.store(bm.u + i * W);
+    s.store(bm.anchor + i * W);
+  }
 #pragma unroll 4
   for (int j = 0; j < m; ++j) s.store(p + (int64_t)j * stride);
   if (blockIdx.y == 0) {
@@ -116,14 +139,22 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
 // 16-byte aligned.  Same arithmetic, one element per thread.
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
-                      __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo) {
+                      __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo, BlockMomentum bm) {
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
   const float mf = (float)m;
   const int64_t i = first + (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (i >= n) return;
   float s = buf[i];
   for (int j = 1; j < m; ++j) s = __fadd_rn(s, buf[(int64_t)j * stride + i]);
-  const float mean = __fdiv_rn(s, mf);
+  float mean = __fdiv_rn(s, mf);
+  if (bm.anchor != nullptr) {
+    const float a = bm.anchor[i];
+    const float G = __fdiv_rn(__fsub_rn(a, mean), bm.lr);
+    const float un = __fadd_rn(__fmul_rn(bm.beta, bm.u[i]), G);
+    bm.u[i] = un;
+    mean = __fsub_rn(a, __fmul_rn(bm.lr, un));
+    bm.anchor[i] = mean;
+  }
   for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
   if (blockIdx.y == 0) {
     if (shadow != nullptr)
@@ -133,16 +164,18 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
   }
 }
 
-template <int W>
+template <int W, bool BM>
 void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
-                __nv_bfloat16* shadow, float* lo) {
+                __nv_bfloat16* shadow, float* lo, const BlockMomentum& bm) {
+#define LS_AVG(M) average_kernel<M, W, BM><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo, bm)
   switch (m) {
-    case 2: average_kernel<2, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
-    case 4: average_kernel<4, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
-    case 8: average_kernel<8, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
-    case 16: average_kernel<16, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
-    default: average_kernel<0, W><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo); break;
+    case 2: LS_AVG(2); break;
+    case 4: LS_AVG(4); break;
+    case 8: LS_AVG(8); break;
+    case 16: LS_AVG(16); break;
+    default: LS_AVG(0); break;
   }
+#undef LS_AVG
 }
 
 inline bool aligned_to(const void* p, size_t a) { return p == nullptr || reinterpret_cast<uintptr_t>(p) % a == 0; }
@@ -150,21 +183,34 @@ inline bool aligned_to(const void* p, size_t a) { return p == nullptr || reinter
 }  // namespace
 
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches) {
+                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches, const BlockMomentum* bmp) {
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
+  BlockMomentum bm{nullptr, nullptr, 0.f, 0.f};
+  if (bmp != nullptr) {
+    if (n_buf != 1 || bmp->anchor == nullptr || bmp->u == nullptr) return cudaErrorInvalidValue;
+    bm = *bmp;
+  }
+  const bool BM = bm.anchor != nullptr;
   // widest slice the addresses allow: 8 floats (32-byte aligned), 4 floats (16-byte), else scalar
   int W = 0;
-  if (aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 && aligned_to(shadow, 16) && aligned_to(lo, 32))
+  if (aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 && aligned_to(shadow, 16) && aligned_to(lo, 32) &&
+      aligned_to(bm.anchor, 32) && aligned_to(bm.u, 32))
     W = 8;
-  else if (aligned_to(base, 16) && stride % 4 == 0 && buf_stride % 4 == 0 && aligned_to(shadow, 8) && aligned_to(lo, 16))
+  else if (aligned_to(base, 16) && stride % 4 == 0 && buf_stride % 4 == 0 && aligned_to(shadow, 8) &&
+           aligned_to(lo, 16) && aligned_to(bm.anchor, 16) && aligned_to(bm.u, 16))
     W = 4;
   const int64_t n_vec = W ? n / W : 0;
   if (n_vec > 0) {
     const int64_t gx = (n_vec + kThreads - 1) / kThreads;
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    if (W == 8) launch_vec<8>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo);
-    else launch_vec<4>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo);
+    if (W == 8) {
+      if (BM) launch_vec<8, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+      else launch_vec<8, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+    } else {
+      if (BM) launch_vec<4, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+      else launch_vec<4, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+    }
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -174,7 +220,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     const int64_t gx = (n - first + kThreads - 1) / kThreads;
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, lo);
+    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, lo, bm);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -188,6 +234,20 @@ extern "C" int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride,
   if (buf_dev == nullptr || m < 1 || P < 0 || stride < P) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(buf_dev) % 4 != 0) return LS_ERR_INVALID_ARG;
   int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
-                             nullptr);
+                             nullptr, nullptr);
+  return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
+extern "C" int ls_block_average_flat(float* buf_dev, float* anchor_dev, float* u_dev, int m, int64_t P, int64_t stride,
+                                     float lr, float beta, void* cuda_stream) {
+  if (buf_dev == nullptr || anchor_dev == nullptr || u_dev == nullptr || m < 1 || P < 0 || stride < P)
+    return LS_ERR_INVALID_ARG;
+  if (!(lr > 0.f) || !isfinite(lr) || !(beta >= 0.f) || !isfinite(beta)) return LS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(buf_dev) % 4 != 0 || reinterpret_cast<uintptr_t>(anchor_dev) % 4 != 0 ||
+      reinterpret_cast<uintptr_t>(u_dev) % 4 != 0)
+    return LS_ERR_INVALID_ARG;
+  ls::BlockMomentum bm{anchor_dev, u_dev, lr, beta};
+  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
+                             nullptr, &bm);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

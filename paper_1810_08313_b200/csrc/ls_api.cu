@@ -25,7 +25,9 @@ static int check_spec(const ls_model_spec* s) {
   if (s->loss == LS_LOSS_MSE_HALF && s->dims[s->n_layers] != 1) return LS_ERR_INVALID_ARG;
   if (s->has_bias != 0 && s->has_bias != 1) return LS_ERR_INVALID_ARG;
   if (s->gemm_dtype != LS_GEMM_FP32 && s->gemm_dtype != LS_GEMM_BF16) return LS_ERR_INVALID_ARG;
-  if (s->momentum_mode < LS_MOMENTUM_AVERAGE || s->momentum_mode > LS_MOMENTUM_RESET) return LS_ERR_INVALID_ARG;
+  if (s->momentum_mode < LS_MOMENTUM_AVERAGE || s->momentum_mode > LS_MOMENTUM_BLOCK) return LS_ERR_INVALID_ARG;
+  if (s->momentum_mode == LS_MOMENTUM_BLOCK && !(s->block_momentum >= 0.f && s->block_momentum < 1.f))
+    return LS_ERR_INVALID_ARG;
   if (!(s->weight_decay == 0.0f)) return isfinite(s->weight_decay) ? LS_ERR_UNSUPPORTED : LS_ERR_INVALID_ARG;
   return LS_OK;
 }
@@ -87,6 +89,10 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   }
   lay.stage_loss_off = take((size_t)kRowOffCap * m * 4);
   lay.err_off = take(256);
+  if (spec->momentum_mode == LS_MOMENTUM_BLOCK) {
+    lay.anchor_off = take((size_t)lay.stride * 4);
+    lay.blocku_off = take((size_t)lay.stride * 4);
+  }
   lay.total = off;
   *out = lay;
   return LS_OK;
@@ -353,12 +359,14 @@ static int average(ls_handle* h) {
   const Layout& lay = h->lay;
   const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
   const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
+  const bool block = h->spec.momentum_mode == LS_MOMENTUM_BLOCK;
   {
     ProfScope ps(h, LS_K_AVG, 0);
+    BlockMomentum bm{anchor_of(h), blocku_of(h), h->lr, h->spec.block_momentum};
     LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                              shadow_of(h), wlo_of(h), h->stream, &h->launches));
+                              shadow_of(h), wlo_of(h), h->stream, &h->launches, block ? &bm : nullptr));
   }
-  if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
+  if (h->mu != 0.f && (h->spec.momentum_mode == LS_MOMENTUM_RESET || block))
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
   return LS_OK;
 }
@@ -602,7 +610,32 @@ int ls_set_params(ls_handle* h, const float* x1_host) {
     LS_CUDA(h, cudaMemcpyAsync(params_of(h) + (int64_t)i * lay.stride, params_of(h), (size_t)lay.stride * 4,
                                cudaMemcpyDeviceToDevice, h->stream));
   LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  if (h->spec.momentum_mode == LS_MOMENTUM_BLOCK) {
+    LS_CUDA(h, cudaMemcpyAsync(anchor_of(h), params_of(h), (size_t)lay.stride * 4, cudaMemcpyDeviceToDevice,
+                               h->stream));
+    LS_CUDA(h, cudaMemsetAsync(blocku_of(h), 0, (size_t)lay.stride * 4, h->stream));
+  }
   rc = refresh_shadow(h);
+  if (rc != LS_OK) return rc;
+  return ls_sync(h);
+}
+
+int ls_set_block_state(ls_handle* h, const float* anchor_host, const float* u_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (h->spec.momentum_mode != LS_MOMENTUM_BLOCK) return LS_ERR_UNSUPPORTED;
+  int rc = LS_OK;
+  if (anchor_host) rc = copy_replica(h, anchor_of(h), const_cast<float*>(anchor_host), true);
+  if (rc == LS_OK && u_host) rc = copy_replica(h, blocku_of(h), const_cast<float*>(u_host), true);
+  if (rc != LS_OK) return rc;
+  return ls_sync(h);
+}
+
+int ls_get_block_state(ls_handle* h, float* anchor_host, float* u_host) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (h->spec.momentum_mode != LS_MOMENTUM_BLOCK) return LS_ERR_UNSUPPORTED;
+  int rc = LS_OK;
+  if (anchor_host) rc = copy_replica(h, anchor_of(h), anchor_host, false);
+  if (rc == LS_OK && u_host) rc = copy_replica(h, blocku_of(h), u_host, false);
   if (rc != LS_OK) return rc;
   return ls_sync(h);
 }

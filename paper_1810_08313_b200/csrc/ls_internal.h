@@ -56,6 +56,7 @@ struct Layout {
   size_t stage_y_off[2] = {0, 0};            // [m][batch] labels / targets
   size_t stage_loss_off = 0;                 // float [kRowOffCap][m]
   size_t err_off = 0;                        // int: device-side error flag (bounded waits that ran out)
+  size_t anchor_off = 0, blocku_off = 0;     // block momentum: period-start model and global buffer, [stride] each
   size_t total = 0;
 };
 
@@ -110,6 +111,8 @@ inline float* mom_of(const ls_handle* h) { return reinterpret_cast<float*>(h->st
 inline __nv_bfloat16* shadow_of(const ls_handle* h) {
   return h->lay.bf16 ? reinterpret_cast<__nv_bfloat16*>(h->state + h->lay.shadow_off) : nullptr;
 }
+inline float* anchor_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.anchor_off); }
+inline float* blocku_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.blocku_off); }
 inline float* wlo_of(const ls_handle* h) {
   return h->lay.bf16 ? nullptr : reinterpret_cast<float*>(h->state + h->lay.shadow_off);
 }
@@ -118,8 +121,15 @@ inline float* wlo_of(const ls_handle* h) {
 // n_buf buffers of m vectors each; buffer b starts at base + b*buf_stride floats,
 // vector j of it at + j*stride.  shadow / lo (optional, same strides) receive the
 // bf16 rounding / the tf32 remainder of the mean of buffer 0.  Returns a cudaError_t.
+// bm (optional, n_buf == 1): block momentum, see average.cu; anchor and u are vectors of n floats.
+struct BlockMomentum {
+  float* anchor;
+  float* u;
+  float lr, beta;
+};
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches);
+                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches,
+                   const BlockMomentum* bm = nullptr);
 
 // ---- fp32-accumulate CUDA-core grouped GEMMs (gemm_simt.cu) ---------------
 struct FwdArgs {           // Z = A W^T + b, optional ReLU

@@ -82,6 +82,72 @@ def test_native_run_matches_oracle_over_three_periods(mode):
     eng.close()
 
 
+@pytest.mark.parametrize("gemm,mu", [("fp32", 0.9), ("fp32", 0.0), ("bf16", 0.9)])
+def test_block_momentum_run_matches_oracle(gemm, mu):
+    """Section 5.3: global momentum buffer applied at every averaging step, local buffers restart.  The
+    averaging step itself is checked to the bit from injected state; the free run within tolerance."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, tau, K, beta = (96, 64, 48, 10), 4, 32, 5, 15, 0.3
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 21)
+    offs = wl.batch_row_offsets(2, K, m, 1024, B)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=mu, batch=B, momentum_mode="block", block_momentum=beta,
+                   gemm_dtype=gemm)
+    xd, yd = to_device(X, y, bf16=(gemm == "bf16"))
+    eng.bind_dataset(xd, yd)
+    # (1) one averaging step from injected state, bit-exact
+    P = spec.n_params
+    st = wl.uniform_flat(5, m + 2, P)
+    xs, anchor, u = st[:m].copy(), st[m].copy(), st[m + 1].copy()
+    eng.set_params(x1)
+    for i in range(m):
+        eng.set_state(i, xs[i], xs[i])
+    eng.set_block_state(anchor, u)
+    eng.average()
+    eng.sync()
+    orc.block_momentum_average(xs, anchor, u, f32(0.05), f32(beta))
+    gx, gv = eng.get_all()
+    ga, gu = eng.get_block_state()
+    for i in range(m):
+        assert np.array_equal(gx[i].view(np.uint32), xs[i].view(np.uint32))
+        if mu != 0.0:
+            assert np.all(gv[i] == 0)
+    assert np.array_equal(ga.view(np.uint32), anchor.view(np.uint32))
+    assert np.array_equal(gu.view(np.uint32), u.view(np.uint32))
+    if gemm == "bf16":
+        eng.close()
+        return
+    # (2) free run from x_1
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(mu), tau, momentum_mode="block", block_beta=f32(beta))
+    eng.set_params(x1)
+    loss_dev = torch.zeros((K, m), dtype=torch.float32, device="cuda")
+    out = eng.run(K, tau, offs, loss_out=loss_dev)
+    eng.sync()
+    assert out["taus"] == ref.taus
+    gx, gv = eng.get_all()
+    ga, gu = eng.get_block_state()
+    for i in range(m):
+        assert max_rel_err_per_tensor(gx[i], ref.params[i], dims, True) <= 1e-4
+    assert max_rel_err_per_tensor(ga, ref.params[0], dims, True) <= 1e-4
+    assert max_rel_err_per_tensor(gu, ref.block_u, dims, True) <= 1e-3
+    got = loss_dev.cpu().numpy()
+    assert np.max(np.abs(got - ref.loss) / ref.loss) <= 1e-4
+    p, v = eng.state_view()
+    assert bool((p[0:1] == p).all())
+    eng.close()
+
+
+def test_block_momentum_handle_argument_checks():
+    from paper_1810_08313_b200 import binding
+    from paper_1810_08313_b200.binding import LocalSGD
+    with pytest.raises(binding.LsError):
+        LocalSGD(2, (16, 8), batch=8, momentum_mode="block", block_momentum=1.0)
+    eng = LocalSGD(2, (16, 8), batch=8, momentum_mode="reset")
+    with pytest.raises(binding.LsError):
+        eng.get_block_state()
+    eng.close()
+
+
 def test_tau1_equals_large_batch_sgd_on_gpu():
     """tau = 1 with m replicas equals one replica trained on the concatenated m*B batch
     (fully synchronous SGD, Section 2 special case), both run on the GPU."""

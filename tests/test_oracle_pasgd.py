@@ -189,3 +189,66 @@ def test_adacomm_intervals_follow_the_rule():
     assert orc.tau_schedule_from_trace(res.F_0, 8, [F for _, F, _ in res.F_trace]) == [t for _, _, t in res.F_trace]
     # periods tile the run exactly
     assert res.avg_points[-1] == K
+
+
+# ---- block momentum (Section 5.3) ---------------------------------------------------------------------
+
+def test_block_momentum_tau1_is_synchronous_momentum_sgd():
+    """tau = 1, no local momentum: G_j is the averaged mini-batch gradient, so block momentum with factor
+    beta is plain momentum SGD on the m-fold batch (torch.optim.SGD(momentum=beta))."""
+    spec, X, y, x1 = _tiny_problem()
+    B, K, m, beta = 8, 10, 4, 0.3
+    offs = wl.batch_row_offsets(2, K, m, X.shape[0], B)
+    res = orc.run_pasgd(spec, x1, X, y, offs, B, lr=float(np.float32(0.05)), mu=0.0, tau=1,
+                        momentum_mode=orc.MOMENTUM_BLOCK, block_beta=float(np.float32(beta)))
+    batches = [np.concatenate([np.arange(int(o), int(o) + B) for o in offs[k]]) for k in range(K)]
+    want = _torch_sgd(spec.dims, True, x1, X, y, batches, float(np.float32(0.05)), float(np.float32(beta)))
+    for i in range(m):
+        assert np.max(np.abs(res.params[i] - want)) / np.max(np.abs(want)) < 5e-6
+
+
+def test_block_momentum_scalar_chain_and_special_cases():
+    rng = np.random.default_rng(8)
+    m, P = 4, 37
+    X = rng.standard_normal((m, P)).astype(np.float32)
+    anchor = rng.standard_normal(P).astype(np.float32)
+    u = rng.standard_normal(P).astype(np.float32)
+    lr, beta = np.float32(0.05), np.float32(0.3)
+    want_x = np.empty(P, np.float32); want_u = np.empty(P, np.float32)
+    for p in range(P):
+        s = np.float32(X[0, p])
+        for j in range(1, m):
+            s = np.float32(s + X[j, p])
+        mean = np.float32(s / np.float32(m))
+        d = np.float32(anchor[p] - mean)
+        G = np.float32(d / lr)
+        un = np.float32(np.float32(beta * u[p]) + G)
+        want_u[p] = un
+        want_x[p] = np.float32(anchor[p] - np.float32(lr * un))
+    Xc, ac, uc = X.copy(), anchor.copy(), u.copy()
+    orc.block_momentum_average(Xc, ac, uc, float(lr), float(beta))
+    for j in range(m):
+        assert np.array_equal(Xc[j].view(np.uint32), want_x.view(np.uint32))
+    assert np.array_equal(ac.view(np.uint32), want_x.view(np.uint32))
+    assert np.array_equal(uc.view(np.uint32), want_u.view(np.uint32))
+    # beta = 0 and an empty buffer: the new model is the plain mean up to the rounding of d / eta * eta
+    Xc, ac, uc = X.copy(), anchor.copy(), np.zeros(P, np.float32)
+    orc.block_momentum_average(Xc, ac, uc, float(lr), 0.0)
+    Xm = X.copy(); orc.average_replicas(Xm)
+    assert np.max(np.abs(Xc[0] - Xm[0])) <= 4 * 2.0 ** -24 * np.max(np.abs(np.concatenate([anchor, Xm[0]])))
+    # no displacement and beta = 1: the model keeps moving along the buffer
+    Xc = np.repeat(anchor[None], m, axis=0).copy(); ac = anchor.copy(); uc = np.ones(P, np.float32)
+    orc.block_momentum_average(Xc, ac, uc, 0.5, 1.0)
+    assert np.allclose(Xc[0], anchor - 0.5, atol=1e-6) and np.allclose(uc, 1.0, atol=1e-6)
+
+
+def test_block_momentum_run_resets_local_buffers_and_synchronizes():
+    spec, X, y, x1 = _tiny_problem()
+    B, K, m, tau = 8, 12, 3, 4
+    offs = wl.batch_row_offsets(3, K, m, X.shape[0], B)
+    res = orc.run_pasgd(spec, x1, X, y, offs, B, 0.05, 0.9, tau, momentum_mode=orc.MOMENTUM_BLOCK, block_beta=0.3)
+    assert np.all(res.momentum == 0)
+    assert np.array_equal(res.params[0], res.params[2])
+    plain = orc.run_pasgd(spec, x1, X, y, offs, B, 0.05, 0.9, tau, momentum_mode=orc.MOMENTUM_RESET)
+    assert not np.array_equal(res.params[0], plain.params[0])       # the global momentum changes the trajectory
+    assert np.any(res.block_u != 0)
