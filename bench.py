@@ -72,12 +72,12 @@ def flops_per_replica_step(w: wl.Workload) -> float:
 
 def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
     """Algorithmic bytes of one weight-gradient + update launch for layer `layer` (all m replicas):
-    read and write W (and v when momentum is on), write the operand copy of W (bf16 rounding, or
-    the fp32 "lo" twin), read the two GEMM operands once (with their lo twins in fp32 models)."""
+    read and write W (and v when momentum is on), write the bf16 copy of W (bf16 models), read the
+    two GEMM operands once."""
     n_out, n_in = layer_shapes(w)[layer]
     bf = w.gemm_dtype == "bf16"
-    per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if bf else 4)
-    operand = (2 if bf else 8) * w.batch * (n_out + n_in)
+    per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if bf else 0)
+    operand = (2 if bf else 4) * w.batch * (n_out + n_in)
     return float(w.m) * (per_param * n_out * n_in + operand)
 
 
@@ -392,6 +392,7 @@ def run_ours(args, w: wl.Workload):
     shares_raw = eng.profile_end()
     tot = sum(v[0] for v in shares_raw.values()) or 1.0
     shares = {f"{c}{l}": round(v[0] / tot, 4) for (c, l), v in sorted(shares_raw.items(), key=lambda kv: -kv[1][0])}
+    kernel_us = {f"{c}{l}": round(v[0] / v[1] * 1e3, 2) for (c, l), v in shares_raw.items() if v[1]}
     dom = max(shares_raw.items(), key=lambda kv: kv[1][0])[0] if shares_raw else ("dw", 0)
 
     # ---- timed region ---------------------------------------------------------
@@ -428,6 +429,7 @@ def run_ours(args, w: wl.Workload):
                          % (xd.numel() * xd.element_size() / 1e6),
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks, "gpu_launches": int(launches), "kernel_time_shares": shares,
+        "kernel_us_per_launch": kernel_us,
         "last_probe_loss": F_t, "next_tau": next_tau,
     }
     if roofline:

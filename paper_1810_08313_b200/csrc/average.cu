@@ -51,8 +51,6 @@ template <> struct Vec<8> {
   }
 };
 
-__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
-
 template <int W>
 __device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&v)[W]) {
   uint32_t u[W / 2];
@@ -73,7 +71,7 @@ __device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&v)[W]
 template <int M, int W, bool BM>
 __global__ void __launch_bounds__(kThreads)
 average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
-               __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo, BlockMomentum bm) {
+               __nv_bfloat16* __restrict__ shadow, BlockMomentum bm) {
   const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (i >= n_vec) return;
   const int m = M > 0 ? M : m_rt;
@@ -123,23 +121,15 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
   }
 #pragma unroll 4
   for (int j = 0; j < m; ++j) s.store(p + (int64_t)j * stride);
-  if (blockIdx.y == 0) {
-    if (shadow != nullptr)
-      for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + i * W, s.v);
-    if (lo != nullptr) {
-      Vec<W> l;
-#pragma unroll
-      for (int e = 0; e < W; ++e) l.v[e] = tf32_lo(s.v[e]);
-      for (int j = 0; j < m; ++j) l.store(lo + (int64_t)j * stride + i * W);
-    }
-  }
+  if (blockIdx.y == 0 && shadow != nullptr)
+    for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + i * W, s.v);
 }
 
 // Scalar path: the ragged tail (n mod W elements) and buffers that are not
 // 16-byte aligned.  Same arithmetic, one element per thread.
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
-                      __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo, BlockMomentum bm) {
+                      __nv_bfloat16* __restrict__ shadow, BlockMomentum bm) {
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
   const float mf = (float)m;
   const int64_t i = first + (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -156,18 +146,14 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
     bm.anchor[i] = mean;
   }
   for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
-  if (blockIdx.y == 0) {
-    if (shadow != nullptr)
-      for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + i] = __float2bfloat16_rn(mean);
-    if (lo != nullptr)
-      for (int j = 0; j < m; ++j) lo[(int64_t)j * stride + i] = tf32_lo(mean);
-  }
+  if (blockIdx.y == 0 && shadow != nullptr)
+    for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + i] = __float2bfloat16_rn(mean);
 }
 
 template <int W, bool BM>
 void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
-                __nv_bfloat16* shadow, float* lo, const BlockMomentum& bm) {
-#define LS_AVG(M) average_kernel<M, W, BM><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, lo, bm)
+                __nv_bfloat16* shadow, const BlockMomentum& bm) {
+#define LS_AVG(M) average_kernel<M, W, BM><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, bm)
   switch (m) {
     case 2: LS_AVG(2); break;
     case 4: LS_AVG(4); break;
@@ -183,7 +169,7 @@ inline bool aligned_to(const void* p, size_t a) { return p == nullptr || reinter
 }  // namespace
 
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches, const BlockMomentum* bmp) {
+                   __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches, const BlockMomentum* bmp) {
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
   BlockMomentum bm{nullptr, nullptr, 0.f, 0.f};
   if (bmp != nullptr) {
@@ -193,11 +179,11 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
   const bool BM = bm.anchor != nullptr;
   // widest slice the addresses allow: 8 floats (32-byte aligned), 4 floats (16-byte), else scalar
   int W = 0;
-  if (aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 && aligned_to(shadow, 16) && aligned_to(lo, 32) &&
+  if (aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 && aligned_to(shadow, 16) &&
       aligned_to(bm.anchor, 32) && aligned_to(bm.u, 32))
     W = 8;
   else if (aligned_to(base, 16) && stride % 4 == 0 && buf_stride % 4 == 0 && aligned_to(shadow, 8) &&
-           aligned_to(lo, 16) && aligned_to(bm.anchor, 16) && aligned_to(bm.u, 16))
+           aligned_to(bm.anchor, 16) && aligned_to(bm.u, 16))
     W = 4;
   const int64_t n_vec = W ? n / W : 0;
   if (n_vec > 0) {
@@ -205,11 +191,11 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
     if (W == 8) {
-      if (BM) launch_vec<8, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
-      else launch_vec<8, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+      if (BM) launch_vec<8, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm);
+      else launch_vec<8, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm);
     } else {
-      if (BM) launch_vec<4, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
-      else launch_vec<4, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, lo, bm);
+      if (BM) launch_vec<4, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm);
+      else launch_vec<4, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm);
     }
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
@@ -220,7 +206,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     const int64_t gx = (n - first + kThreads - 1) / kThreads;
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, lo, bm);
+    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, bm);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -233,8 +219,8 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
 extern "C" int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride, void* cuda_stream) {
   if (buf_dev == nullptr || m < 1 || P < 0 || stride < P) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(buf_dev) % 4 != 0) return LS_ERR_INVALID_ARG;
-  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
-                             nullptr, nullptr);
+  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr,
+                             nullptr);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
@@ -247,7 +233,7 @@ extern "C" int ls_block_average_flat(float* buf_dev, float* anchor_dev, float* u
       reinterpret_cast<uintptr_t>(u_dev) % 4 != 0)
     return LS_ERR_INVALID_ARG;
   ls::BlockMomentum bm{anchor_dev, u_dev, lr, beta};
-  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
-                             nullptr, &bm);
+  int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr,
+                             &bm);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

@@ -139,18 +139,10 @@ gemm_kernel(const TA* A, int64_t a_gstride, const int64_t* a_row_off, int64_t ld
 
 // ---- epilogues ---------------------------------------------------------------
 
-// x - tf32(x): the part of an fp32 value that a tf32 read drops (kept in a twin array for the tensor-core kernels)
-__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
-__device__ __forceinline__ void store_lo(float* lo, int64_t at, const float (&o)[4], int nv, bool vec) {
-  if (lo == nullptr) return;
-  if (vec && nv == 4) *reinterpret_cast<float4*>(lo + at) = make_float4(tf32_lo(o[0]), tf32_lo(o[1]), tf32_lo(o[2]), tf32_lo(o[3]));
-  else for (int s = 0; s < nv; ++s) lo[at + s] = tf32_lo(o[s]);
-}
-
 template <typename TC>
 struct EpiFwd {
   const float* bias; int64_t bias_gstride;
-  TC* C; float* Clo; int M, N; int relu; bool vec;
+  TC* C; int M, N; int relu; bool vec;
   __device__ __forceinline__ void operator()(int g, int i, int j, const float (&acc)[4], int nv) const {
     float o[4];
 #pragma unroll
@@ -163,13 +155,12 @@ struct EpiFwd {
     TC* p = C + at;
     if (vec && nv == 4) store_out4(p, o);
     else for (int s = 0; s < nv; ++s) store_out(p + s, o[s]);
-    store_lo(Clo, at, o, nv, vec);
   }
 };
 
 template <typename TC>
 struct EpiDx {
-  const TC* act; TC* C; float* Clo; int M, N; bool vec;
+  const TC* act; TC* C; int M, N; bool vec;
   __device__ __forceinline__ void operator()(int g, int i, int j, const float (&acc)[4], int nv) const {
     const int64_t at = ((int64_t)g * M + i) * N + j;
     float o[4];
@@ -177,12 +168,11 @@ struct EpiDx {
     for (int s = 0; s < 4; ++s) o[s] = (s < nv && to_f(act[at + s]) > 0.f) ? acc[s] : 0.f;
     if (vec && nv == 4) store_out4(C + at, o);
     else for (int s = 0; s < nv; ++s) store_out(C + at + s, o[s]);
-    store_lo(Clo, at, o, nv, vec);
   }
 };
 
 struct EpiDw {
-  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; int64_t gstride; int N; float lr, mu; bool vec;
+  float* W; float* V; __nv_bfloat16* Wb; int64_t gstride; int N; float lr, mu; bool vec;
   __device__ __forceinline__ void operator()(int g, int i, int j, const float (&acc)[4], int nv) const {
     const int64_t at = (int64_t)g * gstride + (int64_t)i * N + j;
     float w[4], v[4];
@@ -209,7 +199,6 @@ struct EpiDw {
         if (Wb != nullptr) Wb[at + s] = __float2bfloat16_rn(w[s]);
       }
     }
-    store_lo(Wlo, at, w, nv, vec);
   }
 };
 
@@ -229,8 +218,8 @@ template <typename TA, typename TW, typename TC>
 int fwd_typed(const FwdArgs& a, cudaStream_t st) {
   const TA* A = static_cast<const TA*>(a.A);
   const TW* W = static_cast<const TW*>(a.W);
-  EpiFwd<TC> epi{a.bias, a.bias_gstride, static_cast<TC*>(a.C), sizeof(TC) == 4 ? a.Clo : nullptr, a.M, a.N, a.relu,
-                 aligned(a.C, 4 * sizeof(TC)) && (a.Clo == nullptr || aligned(a.Clo, 16)) && a.N % 4 == 0};
+  EpiFwd<TC> epi{a.bias, a.bias_gstride, static_cast<TC*>(a.C), a.M, a.N, a.relu,
+                 aligned(a.C, 4 * sizeof(TC)) && a.N % 4 == 0};
   const int64_t a_gs = (int64_t)a.M * a.K;
   gemm_kernel<TA, true, TW, true, EpiFwd<TC>><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
       A, a_gs, a.row_off, a.K, can_vec<TA>(A, a.K, a_gs), W, a.w_gstride, nullptr, a.K,
@@ -242,9 +231,8 @@ template <typename T>
 int dx_typed(const DxArgs& a, cudaStream_t st) {
   const T* dZ = static_cast<const T*>(a.dZ);
   const T* W = static_cast<const T*>(a.W);
-  EpiDx<T> epi{static_cast<const T*>(a.act), static_cast<T*>(a.C), sizeof(T) == 4 ? a.Clo : nullptr, a.M, a.N,
-               aligned(a.C, 4 * sizeof(T)) && aligned(a.act, 4 * sizeof(T)) && (a.Clo == nullptr || aligned(a.Clo, 16)) &&
-                   a.N % 4 == 0};
+  EpiDx<T> epi{static_cast<const T*>(a.act), static_cast<T*>(a.C), a.M, a.N,
+               aligned(a.C, 4 * sizeof(T)) && aligned(a.act, 4 * sizeof(T)) && a.N % 4 == 0};
   const int64_t a_gs = (int64_t)a.M * a.K;
   gemm_kernel<T, true, T, false, EpiDx<T>><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
       dZ, a_gs, nullptr, a.K, can_vec<T>(dZ, a.K, a_gs), W, a.w_gstride, nullptr, a.N,
@@ -256,9 +244,9 @@ template <typename T>
 int dw_typed(const DwArgs& a, cudaStream_t st) {
   const T* dZ = static_cast<const T*>(a.dZ);
   const T* A = static_cast<const T*>(a.A);
-  EpiDw epi{a.W, a.V, a.Wb, a.Wlo, a.w_gstride, a.N, a.lr, a.mu,
-            aligned(a.W, 16) && aligned(a.V, 16) && (a.Wb == nullptr || aligned(a.Wb, 8)) &&
-                (a.Wlo == nullptr || aligned(a.Wlo, 16)) && a.N % 4 == 0 && a.w_gstride % 4 == 0};
+  EpiDw epi{a.W, a.V, a.Wb, a.w_gstride, a.N, a.lr, a.mu,
+            aligned(a.W, 16) && aligned(a.V, 16) && (a.Wb == nullptr || aligned(a.Wb, 8)) && a.N % 4 == 0 &&
+                a.w_gstride % 4 == 0};
   const int64_t dz_gs = (int64_t)a.B * a.M, a_gs = (int64_t)a.B * a.N;
   gemm_kernel<T, false, T, false, EpiDw><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
       dZ, dz_gs, nullptr, a.M, can_vec<T>(dZ, a.M, dz_gs), A, a_gs, a.row_off, a.N, can_vec<T>(A, a.N, a_gs),

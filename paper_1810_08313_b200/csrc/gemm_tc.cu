@@ -6,15 +6,17 @@
 //   warp 1      allocates tensor memory, issues tcgen05.mma (one elected thread), accumulator in TMEM
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (warp w owns TMEM lanes 32*(w%4)..+31) and apply
 //                 forward   Z = A W^T + b, relu                            (evaluating f, Section 2)
-//                 backward  dZ_prev = (dZ W) * 1[act > 0]
+//                 backward  dZ_prev = (dZ W) * 1[act > 0]; when the tile holds the whole mini-batch, also the
+//                           bias update of the layer below from the column sums of dZ_prev
 //                 update    G = dZ^T A; v <- mu v + G; W <- W - eta v      (Section 2 mini-batch SGD
 //                           update, Section 5.3 momentum); G never leaves the SM
 //
 // Two operand formats:
 //   bf16   one tcgen05.mma kind::f16 per 16 elements of K; outputs rounded to bf16.
 //   fp32   every fp32 operand x is used as the pair (hi, lo): hi is x itself, of which the tensor
-//          core reads the upper 19 bits (tf32), lo = x - tf32(x) lives in a second array that the
-//          producing kernel wrote next to x.  Three kind::tf32 MMAs per 8 elements of K
+//          core reads the upper 19 bits (tf32); lo = x - tf32(x) is written by two splitter warps
+//          (warps 6-7) from each stage that TMA has filled into a second, shorter ring of shared
+//          memory, in the same (swizzled) layout.  Three kind::tf32 MMAs per 8 elements of K
 //          (lo*hi + hi*lo + hi*hi) give products accurate to about 2^-21, accumulated in fp32.
 //          The tensor core's fp32 accumulation truncates, which biases a long sum; the forward and
 //          backward kernels therefore restart the TMEM accumulator every kChunkStages stages (two
@@ -42,7 +44,9 @@ using namespace ptx;
 
 constexpr int BM = 128;            // rows of the output tile = TMEM lanes
 constexpr int KB_BYTES = 128;      // bytes of K per stage row (one swizzle row)
-constexpr int kThreads = 192;
+constexpr int kThreadsBf16 = 192;  // warps 0-5
+constexpr int kThreadsFp32 = 256;  // + two splitter warps
+constexpr int kSplitWarps = 2;
 constexpr int kStageLd = 36;       // floats per staged row (32 + 4 padding) in the update epilogue
 constexpr int kChunkStages = 4;    // fp32 forward/backward: stages per TMEM accumulation chunk (48 MMAs)
 
@@ -56,27 +60,33 @@ struct Operand {
 };
 
 struct Params {
-  Operand a, b, a_lo, b_lo;
+  Operand a, b;
   int M, N, K;               // per group, in elements
   // forward
   const float* bias; int64_t bias_gstride; int relu;
-  // forward / backward output (+ its lo part in fp32 mode), backward mask
-  void* C; float* Clo; const void* act;
+  // forward / backward output, backward mask
+  void* C; const void* act;
+  // backward: bias of the layer below and its momentum (or null), elements between replicas
+  float* dbias; float* dvbias; int64_t dbias_gstride;
   // update
-  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride; float lr, mu;
+  float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride; float lr, mu;
   int* err_flag;
 };
 
+// Shared memory: a ring of STAGES stages filled by TMA (the A and B tiles as they are in memory) and,
+// for fp32 operands, a shorter ring of kLoStages stages that receives their lo parts.
 template <bool TF32, int BN, int STAGES, int MT = 1>
 struct Smem {
-  static constexpr int kTiles = TF32 ? 2 : 1;      // hi and lo copies of each operand tile
+  static constexpr int kLoStages = TF32 ? 2 : 0;
   static constexpr int kABytes = MT * BM * KB_BYTES;   // MT row blocks of 128 share one B tile
   static constexpr int kBBytes = BN * KB_BYTES;
-  static constexpr int kStageBytes = kTiles * (kABytes + kBBytes);
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kRingBytes = (STAGES + kLoStages) * kStageBytes;
   // the update epilogue stages its 32x32 blocks in stage 0, which is free once the accumulator is complete
-  static constexpr int kBarBytes = (2 * STAGES + 4) * 8 + 16;
-  static constexpr int kTotal = 1024 + STAGES * kStageBytes + kBarBytes;
+  static constexpr int kBarBytes = (2 * STAGES + 2 * 2 + 4) * 8 + 16;
+  static constexpr int kTotal = 1024 + kRingBytes + kBarBytes;
   static_assert(4 * 32 * kStageLd * 4 <= kStageBytes, "staging must fit in one stage");
+  static_assert((4 * 32 * kStageLd + MT * 4 * BN) * 4 <= kRingBytes, "column-sum scratch of the backward epilogue");
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
 
@@ -101,10 +111,6 @@ __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uin
   }
 }
 
-// The part of x that a tf32 read keeps (upper 19 bits) and the remainder.
-__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
-__device__ __forceinline__ float tf32_lo(float x) { return x - tf32_hi(x); }
-
 // one 32-byte (whole sector) store; p must be 32-byte aligned
 __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
   asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
@@ -112,21 +118,17 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
                : "memory");
 }
 
-// Store 32 consecutive outputs of one row (bf16, or fp32 plus the lo parts) in whole 32-byte sectors.
+// Store 32 consecutive outputs of one row (bf16 or fp32) in whole 32-byte sectors.
 template <bool TF32>
-__device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, const float (&o)[32]) {
+__device__ __forceinline__ void store_row32(void* C, int64_t at, const float (&o)[32]) {
   if (TF32) {
     float* c = static_cast<float*>(C) + at;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      uint32_t hi[8], lo[8];
+      uint32_t hi[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        hi[e] = __float_as_uint(o[8 * i + e]);
-        lo[e] = __float_as_uint(tf32_lo(o[8 * i + e]));
-      }
+      for (int e = 0; e < 8; ++e) hi[e] = __float_as_uint(o[8 * i + e]);
       st_global_v8(c + 8 * i, hi);
-      st_global_v8(Clo + at + 8 * i, lo);
     }
   } else {
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(C) + at;
@@ -146,9 +148,8 @@ __device__ __forceinline__ void store_row32(void* C, float* Clo, int64_t at, con
 // MT = 2: the CTA computes two 128-row blocks (a 256 x BN tile) from one B tile in shared memory, with two
 // TMEM accumulators: a third less operand traffic from L2 per flop, which is what bounds these kernels.
 template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLIT, int MT>
-__global__ void __launch_bounds__(kThreads, (Smem<TF32, BN, STAGES, MT>::kTotal <= 113 * 1024) ? 2 : 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo, const Params p) {
+__global__ void __launch_bounds__(TF32 ? kThreadsFp32 : kThreadsBf16, (Smem<TF32, BN, STAGES, MT>::kTotal <= 113 * 1024) ? 2 : 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
   using L = Smem<TF32, BN, STAGES, MT>;
   constexpr int EB = TF32 ? 4 : 2;             // bytes per operand element
   constexpr int ELEMS = KB_BYTES / EB;         // K elements per stage
@@ -160,17 +161,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr uint32_t TMEM_COLS = CHUNKED ? 2 * BN : MT * BN;
   static_assert(MT == 1 || (!CHUNKED && !A_MN && EPI != EPI_DW && MT * BN <= 512), "two row blocks: bf16 forward/backward");
   static_assert(SPLIT == 1 || CHUNKED, "split-K needs the register-resident partial sums");
-  static_assert(SPLIT == 1 || BN * BM * 4 <= STAGES * L::kStageBytes, "exchange buffer");
+  static_assert(SPLIT == 1 || BN * BM * 4 <= L::kRingBytes, "exchange buffer");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
   float* staging = reinterpret_cast<float*>(smem);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * L::kStageBytes);
+  float* colsum = staging + 4 * 32 * kStageLd;      // [MT * 4][BN] partial column sums (backward epilogue)
+  uint8_t* lo_base = smem + STAGES * L::kStageBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kRingBytes);
   uint64_t* empty = full + STAGES;
   uint64_t* acc_full = empty + STAGES;      // [2] accumulator (chunk) complete
   uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the 4 epilogue warps
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* lo_full = acc_empty + 2;         // [2] fp32: lo parts of a stage written
+  uint64_t* lo_empty = lo_full + 2;          // [2] ... and read by the tensor core
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(lo_empty + 2);
+  constexpr int LS = L::kLoStages > 0 ? L::kLoStages : 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.z;
@@ -181,11 +187,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4);
+      mbar_init(&lo_full[b], kSplitWarps); mbar_init(&lo_empty[b], 1);
+    }
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
-    if (TF32) { prefetch_tmap(&tmAlo); prefetch_tmap(&tmBlo); }
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TMEM_COLS);
@@ -214,13 +222,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int k0 = (kb0 + kb) * ELEMS;
         issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM * MT, k0);
         issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, k0);
-        if (TF32) {
-          uint8_t* sal = sb + L::kBBytes;
-          uint8_t* sbl = sal + L::kABytes;
-          issue_tile<ELEMS>(sal, &tmAlo, &full[s], p.a_lo, g, A_MN, m0, BM * MT, k0);
-          issue_tile<ELEMS>(sbl, &tmBlo, &full[s], p.b_lo, g, B_MN, n0, BN, k0);
-        }
       }
+    }
+  } else if (TF32 && warp >= 6) {
+    // ---- splitter warps (fp32): lo = x - tf32(x) of both tiles of the stage, element by element, so
+    // the copy has the layout (swizzle included) of the tile it comes from
+    const int tid = threadIdx.x - 6 * 32;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES, sl = kb % LS;
+      bool got = mbar_wait(&full[s], (kb / STAGES) & 1);
+      if (got && kb >= LS) got = mbar_wait(&lo_empty[sl], ((kb / LS) - 1) & 1);
+      if (!__all_sync(0xffffffffu, got)) {
+        if (lane == 0) atomicExch(p.err_flag, 5);
+        break;
+      }
+      static_assert(L::kStageBytes % (8 * 16 * kSplitWarps * 32) == 0, "whole batches of pieces");
+      split_lo_smem(smem_u32(stage_base + s * L::kStageBytes), smem_u32(lo_base + sl * L::kStageBytes),
+                    L::kStageBytes, tid, kSplitWarps * 32);
+      fence_proxy_async_smem();     // the tensor core reads shared memory through the async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&lo_full[sl]);
     }
   } else if (warp == 1) {
     if (elect_one()) {
@@ -234,10 +255,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           break;
         }
         if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { atomicExch(p.err_flag, 2); break; }
+        if (TF32 && !mbar_wait(&lo_full[kb % LS], (kb / LS) & 1)) { atomicExch(p.err_flag, 6); break; }
         tc_fence_after_sync();
         const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
         const uint32_t b_addr = a_addr + L::kABytes;
-        const uint32_t alo_addr = b_addr + L::kBBytes;
+        const uint32_t alo_addr = smem_u32(lo_base + (kb % LS) * L::kStageBytes);
         const uint32_t blo_addr = alo_addr + L::kABytes;
 #pragma unroll
         for (int k = 0; k < ELEMS / MMA_K; ++k) {
@@ -269,11 +291,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+        if (TF32) mma_commit(&lo_empty[kb % LS]);
         if (CHUNKED ? (kb % CS == CS - 1 || kb == num_kb - 1) : (kb == num_kb - 1))
           mma_commit(&acc_full[chunk & 1]);     // this accumulator is complete
       }
     }
-  } else {
+  } else if (warp < 6) {
     // ---- epilogue warps: collect the accumulator(s) ------------------------------
     if (CHUNKED) {
       // add the partial accumulators in registers (this thread owns one output row) as they complete
@@ -314,7 +337,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   if (SPLIT > 1) {
     cluster_sync_all();
-    if (warp >= 2 && rank == 0 && ok) {
+    if (warp >= 2 && warp < 6 && rank == 0 && ok) {
       const uint32_t mine = smem_u32(reinterpret_cast<float*>(smem) + q * 32 + lane);
       for (int r = 1; r < SPLIT; ++r) {
         const uint32_t remote = map_to_rank(mine, (uint32_t)r);
@@ -324,7 +347,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     cluster_sync_all();      // the other CTAs stay alive until rank 0 has read their rows
   }
-  if (warp >= 2) {
+  if (warp >= 2 && warp < 6) {
     if (ok && (SPLIT == 1 || rank == 0)) {
 #pragma unroll
       for (int cc32 = 0; cc32 < MT * (BN / 32); ++cc32) {
@@ -348,7 +371,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (bias) v += __ldg(bias + i);
             o[i] = (p.relu && !(v > 0.f)) ? 0.f : v;
           }
-          store_row32<TF32>(p.C, p.Clo, ((int64_t)g * p.M + row) * p.N + col, o);
+          store_row32<TF32>(p.C, ((int64_t)g * p.M + row) * p.N + col, o);
         } else if (EPI == EPI_DX) {
           const int64_t at = ((int64_t)g * p.M + row) * p.N + col;
           float o[32];
@@ -377,7 +400,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
-          store_row32<TF32>(p.C, p.Clo, at, o);
+          store_row32<TF32>(p.C, at, o);
+          if (p.dbias != nullptr) {
+            // column sums over this warp's 32 rows, through a padded 32 x 33 transpose in the (now idle)
+            // stage memory; lane i ends up with column i
+            float* tile = staging + (warp - 2) * (32 * 33);
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = o[i];
+            __syncwarp();
+            float cs = 0.f;
+#pragma unroll
+            for (int r = 0; r < 32; ++r) cs += tile[r * 33 + lane];
+            colsum[(mt * 4 + q) * BN + c * 32 + lane] = cs;
+          }
         } else {
           // transpose the 32x32 block through shared memory so that global accesses run along rows
           float* st = staging + (warp - 2) * 32 * kStageLd;
@@ -414,10 +450,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             *reinterpret_cast<float4*>(p.W + at) = make_float4(ws[0], ws[1], ws[2], ws[3]);
             if (p.mu != 0.f) *reinterpret_cast<float4*>(p.V + at) = make_float4(vs[0], vs[1], vs[2], vs[3]);
-            if (TF32) {
-              *reinterpret_cast<float4*>(p.Wlo + at) =
-                  make_float4(tf32_lo(ws[0]), tf32_lo(ws[1]), tf32_lo(ws[2]), tf32_lo(ws[3]));
-            } else if (p.Wb != nullptr) {
+            if (!TF32 && p.Wb != nullptr) {
               __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
               __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
               uint2 u;
@@ -428,6 +461,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
           __syncwarp();
         }
+      }
+    }
+    if (EPI == EPI_DX && p.dbias != nullptr && (SPLIT == 1 || rank == 0)) {
+      // all four epilogue warps (and only they) meet here; then one thread per column adds the partial
+      // sums in a fixed order and applies v <- mu v + g, b <- b - eta v
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int t = threadIdx.x - 64; t < BN; t += 128) {
+        float gsum = 0.f;
+#pragma unroll
+        for (int i = 0; i < MT * 4; ++i) gsum += colsum[i * BN + t];
+        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
+        float step = gsum;
+        if (p.mu != 0.f) {
+          step = fmaf(p.mu, p.dvbias[at], gsum);
+          p.dvbias[at] = step;
+        }
+        p.dbias[at] = fmaf(-p.lr, step, p.dbias[at]);
       }
     }
     tc_fence_before_sync();
@@ -469,16 +519,14 @@ int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_
     configured = true;
   }
   dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / (BM * MT)), (unsigned)groups);
-  const CUtensorMap* alo = TF32 ? mp.a_lo : mp.a;
-  const CUtensorMap* blo = TF32 ? mp.b_lo : mp.b;
   if (SPLIT == 1) {
-    kern<<<grid, kThreads, L::kTotal, st>>>(*mp.a, *mp.b, *alo, *blo, p);
+    kern<<<grid, TF32 ? kThreadsFp32 : kThreadsBf16, L::kTotal, st>>>(*mp.a, *mp.b, p);
     return cudaGetLastError();
   }
   // the SPLIT CTAs that share an output tile form one cluster along x
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(TF32 ? kThreadsFp32 : kThreadsBf16);
   cfg.dynamicSmemBytes = L::kTotal;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -488,7 +536,7 @@ int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, *mp.a, *mp.b, *alo, *blo, p);
+  return cudaLaunchKernelEx(&cfg, kern, *mp.a, *mp.b, p);
 }
 
 // fp32 forward / backward: tile width and K split.  128-wide tiles when N allows; K is split over a
@@ -501,9 +549,9 @@ int launch_fp32(const TcOperandMaps& mp, const Params& p, int groups, cudaStream
   int split = 1;
   while (split < 4 && tiles * split * 2 <= 148 && num_kb % (split * 2) == 0 && num_kb / (split * 2) >= 8) split *= 2;
   if (bn == 128) {
-    if (split == 4) return launch_one<true, 128, A_MN, B_MN, EPI, 3, 4>(mp, p, groups, st);
-    if (split == 2) return launch_one<true, 128, A_MN, B_MN, EPI, 3, 2>(mp, p, groups, st);
-    return launch_one<true, 128, A_MN, B_MN, EPI, 3, 1>(mp, p, groups, st);
+    if (split == 4) return launch_one<true, 128, A_MN, B_MN, EPI, 4, 4>(mp, p, groups, st);
+    if (split == 2) return launch_one<true, 128, A_MN, B_MN, EPI, 4, 2>(mp, p, groups, st);
+    return launch_one<true, 128, A_MN, B_MN, EPI, 4, 1>(mp, p, groups, st);
   }
   if (split == 4) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 4>(mp, p, groups, st);
   if (split == 2) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 2>(mp, p, groups, st);
@@ -547,6 +595,13 @@ int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64
   return make_map(out, base, true, false, true, 3, rows, cols, groups, gstride);
 }
 
+// The backward kernel can finish the bias update when one CTA holds every row of its columns: M is one
+// row block, or two with the 256-row bf16 tile.
+bool tc_dx_fuses_bias(bool fp32, int M, int N) {
+  if (M == BM) return true;
+  return !fp32 && M == 2 * BM && N % 256 == 0;
+}
+
 // M output rows, N output columns, K contraction length of one group.
 bool tc_shape_ok(bool fp32, int M, int N, int K) {
   if (M <= 0 || N <= 0 || K <= 0 || M % BM != 0) return false;
@@ -556,11 +611,10 @@ bool tc_shape_ok(bool fp32, int M, int N, int K) {
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
   p.a = Operand{a.row_off, a.M, 0, 0, 0};
-  p.a_lo = Operand{nullptr, a.M, 0, 0, 0};
-  p.b = p.b_lo = Operand{nullptr, 0, a.w_z0, a.w_zstep, 1};
+  p.b = Operand{nullptr, 0, a.w_z0, a.w_zstep, 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.bias = a.bias; p.bias_gstride = a.bias_gstride; p.relu = a.relu;
-  p.C = a.C; p.Clo = a.Clo; p.err_flag = a.err_flag;
+  p.C = a.C; p.err_flag = a.err_flag;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);
@@ -570,10 +624,13 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
 
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
-  p.a = p.a_lo = Operand{nullptr, a.M, 0, 0, 0};
-  p.b = p.b_lo = Operand{nullptr, 0, 0, 1, 1};
+  p.a = Operand{nullptr, a.M, 0, 0, 0};
+  p.b = Operand{nullptr, 0, 0, 1, 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
-  p.C = a.C; p.Clo = a.Clo; p.act = a.act; p.err_flag = a.err_flag;
+  p.C = a.C; p.act = a.act; p.err_flag = a.err_flag;
+  if (a.bias != nullptr && tc_dx_fuses_bias(a.fp32, a.M, a.N)) {
+    p.dbias = a.bias; p.dvbias = a.vbias; p.dbias_gstride = a.bias_gstride; p.lr = a.lr; p.mu = a.mu;
+  }
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 3, 1, 2>(a.maps, p, a.groups, st);
@@ -583,16 +640,15 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
 
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
-  p.a = p.a_lo = Operand{nullptr, a.B, 0, 0, 0};
+  p.a = Operand{nullptr, a.B, 0, 0, 0};
   p.b = Operand{a.row_off, a.B, 0, 0, 0};
-  p.b_lo = Operand{nullptr, a.B, 0, 0, 0};
   p.M = a.M; p.N = a.N; p.K = a.B;
-  p.W = a.W; p.V = a.V; p.Wb = a.Wb; p.Wlo = a.Wlo; p.w_gstride = a.w_gstride; p.lr = a.lr; p.mu = a.mu;
+  p.W = a.W; p.V = a.V; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.lr = a.lr; p.mu = a.mu;
   p.err_flag = a.err_flag;
   if (launches) ++*launches;
   if (a.fp32) {
-    if (a.N % 128 == 0) return launch_one<true, 128, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
-    return launch_one<true, 64, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
+    if (a.N % 128 == 0) return launch_one<true, 128, true, true, EPI_DW, 4>(a.maps, p, a.groups, st);
+    return launch_one<true, 64, true, true, EPI_DW, 4>(a.maps, p, a.groups, st);
   }
   return launch_one<false, 128, true, true, EPI_DW, 3>(a.maps, p, a.groups, st);
 }

@@ -24,7 +24,6 @@ constexpr int kColsPerCta = 64;        // head_bwd: 32 lanes x 2 columns, 8 row 
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
-__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ void put(float* p, float v) { *p = v; }
 __device__ __forceinline__ void put(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
@@ -183,9 +182,10 @@ __device__ __forceinline__ void store2(__nv_bfloat16* p, float a, float b) {
 template <typename TA>
 __global__ void __launch_bounds__(kThreads, 2)
 head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
-                float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb, float* __restrict__ Wlo,
+                float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb,
                 float* __restrict__ bias, float* __restrict__ vbias, int64_t w_gstride, TA* __restrict__ dPrev,
-                float* __restrict__ dPrevLo, int B, int C, int K, float lr, float mu, int pair_ok) {
+                float* __restrict__ pbias, float* __restrict__ pvbias, int B, int C, int K, float lr, float mu,
+                int pair_ok) {
   extern __shared__ float sm[];
   float* dz = sm;                                   // [B][C]
   float* part = sm + (size_t)B * C;                 // [8][CMAX][kColsPerCta]
@@ -202,6 +202,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     wreg[c][1] = (c < C && in1) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k + 1] : 0.f;
     gw[c][0] = gw[c][1] = 0.f;
   }
+  float cs0 = 0.f, cs1 = 0.f;     // column sums of dPrev over this thread's rows (bias gradient of the layer below)
   for (int i = threadIdx.x; i < B * C; i += kThreads) dz[i] = dZ[(int64_t)g * B * C + i];
   __syncthreads();
 
@@ -234,14 +235,14 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
           }
         if (dPrev != nullptr) {
           const float o0 = av[u][0] > 0.f ? da0 : 0.f, o1 = av[u][1] > 0.f ? da1 : 0.f;
+          cs0 += o0;
+          cs1 += o1;
           const int64_t at = ((int64_t)g * B + b) * K + k;
           if (pair_ok) {
             store2(dPrev + at, o0, o1);
-            if (dPrevLo != nullptr) store2(dPrevLo + at, tf32_lo(o0), tf32_lo(o1));
           } else {
             put(dPrev + at, o0);
             if (in1) put(dPrev + at + 1, o1);
-            if (dPrevLo != nullptr) { dPrevLo[at] = tf32_lo(o0); if (in1) dPrevLo[at + 1] = tf32_lo(o1); }
           }
         }
       }
@@ -271,7 +272,6 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     const float w = fmaf(-lr, step, W[at]);
     W[at] = w;
     if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
-    if (Wlo != nullptr) Wlo[at] = tf32_lo(w);
   }
   if (blockIdx.x == 0 && bias != nullptr && threadIdx.x < C) {
     const int c = threadIdx.x;
@@ -284,6 +284,26 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
       vbias[at] = step;
     }
     bias[at] = fmaf(-lr, step, bias[at]);
+  }
+  if (pbias != nullptr) {
+    // bias of the layer below: its gradient is the column sum of dPrev, complete inside this CTA
+    __syncthreads();
+    part[ry * kColsPerCta + cx * 2] = cs0;
+    part[ry * kColsPerCta + cx * 2 + 1] = cs1;
+    __syncthreads();
+    const int kk = blockIdx.x * kColsPerCta + threadIdx.x;
+    if (threadIdx.x < kColsPerCta && kk < K) {
+      float s = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) s += part[r * kColsPerCta + threadIdx.x];
+      const int64_t at = (int64_t)g * w_gstride + kk;
+      float step = s;
+      if (mu != 0.f) {
+        step = fmaf(mu, pvbias[at], s);
+        pvbias[at] = step;
+      }
+      pbias[at] = fmaf(-lr, step, pbias[at]);
+    }
   }
 }
 
@@ -313,8 +333,7 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * kColsPerCta) * sizeof(float);
   const size_t esz = a_bf16 ? 2 : 4;
   const int pair_ok = (a.K % 2 == 0) && reinterpret_cast<uintptr_t>(a.A) % (2 * esz) == 0 &&
-                      (a.dPrev == nullptr || reinterpret_cast<uintptr_t>(a.dPrev) % (2 * esz) == 0) &&
-                      (a.dPrevLo == nullptr || reinterpret_cast<uintptr_t>(a.dPrevLo) % 8 == 0);
+                      (a.dPrev == nullptr || reinterpret_cast<uintptr_t>(a.dPrev) % (2 * esz) == 0);
   if (a_bf16) {
     auto kern = head_bwd_kernel<__nv_bfloat16>;
     static bool configured = false;
@@ -323,9 +342,9 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
       if (e != cudaSuccess) return e;
       configured = true;
     }
-    kern<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo,
-                                       a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev), nullptr, a.B,
-                                       a.C, a.K, a.lr, a.mu, pair_ok);
+    kern<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb,
+                                       a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev),
+                                       a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
   } else {
     auto kern = head_bwd_kernel<float>;
     static bool configured = false;
@@ -334,9 +353,9 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
       if (e != cudaSuccess) return e;
       configured = true;
     }
-    kern<<<grid, kThreads, smem, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.Wlo, a.bias,
-                                       a.vbias, a.w_gstride, static_cast<float*>(a.dPrev), a.dPrevLo, a.B, a.C, a.K,
-                                       a.lr, a.mu, pair_ok);
+    kern<<<grid, kThreads, smem, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.bias,
+                                       a.vbias, a.w_gstride, static_cast<float*>(a.dPrev),
+                                       a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
   }
   return cudaGetLastError();
 }

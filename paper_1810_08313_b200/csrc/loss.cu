@@ -16,19 +16,17 @@ namespace {
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ void put(float* p, float v) { *p = v; }
 __device__ __forceinline__ void put(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 template <typename TD>
 __global__ void __launch_bounds__(kThreads)
 loss_kernel(const float* __restrict__ logits, const void* __restrict__ y, const int64_t* __restrict__ row_off,
-            TD* __restrict__ dZ, float* __restrict__ dZlo, float* __restrict__ loss_out, int B, int C, int kind) {
+            TD* __restrict__ dZ, float* __restrict__ loss_out, int B, int C, int kind) {
   __shared__ float red[kThreads];
   const int g = blockIdx.x;
   const float* z = logits + (int64_t)g * B * C;
   TD* dz = dZ ? dZ + (int64_t)g * B * C : nullptr;
-  float* dzlo = (dZ && dZlo) ? dZlo + (int64_t)g * B * C : nullptr;
   const int64_t r0 = row_off[g];
   const float invB = 1.0f / (float)B;
   float part = 0.f;
@@ -48,7 +46,6 @@ loss_kernel(const float* __restrict__ logits, const void* __restrict__ y, const 
           const float p = expf(zb[c] - mx) * inv;
           const float d = (p - (c == label ? 1.f : 0.f)) * invB;
           put(dz + (int64_t)b * C + c, d);
-          if (dzlo) dzlo[(int64_t)b * C + c] = tf32_lo(d);
         }
       }
     } else {
@@ -56,7 +53,6 @@ loss_kernel(const float* __restrict__ logits, const void* __restrict__ y, const 
       const float r = zb[0] - t;
       part += 0.5f * r * r;
       if (dz) put(dz + b, r * invB);
-      if (dzlo) dzlo[b] = tf32_lo(r * invB);
     }
   }
   red[threadIdx.x] = part;
@@ -107,53 +103,15 @@ to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, i
   for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
-__global__ void __launch_bounds__(kThreads)
-split_lo_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
-  const int64_t step = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) dst[i] = tf32_lo(src[i]);
-}
-
-// one block per mini-batch row
-__global__ void __launch_bounds__(kThreads)
-gather_lo_kernel(const float* __restrict__ X, const int64_t* __restrict__ row_off, float* __restrict__ dst, int B, int d) {
-  const int g = blockIdx.y, b = blockIdx.x;
-  const float* src = X + (row_off[g] + b) * (int64_t)d;
-  float* out = dst + ((int64_t)g * B + b) * d;
-  if (d % 4 == 0) {
-    for (int i = threadIdx.x; i < d / 4; i += kThreads) {
-      const float4 v = reinterpret_cast<const float4*>(src)[i];
-      reinterpret_cast<float4*>(out)[i] = make_float4(tf32_lo(v.x), tf32_lo(v.y), tf32_lo(v.z), tf32_lo(v.w));
-    }
-  } else {
-    for (int i = threadIdx.x; i < d; i += kThreads) out[i] = tf32_lo(src[i]);
-  }
-}
-
 }  // namespace
-
-int launch_split_lo(const float* src, float* dst, int64_t n, cudaStream_t st, int64_t* launches) {
-  if (n <= 0) return cudaSuccess;
-  if (launches) ++*launches;
-  int64_t gx = (n + kThreads - 1) / kThreads;
-  if (gx > 148 * 16) gx = 148 * 16;
-  split_lo_kernel<<<(unsigned)gx, kThreads, 0, st>>>(src, dst, n);
-  return cudaGetLastError();
-}
-
-int launch_gather_lo(const float* X, const int64_t* row_off, float* dst, int groups, int B, int d, cudaStream_t st,
-                     int64_t* launches) {
-  if (launches) ++*launches;
-  gather_lo_kernel<<<dim3((unsigned)B, (unsigned)groups), kThreads, 0, st>>>(X, row_off, dst, B, d);
-  return cudaGetLastError();
-}
 
 int launch_loss(const LossArgs& a, bool dz_bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
   if (dz_bf16)
     loss_kernel<__nv_bfloat16><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<__nv_bfloat16*>(a.dZ),
-                                                              nullptr, a.loss_out, a.B, a.C, a.loss_kind);
+                                                              a.loss_out, a.B, a.C, a.loss_kind);
   else
-    loss_kernel<float><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<float*>(a.dZ), a.dZlo,
+    loss_kernel<float><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<float*>(a.dZ),
                                                       a.loss_out, a.B, a.C, a.loss_kind);
   return cudaGetLastError();
 }

@@ -66,16 +66,13 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   auto take = [&](size_t bytes) { size_t at = off; off = round_up_sz(off + bytes, A); return at; };
   lay.params_off = take((size_t)m * lay.stride * 4);
   lay.mom_off = take((size_t)m * lay.stride * 4);
-  lay.shadow_off = take((size_t)m * lay.stride * (lay.bf16 ? 2 : 4));
+  if (lay.bf16) lay.shadow_off = take((size_t)m * lay.stride * 2);
   for (int l = 1; l < lay.L; ++l) {
     lay.act_off[l] = take((size_t)m * batch * lay.dims[l] * esz);
-    if (!lay.bf16) lay.actlo_off[l] = take((size_t)m * batch * lay.dims[l] * 4);
   }
   for (int s = 0; s < 2; ++s) {
     lay.dz_off[s] = take((size_t)m * batch * lay.max_width * esz);
-    if (!lay.bf16) lay.dzlo_off[s] = take((size_t)m * batch * lay.max_width * 4);
   }
-  if (!lay.bf16) lay.xlo_off = take((size_t)m * batch * lay.dims[0] * 4);
   lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.dzl_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.rowloss_off = take((size_t)LS_MAX_REPLICAS * batch * 4);
@@ -129,21 +126,11 @@ struct ProfScope {
   }
 };
 
-// Refresh the operand copies of the weights (bf16 rounding, or the lo twin of fp32 models).
+// Refresh the bf16 operand copies of the weights (bf16 models).
 static int refresh_shadow(ls_handle* h) {
   const int64_t n = (int64_t)h->lay.m * h->lay.stride;
   if (h->lay.bf16) LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), n, h->stream, &h->launches));
-  else LS_CUDA(h, launch_split_lo(params_of(h), wlo_of(h), n, h->stream, &h->launches));
   return LS_OK;
-}
-
-static inline float* lo_at(const ls_handle* h, size_t off) {
-  return h->lay.bf16 ? nullptr : reinterpret_cast<float*>(h->state + off);
-}
-// fp32 models: does any tensor-core kernel read the mini-batch rows (layer 1 forward or update)?
-static inline bool needs_x_lo(const Layout& lay) {
-  return !lay.bf16 && ((lay.L > 1 && tc_shape_ok(true, lay.batch, lay.dims[1], lay.dims[0])) ||
-                       tc_shape_ok(true, lay.dims[1], lay.dims[0], lay.batch));
 }
 
 // One forward pass of `groups` mini-batches.  Group g reads rows
@@ -160,9 +147,6 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
   const bool bf = lay.bf16;
   const float* P = params_of(h) + replica0 * lay.stride;
   const __nv_bfloat16* S = bf ? shadow_of(h) + replica0 * lay.stride : nullptr;
-  if (needs_x_lo(lay))
-    LS_CUDA(h, launch_gather_lo(static_cast<const float*>(x), row_off_dev, lo_at(h, lay.xlo_off), groups, lay.batch,
-                                lay.dims[0], h->stream, &h->launches));
   for (int l = 0; l < lay.L; ++l) {
     if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
       // narrow output layer: product, loss and dZ in one kernel
@@ -185,10 +169,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       TcFwdArgs t;
       t.fp32 = !bf;
       t.maps.a = (l == 0) ? xmap.k : &h->maps.act[l];
-      t.maps.a_lo = (l == 0) ? &h->maps.x_lo : &h->maps.act_lo[l];
       t.maps.b = &h->maps.w[l];
-      t.maps.b_lo = &h->maps.w_lo[l];
-      t.Clo = lo_at(h, lay.actlo_off[l + 1]);
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.w_z0 = (int)replica0; t.w_zstep = w_gstride != 0 ? 1 : 0;
       t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
@@ -209,7 +190,6 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
     a.bias_gstride = w_gstride;
     const bool last = (l == lay.L - 1);
     a.C = last ? (void*)(h->state + lay.logits_off) : (void*)(h->state + lay.act_off[l + 1]);
-    a.Clo = last ? nullptr : lo_at(h, lay.actlo_off[l + 1]);
     a.M = lay.batch; a.N = lay.dims[l + 1]; a.K = lay.dims[l]; a.groups = groups;
     a.relu = last ? 0 : 1;
     ProfScope ps(h, LS_K_FWD, l);
@@ -219,7 +199,6 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
   la.logits = reinterpret_cast<const float*>(h->state + lay.logits_off);
   la.y = y; la.row_off = row_off_dev;
   la.dZ = want_dz ? (void*)(h->state + lay.dz_off[0]) : nullptr;
-  la.dZlo = want_dz ? lo_at(h, lay.dzlo_off[0]) : nullptr;
   la.loss_out = loss_out;
   la.B = lay.batch; la.C = lay.dims[lay.L]; la.groups = groups; la.loss_kind = h->spec.loss;
   ProfScope ps(h, LS_K_LOSS, 0);
@@ -236,6 +215,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
   if (rc != LS_OK) return rc;
   int cur = 0;
+  bool bias_done[LS_MAX_LAYERS] = {false};     // bias l already updated by the kernel that produced dZ_l
   for (int l = lay.L - 1; l >= 0; --l) {
     void* dZ = h->state + lay.dz_off[cur];
     if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
@@ -246,12 +226,13 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       a.dZ = reinterpret_cast<const float*>(h->state + lay.dzl_off);
       a.W = params_of(h) + lay.w_off[l]; a.V = mom_of(h) + lay.w_off[l];
       a.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
-      a.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
       a.bias = lay.has_bias ? params_of(h) + lay.b_off[l] : nullptr;
       a.vbias = mom_of(h) + lay.b_off[l];
       a.w_gstride = lay.stride;
       a.dPrev = (l > 0) ? (void*)(h->state + lay.dz_off[cur ^ 1]) : nullptr;
-      a.dPrevLo = (l > 0) ? lo_at(h, lay.dzlo_off[cur ^ 1]) : nullptr;
+      a.pbias = (l > 0 && lay.has_bias) ? params_of(h) + lay.b_off[l - 1] : nullptr;
+      a.pvbias = mom_of(h) + (l > 0 ? lay.b_off[l - 1] : 0);
+      if (a.pbias != nullptr) bias_done[l - 1] = true;
       a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = lay.m;
       a.lr = h->lr; a.mu = h->mu;
       ProfScope ps(h, LS_K_DW, l);
@@ -264,13 +245,16 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       TcDxArgs t;
       t.fp32 = !bf;
       t.maps.a = &h->maps.dz[l];
-      t.maps.a_lo = &h->maps.dz_lo[l];
       t.maps.b = &mn.w[l];
-      t.maps.b_lo = &mn.w_lo[l];
       t.act = h->state + lay.act_off[l];
       t.C = h->state + lay.dz_off[cur ^ 1];
-      t.Clo = lo_at(h, lay.dzlo_off[cur ^ 1]);
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
+      t.bias = nullptr; t.vbias = nullptr; t.bias_gstride = lay.stride; t.lr = h->lr; t.mu = h->mu;
+      if (lay.has_bias && tc_dx_fuses_bias(!bf, t.M, t.N)) {
+        t.bias = params_of(h) + lay.b_off[l - 1];
+        t.vbias = mom_of(h) + lay.b_off[l - 1];
+        bias_done[l - 1] = true;
+      }
       t.err_flag = err_flag_of(h);
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_tc_dx(t, h->stream, &h->launches));
@@ -281,7 +265,6 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       d.w_gstride = lay.stride;
       d.act = h->state + lay.act_off[l];
       d.C = h->state + lay.dz_off[cur ^ 1];
-      d.Clo = lo_at(h, lay.dzlo_off[cur ^ 1]);
       d.M = lay.batch; d.N = lay.dims[l]; d.K = lay.dims[l + 1]; d.groups = lay.m;
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
@@ -290,14 +273,11 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       TcUpdateArgs t;
       t.fp32 = !bf;
       t.maps.a = &mn.dz[l];
-      t.maps.a_lo = &mn.dz_lo[l];
       t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
-      t.maps.b_lo = (l == 0) ? &mn.x_lo : &mn.act_lo[l];
       t.mapW = &h->maps.wf[l];
       t.mapV = &h->maps.vf[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
-      t.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
       t.w_gstride = lay.stride;
       t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
       t.lr = h->lr; t.mu = h->mu;
@@ -308,14 +288,11 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       TcDwArgs t;
       t.fp32 = !bf;
       t.maps.a = &mn.dz[l];
-      t.maps.a_lo = &mn.dz_lo[l];
       t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
-      t.maps.b_lo = (l == 0) ? &mn.x_lo : &mn.act_lo[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.W = params_of(h) + lay.w_off[l];
       t.V = mom_of(h) + lay.w_off[l];
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
-      t.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
       t.w_gstride = lay.stride;
       t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
       t.lr = h->lr; t.mu = h->mu;
@@ -330,7 +307,6 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
     w.W = params_of(h) + lay.w_off[l];
     w.V = mom_of(h) + lay.w_off[l];
     w.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
-    w.Wlo = bf ? nullptr : wlo_of(h) + lay.w_off[l];
     w.w_gstride = lay.stride;
     w.M = lay.dims[l + 1]; w.N = lay.dims[l]; w.B = lay.batch; w.groups = lay.m;
     w.lr = h->lr; w.mu = h->mu;
@@ -339,7 +315,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       LS_CUDA(h, launch_dw(w, bf, h->stream, &h->launches));
     }
     }
-    if (lay.has_bias) {
+    if (lay.has_bias && !bias_done[l]) {
       BiasArgs b;
       b.dZ = dZ;
       b.bias = params_of(h) + lay.b_off[l];
@@ -364,7 +340,7 @@ static int average(ls_handle* h) {
     ProfScope ps(h, LS_K_AVG, 0);
     BlockMomentum bm{anchor_of(h), blocku_of(h), h->lr, h->spec.block_momentum};
     LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                              shadow_of(h), wlo_of(h), h->stream, &h->launches, block ? &bm : nullptr));
+                              shadow_of(h), h->stream, &h->launches, block ? &bm : nullptr));
   }
   if (h->mu != 0.f && (h->spec.momentum_mode == LS_MOMENTUM_RESET || block))
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
@@ -509,16 +485,13 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
         if (lay.dims[l] % q == 0) {
           const void* wsrc = f ? (const void*)(params_of(h) + lay.w_off[l]) : (const void*)(shadow_of(h) + lay.w_off[l]);
           ok(tc_make_map_3d(&mp.w[l], wsrc, f, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
-          if (f) ok(tc_make_map_3d(&mp.w_lo[l], wlo_of(h) + lay.w_off[l], true, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
           if (l >= 1) {
             ok(tc_make_map_2d(&mp.act[l], h->state + lay.act_off[l], f, mn, rows, lay.dims[l]));
-            if (f) ok(tc_make_map_2d(&mp.act_lo[l], h->state + lay.actlo_off[l], true, mn, rows, lay.dims[l]));
           }
         }
         if (lay.dims[l + 1] % q == 0) {
           const int buf = (lay.L - 1 - l) & 1;
           ok(tc_make_map_2d(&mp.dz[l], h->state + lay.dz_off[buf], f, mn, rows, lay.dims[l + 1]));
-          if (f) ok(tc_make_map_2d(&mp.dz_lo[l], h->state + lay.dzlo_off[buf], true, mn, rows, lay.dims[l + 1]));
         }
       }
       if (!mn) {
@@ -531,7 +504,6 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
       if (lay.dims[0] % q == 0) {
         for (int s = 0; s < 2; ++s)
           ok(tc_make_map_2d(&mp.x_stage[s], h->state + lay.stage_x_off[s], f, mn, rows, lay.dims[0]));
-        if (f) ok(tc_make_map_2d(&mp.x_lo, h->state + lay.xlo_off, true, mn, rows, lay.dims[0]));
       }
     }
   }

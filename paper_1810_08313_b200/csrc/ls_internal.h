@@ -20,10 +20,9 @@ constexpr int64_t kAlignFloats = 64;   // every tensor and every replica starts 
 // same for the fp32 master copy, the momentum buffer and the operand copy);
 // offsets inside the state block are in bytes.
 //
-// Operand copies.  bf16 models keep a bf16 rounding of the weights.  fp32 models keep, for every
-// tensor that can be a matrix-product operand (weights, layer inputs, dZ, the gathered mini-batch),
-// a "lo" twin holding x - tf32(x): the tensor-core kernels read x as its tf32 upper part and add
-// the lo products (see gemm_tc.cu).  Whoever writes such a tensor writes its twin.
+// Operand copies.  bf16 models keep a bf16 rounding of the weights; whoever writes the weights writes
+// the copy.  fp32 models need none: the tensor-core kernels split every fp32 operand tile into its
+// tf32 upper part and the remainder in shared memory (see gemm_tc.cu).
 struct Layout {
   int L = 0;
   int dims[LS_MAX_LAYERS + 1] = {0};
@@ -39,12 +38,9 @@ struct Layout {
   int64_t w_flat[LS_MAX_LAYERS] = {0}; // offsets in the flat interface layout
   int64_t b_flat[LS_MAX_LAYERS] = {0};
   size_t params_off = 0, mom_off = 0;
-  size_t shadow_off = 0;                     // bf16 [m][stride] (bf16 models) or float lo twin [m][stride] (fp32)
+  size_t shadow_off = 0;                     // bf16 [m][stride] copy of the weights (bf16 models)
   size_t act_off[LS_MAX_LAYERS + 1] = {0};   // post-ReLU activations = inputs of layers 1..L-1
-  size_t actlo_off[LS_MAX_LAYERS + 1] = {0}; // their lo twins (fp32 models)
   size_t dz_off[2] = {0, 0};                 // ping-pong gradient buffers [m][batch][max_width]
-  size_t dzlo_off[2] = {0, 0};
-  size_t xlo_off = 0;                        // lo twin of the current mini-batches [m][batch][dims[0]] (fp32 models)
   size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
   size_t dzl_off = 0;                        // fp32 dZ of a narrow output layer [m][batch][dims[L]]
   size_t rowloss_off = 0;                    // per-sample losses [LS_MAX_REPLICAS][batch]
@@ -65,14 +61,12 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out);
 }  // namespace ls
 
 // TMA descriptors of the tensors the tensor-core kernels read (built once per handle).
-// The *_lo maps are used by fp32 models only.
 struct alignas(64) TcMaps {
-  CUtensorMap w[LS_MAX_LAYERS], w_lo[LS_MAX_LAYERS];      // weights as operands, 3-D [replica][out][in]
-  CUtensorMap act[LS_MAX_LAYERS], act_lo[LS_MAX_LAYERS];  // input of layer l >= 1, 2-D [m*batch][dims[l]]
-  CUtensorMap dz[LS_MAX_LAYERS], dz_lo[LS_MAX_LAYERS];    // dZ_l, 2-D [m*batch][dims[l+1]]
+  CUtensorMap w[LS_MAX_LAYERS];                           // weights as operands, 3-D [replica][out][in]
+  CUtensorMap act[LS_MAX_LAYERS];                         // input of layer l >= 1, 2-D [m*batch][dims[l]]
+  CUtensorMap dz[LS_MAX_LAYERS];                          // dZ_l, 2-D [m*batch][dims[l+1]]
   CUtensorMap x_data;                                     // bound dataset, 2-D [n_rows][dims[0]]
   CUtensorMap x_stage[2];                                 // staging buffers of host batches
-  CUtensorMap x_lo;                                       // lo twin of the current mini-batches
   CUtensorMap wf[LS_MAX_LAYERS], vf[LS_MAX_LAYERS];       // fp32 master weights / momentum, 32 x 32 blocks
 };
 
@@ -113,14 +107,11 @@ inline __nv_bfloat16* shadow_of(const ls_handle* h) {
 }
 inline float* anchor_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.anchor_off); }
 inline float* blocku_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.blocku_off); }
-inline float* wlo_of(const ls_handle* h) {
-  return h->lay.bf16 ? nullptr : reinterpret_cast<float*>(h->state + h->lay.shadow_off);
-}
 
 // ---- averaging (average.cu) ---------------------------------------------
 // n_buf buffers of m vectors each; buffer b starts at base + b*buf_stride floats,
-// vector j of it at + j*stride.  shadow / lo (optional, same strides) receive the
-// bf16 rounding / the tf32 remainder of the mean of buffer 0.  Returns a cudaError_t.
+// vector j of it at + j*stride.  shadow (optional, same strides) receives the
+// bf16 rounding of the mean of buffer 0.  Returns a cudaError_t.
 // bm (optional, n_buf == 1): block momentum, see average.cu; anchor and u are vectors of n floats.
 struct BlockMomentum {
   float* anchor;
@@ -128,7 +119,7 @@ struct BlockMomentum {
   float lr, beta;
 };
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
-                   __nv_bfloat16* shadow, float* lo, cudaStream_t st, int64_t* launches,
+                   __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
                    const BlockMomentum* bm = nullptr);
 
 // ---- fp32-accumulate CUDA-core grouped GEMMs (gemm_simt.cu) ---------------
@@ -140,7 +131,6 @@ struct FwdArgs {           // Z = A W^T + b, optional ReLU
   const float* bias;       // fp32 master bias of group 0 or null
   int64_t bias_gstride;
   void* C;                 // [groups][M][N]
-  float* Clo;              // lo twin of C (fp32 outputs) or null
   int M, N, K, groups;
   int relu;
 };
@@ -150,7 +140,6 @@ struct DxArgs {            // dZ_prev = (dZ W) * 1[act > 0]
   int64_t w_gstride;
   const void* act;         // [groups][M][N] post-ReLU activation of the previous layer
   void* C;                 // [groups][M][N]
-  float* Clo;
   int M, N, K, groups;
 };
 struct DwArgs {            // G = dZ^T A ; v = mu v + G ; W -= lr v ; operand copy of W
@@ -160,7 +149,6 @@ struct DwArgs {            // G = dZ^T A ; v = mu v + G ; W -= lr v ; operand co
   float* W;                // fp32 master [M][N] of group 0
   float* V;                // momentum, same layout (unused when mu == 0)
   __nv_bfloat16* Wb;       // bf16 copy or null
-  float* Wlo;              // lo twin or null
   int64_t w_gstride;
   int M, N, B, groups;
   float lr, mu;
@@ -175,7 +163,6 @@ struct LossArgs {
   const void* y;           // int32 labels or float targets of the bound rows
   const int64_t* row_off;  // device, per group first row in y
   void* dZ;                // [groups][B][C] or null (forward only)
-  float* dZlo;             // lo twin (fp32 dZ) or null
   float* loss_out;         // [groups] or null
   int B, C, groups;
   int loss_kind;
@@ -204,8 +191,10 @@ struct HeadFwdArgs {
 struct HeadBwdArgs {
   const void* A; const int64_t* a_row_off;
   const float* dZ;
-  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; float* bias; float* vbias; int64_t w_gstride;
-  void* dPrev; float* dPrevLo;               // dZ of the layer below [groups][B][K] (+ lo twin) or null
+  float* W; float* V; __nv_bfloat16* Wb; float* bias; float* vbias; int64_t w_gstride;
+  void* dPrev;                               // dZ of the layer below [groups][B][K] or null
+  float* pbias; float* pvbias;               // bias / its momentum of the layer below (updated from the column
+                                             // sums of dPrev) or null; replica stride w_gstride
   int B, C, K, groups;
   float lr, mu;
 };
@@ -215,11 +204,6 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
 
 // fp32 -> bf16 copy of n elements (refresh of the weight copies)
 int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches);
-// dst = src - tf32(src) for n elements (refresh of the lo twins)
-int launch_split_lo(const float* src, float* dst, int64_t n, cudaStream_t st, int64_t* launches);
-// lo twin of the mini-batches: dst[g][b][:] = lo(X[row_off[g] + b][:]) for g < groups, b < B
-int launch_gather_lo(const float* X, const int64_t* row_off, float* dst, int groups, int B, int d, cudaStream_t st,
-                     int64_t* launches);
 
 // ---- tcgen05 grouped GEMMs (gemm_tc.cu) -------------------------------------
 int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols);
@@ -229,7 +213,7 @@ int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64
                          int64_t gstride);
 bool tc_shape_ok(bool fp32, int M, int N, int K);   // output rows, output columns, contraction length
 struct TcOperandMaps {
-  const CUtensorMap *a, *b, *a_lo, *b_lo;   // lo maps: fp32 only
+  const CUtensorMap *a, *b;
 };
 struct TcFwdArgs {
   TcOperandMaps maps;        // a: [rows][K] input (dataset rows through row_off, else group g at row g*M); b: weights
@@ -237,22 +221,27 @@ struct TcFwdArgs {
   const int64_t* row_off;
   int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
   const float* bias; int64_t bias_gstride;
-  void* C; float* Clo;       // [groups][M][N] bf16, or fp32 + lo twin
+  void* C;                   // [groups][M][N] bf16 or fp32
   int M, N, K, groups, relu;
   int* err_flag;
 };
 struct TcDxArgs {
   TcOperandMaps maps;        // a: dZ_l [groups*M][K]; b: weights
   bool fp32;
-  const void* act; void* C; float* Clo;
+  const void* act; void* C;
   int M, N, K, groups;
+  // bias / its momentum of the layer that produced `act` (group 0; replica stride bias_gstride): updated
+  // from the column sums of C inside the kernel when tc_dx_fuses_bias(); else null
+  float* bias; float* vbias; int64_t bias_gstride; float lr, mu;
   int* err_flag;
 };
+// whether launch_tc_dx can also apply the bias update (every output tile holds all M rows)
+bool tc_dx_fuses_bias(bool fp32, int M, int N);
 struct TcDwArgs {
   TcOperandMaps maps;        // a: dZ_l [groups*B][M]; b: layer input [rows][N]
   bool fp32;
   const int64_t* row_off;
-  float* W; float* V; __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride;
+  float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride;
   int M, N, B, groups;
   float lr, mu;
   int* err_flag;
@@ -264,7 +253,7 @@ struct TcUpdateArgs {
   const CUtensorMap* mapV;   // momentum, same shape
   bool fp32;
   const int64_t* row_off;
-  __nv_bfloat16* Wb; float* Wlo; int64_t w_gstride;
+  __nv_bfloat16* Wb; int64_t w_gstride;
   int M, N, B, groups;
   float lr, mu;
   int* err_flag;

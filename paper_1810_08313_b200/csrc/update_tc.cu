@@ -5,12 +5,14 @@
 //     v <- mu v + G ;  W <- W - eta v ;  refresh the operand copy of W
 //
 // The gradient never leaves the SM.  The kernel is bound by the read-modify-write
-// of W and v (16 bytes per parameter with momentum, plus the operand copy), so it
+// of W and v (16 bytes per parameter with momentum, plus the bf16 copy of a bf16 model), so it
 // is built as a stream: one CTA per SM walks over output tiles, and
 //
 //   warp 0      TMA producer of the dZ / A operand tiles (ring of stages)
 //   warp 1      tcgen05.mma issuer; two TMEM accumulators, so the products of tile t+1
 //               overlap the update of tile t
+//   warps 2-3   fp32 models: write lo = x - tf32(x) of each operand stage beside it in shared
+//               memory (three tf32 MMAs per product: lo*hi + hi*lo + hi*hi)
 //   warps 4-7   update warps.  Each owns 32 rows of the tile and a private ring of
 //               shared-memory slots: TMA loads bring its 32 x 32 blocks of W and v in
 //               (issued up to a whole tile ahead), the warp adds the TMEM gradient in
@@ -38,18 +40,19 @@ struct UParams {
   int rows_per_group;                  // = batch
   float lr, mu;
   __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
-  float* Wlo;                          // lo twin of W (fp32 models) or null
   int64_t w_gstride;                   // elements between replicas
   int* err_flag;
 };
 
+// Operand stages are filled by TMA; fp32 models add one buffer for the lo parts of the stage in use.
 template <bool TF32, int STAGES, int R>
 struct USmem {
-  static constexpr int kTiles = TF32 ? 2 : 1;
-  static constexpr int kStageBytes = kTiles * (BM + BN) * KB_BYTES;
+  static constexpr int kLoStages = TF32 ? 1 : 0;
+  static constexpr int kStageBytes = (BM + BN) * KB_BYTES;
+  static constexpr int kOperandBytes = (STAGES + kLoStages) * kStageBytes;
   static constexpr int kRingBytes = 4 * R * kSlotBytes;
-  static constexpr int kBars = 2 * STAGES + 4 + 4 * R;
-  static constexpr int kTotal = 1024 + STAGES * kStageBytes + kRingBytes + kBars * 8 + 16;
+  static constexpr int kBars = 2 * STAGES + 2 + 4 + 4 * R;
+  static constexpr int kTotal = 1024 + kOperandBytes + kRingBytes + kBars * 8 + 16;
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
 
@@ -72,7 +75,6 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
                "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                : "memory");
 }
-__device__ __forceinline__ float tf32_lo(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
 template <int ELEMS>
 __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, int tile0, int extent,
@@ -85,7 +87,6 @@ __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, 
 template <bool TF32, int STAGES, int R>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmAlo, const __grid_constant__ CUtensorMap tmBlo,
                  const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmV, const UParams p) {
   using L = USmem<TF32, STAGES, R>;
   constexpr int EB = TF32 ? 4 : 2;
@@ -95,18 +96,21 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN);
   constexpr uint32_t SW = TF32 ? kSwizzle128B_32B : kSwizzle128B;
   constexpr uint32_t SBO = TF32 ? 512 : 1024;
-  constexpr int kABytes = BM * KB_BYTES, kBBytes = BN * KB_BYTES;
+  constexpr int kABytes = BM * KB_BYTES;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  uint8_t* ring_base = smem + STAGES * L::kStageBytes;
+  uint8_t* lo_buf = smem + STAGES * L::kStageBytes;
+  uint8_t* ring_base = smem + L::kOperandBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(ring_base + L::kRingBytes);
   uint64_t* empty = full + STAGES;
   uint64_t* tmem_full = empty + STAGES;       // [2]
   uint64_t* tmem_empty = tmem_full + 2;       // [2]
   uint64_t* wv_full = tmem_empty + 2;         // [4][R]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wv_full + 4 * R);
+  uint64_t* lo_full = wv_full + 4 * R;        // fp32: lo parts of the current stage written ...
+  uint64_t* lo_empty = lo_full + 1;           // ... and read by the tensor core
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(lo_empty + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = p.M / BM, n_tiles = p.N / BN;
@@ -117,11 +121,11 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(lo_full, 2); mbar_init(lo_empty, 1);
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
     for (int i = 0; i < 4 * R; ++i) mbar_init(&wv_full[i], 1);
     fence_mbar_init();
     prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmW); prefetch_tmap(&tmV);
-    if (TF32) { prefetch_tmap(&tmAlo); prefetch_tmap(&tmBlo); }
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 2 * BN);
@@ -150,12 +154,26 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           uint8_t* sb = sa + kABytes;
           issue_mn_tile<ELEMS>(sa, &tmA, &full[s], m0, BM, a_row + kb * ELEMS);
           issue_mn_tile<ELEMS>(sb, &tmB, &full[s], n0, BN, b_row + kb * ELEMS);
-          if (TF32) {
-            issue_mn_tile<ELEMS>(sb + kBBytes, &tmAlo, &full[s], m0, BM, a_row + kb * ELEMS);
-            issue_mn_tile<ELEMS>(sb + kBBytes + kABytes, &tmBlo, &full[s], n0, BN, a_row + kb * ELEMS);
-          }
         }
       }
+    }
+  } else if (TF32 && (warp == 2 || warp == 3)) {
+    // ---- splitter warps: the lo copy has the layout of the tile it comes from ------------
+    const int tid = threadIdx.x - 64;
+    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total_it = my_tiles * num_kb;
+    for (int it = 0; it < total_it; ++it) {
+      const int s = it % STAGES;
+      bool got = mbar_wait(&full[s], (it / STAGES) & 1);
+      if (got && it >= 1) got = mbar_wait(lo_empty, (it - 1) & 1);
+      if (!__all_sync(0xffffffffu, got)) {
+        if (lane == 0) atomicExch(p.err_flag, 16);
+        break;
+      }
+      split_lo_smem(smem_u32(stage_base + s * L::kStageBytes), smem_u32(lo_buf), L::kStageBytes, tid, 64);
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(lo_full);
     }
   } else if (warp == 1) {
     // ---- MMA issuer -----------------------------------------------------------------
@@ -170,6 +188,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&full[s], (it / STAGES) & 1)) { atomicExch(p.err_flag, 13); ok = false; break; }
+          if (TF32 && !mbar_wait(lo_full, it & 1)) { atomicExch(p.err_flag, 17); ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
           const uint32_t b_addr = a_addr + kABytes;
@@ -180,8 +199,8 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t db = make_smem_desc(b_addr + adv, CHUNK_BYTES, SBO, SW);
             const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
             if (TF32) {
-              const uint64_t dal = make_smem_desc(b_addr + kBBytes + adv, CHUNK_BYTES, SBO, SW);
-              const uint64_t dbl = make_smem_desc(b_addr + kBBytes + kABytes + adv, CHUNK_BYTES, SBO, SW);
+              const uint64_t dal = make_smem_desc(smem_u32(lo_buf) + adv, CHUNK_BYTES, SBO, SW);
+              const uint64_t dbl = make_smem_desc(smem_u32(lo_buf) + kABytes + adv, CHUNK_BYTES, SBO, SW);
               mma_tf32(d_tmem, dal, db, IDESC, acc);
               mma_tf32(d_tmem, da, dbl, IDESC, 1u);
               mma_tf32(d_tmem, da, db, IDESC, 1u);
@@ -190,6 +209,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
           mma_commit(&empty[s]);
+          if (TF32) mma_commit(lo_empty);
         }
         if (ok) mma_commit(&tmem_full[buf]);
       }
@@ -264,11 +284,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           *reinterpret_cast<float4*>(slot + off) = make_float4(ws[0], ws[1], ws[2], ws[3]);
           if (has_v) *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) = make_float4(vs[0], vs[1], vs[2], vs[3]);
           // operand copy of the new weights, collected so that it leaves in whole 32-byte sectors
-          if (TF32) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) cp[(jj & 1) * 4 + e] = __float_as_uint(tf32_lo(ws[e]));
-            if (jj & 1) st_global_v8(p.Wlo + at + (jj - 1) * 4, cp);
-          } else if (p.Wb != nullptr) {
+          if (!TF32 && p.Wb != nullptr) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
             __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
             cp[(jj & 3) * 2] = *reinterpret_cast<uint32_t*>(&lo);
@@ -325,12 +341,10 @@ int launch_update(const TcUpdateArgs& a, cudaStream_t st) {
   UParams p{};
   p.M = a.M; p.N = a.N; p.K = a.B; p.groups = a.groups;
   p.b_row_off = a.row_off; p.rows_per_group = a.B;
-  p.lr = a.lr; p.mu = a.mu; p.Wb = a.Wb; p.Wlo = a.Wlo; p.w_gstride = a.w_gstride; p.err_flag = a.err_flag;
+  p.lr = a.lr; p.mu = a.mu; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.err_flag = a.err_flag;
   const int total = (a.M / BM) * (a.N / BN) * a.groups;
   const int grid = total < num_sms() ? total : num_sms();
-  const CUtensorMap* alo = TF32 ? a.maps.a_lo : a.maps.a;
-  const CUtensorMap* blo = TF32 ? a.maps.b_lo : a.maps.b;
-  kern<<<grid, kThreads, L::kTotal, st>>>(*a.maps.a, *a.maps.b, *alo, *blo, *a.mapW, *a.mapV, p);
+  kern<<<grid, kThreads, L::kTotal, st>>>(*a.maps.a, *a.maps.b, *a.mapW, *a.mapV, p);
   return cudaGetLastError();
 }
 
@@ -342,7 +356,7 @@ bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
 
 int launch_tc_update(const TcUpdateArgs& a, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
-  if (a.fp32) return launch_update<true, 2, 3>(a, st);
+  if (a.fp32) return launch_update<true, 3, 3>(a, st);
   return launch_update<false, 3, 4>(a, st);
 }
 
