@@ -72,6 +72,8 @@ template <int M, int W, bool BM>
 __global__ void __launch_bounds__(kThreads)
 average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
                __nv_bfloat16* __restrict__ shadow, BlockMomentum bm) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (i >= n_vec) return;
   const int m = M > 0 ? M : m_rt;
@@ -130,6 +132,8 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
                       __nv_bfloat16* __restrict__ shadow, BlockMomentum bm) {
+  grid_dep_wait();
+  grid_dep_launch();
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
   const float mf = (float)m;
   const int64_t i = first + (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -153,7 +157,7 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
 template <int W, bool BM>
 void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
                 __nv_bfloat16* shadow, const BlockMomentum& bm) {
-#define LS_AVG(M) average_kernel<M, W, BM><<<grid, kThreads, 0, st>>>(base, buf_stride, m, n_vec, stride, shadow, bm)
+#define LS_AVG(M) launch_dep(average_kernel<M, W, BM>, grid, dim3(kThreads), 0, st, 1, base, buf_stride, m, n_vec, stride, shadow, bm)
   switch (m) {
     case 2: LS_AVG(2); break;
     case 4: LS_AVG(4); break;
@@ -206,7 +210,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     const int64_t gx = (n - first + kThreads - 1) / kThreads;
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
-    average_scalar_kernel<<<grid, kThreads, 0, st>>>(base, buf_stride, m, first, n, stride, shadow, bm);
+    launch_dep(average_scalar_kernel, grid, dim3(kThreads), 0, st, 1, base, buf_stride, m, first, n, stride, shadow, bm);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

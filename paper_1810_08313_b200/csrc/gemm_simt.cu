@@ -92,6 +92,8 @@ gemm_kernel(const TA* A, int64_t a_gstride, const int64_t* a_row_off, int64_t ld
   static_assert(BM == BN, "square tiles");
   __shared__ __align__(16) float As[BK][BM + PAD];
   __shared__ __align__(16) float Bs[BK][BN + PAD];
+  grid_dep_wait();
+  grid_dep_launch();
   const int g = blockIdx.z;
   const int i0 = blockIdx.y * BM, j0 = blockIdx.x * BN;
   const int tid = threadIdx.x;
@@ -221,10 +223,9 @@ int fwd_typed(const FwdArgs& a, cudaStream_t st) {
   EpiFwd<TC> epi{a.bias, a.bias_gstride, static_cast<TC*>(a.C), a.M, a.N, a.relu,
                  aligned(a.C, 4 * sizeof(TC)) && a.N % 4 == 0};
   const int64_t a_gs = (int64_t)a.M * a.K;
-  gemm_kernel<TA, true, TW, true, EpiFwd<TC>><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
-      A, a_gs, a.row_off, a.K, can_vec<TA>(A, a.K, a_gs), W, a.w_gstride, nullptr, a.K,
-      can_vec<TW>(W, a.K, a.w_gstride), a.M, a.N, a.K, epi);
-  return cudaGetLastError();
+  return launch_dep(gemm_kernel<TA, true, TW, true, EpiFwd<TC>>, grid_for(a.M, a.N, a.groups), dim3(kThreads), 0, st, 1,
+                    A, a_gs, a.row_off, a.K, can_vec<TA>(A, a.K, a_gs), W, a.w_gstride, nullptr, a.K,
+                    can_vec<TW>(W, a.K, a.w_gstride), a.M, a.N, a.K, epi);
 }
 
 template <typename T>
@@ -234,10 +235,9 @@ int dx_typed(const DxArgs& a, cudaStream_t st) {
   EpiDx<T> epi{static_cast<const T*>(a.act), static_cast<T*>(a.C), a.M, a.N,
                aligned(a.C, 4 * sizeof(T)) && aligned(a.act, 4 * sizeof(T)) && a.N % 4 == 0};
   const int64_t a_gs = (int64_t)a.M * a.K;
-  gemm_kernel<T, true, T, false, EpiDx<T>><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
-      dZ, a_gs, nullptr, a.K, can_vec<T>(dZ, a.K, a_gs), W, a.w_gstride, nullptr, a.N,
-      can_vec<T>(W, a.N, a.w_gstride), a.M, a.N, a.K, epi);
-  return cudaGetLastError();
+  return launch_dep(gemm_kernel<T, true, T, false, EpiDx<T>>, grid_for(a.M, a.N, a.groups), dim3(kThreads), 0, st, 1,
+                    dZ, a_gs, nullptr, a.K, can_vec<T>(dZ, a.K, a_gs), W, a.w_gstride, nullptr, a.N,
+                    can_vec<T>(W, a.N, a.w_gstride), a.M, a.N, a.K, epi);
 }
 
 template <typename T>
@@ -248,10 +248,9 @@ int dw_typed(const DwArgs& a, cudaStream_t st) {
             aligned(a.W, 16) && aligned(a.V, 16) && (a.Wb == nullptr || aligned(a.Wb, 8)) && a.N % 4 == 0 &&
                 a.w_gstride % 4 == 0};
   const int64_t dz_gs = (int64_t)a.B * a.M, a_gs = (int64_t)a.B * a.N;
-  gemm_kernel<T, false, T, false, EpiDw><<<grid_for(a.M, a.N, a.groups), kThreads, 0, st>>>(
-      dZ, dz_gs, nullptr, a.M, can_vec<T>(dZ, a.M, dz_gs), A, a_gs, a.row_off, a.N, can_vec<T>(A, a.N, a_gs),
-      a.M, a.N, a.B, epi);
-  return cudaGetLastError();
+  return launch_dep(gemm_kernel<T, false, T, false, EpiDw>, grid_for(a.M, a.N, a.groups), dim3(kThreads), 0, st, 1,
+                    dZ, dz_gs, nullptr, a.M, can_vec<T>(dZ, a.M, dz_gs), A, a_gs, a.row_off, a.N,
+                    can_vec<T>(A, a.N, a_gs), a.M, a.N, a.B, epi);
 }
 
 }  // namespace

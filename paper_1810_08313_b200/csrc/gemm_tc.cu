@@ -203,6 +203,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();        // everything above overlapped the previous kernel; its results are needed from here on
+  grid_dep_launch();
 
   // epilogue-warp state (warps 2-5): this thread owns output row `row`
   const int q = warp & 3;
@@ -519,24 +521,7 @@ int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_
     configured = true;
   }
   dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / (BM * MT)), (unsigned)groups);
-  if (SPLIT == 1) {
-    kern<<<grid, TF32 ? kThreadsFp32 : kThreadsBf16, L::kTotal, st>>>(*mp.a, *mp.b, p);
-    return cudaGetLastError();
-  }
-  // the SPLIT CTAs that share an output tile form one cluster along x
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = dim3(TF32 ? kThreadsFp32 : kThreadsBf16);
-  cfg.dynamicSmemBytes = L::kTotal;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = SPLIT;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, *mp.a, *mp.b, p);
+  return launch_dep(kern, grid, dim3(TF32 ? kThreadsFp32 : kThreadsBf16), L::kTotal, st, SPLIT, *mp.a, *mp.b, p);
 }
 
 // fp32 forward / backward: tile width and K split.  128-wide tiles when N allows; K is split over a

@@ -51,6 +51,8 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   __shared__ float zs[kRowsPerCta][CMAX];
   __shared__ unsigned int is_last;
   __shared__ float red[kThreads];
+  grid_dep_wait();
+  grid_dep_launch();
   const int g = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
@@ -189,6 +191,8 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   extern __shared__ float sm[];
   float* dz = sm;                                   // [B][C]
   float* part = sm + (size_t)B * C;                 // [8][CMAX][kColsPerCta]
+  grid_dep_wait();
+  grid_dep_launch();
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int k = blockIdx.x * kColsPerCta + cx * 2;  // this thread's columns k, k + 1
@@ -317,14 +321,12 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   const int vec_ok = (a.K % 4 == 0) && (reinterpret_cast<uintptr_t>(a.A) % 16 == 0) &&
                      (reinterpret_cast<uintptr_t>(a.W) % 16 == 0) && (a.w_gstride % 4 == 0);
   if (a_bf16)
-    head_fwd_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W,
-                                                             a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss,
-                                                             a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
-  else
-    head_fwd_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.W, a.w_gstride,
-                                                      a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out,
-                                                      a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
-  return cudaGetLastError();
+    return launch_dep(head_fwd_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, st, 1,
+                      static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off,
+                      a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
+  return launch_dep(head_fwd_kernel<float>, grid, dim3(kThreads), 0, st, 1, static_cast<const float*>(a.A),
+                    a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters,
+                    a.B, a.C, a.K, a.loss_kind, vec_ok);
 }
 
 int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
@@ -342,9 +344,9 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
       if (e != cudaSuccess) return e;
       configured = true;
     }
-    kern<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb,
-                                       a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev),
-                                       a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
+    return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const __nv_bfloat16*>(a.A), a.a_row_off,
+                      a.dZ, a.W, a.V, a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev),
+                      a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
   } else {
     auto kern = head_bwd_kernel<float>;
     static bool configured = false;
@@ -353,11 +355,10 @@ int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
       if (e != cudaSuccess) return e;
       configured = true;
     }
-    kern<<<grid, kThreads, smem, st>>>(static_cast<const float*>(a.A), a.a_row_off, a.dZ, a.W, a.V, a.Wb, a.bias,
-                                       a.vbias, a.w_gstride, static_cast<float*>(a.dPrev),
-                                       a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
+    return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const float*>(a.A), a.a_row_off, a.dZ,
+                      a.W, a.V, a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<float*>(a.dPrev),
+                      a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace ls

@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(kThreads)
 loss_kernel(const float* __restrict__ logits, const void* __restrict__ y, const int64_t* __restrict__ row_off,
             TD* __restrict__ dZ, float* __restrict__ loss_out, int B, int C, int kind) {
   __shared__ float red[kThreads];
+  grid_dep_wait();
+  grid_dep_launch();
   const int g = blockIdx.x;
   const float* z = logits + (int64_t)g * B * C;
   TD* dz = dZ ? dZ + (int64_t)g * B * C : nullptr;
@@ -71,6 +73,8 @@ bias_kernel(const TD* __restrict__ dZ, float* __restrict__ bias, float* __restri
   // 32 columns x 8 row slices per block: each thread adds every 8th row, then the 8 partial sums of a
   // column are added in slice order
   __shared__ float part[8][32];
+  grid_dep_wait();
+  grid_dep_launch();
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + cx;
@@ -108,24 +112,20 @@ to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, i
 int launch_loss(const LossArgs& a, bool dz_bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
   if (dz_bf16)
-    loss_kernel<__nv_bfloat16><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<__nv_bfloat16*>(a.dZ),
-                                                              a.loss_out, a.B, a.C, a.loss_kind);
-  else
-    loss_kernel<float><<<a.groups, kThreads, 0, st>>>(a.logits, a.y, a.row_off, static_cast<float*>(a.dZ),
-                                                      a.loss_out, a.B, a.C, a.loss_kind);
-  return cudaGetLastError();
+    return launch_dep(loss_kernel<__nv_bfloat16>, dim3(a.groups), dim3(kThreads), 0, st, 1, a.logits, a.y, a.row_off,
+                      static_cast<__nv_bfloat16*>(a.dZ), a.loss_out, a.B, a.C, a.loss_kind);
+  return launch_dep(loss_kernel<float>, dim3(a.groups), dim3(kThreads), 0, st, 1, a.logits, a.y, a.row_off,
+                    static_cast<float*>(a.dZ), a.loss_out, a.B, a.C, a.loss_kind);
 }
 
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
   dim3 grid((unsigned)((a.N + 31) / 32), (unsigned)a.groups);
   if (bf16)
-    bias_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(a.dZ), a.bias, a.vbias,
-                                                          a.gstride, a.B, a.N, a.lr, a.mu);
-  else
-    bias_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(a.dZ), a.bias, a.vbias, a.gstride, a.B, a.N,
-                                                  a.lr, a.mu);
-  return cudaGetLastError();
+    return launch_dep(bias_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, st, 1,
+                      static_cast<const __nv_bfloat16*>(a.dZ), a.bias, a.vbias, a.gstride, a.B, a.N, a.lr, a.mu);
+  return launch_dep(bias_kernel<float>, grid, dim3(kThreads), 0, st, 1, static_cast<const float*>(a.dZ), a.bias,
+                    a.vbias, a.gstride, a.B, a.N, a.lr, a.mu);
 }
 
 int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches) {

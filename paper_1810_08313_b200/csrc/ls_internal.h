@@ -100,6 +100,42 @@ namespace ls {
 
 constexpr uint32_t kMagic = 0x4c53474du;
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel of the step is launched with programmatic stream serialization: its CTAs may become
+// resident while the kernel before it in the stream is still draining, run their prologue (barrier
+// setup, tensor-memory allocation, descriptor prefetch) and then block in grid_dep_wait() until that
+// kernel has completed and its writes are visible.  No kernel touches global memory before the wait,
+// so the results are those of plain stream order; only launch latency and prologues overlap.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... P, typename... A>
+inline cudaError_t launch_dep(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              unsigned cluster_x, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {       // the CTAs that share an output tile form one cluster along x
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...);
+}
+#endif
+
 inline float* params_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.params_off); }
 inline float* mom_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.mom_off); }
 inline __nv_bfloat16* shadow_of(const ls_handle* h) {

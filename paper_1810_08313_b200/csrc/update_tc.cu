@@ -135,6 +135,8 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();        // the prologue above overlapped the previous kernel
+  grid_dep_launch();
 
   if (warp == 0) {
     // ---- operand producer ---------------------------------------------------------
@@ -344,8 +346,7 @@ int launch_update(const TcUpdateArgs& a, cudaStream_t st) {
   p.lr = a.lr; p.mu = a.mu; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.err_flag = a.err_flag;
   const int total = (a.M / BM) * (a.N / BN) * a.groups;
   const int grid = total < num_sms() ? total : num_sms();
-  kern<<<grid, kThreads, L::kTotal, st>>>(*a.maps.a, *a.maps.b, *a.mapW, *a.mapV, p);
-  return cudaGetLastError();
+  return launch_dep(kern, dim3(grid), dim3(kThreads), L::kTotal, st, 1, *a.maps.a, *a.maps.b, *a.mapW, *a.mapV, p);
 }
 
 }  // namespace
