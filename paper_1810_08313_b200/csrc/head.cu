@@ -20,7 +20,6 @@ namespace {
 constexpr int CMAX = 16;
 constexpr int kThreads = 256;
 constexpr int kRowsPerCta = 4;         // head_fwd: rows per CTA (the 8 warps split K)
-constexpr int kColsPerCta = 64;        // head_bwd: 32 lanes x 2 columns, 8 row slices
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -46,7 +45,7 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
                 int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
                 const int64_t* __restrict__ y_row_off, float* __restrict__ dZ, float* __restrict__ row_loss,
                 float* __restrict__ loss_out, unsigned int* __restrict__ counters, int B, int C, int K, int kind,
-                int vec_ok) {
+                int vec_ok, int defer_loss) {
   __shared__ float part[8][kRowsPerCta * CMAX];
   __shared__ float zs[kRowsPerCta][CMAX];
   __shared__ unsigned int is_last;
@@ -60,6 +59,18 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   const int b0 = blockIdx.x * kRowsPerCta;
   const int kchunk = (((K + 7) / 8) + 3) / 4 * 4;
   const int kw0 = warp * kchunk, kw1 = min(K, kw0 + kchunk);
+  // what the end of the kernel needs is requested now, so that it arrives with the operands:
+  // the bias (thread (row, class)) and the label / target of row `warp`
+  float bz = 0.f;
+  if (bias != nullptr && threadIdx.x < kRowsPerCta * CMAX && (threadIdx.x % CMAX) < C)
+    bz = bias[(int64_t)g * w_gstride + (threadIdx.x % CMAX)];
+  int label = 0;
+  float target = 0.f;
+  if (warp < kRowsPerCta && b0 + warp < B) {
+    const int64_t y0 = y_row_off[g];
+    if (kind == LS_LOSS_SOFTMAX_CE) label = static_cast<const int32_t*>(y)[y0 + b0 + warp];
+    else target = static_cast<const float*>(y)[y0 + b0 + warp];
+  }
 
   float acc[kRowsPerCta][CMAX];
 #pragma unroll
@@ -75,14 +86,14 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
         else a[r][0] = a[r][1] = a[r][2] = a[r][3] = 0.f;
       }
 #pragma unroll
-      for (int c = 0; c < CMAX; ++c)
-        if (c < C) {
-          float w[4];
-          load4(Wg + (int64_t)c * K + k, w);
+      for (int c = 0; c < CMAX; ++c) {
+        if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
+        float w[4];
+        load4(Wg + (int64_t)c * K + k, w);
 #pragma unroll
-          for (int r = 0; r < kRowsPerCta; ++r)
-            acc[r][c] = fmaf(a[r][3], w[3], fmaf(a[r][2], w[2], fmaf(a[r][1], w[1], fmaf(a[r][0], w[0], acc[r][c]))));
-        }
+        for (int r = 0; r < kRowsPerCta; ++r)
+          acc[r][c] = fmaf(a[r][3], w[3], fmaf(a[r][2], w[2], fmaf(a[r][1], w[1], fmaf(a[r][0], w[0], acc[r][c]))));
+      }
     }
   } else {
     for (int k = kw0 + lane; k < kw1; k += 32) {
@@ -115,7 +126,7 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     if (c < C) {
 #pragma unroll
       for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
-      if (bias) s += bias[(int64_t)g * w_gstride + c];
+      s += bz;
     }
     zs[r][c] = s;
   }
@@ -124,11 +135,9 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   if (warp < kRowsPerCta && b0 + warp < B) {
     // warp r finishes row r: lane c holds class c
     const int b = b0 + warp;
-    const int64_t y0 = y_row_off[g];
     const float z = (lane < C) ? zs[warp][lane] : -INFINITY;
     float loss, d;
     if (kind == LS_LOSS_SOFTMAX_CE) {
-      const int label = static_cast<const int32_t*>(y)[y0 + b];
       float mx = z;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -140,14 +149,16 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
       loss = (mx + logf(sum)) - ((label >= 0 && label < C) ? zy : mx);
       d = (e / sum - (lane == label ? 1.f : 0.f)) * invB;
     } else {
-      const float res = zs[warp][0] - static_cast<const float*>(y)[y0 + b];
+      const float res = zs[warp][0] - target;
       loss = 0.5f * res * res;
       d = res * invB;
     }
     if (lane == 0) row_loss[(int64_t)g * B + b] = loss;
     if (dZ != nullptr && lane < C) dZ[((int64_t)g * B + b) * C + lane] = d;
   }
-  // the last CTA of this replica adds the row losses in row order
+  // training steps leave the mean of the row losses to the backward kernel of this layer
+  if (defer_loss) return;
+  // the last CTA of this replica adds the row losses
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) is_last = (atomicInc(&counters[g], gridDim.x - 1) == gridDim.x - 1) ? 1u : 0u;
@@ -166,147 +177,215 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   }
 }
 
-__device__ __forceinline__ void load2(const float* p, float (&r)[2]) {
+__device__ __forceinline__ void load_cols(const float* p, float (&r)[1]) { r[0] = *p; }
+__device__ __forceinline__ void load_cols(const __nv_bfloat16* p, float (&r)[1]) { r[0] = __bfloat162float(*p); }
+__device__ __forceinline__ void load_cols(const float* p, float (&r)[2]) {
   const float2 v = *reinterpret_cast<const float2*>(p);
   r[0] = v.x; r[1] = v.y;
 }
-__device__ __forceinline__ void load2(const __nv_bfloat16* p, float (&r)[2]) {
+__device__ __forceinline__ void load_cols(const __nv_bfloat16* p, float (&r)[2]) {
   const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(p);
   r[0] = __low2float(v); r[1] = __high2float(v);
 }
-__device__ __forceinline__ void store2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
-__device__ __forceinline__ void store2(__nv_bfloat16* p, float a, float b) {
-  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b);
+__device__ __forceinline__ void store_cols(float* p, const float (&r)[1]) { *p = r[0]; }
+__device__ __forceinline__ void store_cols(__nv_bfloat16* p, const float (&r)[1]) { *p = __float2bfloat16_rn(r[0]); }
+__device__ __forceinline__ void store_cols(float* p, const float (&r)[2]) {
+  *reinterpret_cast<float2*>(p) = make_float2(r[0], r[1]);
+}
+__device__ __forceinline__ void store_cols(__nv_bfloat16* p, const float (&r)[2]) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(r[0], r[1]);
 }
 
-// One CTA = kColsPerCta (64) columns of the layer input of one replica: 32 lanes x 2 adjacent columns,
-// 8 warps = 8 interleaved row slices.  pair_ok: K is even and the pointers are aligned for 2-element accesses.
-template <typename TA>
+// One CTA = 32 * VEC columns of the layer input of one replica (VEC adjacent columns per lane); the 8
+// warps take interleaved rows.  VEC = 2 needs K even and 2-element alignment and is used when it still
+// leaves a CTA for every SM.  Every global operand the CTA needs (its columns of W, the W / v elements
+// it will update, the biases, the first rows of A) is requested before the first wait, so the kernel
+// costs about one memory round trip plus the arithmetic.  The CTA of column block 0 also adds the row
+// losses that head_fwd_kernel left behind (training steps) into the mini-batch mean.
+template <typename TA, int VEC>
 __global__ void __launch_bounds__(kThreads, 2)
 head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
                 float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb,
                 float* __restrict__ bias, float* __restrict__ vbias, int64_t w_gstride, TA* __restrict__ dPrev,
-                float* __restrict__ pbias, float* __restrict__ pvbias, int B, int C, int K, float lr, float mu,
-                int pair_ok) {
+                float* __restrict__ pbias, float* __restrict__ pvbias, const float* __restrict__ row_loss,
+                float* __restrict__ loss_out, int B, int C, int K, float lr, float mu) {
+  constexpr int COLS = 32 * VEC;
+  constexpr int kTrip = 16 / VEC;                   // rows per thread per trip
+  constexpr int kUpd = (CMAX * COLS) / kThreads;    // elements of the C x COLS block per thread, at most
   extern __shared__ float sm[];
   float* dz = sm;                                   // [B][C]
-  float* part = sm + (size_t)B * C;                 // [8][CMAX][kColsPerCta]
+  float* part = sm + (size_t)B * C;                 // [8][CMAX][COLS]
   grid_dep_wait();
   grid_dep_launch();
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int k = blockIdx.x * kColsPerCta + cx * 2;  // this thread's columns k, k + 1
-  const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
-  const bool in0 = k < K, in1 = k + 1 < K;
-
-  float wreg[CMAX][2], gw[CMAX][2];
+  const int k = blockIdx.x * COLS + cx * VEC;       // this thread's first column
+  bool in[VEC];
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    wreg[c][0] = (c < C && in0) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k] : 0.f;
-    wreg[c][1] = (c < C && in1) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k + 1] : 0.f;
-    gw[c][0] = gw[c][1] = 0.f;
+  for (int v = 0; v < VEC; ++v) in[v] = k + v < K;
+  const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
+
+  // ---- requests --------------------------------------------------------------------------------
+  float wreg[CMAX][VEC];
+#pragma unroll
+  for (int c = 0; c < CMAX; ++c)
+#pragma unroll
+    for (int v = 0; v < VEC; ++v)
+      wreg[c][v] = (c < C && in[v]) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k + v] : 0.f;
+  // update phase: thread t finishes elements t, t + 256, ... of the C x COLS block, element = (class, column)
+  float wu[kUpd], vu[kUpd];
+#pragma unroll
+  for (int i = 0; i < kUpd; ++i) {
+    const int t = threadIdx.x + i * kThreads;
+    const int kk = blockIdx.x * COLS + (t % COLS);
+    wu[i] = vu[i] = 0.f;
+    if (t < C * COLS && kk < K) {
+      const int64_t at = (int64_t)g * w_gstride + (int64_t)(t / COLS) * K + kk;
+      wu[i] = W[at];
+      if (mu != 0.f) vu[i] = V[at];
+    }
   }
-  float cs0 = 0.f, cs1 = 0.f;     // column sums of dPrev over this thread's rows (bias gradient of the layer below)
+  float b_own = 0.f, vb_own = 0.f, b_prev = 0.f, vb_prev = 0.f;
+  const bool own_bias = blockIdx.x == 0 && bias != nullptr && threadIdx.x < C;
+  const int kp = blockIdx.x * COLS + threadIdx.x;
+  const bool prev_bias = pbias != nullptr && threadIdx.x < COLS && kp < K;
+  if (own_bias) {
+    b_own = bias[(int64_t)g * w_gstride + threadIdx.x];
+    if (mu != 0.f) vb_own = vbias[(int64_t)g * w_gstride + threadIdx.x];
+  }
+  if (prev_bias) {
+    b_prev = pbias[(int64_t)g * w_gstride + kp];
+    if (mu != 0.f) vb_prev = pvbias[(int64_t)g * w_gstride + kp];
+  }
+  float av[kTrip][VEC];
+#pragma unroll
+  for (int u = 0; u < kTrip; ++u) {
+    const int b = ry + 8 * u;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) av[u][v] = 0.f;
+    if (b < B && in[0]) {
+      if (VEC == 1 || in[VEC - 1]) load_cols(Ag + (int64_t)b * K + k, av[u]);
+      else av[u][0] = to_f(Ag[(int64_t)b * K + k]);
+    }
+  }
+  if (blockIdx.x == 0 && ry == 7 && loss_out != nullptr) {
+    // mean of the row losses: lane-strided partial sums, then a butterfly
+    float p = 0.f;
+    for (int b = cx; b < B; b += 32) p += row_loss[(int64_t)g * B + b];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
+    if (cx == 0) loss_out[g] = p * (1.0f / (float)B);
+  }
   for (int i = threadIdx.x; i < B * C; i += kThreads) dz[i] = dZ[(int64_t)g * B * C + i];
   __syncthreads();
 
-  if (in0) {
-    for (int bb = ry; bb < B; bb += 64) {
-      // eight rows per trip so that eight loads of A are in flight
-      float av[8][2];
+  // ---- both gradients in one pass over the rows ------------------------------------------------------
+  float gw[CMAX][VEC];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        av[u][0] = av[u][1] = 0.f;
-        if (bb + 8 * u < B) {
-          const TA* src = Ag + (int64_t)(bb + 8 * u) * K + k;
-          if (pair_ok) load2(src, av[u]);
-          else { av[u][0] = to_f(src[0]); if (in1) av[u][1] = to_f(src[1]); }
+  for (int c = 0; c < CMAX; ++c)
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) gw[c][v] = 0.f;
+  float cs[VEC];      // column sums of dPrev over this thread's rows (bias gradient of the layer below)
+#pragma unroll
+  for (int v = 0; v < VEC; ++v) cs[v] = 0.f;
+  for (int bb = 0; bb < B; bb += 8 * kTrip) {
+    if (bb > 0) {
+#pragma unroll
+      for (int u = 0; u < kTrip; ++u) {
+        const int b = bb + ry + 8 * u;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) av[u][v] = 0.f;
+        if (b < B && in[0]) {
+          if (VEC == 1 || in[VEC - 1]) load_cols(Ag + (int64_t)b * K + k, av[u]);
+          else av[u][0] = to_f(Ag[(int64_t)b * K + k]);
         }
       }
+    }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int b = bb + 8 * u;
-        if (b >= B) break;
-        float da0 = 0.f, da1 = 0.f;
+    for (int u = 0; u < kTrip; ++u) {
+      const int b = bb + ry + 8 * u;
+      if (b >= B) break;
+      float da[VEC];
 #pragma unroll
-        for (int c = 0; c < CMAX; ++c)
-          if (c < C) {
-            const float d = dz[b * C + c];
-            gw[c][0] = fmaf(d, av[u][0], gw[c][0]);
-            gw[c][1] = fmaf(d, av[u][1], gw[c][1]);
-            da0 = fmaf(d, wreg[c][0], da0);
-            da1 = fmaf(d, wreg[c][1], da1);
-          }
-        if (dPrev != nullptr) {
-          const float o0 = av[u][0] > 0.f ? da0 : 0.f, o1 = av[u][1] > 0.f ? da1 : 0.f;
-          cs0 += o0;
-          cs1 += o1;
-          const int64_t at = ((int64_t)g * B + b) * K + k;
-          if (pair_ok) {
-            store2(dPrev + at, o0, o1);
-          } else {
-            put(dPrev + at, o0);
-            if (in1) put(dPrev + at + 1, o1);
-          }
+      for (int v = 0; v < VEC; ++v) da[v] = 0.f;
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c) {
+        if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
+        const float d = dz[b * C + c];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+          gw[c][v] = fmaf(d, av[u][v], gw[c][v]);
+          da[v] = fmaf(d, wreg[c][v], da[v]);
         }
+      }
+      if (dPrev != nullptr && in[0]) {
+        float o[VEC];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+          o[v] = av[u][v] > 0.f ? da[v] : 0.f;
+          cs[v] += o[v];
+        }
+        TA* dst = dPrev + ((int64_t)g * B + b) * K + k;
+        if (VEC == 1 || in[VEC - 1]) store_cols(dst, o);
+        else put(dst, o[0]);
       }
     }
   }
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    part[(ry * CMAX + c) * kColsPerCta + cx * 2] = gw[c][0];
-    part[(ry * CMAX + c) * kColsPerCta + cx * 2 + 1] = gw[c][1];
-  }
+  for (int c = 0; c < CMAX; ++c)
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) part[(ry * CMAX + c) * COLS + cx * VEC + v] = gw[c][v];
   __syncthreads();
-  // 8 warps x 64 columns: thread t < 64 * C finishes column t % 64 of output row t / 64 ... done by all
-  // threads in a strided loop so that the V / W accesses are coalesced along k
-  for (int t = threadIdx.x; t < C * kColsPerCta; t += kThreads) {
-    const int c = t / kColsPerCta, col = t % kColsPerCta;
-    const int kk = blockIdx.x * kColsPerCta + col;
-    if (kk >= K) continue;
-    float s = 0.f;
+  // ---- G = sum of the 8 row slices (in slice order); v <- mu v + G; W <- W - eta v -------------------
 #pragma unroll
-    for (int r = 0; r < 8; ++r) s += part[(r * CMAX + c) * kColsPerCta + col];
-    const int64_t at = (int64_t)g * w_gstride + (int64_t)c * K + kk;
-    float step = s;
-    if (mu != 0.f) {
-      step = fmaf(mu, V[at], s);
-      V[at] = step;
+  for (int i = 0; i < kUpd; ++i) {
+    const int t = threadIdx.x + i * kThreads;
+    const int c = t / COLS, col = t % COLS;
+    const int kk = blockIdx.x * COLS + col;
+    if (t < C * COLS && kk < K) {
+      float s = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) s += part[(r * CMAX + c) * COLS + col];
+      const int64_t at = (int64_t)g * w_gstride + (int64_t)c * K + kk;
+      float step = s;
+      if (mu != 0.f) {
+        step = fmaf(mu, vu[i], s);
+        V[at] = step;
+      }
+      const float w = fmaf(-lr, step, wu[i]);
+      W[at] = w;
+      if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
     }
-    const float w = fmaf(-lr, step, W[at]);
-    W[at] = w;
-    if (Wb != nullptr) Wb[at] = __float2bfloat16_rn(w);
   }
-  if (blockIdx.x == 0 && bias != nullptr && threadIdx.x < C) {
+  if (own_bias) {
     const int c = threadIdx.x;
     float s = 0.f;
     for (int b = 0; b < B; ++b) s += dz[b * C + c];
     const int64_t at = (int64_t)g * w_gstride + c;
     float step = s;
     if (mu != 0.f) {
-      step = fmaf(mu, vbias[at], s);
+      step = fmaf(mu, vb_own, s);
       vbias[at] = step;
     }
-    bias[at] = fmaf(-lr, step, bias[at]);
+    bias[at] = fmaf(-lr, step, b_own);
   }
   if (pbias != nullptr) {
     // bias of the layer below: its gradient is the column sum of dPrev, complete inside this CTA
     __syncthreads();
-    part[ry * kColsPerCta + cx * 2] = cs0;
-    part[ry * kColsPerCta + cx * 2 + 1] = cs1;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) part[ry * COLS + cx * VEC + v] = cs[v];
     __syncthreads();
-    const int kk = blockIdx.x * kColsPerCta + threadIdx.x;
-    if (threadIdx.x < kColsPerCta && kk < K) {
+    if (prev_bias) {
       float s = 0.f;
 #pragma unroll
-      for (int r = 0; r < 8; ++r) s += part[r * kColsPerCta + threadIdx.x];
-      const int64_t at = (int64_t)g * w_gstride + kk;
+      for (int r = 0; r < 8; ++r) s += part[r * COLS + threadIdx.x];
+      const int64_t at = (int64_t)g * w_gstride + kp;
       float step = s;
       if (mu != 0.f) {
-        step = fmaf(mu, pvbias[at], s);
+        step = fmaf(mu, vb_prev, s);
         pvbias[at] = step;
       }
-      pbias[at] = fmaf(-lr, step, pbias[at]);
+      pbias[at] = fmaf(-lr, step, b_prev);
     }
   }
 }
@@ -323,42 +402,38 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   if (a_bf16)
     return launch_dep(head_fwd_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, st, 1,
                       static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off,
-                      a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok);
+                      a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok, a.defer_loss);
   return launch_dep(head_fwd_kernel<float>, grid, dim3(kThreads), 0, st, 1, static_cast<const float*>(a.A),
                     a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters,
-                    a.B, a.C, a.K, a.loss_kind, vec_ok);
+                    a.B, a.C, a.K, a.loss_kind, vec_ok, a.defer_loss);
+}
+
+template <typename TA, int VEC>
+int launch_head_bwd_t(const HeadBwdArgs& a, cudaStream_t st) {
+  auto kern = head_bwd_kernel<TA, VEC>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  constexpr int COLS = 32 * VEC;
+  dim3 grid((unsigned)((a.K + COLS - 1) / COLS), (unsigned)a.groups);
+  const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * COLS) * sizeof(float);
+  return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const TA*>(a.A), a.a_row_off, a.dZ, a.W, a.V,
+                    a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<TA*>(a.dPrev), a.dPrev ? a.pbias : nullptr,
+                    a.pvbias, a.row_loss, a.loss_out, a.B, a.C, a.K, a.lr, a.mu);
 }
 
 int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
-  dim3 grid((unsigned)((a.K + kColsPerCta - 1) / kColsPerCta), (unsigned)a.groups);
-  const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * kColsPerCta) * sizeof(float);
   const size_t esz = a_bf16 ? 2 : 4;
-  const int pair_ok = (a.K % 2 == 0) && reinterpret_cast<uintptr_t>(a.A) % (2 * esz) == 0 &&
-                      (a.dPrev == nullptr || reinterpret_cast<uintptr_t>(a.dPrev) % (2 * esz) == 0);
-  if (a_bf16) {
-    auto kern = head_bwd_kernel<__nv_bfloat16>;
-    static bool configured = false;
-    if (!configured) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-      if (e != cudaSuccess) return e;
-      configured = true;
-    }
-    return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const __nv_bfloat16*>(a.A), a.a_row_off,
-                      a.dZ, a.W, a.V, a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<__nv_bfloat16*>(a.dPrev),
-                      a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
-  } else {
-    auto kern = head_bwd_kernel<float>;
-    static bool configured = false;
-    if (!configured) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-      if (e != cudaSuccess) return e;
-      configured = true;
-    }
-    return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const float*>(a.A), a.a_row_off, a.dZ,
-                      a.W, a.V, a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<float*>(a.dPrev),
-                      a.dPrev ? a.pbias : nullptr, a.pvbias, a.B, a.C, a.K, a.lr, a.mu, pair_ok);
-  }
+  // two columns per lane when the pointers allow it and there is still a CTA for every SM
+  const bool pair = (a.K % 2 == 0) && reinterpret_cast<uintptr_t>(a.A) % (2 * esz) == 0 &&
+                    (a.dPrev == nullptr || reinterpret_cast<uintptr_t>(a.dPrev) % (2 * esz) == 0) &&
+                    (int64_t)((a.K + 63) / 64) * a.groups >= 148;
+  if (a_bf16) return pair ? launch_head_bwd_t<__nv_bfloat16, 2>(a, st) : launch_head_bwd_t<__nv_bfloat16, 1>(a, st);
+  return pair ? launch_head_bwd_t<float, 2>(a, st) : launch_head_bwd_t<float, 1>(a, st);
 }
 
 }  // namespace ls
@@ -419,5 +494,6 @@ extern "C" int ls_linear_loss_static(const float* W_dev, const float* bias_dev, 
   a.dZ = nullptr;
   a.row_loss = sc->row_loss; a.loss_out = chunk_loss_dev; a.counters = sc->counters;
   a.B = chunk_rows; a.C = d_out; a.K = d_in; a.groups = (int)chunks; a.loss_kind = loss;
+  a.defer_loss = 0;
   return launch_head_fwd(a, false, st, nullptr) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

@@ -161,6 +161,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       a.loss_out = loss_out;
       a.counters = reinterpret_cast<unsigned int*>(h->state + lay.headcnt_off);
       a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = groups; a.loss_kind = h->spec.loss;
+      a.defer_loss = want_dz ? 1 : 0;       // a training step: the backward kernel of this layer forms the mean
       ProfScope ps(h, LS_K_FWD, l);
       LS_CUDA(h, launch_head_fwd(a, bf, h->stream, &h->launches));
       return LS_OK;
@@ -233,6 +234,8 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       a.pbias = (l > 0 && lay.has_bias) ? params_of(h) + lay.b_off[l - 1] : nullptr;
       a.pvbias = mom_of(h) + (l > 0 ? lay.b_off[l - 1] : 0);
       if (a.pbias != nullptr) bias_done[l - 1] = true;
+      a.row_loss = reinterpret_cast<const float*>(h->state + lay.rowloss_off);
+      a.loss_out = loss_out;
       a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = lay.m;
       a.lr = h->lr; a.mu = h->mu;
       ProfScope ps(h, LS_K_DW, l);

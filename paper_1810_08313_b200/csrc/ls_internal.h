@@ -223,6 +223,7 @@ struct HeadFwdArgs {
   float* dZ;                                 // [groups][B][C] or null (forward only)
   float* row_loss; float* loss_out; unsigned int* counters;
   int B, C, K, groups, loss_kind;
+  int defer_loss;                            // 1: only write row_loss; the backward kernel forms loss_out
 };
 struct HeadBwdArgs {
   const void* A; const int64_t* a_row_off;
@@ -231,6 +232,7 @@ struct HeadBwdArgs {
   void* dPrev;                               // dZ of the layer below [groups][B][K] or null
   float* pbias; float* pvbias;               // bias / its momentum of the layer below (updated from the column
                                              // sums of dPrev) or null; replica stride w_gstride
+  const float* row_loss; float* loss_out;    // row losses left by the forward kernel and where their mean goes, or null
   int B, C, K, groups;
   float lr, mu;
 };
