@@ -23,9 +23,10 @@
 //          accumulators, double-buffered) and the epilogue warps add the partial sums in registers
 //          with round-to-nearest while the next chunk is being multiplied.
 //          When a layer has too few output tiles to occupy the GPU (small batch x width), K is split
-//          over a thread-block cluster of 2 or 4 CTAs: every CTA sums its K slice as above, the
-//          partial rows are exchanged through distributed shared memory and added in rank order by
-//          the rank-0 CTA, which then runs the epilogue.  No atomics, so the result is reproducible.
+//          over a thread-block cluster of 2 or 4 CTAs: every CTA sums its K slice as above and leaves
+//          its partial tile in shared memory; then CTA r adds, in rank order, the partial sums of
+//          columns [r BN/S, (r+1) BN/S) through distributed shared memory and runs the epilogue for
+//          them (a reduce-scatter).  No atomics, so the result is reproducible.
 //
 // Operands are read in place whatever their orientation: a K-major operand
 // ([rows][K], K contiguous) and an MN-major operand ([K][rows], rows contiguous)
@@ -162,6 +163,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   static_assert(MT == 1 || (!CHUNKED && !A_MN && EPI != EPI_DW && MT * BN <= 512), "two row blocks: bf16 forward/backward");
   static_assert(SPLIT == 1 || CHUNKED, "split-K needs the register-resident partial sums");
   static_assert(SPLIT == 1 || BN * BM * 4 <= L::kRingBytes, "exchange buffer");
+  constexpr int CPR = BN / SPLIT;              // columns that each CTA of the cluster finishes
+  static_assert(CPR % 32 == 0, "whole 32-column blocks per CTA");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -329,9 +332,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after_sync();
     }
     if (!ok && lane == 0) atomicExch(p.err_flag, 3);
-    if (SPLIT > 1 && rank != 0 && ok) {
+    if (SPLIT > 1 && ok) {
       // every load of this CTA has been consumed and every MMA has completed: the stage buffers are
-      // free, and hold this CTA's partial rows for rank 0 ([column][row], so lanes are conflict-free)
+      // free, and hold this CTA's partial tile for the cluster ([column][row], so lanes are conflict-free)
       float* xbuf = reinterpret_cast<float*>(smem);
 #pragma unroll
       for (int i = 0; i < (CHUNKED ? BN : 1); ++i) xbuf[i * BM + q * 32 + lane] = sum[i];
@@ -339,21 +342,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   if (SPLIT > 1) {
     cluster_sync_all();
-    if (warp >= 2 && warp < 6 && rank == 0 && ok) {
-      const uint32_t mine = smem_u32(reinterpret_cast<float*>(smem) + q * 32 + lane);
-      for (int r = 1; r < SPLIT; ++r) {
+    if (warp >= 2 && warp < 6 && ok) {
+      // this CTA's columns, added in rank order whoever adds them
+      const uint32_t mine = smem_u32(reinterpret_cast<float*>(smem) + (rank * CPR) * BM + q * 32 + lane);
+#pragma unroll
+      for (int r = 0; r < SPLIT; ++r) {
         const uint32_t remote = map_to_rank(mine, (uint32_t)r);
 #pragma unroll
-        for (int i = 0; i < (CHUNKED ? BN : 1); ++i) sum[i] += ld_cluster_f32(remote + (uint32_t)(i * BM * 4));
+        for (int i = 0; i < (CHUNKED ? CPR : 1); ++i) {
+          const float v = ld_cluster_f32(remote + (uint32_t)(i * BM * 4));
+          sum[i] = (r == 0) ? v : sum[i] + v;
+        }
       }
     }
-    cluster_sync_all();      // the other CTAs stay alive until rank 0 has read their rows
+    cluster_sync_all();      // every CTA stays alive until the others have read its tile
   }
   if (warp >= 2 && warp < 6) {
-    if (ok && (SPLIT == 1 || rank == 0)) {
+    if (ok) {
 #pragma unroll
-      for (int cc32 = 0; cc32 < MT * (BN / 32); ++cc32) {
-        const int mt = cc32 / (BN / 32), c = cc32 % (BN / 32);
+      for (int cc32 = 0; cc32 < MT * (CPR / 32); ++cc32) {
+        const int mt = cc32 / (CPR / 32), c = cc32 % (CPR / 32);
         const int row = row0 + mt * BM;          // output row this thread owns in row block mt
         uint32_t r[32];
         if (CHUNKED) {
@@ -363,7 +371,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tmem_ld_32x32(taddr + mt * BN + c * 32, r);
           tmem_ld_wait();
         }
-        const int col = n0 + c * 32;
+        const int col = n0 + rank * CPR + c * 32;
         if (EPI == EPI_FWD) {
           float o[32];
           const float* bias = p.bias ? p.bias + (int64_t)g * p.bias_gstride + col : nullptr;
@@ -465,15 +473,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
     }
-    if (EPI == EPI_DX && p.dbias != nullptr && (SPLIT == 1 || rank == 0)) {
+    if (EPI == EPI_DX && p.dbias != nullptr) {
       // all four epilogue warps (and only they) meet here; then one thread per column adds the partial
       // sums in a fixed order and applies v <- mu v + g, b <- b - eta v
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      for (int t = threadIdx.x - 64; t < BN; t += 128) {
+      for (int t = threadIdx.x - 64; t < CPR; t += 128) {
         float gsum = 0.f;
 #pragma unroll
         for (int i = 0; i < MT * 4; ++i) gsum += colsum[i * BN + t];
-        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
+        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + rank * CPR + t;
         float step = gsum;
         if (p.mu != 0.f) {
           step = fmaf(p.mu, p.dvbias[at], gsum);
@@ -532,13 +540,14 @@ int launch_fp32(const TcOperandMaps& mp, const Params& p, int groups, cudaStream
   const int tiles = (p.M / BM) * (p.N / bn) * groups;
   const int num_kb = p.K / 32;
   int split = 1;
-  while (split < 4 && tiles * split * 2 <= 148 && num_kb % (split * 2) == 0 && num_kb / (split * 2) >= 8) split *= 2;
+  const int max_split = bn == 128 ? 4 : 2;      // every CTA of the cluster finishes at least 32 columns
+  while (split < max_split && tiles * split * 2 <= 148 && num_kb % (split * 2) == 0 && num_kb / (split * 2) >= 4)
+    split *= 2;
   if (bn == 128) {
     if (split == 4) return launch_one<true, 128, A_MN, B_MN, EPI, 4, 4>(mp, p, groups, st);
     if (split == 2) return launch_one<true, 128, A_MN, B_MN, EPI, 4, 2>(mp, p, groups, st);
     return launch_one<true, 128, A_MN, B_MN, EPI, 4, 1>(mp, p, groups, st);
   }
-  if (split == 4) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 4>(mp, p, groups, st);
   if (split == 2) return launch_one<true, 64, A_MN, B_MN, EPI, 4, 2>(mp, p, groups, st);
   return launch_one<true, 64, A_MN, B_MN, EPI, 4, 1>(mp, p, groups, st);
 }
