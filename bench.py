@@ -70,15 +70,33 @@ def flops_per_replica_step(w: wl.Workload) -> float:
     return f
 
 
-def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
-    """Algorithmic bytes of one weight-gradient + update launch for layer `layer` (all m replicas):
-    read and write W (and v when momentum is on), write the bf16 copy of W (bf16 models), read the
-    two GEMM operands once."""
-    n_out, n_in = layer_shapes(w)[layer]
+def streamed_update_layers(w: wl.Workload):
+    """Layers whose weight update runs on the streaming tensor-core kernel: all of them go into one launch."""
     bf = w.gemm_dtype == "bf16"
-    per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if bf else 0)
-    operand = (2 if bf else 4) * w.batch * (n_out + n_in)
-    return float(w.m) * (per_param * n_out * n_in + operand)
+    out = []
+    for l, (n_out, n_in) in enumerate(layer_shapes(w)):
+        last = l == len(w.dims) - 2
+        if last and n_out <= 16:
+            continue
+        if n_out % 128 == 0 and n_in % 128 == 0 and w.batch % (64 if bf else 32) == 0:
+            out.append(l)
+    return out
+
+
+def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
+    """Algorithmic bytes of the weight-gradient + update launch that covers layer `layer` (all m replicas):
+    read and write W (and v when momentum is on), write the bf16 copy of W (bf16 models), read the
+    two GEMM operands once; summed over the layers that share the launch."""
+    bf = w.gemm_dtype == "bf16"
+    merged = streamed_update_layers(w)
+    layers = merged if layer in merged else [layer]
+    total = 0.0
+    for l in layers:
+        n_out, n_in = layer_shapes(w)[l]
+        per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if bf else 0)
+        operand = (2 if bf else 4) * w.batch * (n_out + n_in)
+        total += float(w.m) * (per_param * n_out * n_in + operand)
+    return total
 
 
 def uses_tensor_cores(w: wl.Workload, cls: str, layer: int) -> bool:
@@ -136,7 +154,9 @@ def roofline_for(dom, dur_s: float, w: wl.Workload, peaks, clocks):
     if cls == "dw" and tc:
         by = update_bytes_per_launch(w, layer)
         ach = by / dur_s / 1e9
-        return {"kernel": f"weight gradient + update, layer {layer} (tcgen05, streaming)", "bound": "hbm",
+        merged = streamed_update_layers(w)
+        which = f"layers {merged}" if layer in merged and len(merged) > 1 else f"layer {layer}"
+        return {"kernel": f"weight gradient + update, {which} in one launch (tcgen05, streaming)", "bound": "hbm",
                 "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                 "traffic": traffic, "peak_source": src, "ms_per_launch": ms}
     n_out, n_in = layer_shapes(w)[layer]

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -70,9 +71,7 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   for (int l = 1; l < lay.L; ++l) {
     lay.act_off[l] = take((size_t)m * batch * lay.dims[l] * esz);
   }
-  for (int s = 0; s < 2; ++s) {
-    lay.dz_off[s] = take((size_t)m * batch * lay.max_width * esz);
-  }
+  for (int l = 0; l < lay.L; ++l) lay.dz_off[l] = take((size_t)m * batch * lay.dims[l + 1] * esz);
   lay.logits_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.dzl_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.rowloss_off = take((size_t)LS_MAX_REPLICAS * batch * 4);
@@ -199,7 +198,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
   LossArgs la;
   la.logits = reinterpret_cast<const float*>(h->state + lay.logits_off);
   la.y = y; la.row_off = row_off_dev;
-  la.dZ = want_dz ? (void*)(h->state + lay.dz_off[0]) : nullptr;
+  la.dZ = want_dz ? (void*)(h->state + lay.dz_off[lay.L - 1]) : nullptr;
   la.loss_out = loss_out;
   la.B = lay.batch; la.C = lay.dims[lay.L]; la.groups = groups; la.loss_kind = h->spec.loss;
   ProfScope ps(h, LS_K_LOSS, 0);
@@ -215,10 +214,13 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   const TcMaps& mn = bf ? h->maps : h->maps_mn;     // descriptors for MN-major reads
   int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
   if (rc != LS_OK) return rc;
-  int cur = 0;
   bool bias_done[LS_MAX_LAYERS] = {false};     // bias l already updated by the kernel that produced dZ_l
+  // Weight updates that run on the streaming tensor-core kernel are collected and launched together after
+  // the last data gradient: they are independent of one another, and dZ_l / the layer inputs stay in place.
+  TcUpdateArgs upd[LS_MAX_LAYERS];
+  int n_upd = 0;
   for (int l = lay.L - 1; l >= 0; --l) {
-    void* dZ = h->state + lay.dz_off[cur];
+    void* dZ = h->state + lay.dz_off[l];
     if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
       // narrow output layer: both gradients, the update and the bias in one pass over its input
       HeadBwdArgs a;
@@ -230,7 +232,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       a.bias = lay.has_bias ? params_of(h) + lay.b_off[l] : nullptr;
       a.vbias = mom_of(h) + lay.b_off[l];
       a.w_gstride = lay.stride;
-      a.dPrev = (l > 0) ? (void*)(h->state + lay.dz_off[cur ^ 1]) : nullptr;
+      a.dPrev = (l > 0) ? (void*)(h->state + lay.dz_off[l - 1]) : nullptr;
       a.pbias = (l > 0 && lay.has_bias) ? params_of(h) + lay.b_off[l - 1] : nullptr;
       a.pvbias = mom_of(h) + (l > 0 ? lay.b_off[l - 1] : 0);
       if (a.pbias != nullptr) bias_done[l - 1] = true;
@@ -240,7 +242,6 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       a.lr = h->lr; a.mu = h->mu;
       ProfScope ps(h, LS_K_DW, l);
       LS_CUDA(h, launch_head_bwd(a, bf, h->stream, &h->launches));
-      cur ^= 1;
       continue;
     }
     if (l > 0 && tc_shape_ok(!bf, lay.batch, lay.dims[l], lay.dims[l + 1])) {
@@ -250,7 +251,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.maps.a = &h->maps.dz[l];
       t.maps.b = &mn.w[l];
       t.act = h->state + lay.act_off[l];
-      t.C = h->state + lay.dz_off[cur ^ 1];
+      t.C = h->state + lay.dz_off[l - 1];
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
       t.bias = nullptr; t.vbias = nullptr; t.bias_gstride = lay.stride; t.lr = h->lr; t.mu = h->mu;
       if (lay.has_bias && tc_dx_fuses_bias(!bf, t.M, t.N)) {
@@ -267,13 +268,13 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       d.W = bf ? (const void*)(shadow_of(h) + lay.w_off[l]) : (const void*)(params_of(h) + lay.w_off[l]);
       d.w_gstride = lay.stride;
       d.act = h->state + lay.act_off[l];
-      d.C = h->state + lay.dz_off[cur ^ 1];
+      d.C = h->state + lay.dz_off[l - 1];
       d.M = lay.batch; d.N = lay.dims[l]; d.K = lay.dims[l + 1]; d.groups = lay.m;
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_dx(d, bf, h->stream, &h->launches));
     }
     if (tc_update_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
-      TcUpdateArgs t;
+      TcUpdateArgs& t = upd[n_upd++];
       t.fp32 = !bf;
       t.maps.a = &mn.dz[l];
       t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
@@ -285,8 +286,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.M = lay.dims[l + 1]; t.N = lay.dims[l]; t.B = lay.batch; t.groups = lay.m;
       t.lr = h->lr; t.mu = h->mu;
       t.err_flag = err_flag_of(h);
-      ProfScope ps(h, LS_K_DW, l);
-      LS_CUDA(h, launch_tc_update(t, h->stream, &h->launches));
+      t.layer = l;
     } else if (tc_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
       TcDwArgs t;
       t.fp32 = !bf;
@@ -329,7 +329,15 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       ProfScope ps(h, LS_K_BIAS, l);
       LS_CUDA(h, launch_bias(b, bf, h->stream, &h->launches));
     }
-    cur ^= 1;
+  }
+  // largest layer first, so that the short tiles fill the end of the list
+  std::sort(upd, upd + n_upd, [](const TcUpdateArgs& x, const TcUpdateArgs& y) {
+    return (int64_t)x.M * x.N > (int64_t)y.M * y.N;
+  });
+  for (int i = 0; i < n_upd; i += tc_update_max_layers()) {
+    const int n = std::min(n_upd - i, tc_update_max_layers());
+    ProfScope ps(h, LS_K_DW, upd[i].layer);
+    LS_CUDA(h, launch_tc_update(upd + i, n, h->stream, &h->launches));
   }
   return LS_OK;
 }
@@ -493,8 +501,7 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
           }
         }
         if (lay.dims[l + 1] % q == 0) {
-          const int buf = (lay.L - 1 - l) & 1;
-          ok(tc_make_map_2d(&mp.dz[l], h->state + lay.dz_off[buf], f, mn, rows, lay.dims[l + 1]));
+          ok(tc_make_map_2d(&mp.dz[l], h->state + lay.dz_off[l], f, mn, rows, lay.dims[l + 1]));
         }
       }
       if (!mn) {

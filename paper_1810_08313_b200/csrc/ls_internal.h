@@ -40,7 +40,7 @@ struct Layout {
   size_t params_off = 0, mom_off = 0;
   size_t shadow_off = 0;                     // bf16 [m][stride] copy of the weights (bf16 models)
   size_t act_off[LS_MAX_LAYERS + 1] = {0};   // post-ReLU activations = inputs of layers 1..L-1
-  size_t dz_off[2] = {0, 0};                 // ping-pong gradient buffers [m][batch][max_width]
+  size_t dz_off[LS_MAX_LAYERS] = {0};        // dZ_l = gradient w.r.t. the output of layer l, [m][batch][dims[l+1]]
   size_t logits_off = 0;                     // [m][batch][dims[L]] fp32
   size_t dzl_off = 0;                        // fp32 dZ of a narrow output layer [m][batch][dims[L]]
   size_t rowloss_off = 0;                    // per-sample losses [LS_MAX_REPLICAS][batch]
@@ -295,9 +295,12 @@ struct TcUpdateArgs {
   int M, N, B, groups;
   float lr, mu;
   int* err_flag;
+  int layer;                 // which layer of the model this is (bookkeeping of the caller)
 };
 bool tc_update_shape_ok(bool fp32, int M, int N, int B);
-int launch_tc_update(const TcUpdateArgs& a, cudaStream_t st, int64_t* launches);
+int tc_update_max_layers();
+// one launch for the updates of layers[0..n) (n <= tc_update_max_layers(); same batch, replicas, rates, type)
+int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches);
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches);

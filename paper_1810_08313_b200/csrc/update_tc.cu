@@ -4,6 +4,8 @@
 //     G = dZ^T A  (per replica, 128 x 128 tiles on tcgen05, accumulator in TMEM)
 //     v <- mu v + G ;  W <- W - eta v ;  refresh the operand copy of W
 //
+// for every layer whose shapes fill tensor-core tiles, in ONE launch: the updates of different layers do
+// not depend on one another, so their tiles form one list (largest layer first) that the CTAs walk.
 // The gradient never leaves the SM.  The kernel is bound by the read-modify-write
 // of W and v (16 bytes per parameter with momentum, plus the bf16 copy of a bf16 model), so it
 // is built as a stream: one CTA per SM walks over output tiles, and
@@ -34,15 +36,41 @@ constexpr int KB_BYTES = 128;
 constexpr int kThreads = 256;
 constexpr int kSlotBytes = 8192;       // one 32 x 32 fp32 block of W (4 KB) and of v (4 KB)
 
-struct UParams {
-  int M, N, K, groups;                 // per replica: out features, in features, batch
+constexpr int kMaxLayers = 4;          // layers per launch
+
+struct ULayer {
+  int N;                               // in features (row length of W)
+  int n_tiles;                         // N / BN
+  int tiles_per_group;                 // (M / BM) * (N / BN)
+  int tile_begin;                      // first tile of this layer in the launch's list
   const int64_t* b_row_off;            // layer input = dataset rows: first row of replica g, else null
+  __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
+};
+struct UParams {
+  ULayer layer[kMaxLayers];
+  int n_layers, total_tiles;
+  int K, groups;                       // batch, replicas
   int rows_per_group;                  // = batch
   float lr, mu;
-  __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
   int64_t w_gstride;                   // elements between replicas
   int* err_flag;
 };
+// dZ_l (a), layer input (b), weights and momentum (w, v) of every layer of the launch
+struct alignas(64) UMaps {
+  CUtensorMap a[kMaxLayers], b[kMaxLayers], w[kMaxLayers], v[kMaxLayers];
+};
+
+struct Tile { int layer, g, m0, n0; };
+__device__ __forceinline__ Tile decode_tile(const UParams& p, int t) {
+  int l = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxLayers; ++i)
+    if (i < p.n_layers && t >= p.layer[i].tile_begin) l = i;
+  const int r = t - p.layer[l].tile_begin;
+  const int tpg = p.layer[l].tiles_per_group, nt = p.layer[l].n_tiles;
+  const int g = r / tpg, rem = r % tpg;
+  return Tile{l, g, (rem / nt) * BM, (rem % nt) * BN};
+}
 
 // Operand stages are filled by TMA; fp32 models add one buffer for the lo parts of the stage in use.
 template <bool TF32, int STAGES, int R>
@@ -86,8 +114,7 @@ __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, 
 
 template <bool TF32, int STAGES, int R>
 __global__ void __launch_bounds__(kThreads, 1)
-tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmV, const UParams p) {
+tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UParams p) {
   using L = USmem<TF32, STAGES, R>;
   constexpr int EB = TF32 ? 4 : 2;
   constexpr int ELEMS = KB_BYTES / EB;          // K elements per stage
@@ -113,9 +140,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(lo_empty + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tiles = p.M / BM, n_tiles = p.N / BN;
-  const int tiles_per_group = m_tiles * n_tiles;
-  const int total_tiles = tiles_per_group * p.groups;
+  const int total_tiles = p.total_tiles;
   const int num_kb = p.K / ELEMS;
   const bool has_v = p.mu != 0.f;
 
@@ -125,7 +150,9 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
     for (int i = 0; i < 4 * R; ++i) mbar_init(&wv_full[i], 1);
     fence_mbar_init();
-    prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmW); prefetch_tmap(&tmV);
+    for (int l = 0; l < p.n_layers; ++l) {
+      prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
+    }
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 2 * BN);
@@ -144,18 +171,20 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int g = t / tiles_per_group, rem = t % tiles_per_group;
-        const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
-        const int a_row = g * p.rows_per_group;
-        const int b_row = p.b_row_off ? (int)p.b_row_off[g] : a_row;
+        const Tile tl = decode_tile(p, t);
+        const int a_row = tl.g * p.rows_per_group;
+        const int64_t* b_off = p.layer[tl.layer].b_row_off;
+        const int b_row = b_off ? (int)b_off[tl.g] : a_row;
+        const CUtensorMap* tmA = &maps.a[tl.layer];
+        const CUtensorMap* tmB = &maps.b[tl.layer];
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1)) { atomicExch(p.err_flag, 11); ok = false; break; }
           mbar_expect_tx(&full[s], L::kStageBytes);
           uint8_t* sa = stage_base + s * L::kStageBytes;
           uint8_t* sb = sa + kABytes;
-          issue_mn_tile<ELEMS>(sa, &tmA, &full[s], m0, BM, a_row + kb * ELEMS);
-          issue_mn_tile<ELEMS>(sb, &tmB, &full[s], n0, BN, b_row + kb * ELEMS);
+          issue_mn_tile<ELEMS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * ELEMS);
+          issue_mn_tile<ELEMS>(sb, tmB, &full[s], tl.n0, BN, b_row + kb * ELEMS);
         }
       }
     }
@@ -227,13 +256,12 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // chunk j of this CTA: tile ordinal j / 4, column block j % 4; rows q*32.. of the tile
     auto load_chunk = [&](int j) {
       if (j >= my_chunks) return;
-      const int t = blockIdx.x + (j >> 2) * gridDim.x;
-      const int g = t / tiles_per_group, rem = t % tiles_per_group;
-      const int y = (rem / n_tiles) * BM + q * 32, x = (rem % n_tiles) * BN + (j & 3) * 32;
+      const Tile tl = decode_tile(p, blockIdx.x + (j >> 2) * gridDim.x);
+      const int y = tl.m0 + q * 32, x = tl.n0 + (j & 3) * 32;
       uint8_t* slot = my_ring + (j % R) * kSlotBytes;
       mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
-      tma_load_3d(slot, &tmW, &my_full[j % R], x, y, g);
-      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &tmV, &my_full[j % R], x, y, g);
+      tma_load_3d(slot, &maps.w[tl.layer], &my_full[j % R], x, y, tl.g);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.v[tl.layer], &my_full[j % R], x, y, tl.g);
     };
     if (lane == 0)
       for (int j = 0; j < R; ++j) load_chunk(j);
@@ -242,9 +270,10 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     bool ok = true;
     int j = 0;
     for (int n = 0; n < my_tiles && ok; ++n) {
-      const int t = blockIdx.x + n * gridDim.x;
-      const int g = t / tiles_per_group, rem = t % tiles_per_group;
-      const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+      const Tile tl = decode_tile(p, blockIdx.x + n * gridDim.x);
+      const int g = tl.g, m0 = tl.m0, n0 = tl.n0;
+      const int ldw = p.layer[tl.layer].N;
+      __nv_bfloat16* Wb = p.layer[tl.layer].Wb;
       const int buf = n & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (n >> 1) & 1));
       if (!ok) { if (lane == 0) atomicExch(p.err_flag, 14); break; }
@@ -264,7 +293,7 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         if (!ok) { if (lane == 0) atomicExch(p.err_flag, 15); break; }
         // this thread's row of the 32 x 32 block; 16-byte pieces are XOR-swizzled by the row (128-byte swizzle)
-        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * p.N + n0 + c * 32;
+        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * ldw + n0 + c * 32;
         uint32_t cp[8];
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
@@ -286,12 +315,12 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           *reinterpret_cast<float4*>(slot + off) = make_float4(ws[0], ws[1], ws[2], ws[3]);
           if (has_v) *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) = make_float4(vs[0], vs[1], vs[2], vs[3]);
           // operand copy of the new weights, collected so that it leaves in whole 32-byte sectors
-          if (!TF32 && p.Wb != nullptr) {
+          if (!TF32 && Wb != nullptr) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
             __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
             cp[(jj & 3) * 2] = *reinterpret_cast<uint32_t*>(&lo);
             cp[(jj & 3) * 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
-            if ((jj & 3) == 3) st_global_v8(p.Wb + at + (jj - 3) * 4, cp);
+            if ((jj & 3) == 3) st_global_v8(Wb + at + (jj - 3) * 4, cp);
           }
         }
         // make the in-place update visible to the bulk-copy engine, then write the blocks back
@@ -299,8 +328,8 @@ tc_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
         if (lane == 0) {
           const int y = m0 + q * 32, x = n0 + c * 32;
-          tma_store_3d(&tmW, slot, x, y, g);
-          if (has_v) tma_store_3d(&tmV, slot + kSlotBytes / 2, x, y, g);
+          tma_store_3d(&maps.w[tl.layer], slot, x, y, g);
+          if (has_v) tma_store_3d(&maps.v[tl.layer], slot + kSlotBytes / 2, x, y, g);
           bulk_commit();
           // the slot used one chunk ago is free once its store has read shared memory: refill it
           bulk_wait_read<1>();
@@ -331,7 +360,7 @@ int num_sms() {
 }
 
 template <bool TF32, int STAGES, int R>
-int launch_update(const TcUpdateArgs& a, cudaStream_t st) {
+int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   using L = USmem<TF32, STAGES, R>;
   auto kern = tc_update_kernel<TF32, STAGES, R>;
   static bool configured = false;
@@ -340,13 +369,30 @@ int launch_update(const TcUpdateArgs& a, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  const TcUpdateArgs& a0 = layers[0];
   UParams p{};
-  p.M = a.M; p.N = a.N; p.K = a.B; p.groups = a.groups;
-  p.b_row_off = a.row_off; p.rows_per_group = a.B;
-  p.lr = a.lr; p.mu = a.mu; p.Wb = a.Wb; p.w_gstride = a.w_gstride; p.err_flag = a.err_flag;
-  const int total = (a.M / BM) * (a.N / BN) * a.groups;
+  UMaps maps;
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const TcUpdateArgs& a = layers[i];
+    ULayer& l = p.layer[i];
+    l.N = a.N;
+    l.n_tiles = a.N / BN;
+    l.tiles_per_group = (a.M / BM) * (a.N / BN);
+    l.tile_begin = total;
+    l.b_row_off = a.row_off;
+    l.Wb = a.Wb;
+    total += l.tiles_per_group * a.groups;
+    maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
+  }
+  for (int i = n; i < kMaxLayers; ++i) {     // unused slots hold valid descriptors
+    maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
+  }
+  p.n_layers = n; p.total_tiles = total;
+  p.K = a0.B; p.groups = a0.groups; p.rows_per_group = a0.B;
+  p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
   const int grid = total < num_sms() ? total : num_sms();
-  return launch_dep(kern, dim3(grid), dim3(kThreads), L::kTotal, st, 1, *a.maps.a, *a.maps.b, *a.mapW, *a.mapV, p);
+  return launch_dep(kern, dim3(grid), dim3(kThreads), L::kTotal, st, 1, maps, p);
 }
 
 }  // namespace
@@ -355,10 +401,14 @@ bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
   return M > 0 && N > 0 && B > 0 && M % BM == 0 && N % BN == 0 && B % (fp32 ? 32 : 64) == 0;
 }
 
-int launch_tc_update(const TcUpdateArgs& a, cudaStream_t st, int64_t* launches) {
+int tc_update_max_layers() { return kMaxLayers; }
+
+// layers[0..n): same batch, replica count, rates and element type; the largest layer should come first
+int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
+  if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   if (launches) ++*launches;
-  if (a.fp32) return launch_update<true, 3, 3>(a, st);
-  return launch_update<false, 3, 4>(a, st);
+  if (layers[0].fp32) return launch_update<true, 3, 3>(layers, n, st);
+  return launch_update<false, 3, 4>(layers, n, st);
 }
 
 }  // namespace ls

@@ -27,9 +27,13 @@ def test_work_models():
     w2, w3 = wl.WORKLOADS["c2_mlp_fp32"], wl.WORKLOADS["c3_mlp_bf16"]
     assert abs(bench.flops_per_replica_step(w2) / 1e9 - 1.010) < 0.01      # 1.01 GFLOP per replica-step
     assert abs(bench.flops_per_replica_step(w3) / 1e9 - 19.36) < 0.05      # 19.36 GFLOP per replica-step
-    # update kernel, bf16 workload, layer 0: 18 bytes per parameter per replica plus the two operand tiles
+    # update kernel, bf16 workload: layers 0-2 share one launch; 18 bytes per parameter per replica plus the
+    # two operand tiles of every layer
+    assert bench.streamed_update_layers(w3) == [0, 1, 2] and bench.streamed_update_layers(w2) == [0, 1]
     by = bench.update_bytes_per_launch(w3, 0)
-    assert by == 16 * (18 * 2048 * 3072 + 2 * 256 * (2048 + 3072))
+    assert by == 16 * (18 * 2048 * 3072 + 2 * 256 * (2048 + 3072)) + 2 * 16 * (18 * 2048 * 2048 + 2 * 256 * 4096)
+    # fp32 workload: 16 bytes per parameter, fp32 operands
+    assert bench.update_bytes_per_launch(w2, 1) == 8 * (16 * 512 * 3072 + 4 * 128 * 3584) + 8 * (16 * 512 * 512 + 4 * 128 * 1024)
     assert bench.uses_tensor_cores(w3, "dw", 0) and bench.uses_tensor_cores(w2, "fwd", 0)
     assert not bench.uses_tensor_cores(w2, "fwd", 2) and not bench.uses_tensor_cores(w2, "dw", 2)
     assert not bench.uses_tensor_cores(wl.WORKLOADS["c1_softmax"], "dw", 0)
