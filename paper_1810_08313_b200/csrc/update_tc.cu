@@ -6,6 +6,9 @@
 //
 // for every layer whose shapes fill tensor-core tiles, in ONE launch: the updates of different layers do
 // not depend on one another, so their tiles form one list (largest layer first) that the CTAs walk.
+// Every CTA takes the same number of whole 128 x 128 tiles; the tiles left over after those rounds are cut
+// into column strips (32 columns for fp32, 64 for bf16) that are spread over all CTAs, so that the last
+// round is a fraction of a tile long instead of a whole tile on a few SMs.
 // The gradient never leaves the SM.  The kernel is bound by the read-modify-write
 // of W and v (16 bytes per parameter with momentum, plus the bf16 copy of a bf16 model), so it
 // is built as a stream: one CTA per SM walks over output tiles, and
@@ -49,6 +52,8 @@ struct ULayer {
 struct UParams {
   ULayer layer[kMaxLayers];
   int n_layers, total_tiles;
+  int full_rounds;                     // whole tiles per CTA; tile t of round n on CTA b is b + n * gridDim.x
+  int tail_units;                      // column strips of the left-over tiles, strip u on CTA u % gridDim.x
   int K, groups;                       // batch, replicas
   int rows_per_group;                  // = batch
   float lr, mu;
@@ -61,6 +66,8 @@ struct alignas(64) UMaps {
 };
 
 struct Tile { int layer, g, m0, n0; };
+// A unit of work: 32-column blocks [c0, c0 + nc) of a tile (nc = 4: the whole tile).
+struct Unit { Tile tl; int c0, nc; };
 __device__ __forceinline__ Tile decode_tile(const UParams& p, int t) {
   int l = 0;
 #pragma unroll
@@ -112,6 +119,15 @@ __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, 
     tma_load_2d(static_cast<char*>(dst) + c * ELEMS * KB_BYTES, tm, bar, tile0 + c * ELEMS, row0);
 }
 
+// n-th unit of CTA `b`; SUB strips per left-over tile
+template <int SUB>
+__device__ __forceinline__ Unit decode_unit(const UParams& p, int n, int b, int grid) {
+  if (n < p.full_rounds) return Unit{decode_tile(p, b + n * grid), 0, 4};
+  const int u = b + (n - p.full_rounds) * grid;
+  constexpr int NC = 4 / SUB;
+  return Unit{decode_tile(p, p.full_rounds * grid + u / SUB), (u % SUB) * NC, NC};
+}
+
 template <bool TF32, int STAGES, int R>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UParams p) {
@@ -121,6 +137,9 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
   constexpr int MMA_K = 32 / EB;
   constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
   constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN);
+  constexpr int SUB = TF32 ? 4 : 2;             // column strips per left-over tile (one operand chunk each)
+  constexpr int NCS = 4 / SUB;                  // 32-column blocks per strip
+  constexpr uint32_t IDESC_STRIP = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN / SUB);
   constexpr uint32_t SW = TF32 ? kSwizzle128B_32B : kSwizzle128B;
   constexpr uint32_t SBO = TF32 ? 512 : 1024;
   constexpr int kABytes = BM * KB_BYTES;
@@ -140,8 +159,10 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(lo_empty + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.total_tiles;
   const int num_kb = p.K / ELEMS;
+  const int bx = blockIdx.x, grid = gridDim.x;
+  const int my_strips = bx < p.tail_units ? (p.tail_units - 1 - bx) / grid + 1 : 0;
+  const int my_units = p.full_rounds + my_strips;
   const bool has_v = p.mu != 0.f;
 
   if (threadIdx.x == 0) {
@@ -170,8 +191,9 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
     if (elect_one()) {
       int it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const Tile tl = decode_tile(p, t);
+      for (int n = 0; n < my_units && ok; ++n) {
+        const Unit un = decode_unit<SUB>(p, n, bx, grid);
+        const Tile tl = un.tl;
         const int a_row = tl.g * p.rows_per_group;
         const int64_t* b_off = p.layer[tl.layer].b_row_off;
         const int b_row = b_off ? (int)b_off[tl.g] : a_row;
@@ -180,19 +202,18 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1)) { atomicExch(p.err_flag, 11); ok = false; break; }
-          mbar_expect_tx(&full[s], L::kStageBytes);
+          mbar_expect_tx(&full[s], kABytes + un.nc * 32 * KB_BYTES);
           uint8_t* sa = stage_base + s * L::kStageBytes;
           uint8_t* sb = sa + kABytes;
           issue_mn_tile<ELEMS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * ELEMS);
-          issue_mn_tile<ELEMS>(sb, tmB, &full[s], tl.n0, BN, b_row + kb * ELEMS);
+          issue_mn_tile<ELEMS>(sb, tmB, &full[s], tl.n0 + un.c0 * 32, un.nc * 32, b_row + kb * ELEMS);
         }
       }
     }
   } else if (TF32 && (warp == 2 || warp == 3)) {
     // ---- splitter warps: the lo copy has the layout of the tile it comes from ------------
     const int tid = threadIdx.x - 64;
-    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int total_it = my_tiles * num_kb;
+    const int total_it = my_units * num_kb;
     for (int it = 0; it < total_it; ++it) {
       const int s = it % STAGES;
       bool got = mbar_wait(&full[s], (it / STAGES) & 1);
@@ -209,10 +230,11 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
   } else if (warp == 1) {
     // ---- MMA issuer -----------------------------------------------------------------
     if (elect_one()) {
-      int it = 0, n = 0;
+      int it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++n) {
+      for (int n = 0; n < my_units && ok; ++n) {
         const int buf = n & 1;
+        const uint32_t idesc = n < p.full_rounds ? IDESC : IDESC_STRIP;     // a strip is BN / SUB columns wide
         if (!mbar_wait(&tmem_empty[buf], ((n >> 1) & 1) ^ 1)) { atomicExch(p.err_flag, 12); break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
@@ -232,11 +254,11 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
             if (TF32) {
               const uint64_t dal = make_smem_desc(smem_u32(lo_buf) + adv, CHUNK_BYTES, SBO, SW);
               const uint64_t dbl = make_smem_desc(smem_u32(lo_buf) + kABytes + adv, CHUNK_BYTES, SBO, SW);
-              mma_tf32(d_tmem, dal, db, IDESC, acc);
-              mma_tf32(d_tmem, da, dbl, IDESC, 1u);
-              mma_tf32(d_tmem, da, db, IDESC, 1u);
+              mma_tf32(d_tmem, dal, db, idesc, acc);
+              mma_tf32(d_tmem, da, dbl, idesc, 1u);
+              mma_tf32(d_tmem, da, db, idesc, 1u);
             } else {
-              mma_bf16(d_tmem, da, db, IDESC, acc);
+              mma_bf16(d_tmem, da, db, idesc, acc);
             }
           }
           mma_commit(&empty[s]);
@@ -250,14 +272,18 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
     const int q = warp & 3;
     uint8_t* my_ring = ring_base + q * R * kSlotBytes;
     uint64_t* my_full = wv_full + q * R;
-    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int my_chunks = my_tiles * (BN / 32);
+    const int full_chunks = p.full_rounds * 4;
+    const int my_chunks = full_chunks + my_strips * NCS;
 
-    // chunk j of this CTA: tile ordinal j / 4, column block j % 4; rows q*32.. of the tile
+    // chunk j of this CTA: the 32 x 32 block of rows q*32.. and column block c of unit n, where whole
+    // tiles contribute four chunks each and strips NCS
     auto load_chunk = [&](int j) {
       if (j >= my_chunks) return;
-      const Tile tl = decode_tile(p, blockIdx.x + (j >> 2) * gridDim.x);
-      const int y = tl.m0 + q * 32, x = tl.n0 + (j & 3) * 32;
+      const int n = j < full_chunks ? (j >> 2) : p.full_rounds + (j - full_chunks) / NCS;
+      const Unit un = decode_unit<SUB>(p, n, bx, grid);
+      const Tile tl = un.tl;
+      const int c = j < full_chunks ? (j & 3) : un.c0 + (j - full_chunks) % NCS;
+      const int y = tl.m0 + q * 32, x = tl.n0 + c * 32;
       uint8_t* slot = my_ring + (j % R) * kSlotBytes;
       mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
       tma_load_3d(slot, &maps.w[tl.layer], &my_full[j % R], x, y, tl.g);
@@ -269,8 +295,9 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     bool ok = true;
     int j = 0;
-    for (int n = 0; n < my_tiles && ok; ++n) {
-      const Tile tl = decode_tile(p, blockIdx.x + n * gridDim.x);
+    for (int n = 0; n < my_units && ok; ++n) {
+      const Unit un = decode_unit<SUB>(p, n, bx, grid);
+      const Tile tl = un.tl;
       const int g = tl.g, m0 = tl.m0, n0 = tl.n0;
       const int ldw = p.layer[tl.layer].N;
       __nv_bfloat16* Wb = p.layer[tl.layer].Wb;
@@ -279,13 +306,14 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
       if (!ok) { if (lane == 0) atomicExch(p.err_flag, 14); break; }
       tc_fence_after_sync();
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c, ++j) {
+      for (int ci = 0; ci < un.nc; ++ci, ++j) {
+        const int c = un.c0 + ci;          // column block inside the tile; the accumulator starts at the strip
         uint8_t* slot = my_ring + (j % R) * kSlotBytes;
         uint32_t r[32];
-        tmem_ld_32x32(taddr + buf * BN + c * 32, r);
+        tmem_ld_32x32(taddr + buf * BN + ci * 32, r);
         ok = __all_sync(0xffffffffu, mbar_wait(&my_full[j % R], (j / R) & 1));
         tmem_ld_wait();
-        if (c == BN / 32 - 1) {
+        if (ci == un.nc - 1) {
           // the accumulator has been read: hand the TMEM buffer back to the MMA warp
           tc_fence_before_sync();
           __syncwarp();
@@ -389,6 +417,11 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
   }
   p.n_layers = n; p.total_tiles = total;
+  {
+    const int ctas = total < num_sms() ? total : num_sms();
+    p.full_rounds = total / ctas;
+    p.tail_units = (total - p.full_rounds * ctas) * (TF32 ? 4 : 2);
+  }
   p.K = a0.B; p.groups = a0.groups; p.rows_per_group = a0.B;
   p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
   const int grid = total < num_sms() ? total : num_sms();
@@ -407,8 +440,8 @@ int tc_update_max_layers() { return kMaxLayers; }
 int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   if (launches) ++*launches;
-  if (layers[0].fp32) return launch_update<true, 3, 3>(layers, n, st);
-  return launch_update<false, 3, 4>(layers, n, st);
+  if (layers[0].fp32) return launch_update<true, 2, 4>(layers, n, st);
+  return launch_update<false, 2, 5>(layers, n, st);
 }
 
 }  // namespace ls
