@@ -5,7 +5,11 @@
 //   warp 0      TMA producer: cp.async.bulk.tensor tiles (128-byte swizzle) into a ring of stages
 //   warp 1      allocates tensor memory, issues tcgen05.mma (one elected thread), accumulator in TMEM
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (warp w owns TMEM lanes 32*(w%4)..+31) and apply
-//                 forward   Z = A W^T + b, relu                            (evaluating f, Section 2)
+//                 forward   Z = A W^T + b, relu                            (evaluating f, Section 2);
+//                           when the next layer is the narrow output layer and the tile holds the whole
+//                           mini-batch, also that layer: partial logits of this CTA's columns go to a
+//                           scratch, and the last CTA of the replica to finish adds them in a fixed
+//                           order and forms the per-sample losses and dZ of the output layer
 //                 backward  dZ_prev = (dZ W) * 1[act > 0]; when the tile holds the whole mini-batch, also the
 //                           bias update of the layer below from the column sums of dZ_prev
 //                 update    G = dZ^T A; v <- mu v + G; W <- W - eta v      (Section 2 mini-batch SGD
@@ -48,6 +52,7 @@ constexpr int KB_BYTES = 128;      // bytes of K per stage row (one swizzle row)
 constexpr int kThreadsBf16 = 192;  // warps 0-5
 constexpr int kThreadsFp32 = 256;  // + two splitter warps
 constexpr int kSplitWarps = 2;
+constexpr int kHeadMax = 16;       // outputs of a fused narrow output layer, at most
 constexpr int kStageLd = 36;       // floats per staged row (32 + 4 padding) in the update epilogue
 constexpr int kChunkStages = 4;    // fp32 forward/backward: stages per TMEM accumulation chunk (48 MMAs)
 
@@ -69,6 +74,8 @@ struct Params {
   void* C; const void* act;
   // backward: bias of the layer below and its momentum (or null), elements between replicas
   float* dbias; float* dvbias; int64_t dbias_gstride;
+  // forward: the narrow output layer that follows (hW null: none)
+  TcHead head;
   // update
   float* W; float* V; __nv_bfloat16* Wb; int64_t w_gstride; float lr, mu;
   int* err_flag;
@@ -215,6 +222,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
   float sum[CHUNKED ? BN : 1];
   bool ok = true;
+  // fused output layer: its weights for this CTA's columns ([class][CPR], as float4) and this thread's
+  // labels are requested now and parked in registers until the stage memory is free
+  constexpr int HP = (EPI == EPI_FWD) ? (kHeadMax * CPR / 4 + 127) / 128 : 1;
+  float4 hw_pref[HP];
+  int h_label[EPI == EPI_FWD ? MT : 1];
+  float h_target[EPI == EPI_FWD ? MT : 1];
+  if (EPI == EPI_FWD && warp >= 2 && warp < 6 && p.head.W != nullptr) {
+    const float* hw = p.head.W + (int64_t)g * p.head.w_gstride + n0 + rank * CPR;
+#pragma unroll
+    for (int i = 0; i < HP; ++i) {
+      const int idx = (int)threadIdx.x - 64 + i * 128;
+      const int cls = idx / (CPR / 4), c4 = idx % (CPR / 4);
+      hw_pref[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (cls < p.head.C) hw_pref[i] = __ldg(reinterpret_cast<const float4*>(hw + (int64_t)cls * p.N) + c4);
+    }
+    const int64_t y0 = p.head.y_row_off[g];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      h_label[mt] = 0; h_target[mt] = 0.f;
+      if (p.head.kind == LS_LOSS_SOFTMAX_CE) h_label[mt] = static_cast<const int32_t*>(p.head.y)[y0 + mt * BM + q * 32 + lane];
+      else h_target[mt] = static_cast<const float*>(p.head.y)[y0 + mt * BM + q * 32 + lane];
+    }
+  }
 
   if (warp == 0) {
     if (elect_one()) {
@@ -358,6 +388,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     cluster_sync_all();      // every CTA stays alive until the others have read its tile
   }
   if (warp >= 2 && warp < 6) {
+    // weights of the fused output layer: behind the exchange tile, which other CTAs may still be reading
+    float4* ws4 = reinterpret_cast<float4*>(smem + (SPLIT > 1 ? BN * BM * 4 : 0) + 256);
+    if (EPI == EPI_FWD && p.head.W != nullptr) {
+#pragma unroll
+      for (int i = 0; i < HP; ++i) {
+        const int idx = (int)threadIdx.x - 64 + i * 128;
+        if (idx < kHeadMax * CPR / 4) ws4[idx] = hw_pref[i];
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+    float hl[EPI == EPI_FWD ? MT : 1][kHeadMax];      // partial logits of this thread's row(s)
+#pragma unroll
+    for (int i = 0; i < (EPI == EPI_FWD ? MT : 1); ++i)
+#pragma unroll
+      for (int cls = 0; cls < kHeadMax; ++cls) hl[i][cls] = 0.f;
     if (ok) {
 #pragma unroll
       for (int cc32 = 0; cc32 < MT * (CPR / 32); ++cc32) {
@@ -382,6 +427,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             o[i] = (p.relu && !(v > 0.f)) ? 0.f : v;
           }
           store_row32<TF32>(p.C, ((int64_t)g * p.M + row) * p.N + col, o);
+          if (p.head.W != nullptr) {
+            // logits of the output layer restricted to these 32 columns (of the values as stored)
+            if (!TF32) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __bfloat162float(__float2bfloat16_rn(o[i]));
+            }
+#pragma unroll
+            for (int cls = 0; cls < kHeadMax; ++cls) {
+              if (cls < p.head.C) {           // uniform; the classes are independent chains
+                const float4* w4 = ws4 + (cls * CPR + c * 32) / 4;
+                float a = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float4 w = w4[i];
+                  a = fmaf(o[4 * i + 3], w.w, fmaf(o[4 * i + 2], w.z, fmaf(o[4 * i + 1], w.y, fmaf(o[4 * i], w.x, a))));
+                }
+                hl[mt][cls] += a;
+              }
+            }
+          }
         } else if (EPI == EPI_DX) {
           const int64_t at = ((int64_t)g * p.M + row) * p.N + col;
           float o[32];
@@ -470,6 +535,85 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
           __syncwarp();
+        }
+      }
+    }
+    if (EPI == EPI_FWD && p.head.W != nullptr) {
+      // ---- the output layer, finished by the last CTA of the replica ---------------------------------
+      const TcHead& hd = p.head;
+      const int parts = gridDim.x;                 // CTAs that hold columns of this replica's rows
+      const int tid = q * 32 + lane;               // this thread's row inside a row block (its TMEM lane)
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        float4* dst = reinterpret_cast<float4*>(hd.part + (((int64_t)g * parts + blockIdx.x) * p.M + mt * BM + tid) * kHeadMax);
+#pragma unroll
+        for (int i = 0; i < kHeadMax / 4; ++i)
+          dst[i] = make_float4(hl[mt][4 * i], hl[mt][4 * i + 1], hl[mt][4 * i + 2], hl[mt][4 * i + 3]);
+      }
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      uint32_t* flag = reinterpret_cast<uint32_t*>(smem + (SPLIT > 1 ? BN * BM * 4 : 0));   // idle stage memory
+      if (tid == 0) *flag = (atomicInc(hd.counters + g, (unsigned)parts - 1) == (unsigned)parts - 1) ? 1u : 0u;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*flag != 0u) {
+        __threadfence();
+        const float invB = 1.0f / (float)p.M;
+        float lsum = 0.f;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int b = mt * BM + tid;
+          float z[kHeadMax];
+#pragma unroll
+          for (int cls = 0; cls < kHeadMax; ++cls)
+            z[cls] = (hd.bias != nullptr && cls < hd.C) ? hd.bias[(int64_t)g * hd.w_gstride + cls] : 0.f;
+          for (int pt = 0; pt < parts; ++pt) {          // fixed order: column block by column block
+            const float4* src = reinterpret_cast<const float4*>(hd.part + (((int64_t)g * parts + pt) * p.M + b) * kHeadMax);
+#pragma unroll
+            for (int i = 0; i < kHeadMax / 4; ++i) {
+              const float4 v = __ldcg(src + i);
+              z[4 * i] += v.x; z[4 * i + 1] += v.y; z[4 * i + 2] += v.z; z[4 * i + 3] += v.w;
+            }
+          }
+          float loss;
+          float d[kHeadMax];
+          if (hd.kind == LS_LOSS_SOFTMAX_CE) {
+            const int label = h_label[mt];
+            float mx = z[0];
+#pragma unroll
+            for (int cls = 1; cls < kHeadMax; ++cls) if (cls < hd.C) mx = fmaxf(mx, z[cls]);
+            float sum = 0.f, zy = mx;
+#pragma unroll
+            for (int cls = 0; cls < kHeadMax; ++cls)
+              if (cls < hd.C) {
+                d[cls] = expf(z[cls] - mx);
+                sum += d[cls];
+                if (cls == label) zy = z[cls];
+              }
+            loss = (mx + logf(sum)) - zy;
+#pragma unroll
+            for (int cls = 0; cls < kHeadMax; ++cls)
+              if (cls < hd.C) d[cls] = (d[cls] / sum - (cls == label ? 1.f : 0.f)) * invB;
+          } else {
+            const float res = z[0] - h_target[mt];
+            loss = 0.5f * res * res;
+            d[0] = res * invB;
+          }
+          hd.row_loss[(int64_t)g * p.M + b] = loss;
+          lsum += loss;
+          if (hd.dZ != nullptr) {
+#pragma unroll
+            for (int cls = 0; cls < kHeadMax; ++cls)
+              if (cls < hd.C) hd.dZ[((int64_t)g * p.M + b) * hd.C + cls] = d[cls];
+          }
+        }
+        if (!hd.defer_loss && hd.loss_out != nullptr) {
+          // mean of the row losses: lanes, then the four warps in order
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o2);
+          float* wsum = reinterpret_cast<float*>(flag) + 8;
+          if (lane == 0) wsum[q] = lsum;
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (tid == 0) hd.loss_out[g] = (wsum[0] + wsum[1] + wsum[2] + wsum[3]) * invB;
         }
       }
     }
@@ -589,6 +733,18 @@ int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64
   return make_map(out, base, true, false, true, 3, rows, cols, groups, gstride);
 }
 
+// The forward kernel can also evaluate a narrow output layer that follows when one CTA holds every row of
+// its columns and the layer fits kHeadMax outputs.  Used for one row block (M = 128): with the 256-row
+// bf16 tile the four epilogue warps carry two rows each and the separate output-layer kernel, which
+// spreads the rows over the whole GPU, measured faster.
+bool tc_fwd_fuses_head(bool fp32, int M, int N, int C) {
+  (void)fp32;
+  if (C < 1 || C > kHeadMax || N % 4 != 0) return false;
+  return M == BM;
+}
+// upper bound of the CTAs that share a replica's rows (column blocks of at least 32 columns)
+int tc_fwd_head_parts(int N) { return N / 32; }
+
 // The backward kernel can finish the bias update when one CTA holds every row of its columns: M is one
 // row block, or two with the 256-row bf16 tile.
 bool tc_dx_fuses_bias(bool fp32, int M, int N) {
@@ -609,6 +765,8 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.bias = a.bias; p.bias_gstride = a.bias_gstride; p.relu = a.relu;
   p.C = a.C; p.err_flag = a.err_flag;
+  p.head = a.head;
+  if (p.head.W != nullptr && !tc_fwd_fuses_head(a.fp32, a.M, a.N, p.head.C)) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);

@@ -76,6 +76,9 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   lay.dzl_off = take((size_t)m * batch * lay.dims[lay.L] * 4);
   lay.rowloss_off = take((size_t)LS_MAX_REPLICAS * batch * 4);
   lay.headcnt_off = take((size_t)LS_MAX_REPLICAS * 4);
+  if (lay.L >= 2 && head_shape_ok(batch, lay.dims[lay.L]) &&
+      tc_fwd_fuses_head(!lay.bf16, batch, lay.dims[lay.L - 1], lay.dims[lay.L]))
+    lay.headpart_off = take((size_t)m * tc_fwd_head_parts(lay.dims[lay.L - 1]) * batch * 16 * 4);
   lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
   lay.evaloff_off = take((size_t)kEvalCap * 8);
   lay.evalloss_off = take((size_t)kEvalCap * 4);
@@ -177,8 +180,24 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       t.C = h->state + lay.act_off[l + 1];
       t.M = lay.batch; t.N = lay.dims[l + 1]; t.K = lay.dims[l]; t.groups = groups; t.relu = 1;
       t.err_flag = err_flag_of(h);
+      t.head = TcHead{};
+      const bool fuse_head = l == lay.L - 2 && lay.headpart_off != 0 && groups <= lay.m;
+      if (fuse_head) {
+        // the narrow output layer rides on this kernel: logits, per-sample losses and dZ_L
+        TcHead& hd = t.head;
+        hd.W = P + lay.w_off[lay.L - 1]; hd.w_gstride = w_gstride;
+        hd.bias = lay.has_bias ? P + lay.b_off[lay.L - 1] : nullptr;
+        hd.y = y; hd.y_row_off = row_off_dev;
+        hd.part = reinterpret_cast<float*>(h->state + lay.headpart_off);
+        hd.counters = reinterpret_cast<unsigned int*>(h->state + lay.headcnt_off);
+        hd.dZ = want_dz ? reinterpret_cast<float*>(h->state + lay.dzl_off) : nullptr;
+        hd.row_loss = reinterpret_cast<float*>(h->state + lay.rowloss_off);
+        hd.loss_out = loss_out;
+        hd.C = lay.dims[lay.L]; hd.kind = h->spec.loss; hd.defer_loss = want_dz ? 1 : 0;
+      }
       ProfScope ps(h, LS_K_FWD, l);
       LS_CUDA(h, launch_tc_fwd(t, h->stream, &h->launches));
+      if (fuse_head) return LS_OK;
       continue;
     }
     FwdArgs a;

@@ -45,6 +45,7 @@ struct Layout {
   size_t dzl_off = 0;                        // fp32 dZ of a narrow output layer [m][batch][dims[L]]
   size_t rowloss_off = 0;                    // per-sample losses [LS_MAX_REPLICAS][batch]
   size_t headcnt_off = 0;                    // per-replica CTA counters of the output-layer kernel
+  size_t headpart_off = 0;                   // partial logits of a fused output layer [m][parts][batch][16]
   size_t rowoff_off = 0;                     // int64 [kRowOffCap][m]
   size_t evaloff_off = 0;                    // int64 [kEvalCap]
   size_t evalloss_off = 0;                   // float [kEvalCap]
@@ -253,6 +254,19 @@ bool tc_shape_ok(bool fp32, int M, int N, int K);   // output rows, output colum
 struct TcOperandMaps {
   const CUtensorMap *a, *b;
 };
+// A narrow output layer evaluated by the forward kernel of the layer before it (W null: none).
+struct TcHead {
+  const float* W; int64_t w_gstride; const float* bias;    // [C][N] fp32 master weights, bias or null
+  const void* y; const int64_t* y_row_off;                 // labels / targets and each group's first row
+  float* part;               // scratch [groups][parts][M][16] partial logits, parts <= tc_fwd_head_parts(N)
+  unsigned int* counters;    // [groups], zero before the launch, zero again after it
+  float* dZ;                 // [groups][M][C] or null (forward only)
+  float* row_loss;           // [groups][M]
+  float* loss_out;           // [groups] or null
+  int C, kind, defer_loss;   // defer_loss: leave the mean of the row losses to the backward kernel
+};
+bool tc_fwd_fuses_head(bool fp32, int M, int N, int C);
+int tc_fwd_head_parts(int N);
 struct TcFwdArgs {
   TcOperandMaps maps;        // a: [rows][K] input (dataset rows through row_off, else group g at row g*M); b: weights
   bool fp32;
@@ -260,6 +274,7 @@ struct TcFwdArgs {
   int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
   const float* bias; int64_t bias_gstride;
   void* C;                   // [groups][M][N] bf16 or fp32
+  TcHead head;
   int M, N, K, groups, relu;
   int* err_flag;
 };
