@@ -530,6 +530,36 @@ def run_ours(args, w: wl.Workload):
             del buf
         line["averaging_gbs"] = avg
 
+        # ---- measured throughput against the period, beside the runtime model's speed-up (Section 3.2) -----
+        if args.tau_sweep:
+            sweep = {}
+            n_it = 400
+            so = wl.batch_row_offsets(w.seed + 999, n_it, m, w.n_rows, B)
+            sl = torch.zeros((n_it, m), dtype=torch.float32, device="cuda")
+            for t in (1, 2, 5, 20, 100):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                for rep in range(2):           # first pass warms up
+                    torch.cuda.synchronize()
+                    ev[0].record()
+                    for k0 in range(0, n_it, t):
+                        n = min(t, n_it - k0)
+                        eng.local_steps(n, so[k0:k0 + n], sl[k0:k0 + n])
+                        eng.average()
+                    ev[1].record()
+                    torch.cuda.synchronize()
+                sweep[t] = ev[0].elapsed_time(ev[1]) / n_it          # ms per iteration
+            # Y: time of an iteration without averaging, D: time of one averaging, both from the two ends
+            # of the sweep (T(tau) = Y + D / tau)
+            D_ms = (sweep[1] - sweep[100]) / (1.0 - 1.0 / 100.0)
+            Y_ms = sweep[1] - D_ms
+            alpha = D_ms / Y_ms
+            line["tau_sweep"] = {
+                "ms_per_iteration": {str(t): round(v, 5) for t, v in sweep.items()},
+                "Y_ms": round(Y_ms, 5), "D_ms": round(D_ms, 5), "alpha": round(alpha, 4),
+                "speedup_measured": {str(t): round(sweep[1] / v, 4) for t, v in sweep.items()},
+                "speedup_model": {str(t): round((1 + alpha) / (1 + alpha / t), 4) for t in sweep},
+                "note": "model: (1 + alpha) / (1 + alpha / tau) with alpha = D / Y fitted at tau = 1 and 100"}
+
         # ---- the CPU oracle on the host cores, bounded sample -----------------------------------
         if not args.no_cpu_baseline:
             v, iters, dt = oracle_replica_steps_per_s(w, X[:8192], y[:8192], x1, tau, budget_s=args.cpu_budget,
@@ -554,6 +584,8 @@ def main():
     ap.add_argument("--tau", type=int, default=20)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tau-sweep", action="store_true",
+                    help="also time iterations at tau = 1, 2, 5, 20, 100 and compare with the speed-up model of Section 3.2")
     ap.add_argument("--avg-1b", action="store_true", help="add the 10^9-element point to the averaging sweep (128 GB)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, averaging sweep or CPU baseline")

@@ -256,6 +256,43 @@ int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows,
            int64_t* decision_k, float* decision_F, int32_t* decision_tau, int64_t max_decisions,
            int64_t* n_decisions, float* F0_host);
 
+/* The same run with the intervals of Section 4 as the paper defines them: training is cut into
+ * wall-clock intervals of length T0_ms, and the period is re-chosen at the first averaging point
+ * after each interval boundary (the clock is the host's steady clock, read after the stream has
+ * drained at every averaging point, starting when the first local step is enqueued).  The schedule
+ * depends on how fast the machine is, so it is not reproducible; what is reproducible is that every
+ * logged decision equals adacomm_next_tau(decision_F, F_0, tau_0).  T0_ms <= 0 decides at every
+ * averaging point.  decision_ms (optional, [max_decisions]) receives the elapsed time of each decision. */
+int ls_run_timed(ls_handle* h, int64_t K, int tau_0, double T0_ms, int64_t probe_rows,
+                 const int64_t* row_offset_host, float* loss_dev,
+                 int32_t* period_tau, int64_t max_periods, int64_t* n_periods,
+                 int64_t* decision_k, float* decision_F, int32_t* decision_tau, double* decision_ms,
+                 int64_t max_decisions, int64_t* n_decisions, float* F0_host);
+
+/* ---- runtime model (host only; Sections 2-4) -------------------------------
+ * The delay model and the runtime / error-runtime formulas that motivate the choice of the period.
+ * Pure host functions: no GPU, no handle. */
+enum { LS_DELAY_CONSTANT = 0, LS_DELAY_LOG2 = 1, LS_DELAY_TREE = 2, LS_DELAY_LINEAR = 3 };
+/* D = D0 * s(m) with s(m) = 1, log2 m, 2 log2 m (reduction tree) or m  (Section 2, delay model). */
+int ls_delay(double D0, int m, int scaling, double* D);
+/* E[T_sync] / E[T_P-Avg] = (1 + alpha) / (1 + alpha / tau) for constant Y and D, alpha = D / Y (Section 3.2). */
+int ls_speedup(double alpha, int tau, double* speedup);
+/* Theorem 1: 2 (F1 - Finf) / (lr T) (Y + D / tau) + lr L sigma2 / m + lr^2 L^2 sigma2 (tau - 1). */
+int ls_error_bound(double T, double F1, double Finf, double lr, double L, double sigma2, int m, int tau, double Y,
+                   double D, double* bound);
+/* Theorem 2: tau* = sqrt(2 (F1 - Finf) D / (lr^3 L^2 sigma2 T)). */
+int ls_tau_star(double F1, double Finf, double D, double lr, double L, double sigma2, double T, double* tau);
+/* Monte-Carlo means of the runtime per iteration (Section 3.1) over n_periods periods of tau local
+ * steps of m workers: t_sync_mean of T_sync = max_i Y_i + D (every local step followed by a
+ * broadcast), t_pavg_mean of T_P-Avg = max_i (sum_k Y_ik / tau) + D / tau, on the same draws.
+ * Y_ik is exponential with mean y_mean (exponential != 0) or the constant y_mean.  The draw of
+ * (period p, step k, worker i) is -y_mean ln((x + 0.5) / 2^32), x the first word of
+ * Philox4x32-10(counter = (p lo, p hi, k, i), key = (seed lo, seed hi)). */
+int ls_simulate_runtime(int m, int tau, int64_t n_periods, double y_mean, double D, uint64_t seed, int exponential,
+                        double* t_sync_mean, double* t_pavg_mean);
+/* One block of Philox4x32-10 (Salmon et al., SC'11). */
+int ls_philox4x32_10(const uint32_t counter[4], const uint32_t key[2], uint32_t out[4]);
+
 /* Mean loss of a linear model on device-resident rows, for callers that must not allocate.
  * (The paper has no counterpart: this entry point exists for deployment reasons only.)
  *

@@ -90,6 +90,13 @@ def _lib():
         "ls_average_flat": (C.c_int, [vp, C.c_int, i64, i64, vp]),
         "ls_block_average_flat": (C.c_int, [vp, vp, vp, C.c_int, i64, i64, C.c_float, C.c_float, vp]),
         "ls_set_block_state": (C.c_int, [vp, vp, vp]),
+        "ls_run_timed": (C.c_int, [vp, i64, C.c_int, C.c_double, i64, vp, vp, vp, i64, vp, vp, vp, vp, vp, i64, vp, vp]),
+        "ls_delay": (C.c_int, [C.c_double, C.c_int, C.c_int, vp]),
+        "ls_speedup": (C.c_int, [C.c_double, C.c_int, vp]),
+        "ls_error_bound": (C.c_int, [C.c_double] * 6 + [C.c_int, C.c_int, C.c_double, C.c_double, vp]),
+        "ls_tau_star": (C.c_int, [C.c_double] * 7 + [vp]),
+        "ls_simulate_runtime": (C.c_int, [C.c_int, C.c_int, i64, C.c_double, C.c_double, C.c_uint64, C.c_int, vp, vp]),
+        "ls_philox4x32_10": (C.c_int, [vp, vp, vp]),
         "ls_get_block_state": (C.c_int, [vp, vp, vp]),
         "ls_eval_loss": (C.c_int, [vp, C.c_int, i64, i64, P(f32)]),
         "adacomm_next_tau": (C.c_int, [C.c_double, C.c_double, C.c_int]),
@@ -199,6 +206,52 @@ def block_average_flat(buf, anchor, u, m: int, P: int, lr: float, beta: float, s
         raise ValueError("buffer too small")
     _check(_lib().ls_block_average_flat(buf.data_ptr(), anchor.data_ptr(), u.data_ptr(), int(m), int(P), stride,
                                         float(lr), float(beta), _stream_ptr(stream)), "ls_block_average_flat")
+
+
+# ---- runtime model (host only; Sections 2-4) ----------------------------------------------------------
+DELAY_SCALING = {"constant": 0, "log2": 1, "tree": 2, "linear": 3}
+
+
+def delay(D0: float, m: int, scaling: str = "tree") -> float:
+    out = C.c_double()
+    _check(_lib().ls_delay(float(D0), int(m), DELAY_SCALING[scaling], C.byref(out)), "ls_delay")
+    return out.value
+
+
+def speedup(alpha: float, tau: int) -> float:
+    out = C.c_double()
+    _check(_lib().ls_speedup(float(alpha), int(tau), C.byref(out)), "ls_speedup")
+    return out.value
+
+
+def error_bound(T, F1, Finf, lr, L, sigma2, m, tau, Y, D) -> float:
+    out = C.c_double()
+    _check(_lib().ls_error_bound(float(T), float(F1), float(Finf), float(lr), float(L), float(sigma2), int(m), int(tau),
+                                 float(Y), float(D), C.byref(out)), "ls_error_bound")
+    return out.value
+
+
+def tau_star(F1, Finf, D, lr, L, sigma2, T) -> float:
+    out = C.c_double()
+    _check(_lib().ls_tau_star(float(F1), float(Finf), float(D), float(lr), float(L), float(sigma2), float(T),
+                              C.byref(out)), "ls_tau_star")
+    return out.value
+
+
+def simulate_runtime(m: int, tau: int, n_periods: int, y_mean: float, D: float, seed: int, exponential: bool = True):
+    """(mean T_sync, mean T_P-Avg) per iteration over n_periods periods (Section 3.1)."""
+    a, b = C.c_double(), C.c_double()
+    _check(_lib().ls_simulate_runtime(int(m), int(tau), int(n_periods), float(y_mean), float(D), int(seed),
+                                      int(bool(exponential)), C.byref(a), C.byref(b)), "ls_simulate_runtime")
+    return a.value, b.value
+
+
+def philox4x32_10(counter, key):
+    c = (C.c_uint32 * 4)(*counter)
+    k = (C.c_uint32 * 2)(*key)
+    o = (C.c_uint32 * 4)()
+    _check(_lib().ls_philox4x32_10(c, k, o), "ls_philox4x32_10")
+    return tuple(int(v) for v in o)
 
 
 def linear_loss_static(W, bias, x, y, chunk_rows: int, chunk_loss, loss: str = "softmax_ce", stream=None) -> None:
@@ -369,6 +422,27 @@ class LocalSGD:
         n_p, n_d = n_p.value, n_d.value
         return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
                 "decision_tau": dt[:n_d].tolist(), "F_0": float(F0.value) if interval > 0 else None}
+
+    def run_timed(self, K: int, tau_0: int, T0_ms: float, row_offsets: np.ndarray, probe_rows: int, loss_out=None):
+        """K iterations with AdaComm decisions at wall-clock intervals of T0_ms (Section 4)."""
+        offs = np.ascontiguousarray(row_offsets, dtype=np.int64)
+        if offs.size != K * self.m:
+            raise ValueError("row_offsets must be [K][m]")
+        max_p = int(K) + 1
+        period_tau = np.zeros(max_p, dtype=np.int32)
+        dk = np.zeros(max_p, dtype=np.int64)
+        dF = np.zeros(max_p, dtype=np.float32)
+        dt = np.zeros(max_p, dtype=np.int32)
+        dms = np.zeros(max_p, dtype=np.float64)
+        n_p, n_d, F0 = C.c_int64(), C.c_int64(), C.c_float()
+        lp = None if loss_out is None else loss_out.data_ptr()
+        _check(self.lib.ls_run_timed(self.h, int(K), int(tau_0), float(T0_ms), int(probe_rows), offs.ctypes.data, lp,
+                                     period_tau.ctypes.data, max_p, C.byref(n_p), dk.ctypes.data, dF.ctypes.data,
+                                     dt.ctypes.data, dms.ctypes.data, max_p, C.byref(n_d), C.byref(F0)),
+               "ls_run_timed")
+        n_p, n_d = n_p.value, n_d.value
+        return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
+                "decision_tau": dt[:n_d].tolist(), "decision_ms": dms[:n_d].copy(), "F_0": float(F0.value)}
 
     def profile_begin(self, classes: Sequence[str] = KERNEL_CLASSES, layer: int = -1):
         mask = 0

@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <chrono>
 #include <new>
 #include <vector>
 
@@ -775,7 +776,18 @@ int adacomm_next_tau_refined(double F_t, double F_0, int tau_0, int tau_prev, do
 static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
                     float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
                     float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions,
-                    float* F0_host, const ls_adacomm_opts* opts);
+                    float* F0_host, const ls_adacomm_opts* opts, bool timed = false, double t0_ms = 0.0,
+                    double* decision_ms = nullptr);
+
+int ls_run_timed(ls_handle* h, int64_t K, int tau_0, double T0_ms, int64_t probe_rows, const int64_t* row_offset_host,
+                 float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
+                 float* decision_F, int32_t* decision_tau, double* decision_ms, int64_t max_decisions,
+                 int64_t* n_decisions, float* F0_host) {
+  if (!isfinite(T0_ms)) return LS_ERR_INVALID_ARG;
+  return run_loop(h, K, tau_0, 1, probe_rows, row_offset_host, loss_dev, period_tau, max_periods, n_periods,
+                  decision_k, decision_F, decision_tau, max_decisions, n_decisions, F0_host, nullptr, true, T0_ms,
+                  decision_ms);
+}
 
 int ls_run(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
            float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
@@ -803,7 +815,7 @@ int ls_run_refined(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pro
 static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t probe_rows, const int64_t* row_offset_host,
                     float* loss_dev, int32_t* period_tau, int64_t max_periods, int64_t* n_periods, int64_t* decision_k,
                     float* decision_F, int32_t* decision_tau, int64_t max_decisions, int64_t* n_decisions,
-                    float* F0_host, const ls_adacomm_opts* opts) {
+                    float* F0_host, const ls_adacomm_opts* opts, bool timed, double t0_ms, double* decision_ms) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   if (K < 1 || tau_0 < 1 || interval < 0 || row_offset_host == nullptr) return LS_ERR_INVALID_ARG;
   const Layout& lay = h->lay;
@@ -817,6 +829,7 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
   }
   int64_t k = 0, np = 0, nd = 0, next_interval = 1;
   int tau = tau_0;
+  const auto t_start = std::chrono::steady_clock::now();
   while (k < K) {
     const int steps = (int)((K - k < tau) ? K - k : tau);
     if (period_tau && np < max_periods) period_tau[np] = tau;
@@ -826,7 +839,15 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
     k += steps;
     rc = average(h);
     if (rc != LS_OK) return rc;
-    if (interval > 0 && k >= next_interval * (int64_t)interval) {
+    bool decide = interval > 0 && k >= next_interval * (int64_t)interval;
+    double elapsed_ms = 0.0;
+    if (timed) {
+      // wall-clock intervals (Section 4): the averaging step has to be over before the clock is read
+      LS_CUDA(h, cudaStreamSynchronize(h->stream));
+      elapsed_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_start).count();
+      decide = t0_ms <= 0.0 || elapsed_ms >= (double)next_interval * t0_ms;
+    }
+    if (decide) {
       float F_t = 0.f;
       rc = eval_loss(h, 0, 0, probe_rows, &F_t);
       if (rc != LS_OK) return rc;
@@ -850,9 +871,11 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
         if (decision_k) decision_k[nd] = k;
         if (decision_F) decision_F[nd] = F_t;
         if (decision_tau) decision_tau[nd] = t;
+        if (decision_ms) decision_ms[nd] = elapsed_ms;
       }
       ++nd;
-      next_interval = k / interval + 1;
+      if (timed) next_interval = t0_ms > 0.0 ? (int64_t)floor(elapsed_ms / t0_ms) + 1 : 1;
+      else next_interval = k / interval + 1;
     }
   }
   if (n_periods) *n_periods = np;

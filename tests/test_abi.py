@@ -101,3 +101,38 @@ def test_refined_controller_agrees_with_hand_table_and_oracle():
     assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 0, 0.5, 0, 0.1, 0.1, 0) == binding.LS_ERR_INVALID_ARG
     assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 20, 0.5, -1, 0.1, 0.1, 0) == binding.LS_ERR_INVALID_ARG
     assert lib.adacomm_next_tau_refined(1.0, 1.0, 20, 20, 0.5, 0, 0.1, 0.0, 0) == binding.LS_ERR_INVALID_ARG
+
+
+def test_runtime_model_host_functions_match_the_oracle():
+    """Sections 2-4: delay model, speed-up, Theorems 1-2 and the Monte-Carlo runtime means (host code, no GPU)."""
+    import math
+    from oracle import runtime_model_oracle as rm
+    from paper_1810_08313_b200 import binding
+    assert binding.philox4x32_10((0, 0, 0, 0), (0, 0)) == (0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8)
+    for c, k in [((1, 2, 3, 4), (5, 6)), ((0xFFFFFFFF, 0, 7, 0x80000000), (0xDEADBEEF, 1))]:
+        assert binding.philox4x32_10(c, k) == rm.philox4x32_10(c, k)
+    for name, code in binding.DELAY_SCALING.items():
+        for m in (1, 2, 16, 100):
+            assert binding.delay(0.37, m, name) == rm.delay(0.37, m, code)
+    for alpha, tau in [(0.9, 1), (0.9, 10), (4.0, 100), (0.0, 3)]:
+        assert binding.speedup(alpha, tau) == rm.speedup_constant(alpha, tau)
+    args = (500.0, 1.0, 0.0, 0.08, 1.0, 1.0, 16, 10, 1.0, 1.0)
+    assert abs(binding.error_bound(*args) - rm.error_bound(*args)) <= 1e-15 * rm.error_bound(*args)
+    ts = binding.tau_star(1.0, 0.0, 1.0, 0.08, 1.0, 1.0, 500.0)
+    assert abs(ts - rm.tau_star(1.0, 0.0, 1.0, 0.08, 1.0, 1.0, 500.0)) <= 1e-15 * ts
+    for (m, tau, n, y, D, seed, expo) in [(16, 10, 30, 1.0, 1.0, 7, True), (4, 1, 50, 2.0, 0.5, 2 ** 40 + 3, True),
+                                          (8, 5, 4, 1.5, 0.9, 1, False)]:
+        gs, gp = binding.simulate_runtime(m, tau, n, y, D, seed, expo)
+        ws, wp = rm.simulate(m, tau, n, y, D, seed, expo)
+        assert abs(gs - ws) <= 1e-12 * ws and abs(gp - wp) <= 1e-12 * wp
+    # the harmonic-sum law on the library's own draws (Section 3.2)
+    s, _ = binding.simulate_runtime(16, 1, 20000, 1.0, 0.0, 5, True)
+    assert abs(s - sum(1.0 / i for i in range(1, 17))) < 3 * math.sqrt(1.65 / 20000)
+    lib = binding._lib()
+    out = binding.C.c_double()
+    bad = binding.LS_ERR_INVALID_ARG
+    assert lib.ls_delay(1.0, 0, 0, binding.C.byref(out)) == bad
+    assert lib.ls_delay(1.0, 4, 9, binding.C.byref(out)) == bad
+    assert lib.ls_speedup(0.5, 0, binding.C.byref(out)) == bad
+    assert lib.ls_tau_star(1.0, 0.0, 1.0, 0.0, 1.0, 1.0, 1.0, binding.C.byref(out)) == bad
+    assert lib.ls_simulate_runtime(0, 1, 1, 1.0, 1.0, 1, 1, binding.C.byref(out), binding.C.byref(out)) == bad

@@ -281,3 +281,45 @@ def test_refined_adacomm_run_with_deferred_lr_decay():
         assert t == want
         prev = t
     eng.close()
+
+
+def test_wall_clock_intervals():
+    """Section 4: decisions at wall-clock interval boundaries.  With T0 <= 0 every averaging point decides, which
+    is the iteration scheme with interval 1 and must follow the oracle; with a real T0 the schedule depends on
+    the machine, and what is checked is every decision against the rule and the interval bookkeeping."""
+    import torch
+    from paper_1810_08313_b200 import binding
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims, m, B, tau0, K, probe = (96, 64, 48, 10), 4, 32, 6, 60, 256
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 31)
+    offs = wl.batch_row_offsets(4, K, m, 1024, B)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B)
+    eng.bind_dataset(xd, yd)
+    # (1) every averaging point decides
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(0.9), tau0, adacomm_interval=1, probe_rows=probe)
+    eng.set_params(x1)
+    out = eng.run_timed(K, tau0, 0.0, offs, probe)
+    eng.sync()
+    assert out["taus"] == ref.taus
+    assert out["decision_k"] == [k for k, _, _ in ref.F_trace]
+    assert out["decision_tau"] == [t for _, _, t in ref.F_trace]
+    gx, _ = eng.get_all()
+    assert max_rel_err_per_tensor(gx[0], ref.params[0], dims, True) <= 2e-4
+    # (2) an interval longer than the run: the period never changes
+    eng.set_params(x1)
+    out = eng.run_timed(K, tau0, 1e9, offs, probe)
+    assert out["decision_k"] == [] and out["taus"] == [tau0] * (K // tau0)
+    # (3) a real interval: each decision follows the rule on its logged loss, in a later interval than the last
+    eng.set_params(x1)
+    T0 = 0.25
+    out = eng.run_timed(K, tau0, T0, offs, probe)
+    assert len(out["decision_k"]) >= 1
+    last = 0
+    for F, t, ms in zip(out["decision_F"], out["decision_tau"], out["decision_ms"]):
+        assert t == binding.adacomm_next_tau(float(F), out["F_0"], tau0)
+        assert int(ms // T0) > last or last == 0
+        assert ms >= T0
+        last = int(ms // T0)
+    assert sum(min(t, K) for t in out["taus"]) >= K
+    eng.close()
