@@ -441,7 +441,7 @@ int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (layers[0].fp32) return launch_update<true, 2, 4>(layers, n, st);
-  return launch_update<false, 2, 5>(layers, n, st);
+  return launch_update<false, 1, 6>(layers, n, st);
 }
 
 }  // namespace ls
