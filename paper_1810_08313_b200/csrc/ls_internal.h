@@ -4,6 +4,7 @@
 
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <stdlib.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
@@ -121,9 +122,13 @@ inline cudaError_t launch_dep(void (*kern)(P...), dim3 grid, dim3 block, size_t 
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   unsigned n = 0;
-  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[n].val.programmaticStreamSerializationAllowed = 1;
-  ++n;
+  // LS_DISABLE_PDL=1 in the environment launches every kernel in plain stream order (a diagnostic switch)
+  static const bool pdl = [] { const char* e = getenv("LS_DISABLE_PDL"); return !(e && e[0] == '1'); }();
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
   if (cluster_x > 1) {       // the CTAs that share an output tile form one cluster along x
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = cluster_x;
