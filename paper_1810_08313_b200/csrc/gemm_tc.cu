@@ -697,7 +697,7 @@ int launch_fp32(const TcOperandMaps& mp, const Params& p, int groups, cudaStream
 }
 
 int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, bool block32, int rank, int64_t rows,
-             int64_t cols, int64_t groups, int64_t gstride) {
+             int64_t cols, int64_t groups, int64_t gstride, int box_rows = 0) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
   const cuuint64_t eb = fp32 ? 4 : 2;
@@ -707,11 +707,13 @@ int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, bool bloc
   // K-major reads take boxes of 64 rows; MN-major reads (and the 32 x 32 blocks of the update kernel) of
   // fp32 tensors take 32 rows.  For bf16 both are 64.
   cuuint32_t box[3] = {elems, (fp32 && !mn32 && !block32) ? 64u : elems, 1};
+  if (box_rows > 0) box[1] = (cuuint32_t)box_rows;
   cuuint32_t es[3] = {1, 1, 1};
   CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
                   const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   (fp32 && mn32) ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  block32 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
@@ -721,6 +723,11 @@ int make_map(CUtensorMap* out, const void* base, bool fp32, bool mn32, bool bloc
 // swizzle.  mn32: the fp32 tensor will be read as an MN-major operand (swizzle in 32-byte units).
 int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols) {
   return make_map(out, base, fp32, mn32, false, 2, rows, cols, 1, 0);
+}
+// The same with boxes of box_rows rows (operand stages of the update kernel).
+int tc_make_map_2d_rows(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
+                        int box_rows) {
+  return make_map(out, base, fp32, mn32, false, 2, rows, cols, 1, 0, box_rows);
 }
 // 3-D map over `groups` row-major matrices [rows][cols] that start every gstride elements.
 int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,

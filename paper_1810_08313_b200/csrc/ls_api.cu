@@ -142,7 +142,7 @@ static int refresh_shadow(ls_handle* h) {
 static inline int* err_flag_of(const ls_handle* h) { return reinterpret_cast<int*>(h->state + h->lay.err_off); }
 
 // x maps: [0] for K-major reads, [1] for MN-major reads of the mini-batch rows
-struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; };
+struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; const CUtensorMap* upd; };
 
 static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
                    int groups, int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
@@ -296,8 +296,8 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
     if (tc_update_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
       TcUpdateArgs& t = upd[n_upd++];
       t.fp32 = !bf;
-      t.maps.a = &mn.dz[l];
-      t.maps.b = (l == 0) ? xmap.mn : &mn.act[l];
+      t.maps.a = &h->maps_upd.dz[l];
+      t.maps.b = (l == 0) ? xmap.upd : &h->maps_upd.act[l];
       t.mapW = &h->maps.wf[l];
       t.mapV = &h->maps.vf[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
@@ -396,7 +396,7 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
   const int cap = (lay.L == 1 && head_shape_ok(lay.batch, lay.dims[1])) ? LS_MAX_REPLICAS : lay.m;
   for (int64_t c0 = 0; c0 < chunks; c0 += cap) {
     const int groups = (int)((chunks - c0 < cap) ? chunks - c0 : cap);
-    int rc = forward(h, h->x_dev, XMaps{&h->maps.x_data, &h->maps_mn.x_data}, h->y_dev, off_dev + c0, groups, replica, 0,
+    int rc = forward(h, h->x_dev, XMaps{&h->maps.x_data, &h->maps_mn.x_data, &h->maps_upd.x_data}, h->y_dev, off_dev + c0, groups, replica, 0,
                      false, loss_dev + c0);
     if (rc != LS_OK) return rc;
   }
@@ -421,7 +421,7 @@ static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, fl
                                cudaMemcpyHostToDevice, h->stream));
     for (int s = 0; s < n; ++s) {
       const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
-      int rc = local_step(h, h->x_dev, XMaps{&h->maps.x_data, &mnm.x_data}, h->y_dev, off_dev + (int64_t)s * lay.m,
+      int rc = local_step(h, h->x_dev, XMaps{&h->maps.x_data, &mnm.x_data, &h->maps_upd.x_data}, h->y_dev, off_dev + (int64_t)s * lay.m,
                           loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr);
       if (rc != LS_OK) return rc;
     }
@@ -536,6 +536,17 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
           ok(tc_make_map_2d(&mp.x_stage[s], h->state + lay.stage_x_off[s], f, mn, rows, lay.dims[0]));
       }
     }
+    // the operands of the update kernel: dZ_l and the layer inputs, MN-major, boxes of its stage height
+    const int ur = tc_update_box_rows(f);
+    for (int l = 0; l < lay.L; ++l) {
+      if (l >= 1 && lay.dims[l] % q == 0)
+        ok(tc_make_map_2d_rows(&h->maps_upd.act[l], h->state + lay.act_off[l], f, f, rows, lay.dims[l], ur));
+      if (lay.dims[l + 1] % q == 0)
+        ok(tc_make_map_2d_rows(&h->maps_upd.dz[l], h->state + lay.dz_off[l], f, f, rows, lay.dims[l + 1], ur));
+    }
+    if (lay.dims[0] % q == 0)
+      for (int s = 0; s < 2; ++s)
+        ok(tc_make_map_2d_rows(&h->maps_upd.x_stage[s], h->state + lay.stage_x_off[s], f, f, rows, lay.dims[0], ur));
   }
   if (e != cudaSuccess) {
     h->last_cuda = e;
@@ -682,6 +693,8 @@ int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t 
   if (h->lay.dims[0] % (h->lay.bf16 ? 8 : 4) == 0) {
     LS_CUDA(h, tc_make_map_2d(&h->maps.x_data, x_dev, !h->lay.bf16, false, n_rows, h->lay.dims[0]));
     if (!h->lay.bf16) LS_CUDA(h, tc_make_map_2d(&h->maps_mn.x_data, x_dev, true, true, n_rows, h->lay.dims[0]));
+    LS_CUDA(h, tc_make_map_2d_rows(&h->maps_upd.x_data, x_dev, !h->lay.bf16, !h->lay.bf16, n_rows, h->lay.dims[0],
+                                   tc_update_box_rows(!h->lay.bf16)));
   }
   h->x_dev = x_dev;
   h->y_dev = y_dev;
@@ -724,7 +737,8 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
       LS_CUDA(h, cudaEventRecord(h->ev_copied[slot], h->copy_stream));
       LS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_copied[slot], 0));
       const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
-      int rc = local_step(h, xs, XMaps{&h->maps.x_stage[slot], &mnm.x_stage[slot]}, ys, stage_off,
+      int rc = local_step(h, xs, XMaps{&h->maps.x_stage[slot], &mnm.x_stage[slot], &h->maps_upd.x_stage[slot]}, ys,
+                          stage_off,
                           loss_stage + (int64_t)s * lay.m);
       if (rc != LS_OK) return rc;
       LS_CUDA(h, cudaEventRecord(h->ev_consumed[slot], h->stream));

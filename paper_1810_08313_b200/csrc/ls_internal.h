@@ -75,6 +75,7 @@ struct alignas(64) TcMaps {
 struct ls_handle {
   TcMaps maps;       // for K-major reads (and every read of a bf16 tensor)
   TcMaps maps_mn;    // fp32 models: the same tensors for MN-major reads (swizzle in 32-byte units)
+  TcMaps maps_upd;   // dz / act / x_* as the update kernel reads them (MN-major, boxes of tc_update_box_rows rows)
   uint32_t magic;
   ls::Layout lay;
   ls_model_spec spec;
@@ -251,6 +252,8 @@ int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t
 
 // ---- tcgen05 grouped GEMMs (gemm_tc.cu) -------------------------------------
 int tc_make_map_2d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols);
+int tc_make_map_2d_rows(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
+                        int box_rows);
 int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int64_t rows, int64_t cols,
                    int64_t groups, int64_t gstride);
 int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups,
@@ -319,6 +322,7 @@ struct TcUpdateArgs {
 };
 bool tc_update_shape_ok(bool fp32, int M, int N, int B);
 int tc_update_max_layers();
+int tc_update_box_rows(bool fp32);     // rows of the TMA boxes its operand maps (dZ, layer input) must have
 // one launch for the updates of layers[0..n) (n <= tc_update_max_layers(); same batch, replicas, rates, type)
 int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches);
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);

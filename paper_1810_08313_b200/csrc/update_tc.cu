@@ -40,6 +40,8 @@ constexpr int kThreads = 256;
 constexpr int kSlotBytes = 8192;       // one 32 x 32 fp32 block of W (4 KB) and of v (4 KB)
 
 constexpr int kMaxLayers = 4;          // layers per launch
+constexpr int kRowsFp32 = 16;          // mini-batch rows per operand stage: the TMA boxes of the operand maps
+constexpr int kRowsBf16 = 64;          // are this many rows high (tc_update_box_rows)
 
 struct ULayer {
   int N;                               // in features (row length of W)
@@ -80,10 +82,11 @@ __device__ __forceinline__ Tile decode_tile(const UParams& p, int t) {
 }
 
 // Operand stages are filled by TMA; fp32 models add one buffer for the lo parts of the stage in use.
-template <bool TF32, int STAGES, int R>
+// KS: K-rows (mini-batch rows) per stage.
+template <bool TF32, int STAGES, int R, int KS>
 struct USmem {
   static constexpr int kLoStages = TF32 ? 1 : 0;
-  static constexpr int kStageBytes = (BM + BN) * KB_BYTES;
+  static constexpr int kStageBytes = (BM + BN) * KS * (TF32 ? 4 : 2);
   static constexpr int kOperandBytes = (STAGES + kLoStages) * kStageBytes;
   static constexpr int kRingBytes = 4 * R * kSlotBytes;
   static constexpr int kBars = 2 * STAGES + 2 + 4 + 4 * R;
@@ -111,12 +114,12 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
                : "memory");
 }
 
-template <int ELEMS>
+template <int MNC, int KS>
 __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, int tile0, int extent,
                                               int row0) {
-  // MN-major operand: boxes of 128 bytes (ELEMS MN-elements) x ELEMS K-rows, one per chunk of MN
-  for (int c = 0; c < extent / ELEMS; ++c)
-    tma_load_2d(static_cast<char*>(dst) + c * ELEMS * KB_BYTES, tm, bar, tile0 + c * ELEMS, row0);
+  // MN-major operand: boxes of 128 bytes (MNC MN-elements) x KS K-rows, one per chunk of MN
+  for (int c = 0; c < extent / MNC; ++c)
+    tma_load_2d(static_cast<char*>(dst) + c * KS * KB_BYTES, tm, bar, tile0 + c * MNC, row0);
 }
 
 // n-th unit of CTA `b`; SUB strips per left-over tile
@@ -128,21 +131,22 @@ __device__ __forceinline__ Unit decode_unit(const UParams& p, int n, int b, int 
   return Unit{decode_tile(p, p.full_rounds * grid + u / SUB), (u % SUB) * NC, NC};
 }
 
-template <bool TF32, int STAGES, int R>
+template <bool TF32, int STAGES, int R, int KS>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UParams p) {
-  using L = USmem<TF32, STAGES, R>;
+  using L = USmem<TF32, STAGES, R, KS>;
   constexpr int EB = TF32 ? 4 : 2;
-  constexpr int ELEMS = KB_BYTES / EB;          // K elements per stage
+  constexpr int MNC = KB_BYTES / EB;            // MN elements per operand chunk (one 128-byte row)
   constexpr int MMA_K = 32 / EB;
-  constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
+  constexpr int CHUNK_BYTES = KS * KB_BYTES;
+  static_assert(KS % MMA_K == 0 && KS % 8 == 0, "whole MMAs and swizzle periods per stage");
   constexpr uint32_t IDESC = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN);
   constexpr int SUB = TF32 ? 4 : 2;             // column strips per left-over tile (one operand chunk each)
   constexpr int NCS = 4 / SUB;                  // 32-column blocks per strip
   constexpr uint32_t IDESC_STRIP = make_idesc(TF32 ? 2u : 1u, true, true, BM, BN / SUB);
   constexpr uint32_t SW = TF32 ? kSwizzle128B_32B : kSwizzle128B;
   constexpr uint32_t SBO = TF32 ? 512 : 1024;
-  constexpr int kABytes = BM * KB_BYTES;
+  constexpr int kABytes = BM * KS * EB;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -159,7 +163,7 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(lo_empty + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_kb = p.K / ELEMS;
+  const int num_kb = p.K / KS;
   const int bx = blockIdx.x, grid = gridDim.x;
   const int my_strips = bx < p.tail_units ? (p.tail_units - 1 - bx) / grid + 1 : 0;
   const int my_units = p.full_rounds + my_strips;
@@ -202,11 +206,11 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1)) { atomicExch(p.err_flag, 11); ok = false; break; }
-          mbar_expect_tx(&full[s], kABytes + un.nc * 32 * KB_BYTES);
+          mbar_expect_tx(&full[s], kABytes + un.nc * 32 * KS * EB);
           uint8_t* sa = stage_base + s * L::kStageBytes;
           uint8_t* sb = sa + kABytes;
-          issue_mn_tile<ELEMS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * ELEMS);
-          issue_mn_tile<ELEMS>(sb, tmB, &full[s], tl.n0 + un.c0 * 32, un.nc * 32, b_row + kb * ELEMS);
+          issue_mn_tile<MNC, KS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * KS);
+          issue_mn_tile<MNC, KS>(sb, tmB, &full[s], tl.n0 + un.c0 * 32, un.nc * 32, b_row + kb * KS);
         }
       }
     }
@@ -246,7 +250,7 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
           const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
           const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
-          for (int k = 0; k < ELEMS / MMA_K; ++k) {
+          for (int k = 0; k < KS / MMA_K; ++k) {
             const uint32_t adv = k * MMA_K * KB_BYTES;      // next MMA_K K-rows
             const uint64_t da = make_smem_desc(a_addr + adv, CHUNK_BYTES, SBO, SW);
             const uint64_t db = make_smem_desc(b_addr + adv, CHUNK_BYTES, SBO, SW);
@@ -387,10 +391,10 @@ int num_sms() {
   return sms;
 }
 
-template <bool TF32, int STAGES, int R>
+template <bool TF32, int STAGES, int R, int KS>
 int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
-  using L = USmem<TF32, STAGES, R>;
-  auto kern = tc_update_kernel<TF32, STAGES, R>;
+  using L = USmem<TF32, STAGES, R, KS>;
+  auto kern = tc_update_kernel<TF32, STAGES, R, KS>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
@@ -435,13 +439,14 @@ bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
 }
 
 int tc_update_max_layers() { return kMaxLayers; }
+int tc_update_box_rows(bool fp32) { return fp32 ? kRowsFp32 : kRowsBf16; }
 
 // layers[0..n): same batch, replica count, rates and element type; the largest layer should come first
 int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   if (launches) ++*launches;
-  if (layers[0].fp32) return launch_update<true, 2, 4>(layers, n, st);
-  return launch_update<false, 1, 6>(layers, n, st);
+  if (layers[0].fp32) return launch_update<true, 5, 4, kRowsFp32>(layers, n, st);
+  return launch_update<false, 1, 6, kRowsBf16>(layers, n, st);
 }
 
 }  // namespace ls
