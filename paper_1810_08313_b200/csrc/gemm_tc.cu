@@ -98,24 +98,28 @@ struct Smem {
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
 
+__device__ __forceinline__ int operand_row_base(const Operand& op, int g) {
+  return op.rank3 ? 0 : (int)(op.row_off ? op.row_off[g] : (int64_t)g * op.rows_per_group);
+}
 // Bring one operand tile of `tile_extent` MN-rows x ELEMS K-elements into shared memory as boxes of
 // 128 bytes x ELEMS rows.  K-major: box rows are MN-rows, inner coordinate k0.  MN-major: box rows are
 // K-rows, inner coordinate is the tile start; chunks of ELEMS MN-elements follow each other.
+// row_base = operand_row_base(op, g), read once by the caller (for dataset rows it is a global load).
 template <int ELEMS>
 __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, const Operand& op, int g,
-                                           bool mn_major, int tile0, int tile_extent, int k0) {
+                                           int row_base, bool mn_major, int tile0, int tile_extent, int k0,
+                                           uint64_t pol) {
   // rows per box: a K-major box always holds 64 MN-rows, an MN-major box holds ELEMS K-rows
   const int box_rows = mn_major ? ELEMS : 64;
   const int kChunkBytes = box_rows * KB_BYTES;
-  const int row_base = op.rank3 ? 0 : (int)(op.row_off ? op.row_off[g] : (int64_t)g * op.rows_per_group);
   const int z = op.z0 + g * op.z_step;
   const int n_boxes = mn_major ? tile_extent / ELEMS : tile_extent / 64;
   for (int c = 0; c < n_boxes; ++c) {
     char* d = static_cast<char*>(dst) + c * kChunkBytes;
     const int x = mn_major ? tile0 + c * ELEMS : k0;
     const int y = mn_major ? k0 : tile0 + c * 64;
-    if (op.rank3) tma_load_3d(d, tm, bar, x, y, z);
-    else tma_load_2d(d, tm, bar, x, row_base + y);
+    if (op.rank3) tma_load_3d_hint(d, tm, bar, x, y, z, pol);
+    else tma_load_2d_hint(d, tm, bar, x, row_base + y, pol);
   }
 }
 
@@ -248,6 +252,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == 0) {
     if (elect_one()) {
+      // the A tile (activations, gradients) is re-read by every CTA of its replica, the weight tile by nobody:
+      // L2 keeps the former and lets the latter go first
+      const uint64_t pol_a = l2_policy(2), pol_b = l2_policy(EPI == EPI_DW ? 2 : 1);
+      const int a_base = operand_row_base(p.a, g), b_base = operand_row_base(p.b, g);
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { atomicExch(p.err_flag, 1); break; }
@@ -255,8 +263,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t* sa = stage_base + s * L::kStageBytes;
         uint8_t* sb = sa + L::kABytes;
         const int k0 = (kb0 + kb) * ELEMS;
-        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, A_MN, m0, BM * MT, k0);
-        issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, B_MN, n0, BN, k0);
+        issue_tile<ELEMS>(sa, &tmA, &full[s], p.a, g, a_base, A_MN, m0, BM * MT, k0, pol_a);
+        issue_tile<ELEMS>(sb, &tmB, &full[s], p.b, g, b_base, B_MN, n0, BN, k0, pol_b);
       }
     }
   } else if (TF32 && warp >= 6) {

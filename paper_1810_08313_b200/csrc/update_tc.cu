@@ -116,10 +116,10 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
 
 template <int MNC, int KS>
 __device__ __forceinline__ void issue_mn_tile(void* dst, const CUtensorMap* tm, uint64_t* bar, int tile0, int extent,
-                                              int row0) {
+                                              int row0, uint64_t pol) {
   // MN-major operand: boxes of 128 bytes (MNC MN-elements) x KS K-rows, one per chunk of MN
   for (int c = 0; c < extent / MNC; ++c)
-    tma_load_2d(static_cast<char*>(dst) + c * KS * KB_BYTES, tm, bar, tile0 + c * MNC, row0);
+    tma_load_2d_hint(static_cast<char*>(dst) + c * KS * KB_BYTES, tm, bar, tile0 + c * MNC, row0, pol);
 }
 
 // n-th unit of CTA `b`; SUB strips per left-over tile
@@ -195,6 +195,9 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
     if (elect_one()) {
       int it = 0;
       bool ok = true;
+      // dZ and the layer inputs are re-read by every CTA that shares a row or column of tiles, while the
+      // W / v stream passes through L2 once: keep the operands (measured: 802 -> 782 us on the bf16 MLP)
+      const uint64_t pol = l2_policy(2);
       for (int n = 0; n < my_units && ok; ++n) {
         const Unit un = decode_unit<SUB>(p, n, bx, grid);
         const Tile tl = un.tl;
@@ -209,8 +212,8 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
           mbar_expect_tx(&full[s], kABytes + un.nc * 32 * KS * EB);
           uint8_t* sa = stage_base + s * L::kStageBytes;
           uint8_t* sb = sa + kABytes;
-          issue_mn_tile<MNC, KS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * KS);
-          issue_mn_tile<MNC, KS>(sb, tmB, &full[s], tl.n0 + un.c0 * 32, un.nc * 32, b_row + kb * KS);
+          issue_mn_tile<MNC, KS>(sa, tmA, &full[s], tl.m0, BM, a_row + kb * KS, pol);
+          issue_mn_tile<MNC, KS>(sb, tmB, &full[s], tl.n0 + un.c0 * 32, un.nc * 32, b_row + kb * KS, pol);
         }
       }
     }
