@@ -652,6 +652,216 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// ---- bf16 forward / backward on CTA pairs ----------------------------------------------------------
+// A 256 x 512 output tile per cluster of two CTAs (cta_group::2).  Every tcgen05.mma spans both SMs: a CTA
+// supplies its 128 rows of A and its half (128 of 256 columns) of each of the two B blocks, and keeps its 128
+// rows x 512 columns of the product in its own tensor memory.  Per stage a CTA brings in 48 KB (16 KB of A,
+// 32 KB of B) for 128 x 512 x 64 products, against 64 KB for the same work on one CTA, and the tensor core
+// reads each B element from shared memory once per pair instead of once per row block: the single-CTA kernel
+// is bound by shared-memory bandwidth (TMA writes + operand reads), this one is not.
+//   warp 0   TMA producer (each CTA loads its own parts; completion is counted on the leader's barrier)
+//   warp 1   leader CTA: issues the MMAs; commits arrive on the barriers of both CTAs
+//   warps 2-5 epilogue of this CTA's 128 rows (same arithmetic as tc_gemm_kernel)
+constexpr int kPairStages = 4;
+constexpr int kPairN = 512;          // columns of the pair's tile: two MMA blocks of 256
+struct SmemPair {
+  static constexpr int kABytes = BM * KB_BYTES;                 // this CTA's 128 rows
+  static constexpr int kBBlockBytes = 128 * KB_BYTES;           // this CTA's half of one 256-column block
+  static constexpr int kStageBytes = kABytes + 2 * kBBlockBytes;
+  static constexpr int kRingBytes = kPairStages * kStageBytes;
+  static constexpr int kBarBytes = (2 * kPairStages + 1) * 8 + 16;
+  static constexpr int kTotal = 1024 + kRingBytes + kBarBytes;
+  static_assert((4 * 32 * 33 + 4 * kPairN) * 4 <= kRingBytes, "epilogue scratch");
+  static_assert(kTotal <= 227 * 1024, "shared memory budget");
+};
+
+template <bool B_MN, int EPI>
+__global__ void __launch_bounds__(kThreadsBf16, 1)
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+  using L = SmemPair;
+  constexpr int ELEMS = 64, MMA_K = 16, STAGES = kPairStages;
+  constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
+  constexpr uint32_t IDESC = make_idesc(1u, false, B_MN, 256, 256);
+  constexpr uint32_t TMEM_COLS = kPairN;
+  static_assert(EPI == EPI_FWD || EPI == EPI_DX, "forward / backward only");
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem;
+  float* staging = reinterpret_cast<float*>(smem);            // [4][32 x 33] transposes (backward epilogue)
+  float* colsum = staging + 4 * 32 * 33;                      // [4][kPairN] column sums of this CTA's rows
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kRingBytes);
+  uint64_t* empty = full + STAGES;
+  uint64_t* acc_full = empty + STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();                    // 0: leader
+  const int g = blockIdx.z;
+  const int m0 = blockIdx.y * 256 + rank * BM;                // first row of this CTA
+  const int n0 = (int)(blockIdx.x >> 1) * kPairN;             // first column of the pair
+  const int num_kb = p.K / ELEMS;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    fence_mbar_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  cluster_sync_all();       // both CTAs' barriers exist before either signals the other
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
+
+  if (warp == 0) {
+    if (elect_one()) {
+      const uint64_t pol_a = l2_policy(2), pol_b = l2_policy(1);
+      const int a_base = operand_row_base(p.a, g);
+      const int zb = p.b.z0 + g * p.b.z_step;
+      const uint32_t full_leader = map_to_rank(smem_u32(&full[0]), 0);
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { atomicExch(p.err_flag, 21); break; }
+        if (rank == 0) mbar_expect_tx(&full[s], 2 * L::kStageBytes);      // both CTAs' bytes
+        const uint32_t bar = full_leader + (uint32_t)(s * 8);
+        uint8_t* sa = stage_base + s * L::kStageBytes;
+        uint8_t* sb = sa + L::kABytes;
+        const int k0 = kb * ELEMS;
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+          tma_load_2d_pair(sa + c * CHUNK_BYTES, &tmA, bar, k0, a_base + m0 + c * 64, pol_a);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int nb = n0 + j * 256 + rank * 128;       // this CTA's 128 columns of block j
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            uint8_t* d = sb + j * L::kBBlockBytes + c * CHUNK_BYTES;
+            if (B_MN) tma_load_3d_pair(d, &tmB, bar, nb + c * 64, k0, zb, pol_b);
+            else tma_load_3d_pair(d, &tmB, bar, k0, nb + c * 64, zb, pol_b);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && elect_one()) {
+      bool ok = true;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { atomicExch(p.err_flag, 22); ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
+        const uint32_t b_addr = a_addr + L::kABytes;
+#pragma unroll
+        for (int k = 0; k < ELEMS / MMA_K; ++k) {
+          const uint32_t b_adv = B_MN ? k * MMA_K * KB_BYTES : k * 32;
+          const uint32_t b_lbo = B_MN ? CHUNK_BYTES : 16;
+          const uint64_t da = make_smem_desc(a_addr + k * 32, 16, 1024, kSwizzle128B);
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint64_t db = make_smem_desc(b_addr + j * L::kBBlockBytes + b_adv, b_lbo, 1024, kSwizzle128B);
+            mma_bf16_pair(tmem_base + (uint32_t)(j * 256), da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+          }
+        }
+        mma_commit_pair(&empty[s]);
+      }
+      if (ok) mma_commit_pair(acc_full);
+    }
+  } else {
+    // ---- epilogue of this CTA's 128 rows x 512 columns ------------------------------------------
+    const int q = warp & 3;
+    const int row = m0 + q * 32 + lane;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    bool ok = mbar_wait(acc_full, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after_sync();
+    if (!ok && lane == 0) atomicExch(p.err_flag, 23);
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < kPairN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + c * 32, r);
+        tmem_ld_wait();
+        const int col = n0 + c * 32;
+        const int64_t at = ((int64_t)g * p.M + row) * p.N + col;
+        float o[32];
+        if (EPI == EPI_FWD) {
+          const float* bias = p.bias ? p.bias + (int64_t)g * p.bias_gstride + col : nullptr;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float v = __uint_as_float(r[i]);
+            if (bias) v += __ldg(bias + i);
+            o[i] = (p.relu && !(v > 0.f)) ? 0.f : v;
+          }
+          store_row32<false>(p.C, at, o);
+        } else {
+          const uint4* a4 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) + at);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 u = a4[i];
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
+              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2]) : 0.f;
+              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2 + 1]) : 0.f;
+            }
+          }
+          store_row32<false>(p.C, at, o);
+          if (p.dbias != nullptr) {
+            float* tile = staging + q * (32 * 33);
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = o[i];
+            __syncwarp();
+            float cs = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < 32; ++rr) cs += tile[rr * 33 + lane];
+            colsum[q * kPairN + c * 32 + lane] = cs;
+          }
+        }
+      }
+    }
+    tc_fence_before_sync();
+  }
+  if (EPI == EPI_DX && p.dbias != nullptr) {
+    // bias update of the layer below: column sums over the pair's 256 rows, added in row order (leader's
+    // warps 0-3, then the peer's) by the CTA that owns the column half
+    cluster_sync_all();
+    if (warp >= 2) {
+      const uint32_t mine = smem_u32(colsum);
+      const uint32_t src0 = map_to_rank(mine, 0), src1 = map_to_rank(mine, 1);
+      for (int t = rank * 256 + (int)threadIdx.x - 64; t < rank * 256 + 256; t += 128) {
+        float gsum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gsum += ld_cluster_f32(src0 + (uint32_t)((i * kPairN + t) * 4));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gsum += ld_cluster_f32(src1 + (uint32_t)((i * kPairN + t) * 4));
+        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
+        float step = gsum;
+        if (p.mu != 0.f) {
+          step = fmaf(p.mu, p.dvbias[at], gsum);
+          p.dvbias[at] = step;
+        }
+        p.dbias[at] = fmaf(-p.lr, step, p.dbias[at]);
+      }
+    }
+  }
+  // neither CTA leaves (or frees tensor memory) while the other may still read its shared memory or
+  // receive an arrival from it
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 // ---- host side -----------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -683,6 +893,21 @@ int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_
   dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / (BM * MT)), (unsigned)groups);
   return launch_dep(kern, grid, dim3(TF32 ? kThreadsFp32 : kThreadsBf16), L::kTotal, st, SPLIT, *mp.a, *mp.b, p);
 }
+
+template <bool B_MN, int EPI>
+int launch_pair(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
+  auto kern = tc_gemm_pair_kernel<B_MN, EPI>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPair::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid((unsigned)(p.N / kPairN * 2), (unsigned)(p.M / 256), (unsigned)groups);
+  return launch_dep(kern, grid, dim3(kThreadsBf16), SmemPair::kTotal, st, 2, *mp.a, *mp.b, p);
+}
+// bf16 shapes that the pair kernel covers
+bool pair_shape_ok(int M, int N, int K) { return M % 256 == 0 && N % kPairN == 0 && K % 64 == 0; }
 
 // fp32 forward / backward: tile width and K split.  128-wide tiles when N allows; K is split over a
 // cluster while that keeps the grid within one wave of SMs and every slice keeps whole stages.
@@ -784,6 +1009,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   if (p.head.W != nullptr && !tc_fwd_fuses_head(a.fp32, a.M, a.N, p.head.C)) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
+  if (p.head.W == nullptr && pair_shape_ok(a.M, a.N, a.K)) return launch_pair<false, EPI_FWD>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
@@ -800,6 +1026,7 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   }
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
+  if (pair_shape_ok(a.M, a.N, a.K)) return launch_pair<true, EPI_DX>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);

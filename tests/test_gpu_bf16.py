@@ -38,6 +38,7 @@ def _run_pair(dims, m, B, tau, K, n_rows, seed, mu=0.9, lr=0.05):
     ((256, 256, 128, 10), 2, 128),          # every hidden layer fills tensor-core tiles
     ((200, 136, 72, 10), 3, 48),            # nothing does: CUDA-core kernels with bf16 operands
     ((384, 256, 256, 256, 10), 4, 256),     # the bf16 workload's depth and batch at reduced width
+    ((384, 512, 512, 10), 3, 256),          # 512-wide layers, batch 256: forward / backward on CTA pairs
 ])
 def test_loss_trajectory_three_periods(dims, m, B):
     tau, K = 4, 12
@@ -110,7 +111,9 @@ def test_tensor_core_update_kernel_tight():
 
 
 @pytest.mark.parametrize("dims,m,B", [((256, 256, 128, 10), 2, 128), ((384, 256, 256, 256, 10), 3, 256),
-                                      ((256, 128, 128), 2, 128)])
+                                      ((256, 128, 128), 2, 128),
+                                      ((384, 512, 1024, 10), 3, 256),      # CTA pairs, two and four column tiles
+                                      ((256, 512, 512, 10), 2, 512)])      # CTA pairs, two row tiles per replica
 def test_single_step_gradients_through_relu(dims, m, B):
     """All three tensor-core kernels in one step.  bf16 rounding flips a few ReLU masks, which moves single
     entries by O(10 %) of the largest one; the direction of every tensor's gradient is what is checked."""
