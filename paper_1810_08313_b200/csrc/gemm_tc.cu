@@ -657,27 +657,48 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // supplies its 128 rows of A and its half (128 of 256 columns) of each of the two B blocks, and keeps its 128
 // rows x 512 columns of the product in its own tensor memory.  Per stage a CTA brings in 48 KB (16 KB of A,
 // 32 KB of B) for 128 x 512 x 64 products, against 64 KB for the same work on one CTA, and the tensor core
-// reads each B element from shared memory once per pair instead of once per row block: the single-CTA kernel
-// is bound by shared-memory bandwidth (TMA writes + operand reads), this one is not.
-//   warp 0   TMA producer (each CTA loads its own parts; completion is counted on the leader's barrier)
+// reads each B element from shared memory once per pair instead of once per row block.
+//   warp 0   TMA producer (each CTA loads its own parts; completion is counted on the leader's barrier);
+//            backward: as the stages are used for the last time it also brings this CTA's 128 x 512 block of
+//            the layer's activations (the ReLU mask) into them
 //   warp 1   leader CTA: issues the MMAs; commits arrive on the barriers of both CTAs
-//   warps 2-5 epilogue of this CTA's 128 rows (same arithmetic as tc_gemm_kernel)
+//   warps 2-5 epilogue of this CTA's 128 rows: bias + ReLU (forward) or mask (backward) on the accumulator,
+//            outputs packed to bf16 into the (now idle) stage memory in the layout of a TMA box, and written
+//            with bulk tensor stores of 64 rows x 128 bytes.  (With one st.global per thread and row the
+//            epilogue took as long as half the main loop: 16-32 k cycles against 4-5 k now.)
 constexpr int kPairStages = 4;
 constexpr int kPairN = 512;          // columns of the pair's tile: two MMA blocks of 256
+constexpr int kPairGroups = kPairN / 64;      // 64-column groups of the epilogue (one 128-byte box row each)
 struct SmemPair {
   static constexpr int kABytes = BM * KB_BYTES;                 // this CTA's 128 rows
   static constexpr int kBBlockBytes = 128 * KB_BYTES;           // this CTA's half of one 256-column block
   static constexpr int kStageBytes = kABytes + 2 * kBBlockBytes;
   static constexpr int kRingBytes = kPairStages * kStageBytes;
-  static constexpr int kBarBytes = (2 * kPairStages + 1) * 8 + 16;
+  static constexpr int kBoxBytes = 64 * KB_BYTES;               // epilogue: 64 rows x 64 bf16
+  static constexpr int kOutBytes = 2 * kPairGroups * kBoxBytes; // the CTA's 128 x 512 outputs (and mask) as boxes
+  static constexpr int kTransBytes = 4 * 32 * 33 * 4;           // backward: per-warp transposes for the column sums
+  static constexpr int kColsumBytes = 4 * kPairN * 4;
+  static constexpr int kBars = 2 * kPairStages + 1 + kPairGroups;
+  static constexpr int kBarBytes = kBars * 8 + 16;
   static constexpr int kTotal = 1024 + kRingBytes + kBarBytes;
-  static_assert((4 * 32 * 33 + 4 * kPairN) * 4 <= kRingBytes, "epilogue scratch");
+  static_assert(kOutBytes + kTransBytes + kColsumBytes <= kRingBytes, "epilogue scratch");
+  static_assert(kStageBytes % kBoxBytes == 0, "whole boxes per stage");
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(m)),
+               "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
+}
+
+// tmC: the output [groups*M][N] as boxes of 64 rows x 64 bf16 (128-byte swizzle); tmMask (backward): the
+// activations of the layer, same shape and boxes.
 template <bool B_MN, int EPI>
 __global__ void __launch_bounds__(kThreadsBf16, 1)
-tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmMask, const Params p) {
   using L = SmemPair;
   constexpr int ELEMS = 64, MMA_K = 16, STAGES = kPairStages;
   constexpr int CHUNK_BYTES = ELEMS * KB_BYTES;
@@ -688,26 +709,31 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  float* staging = reinterpret_cast<float*>(smem);            // [4][32 x 33] transposes (backward epilogue)
-  float* colsum = staging + 4 * 32 * 33;                      // [4][kPairN] column sums of this CTA's rows
+  float* staging = reinterpret_cast<float*>(smem + L::kOutBytes);           // [4][32 x 33]
+  float* colsum = reinterpret_cast<float*>(smem + L::kOutBytes + L::kTransBytes);   // [4][kPairN]
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kRingBytes);
   uint64_t* empty = full + STAGES;
   uint64_t* acc_full = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  uint64_t* mask_full = acc_full + 1;                           // [kPairGroups]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mask_full + kPairGroups);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();                    // 0: leader
   const int g = blockIdx.z;
-  const int m0 = blockIdx.y * 256 + rank * BM;                // first row of this CTA
+  const int m0 = blockIdx.y * 256 + rank * BM;                // first row of this CTA inside the replica
   const int n0 = (int)(blockIdx.x >> 1) * kPairN;             // first column of the pair
   const int num_kb = p.K / ELEMS;
+  const int out_row0 = g * p.M + m0;                          // first row of this CTA in the output / mask tensor
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    for (int i = 0; i < kPairGroups; ++i) mbar_init(&mask_full[i], 1);
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    prefetch_tmap(&tmC);
+    if (EPI == EPI_DX) prefetch_tmap(&tmMask);
   }
   if (warp == 1) {
     tmem_alloc_pair(tmem_slot, TMEM_COLS);
@@ -726,9 +752,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int a_base = operand_row_base(p.a, g);
       const int zb = p.b.z0 + g * p.b.z_step;
       const uint32_t full_leader = map_to_rank(smem_u32(&full[0]), 0);
+      bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
-        if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { atomicExch(p.err_flag, 21); break; }
+        if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { atomicExch(p.err_flag, 21); ok = false; break; }
         if (rank == 0) mbar_expect_tx(&full[s], 2 * L::kStageBytes);      // both CTAs' bytes
         const uint32_t bar = full_leader + (uint32_t)(s * 8);
         uint8_t* sa = stage_base + s * L::kStageBytes;
@@ -746,6 +773,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (B_MN) tma_load_3d_pair(d, &tmB, bar, nb + c * 64, k0, zb, pol_b);
             else tma_load_3d_pair(d, &tmB, bar, k0, nb + c * 64, zb, pol_b);
           }
+        }
+      }
+      if (EPI == EPI_DX && ok) {
+        // the mask: box b = (column group b / 2, row half b % 2) goes to bytes [b, b + 1) * 8 KB of the ring;
+        // a stage is overwritten once the MMAs of its last use have completed
+        for (int i = 0; i < kPairGroups; ++i) mbar_expect_tx(&mask_full[i], 2 * L::kBoxBytes);
+        constexpr int kBoxesPerStage = L::kStageBytes / L::kBoxBytes;
+        for (int i = 0; i < STAGES && ok; ++i) {
+          const int s = (num_kb + i) % STAGES;                       // in the order of their last use
+          const int uses = (num_kb - s + STAGES - 1) / STAGES;
+          if (uses > 0 && !mbar_wait(&empty[s], (uses - 1) & 1)) { atomicExch(p.err_flag, 24); ok = false; break; }
+          for (int b = s * kBoxesPerStage; b < (s + 1) * kBoxesPerStage && b < 2 * kPairGroups; ++b)
+            tma_load_2d(smem + b * L::kBoxBytes, &tmMask, &mask_full[b >> 1], n0 + (b >> 1) * 64,
+                        out_row0 + (b & 1) * 64);
         }
       }
     }
@@ -775,8 +816,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else {
     // ---- epilogue of this CTA's 128 rows x 512 columns ------------------------------------------
-    const int q = warp & 3;
-    const int row = m0 + q * 32 + lane;
+    const int q = warp & 3;                  // TMEM lanes 32 q .. 32 q + 31
+    const int half = q >> 1;                 // rows 64 half .. of the CTA: one TMA box with the other warp of the half
+    const int rih = (q & 1) * 32 + lane;     // this thread's row inside the box
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     bool ok = mbar_wait(acc_full, 0);
     ok = __all_sync(0xffffffffu, ok);
@@ -785,49 +827,83 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (ok) {
 #pragma unroll 1
       for (int c = 0; c < kPairN / 32; ++c) {
+        const int grp = c >> 1, sub = c & 1;
+        uint8_t* box = smem + (grp * 2 + half) * L::kBoxBytes;
+        uint8_t* myrow = box + rih * 128;
         uint32_t r[32];
         tmem_ld_32x32(taddr + c * 32, r);
+        if (EPI == EPI_DX && sub == 0 && ok) {
+          // (after a failed wait the loop goes on without the mask, so that every barrier below is still met)
+          ok = __all_sync(0xffffffffu, mbar_wait(&mask_full[grp], 0));
+          if (!ok && lane == 0) atomicExch(p.err_flag, 25);
+        }
         tmem_ld_wait();
         const int col = n0 + c * 32;
-        const int64_t at = ((int64_t)g * p.M + row) * p.N + col;
         float o[32];
         if (EPI == EPI_FWD) {
-          const float* bias = p.bias ? p.bias + (int64_t)g * p.bias_gstride + col : nullptr;
+          const float4* bias4 = p.bias ? reinterpret_cast<const float4*>(p.bias + (int64_t)g * p.bias_gstride + col) : nullptr;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float v = __uint_as_float(r[i]);
-            if (bias) v += __ldg(bias + i);
-            o[i] = (p.relu && !(v > 0.f)) ? 0.f : v;
+          for (int i = 0; i < 8; ++i) {
+            float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (bias4) bv = __ldg(bias4 + i);
+            const float b4[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float v = __uint_as_float(r[4 * i + e]) + b4[e];
+              o[4 * i + e] = (p.relu && !(v > 0.f)) ? 0.f : v;
+            }
           }
-          store_row32<false>(p.C, at, o);
         } else {
-          const uint4* a4 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) + at);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const uint4 u = a4[i];
+            const uint4 u = *reinterpret_cast<const uint4*>(myrow + (((sub * 4 + i) ^ (rih & 7)) << 4));
             const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
+              // a bf16 is positive iff it is non-zero with the sign bit clear
               const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
               o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2]) : 0.f;
               o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2 + 1]) : 0.f;
             }
           }
-          store_row32<false>(p.C, at, o);
-          if (p.dbias != nullptr) {
-            float* tile = staging + q * (32 * 33);
-            __syncwarp();
+        }
+        // 32 outputs = four 16-byte pieces of this thread's box row (pieces are XOR-swizzled by the row)
 #pragma unroll
-            for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = o[i];
-            __syncwarp();
-            float cs = 0.f;
+        for (int i = 0; i < 4; ++i) {
+          uint32_t u[4];
 #pragma unroll
-            for (int rr = 0; rr < 32; ++rr) cs += tile[rr * 33 + lane];
-            colsum[q * kPairN + c * 32 + lane] = cs;
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(o[8 * i + 2 * e], o[8 * i + 2 * e + 1]);
+            u[e] = *reinterpret_cast<uint32_t*>(&t);
+          }
+          *reinterpret_cast<uint4*>(myrow + (((sub * 4 + i) ^ (rih & 7)) << 4)) = make_uint4(u[0], u[1], u[2], u[3]);
+        }
+        if (EPI == EPI_DX && p.dbias != nullptr) {
+          // column sums over this warp's 32 rows (of the values as stored would differ in the last bit: the
+          // sums use the unrounded gradients, like the single-CTA kernel)
+          float* tile = staging + q * (32 * 33);
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = o[i];
+          __syncwarp();
+          float cs = 0.f;
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr) cs += tile[rr * 33 + lane];
+          colsum[q * kPairN + c * 32 + lane] = cs;
+        }
+        if (sub == 1) {
+          // both warps of the half have written the box: hand it to the bulk-copy engine
+          fence_proxy_async_smem();
+          if (half == 0) asm volatile("bar.sync 2, 64;" ::: "memory");
+          else asm volatile("bar.sync 3, 64;" ::: "memory");
+          if ((q & 1) == 0 && lane == 0) {
+            tma_store_2d(&tmC, box, n0 + grp * 64, out_row0 + half * 64);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
         }
       }
     }
+    if ((q & 1) == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before_sync();
   }
   if (EPI == EPI_DX && p.dbias != nullptr) {
@@ -895,7 +971,8 @@ int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_
 }
 
 template <bool B_MN, int EPI>
-int launch_pair(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
+int launch_pair(const TcOperandMaps& mp, const CUtensorMap* c_map, const CUtensorMap* mask_map, const Params& p,
+                int groups, cudaStream_t st) {
   auto kern = tc_gemm_pair_kernel<B_MN, EPI>;
   static bool configured = false;
   if (!configured) {
@@ -904,7 +981,8 @@ int launch_pair(const TcOperandMaps& mp, const Params& p, int groups, cudaStream
     configured = true;
   }
   dim3 grid((unsigned)(p.N / kPairN * 2), (unsigned)(p.M / 256), (unsigned)groups);
-  return launch_dep(kern, grid, dim3(kThreadsBf16), SmemPair::kTotal, st, 2, *mp.a, *mp.b, p);
+  return launch_dep(kern, grid, dim3(kThreadsBf16), SmemPair::kTotal, st, 2, *mp.a, *mp.b, *c_map,
+                    mask_map ? *mask_map : *c_map, p);
 }
 // bf16 shapes that the pair kernel covers
 bool pair_shape_ok(int M, int N, int K) { return M % 256 == 0 && N % kPairN == 0 && K % 64 == 0; }
@@ -1009,7 +1087,8 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   if (p.head.W != nullptr && !tc_fwd_fuses_head(a.fp32, a.M, a.N, p.head.C)) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
-  if (p.head.W == nullptr && pair_shape_ok(a.M, a.N, a.K)) return launch_pair<false, EPI_FWD>(a.maps, p, a.groups, st);
+  if (p.head.W == nullptr && a.c_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
+    return launch_pair<false, EPI_FWD>(a.maps, a.c_map, nullptr, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
@@ -1026,7 +1105,8 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   }
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
-  if (pair_shape_ok(a.M, a.N, a.K)) return launch_pair<true, EPI_DX>(a.maps, p, a.groups, st);
+  if (a.c_map != nullptr && a.act_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
+    return launch_pair<true, EPI_DX>(a.maps, a.c_map, a.act_map, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);
   return launch_one<false, 128, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);

@@ -179,6 +179,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
       t.bias_gstride = w_gstride;
       t.C = h->state + lay.act_off[l + 1];
+      t.c_map = (bf && lay.dims[l + 1] % 8 == 0) ? &h->maps.act[l + 1] : nullptr;
       t.M = lay.batch; t.N = lay.dims[l + 1]; t.K = lay.dims[l]; t.groups = groups; t.relu = 1;
       t.err_flag = err_flag_of(h);
       t.head = TcHead{};
@@ -272,6 +273,8 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.maps.b = &mn.w[l];
       t.act = h->state + lay.act_off[l];
       t.C = h->state + lay.dz_off[l - 1];
+      t.c_map = (bf && lay.dims[l] % 8 == 0) ? &h->maps.dz[l - 1] : nullptr;
+      t.act_map = (bf && lay.dims[l] % 8 == 0) ? &h->maps.act[l] : nullptr;
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
       t.bias = nullptr; t.vbias = nullptr; t.bias_gstride = lay.stride; t.lr = h->lr; t.mu = h->mu;
       if (lay.has_bias && tc_dx_fuses_bias(!bf, t.M, t.N)) {

@@ -282,6 +282,7 @@ struct TcFwdArgs {
   int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
   const float* bias; int64_t bias_gstride;
   void* C;                   // [groups][M][N] bf16 or fp32
+  const CUtensorMap* c_map;  // bf16: C as a 2-D tensor [groups*M][N], boxes of 64 x 64 (pair kernel's stores), or null
   TcHead head;
   int M, N, K, groups, relu;
   int* err_flag;
@@ -290,6 +291,8 @@ struct TcDxArgs {
   TcOperandMaps maps;        // a: dZ_l [groups*M][K]; b: weights
   bool fp32;
   const void* act; void* C;
+  const CUtensorMap* c_map;   // bf16: C and act as 2-D tensors [groups*M][N], boxes of 64 x 64, or null
+  const CUtensorMap* act_map;
   int M, N, K, groups;
   // bias / its momentum of the layer that produced `act` (group 0; replica stride bias_gstride): updated
   // from the column sums of C inside the kernel when tc_dx_fuses_bias(); else null
