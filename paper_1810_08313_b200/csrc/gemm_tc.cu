@@ -679,8 +679,10 @@ struct SmemPair {
   static constexpr int kTransBytes = 4 * 32 * 33 * 4;           // backward: per-warp transposes for the column sums
   static constexpr int kColsumBytes = 4 * kPairN * 4;
   static constexpr int kBars = 2 * kPairStages + 1 + kPairGroups;
-  static constexpr int kBarBytes = kBars * 8 + 16;
-  static constexpr int kTotal = 1024 + kRingBytes + kBarBytes;
+  static constexpr int kBarBytes = (kBars * 8 + 16 + 15) / 16 * 16;
+  static constexpr int kBiasBytes = kPairN * 4;                 // forward: the bias of the tile's columns
+  static constexpr int kTotal = 1024 + kRingBytes + kBarBytes + kBiasBytes;
+  static_assert(kBarBytes % 16 == 0, "bias block alignment");
   static_assert(kOutBytes + kTransBytes + kColsumBytes <= kRingBytes, "epilogue scratch");
   static_assert(kStageBytes % kBoxBytes == 0, "whole boxes per stage");
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
@@ -716,6 +718,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* acc_full = empty + STAGES;
   uint64_t* mask_full = acc_full + 1;                           // [kPairGroups]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mask_full + kPairGroups);
+  float* bias_s = reinterpret_cast<float*>(smem + L::kRingBytes + L::kBarBytes);   // [kPairN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();                    // 0: leader
@@ -746,6 +749,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   grid_dep_wait();
   grid_dep_launch();
 
+  float dx_pb[2] = {0.f, 0.f}, dx_pvb[2] = {0.f, 0.f};   // backward: bias / momentum elements this thread updates
   if (warp == 0) {
     if (elect_one()) {
       const uint64_t pol_a = l2_policy(2), pol_b = l2_policy(1);
@@ -819,37 +823,53 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int q = warp & 3;                  // TMEM lanes 32 q .. 32 q + 31
     const int half = q >> 1;                 // rows 64 half .. of the CTA: one TMA box with the other warp of the half
     const int rih = (q & 1) * 32 + lane;     // this thread's row inside the box
+    const int et = (int)threadIdx.x - 64;    // 0..127 among the epilogue threads
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    // while the products run: the bias of the tile's columns goes to shared memory (forward), and the bias
+    // elements that this thread will update are requested (backward)
+    if (EPI == EPI_FWD) {
+      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + (int64_t)g * p.bias_gstride + n0) + et);
+      reinterpret_cast<float4*>(bias_s)[et] = bv;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    } else if (p.dbias != nullptr) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + rank * 256 + et + i * 128;
+        dx_pb[i] = p.dbias[at];
+        if (p.mu != 0.f) dx_pvb[i] = p.dvbias[at];
+      }
+    }
     bool ok = mbar_wait(acc_full, 0);
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after_sync();
     if (!ok && lane == 0) atomicExch(p.err_flag, 23);
     if (ok) {
-#pragma unroll 1
+      // the accumulator is read one 32-column block ahead of the arithmetic
+      uint32_t r[2][32];
+      tmem_ld_32x32(taddr, r[0]);
+#pragma unroll
       for (int c = 0; c < kPairN / 32; ++c) {
         const int grp = c >> 1, sub = c & 1;
         uint8_t* box = smem + (grp * 2 + half) * L::kBoxBytes;
         uint8_t* myrow = box + rih * 128;
-        uint32_t r[32];
-        tmem_ld_32x32(taddr + c * 32, r);
+        tmem_ld_wait();
+        if (c + 1 < kPairN / 32) tmem_ld_32x32(taddr + (c + 1) * 32, r[(c + 1) & 1]);
         if (EPI == EPI_DX && sub == 0 && ok) {
           // (after a failed wait the loop goes on without the mask, so that every barrier below is still met)
           ok = __all_sync(0xffffffffu, mbar_wait(&mask_full[grp], 0));
           if (!ok && lane == 0) atomicExch(p.err_flag, 25);
         }
-        tmem_ld_wait();
-        const int col = n0 + c * 32;
         float o[32];
         if (EPI == EPI_FWD) {
-          const float4* bias4 = p.bias ? reinterpret_cast<const float4*>(p.bias + (int64_t)g * p.bias_gstride + col) : nullptr;
+          const float4* bias4 = reinterpret_cast<const float4*>(bias_s + c * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (bias4) bv = __ldg(bias4 + i);
+            const float4 bv = bias4[i];
             const float b4[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float v = __uint_as_float(r[4 * i + e]) + b4[e];
+              const float v = __uint_as_float(r[c & 1][4 * i + e]) + b4[e];
               o[4 * i + e] = (p.relu && !(v > 0.f)) ? 0.f : v;
             }
           }
@@ -862,8 +882,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int j = 0; j < 4; ++j) {
               // a bf16 is positive iff it is non-zero with the sign bit clear
               const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
-              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2]) : 0.f;
-              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[i * 8 + j * 2 + 1]) : 0.f;
+              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[c & 1][i * 8 + j * 2]) : 0.f;
+              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[c & 1][i * 8 + j * 2 + 1]) : 0.f;
             }
           }
         }
@@ -879,8 +899,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           *reinterpret_cast<uint4*>(myrow + (((sub * 4 + i) ^ (rih & 7)) << 4)) = make_uint4(u[0], u[1], u[2], u[3]);
         }
         if (EPI == EPI_DX && p.dbias != nullptr) {
-          // column sums over this warp's 32 rows (of the values as stored would differ in the last bit: the
-          // sums use the unrounded gradients, like the single-CTA kernel)
+          // column sums over this warp's 32 rows, of the unrounded gradients like the single-CTA kernel
           float* tile = staging + q * (32 * 33);
           __syncwarp();
 #pragma unroll
@@ -913,7 +932,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp >= 2) {
       const uint32_t mine = smem_u32(colsum);
       const uint32_t src0 = map_to_rank(mine, 0), src1 = map_to_rank(mine, 1);
-      for (int t = rank * 256 + (int)threadIdx.x - 64; t < rank * 256 + 256; t += 128) {
+#pragma unroll
+      for (int i2 = 0; i2 < 2; ++i2) {
+        const int t = rank * 256 + (int)threadIdx.x - 64 + i2 * 128;
         float gsum = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) gsum += ld_cluster_f32(src0 + (uint32_t)((i * kPairN + t) * 4));
@@ -922,10 +943,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
         float step = gsum;
         if (p.mu != 0.f) {
-          step = fmaf(p.mu, p.dvbias[at], gsum);
+          step = fmaf(p.mu, dx_pvb[i2], gsum);
           p.dvbias[at] = step;
         }
-        p.dbias[at] = fmaf(-p.lr, step, p.dbias[at]);
+        p.dbias[at] = fmaf(-p.lr, step, dx_pb[i2]);
       }
     }
   }
