@@ -39,7 +39,10 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&r)[4]) {
 
 // One CTA = kRowsPerCta (4) mini-batch rows of one replica.  The 8 warps split K; partial dot products are
 // combined lane-wise by a butterfly and warp-wise through shared memory in warp order.
-template <typename TA>
+// CT: the number of outputs when it is known at compile time (10 classes, 1 regression output), else 0.  With
+// a run-time count the class loops need an early exit, and a load behind a branch cannot be issued before
+// the branch: the loads of the classes then go out one round trip at a time.
+template <typename TA, int CT>
 __global__ void __launch_bounds__(kThreads, 2)
 head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ W,
                 int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
@@ -72,11 +75,12 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     else target = static_cast<const float*>(y)[y0 + b0 + warp];
   }
 
-  float acc[kRowsPerCta][CMAX];
+  constexpr int CU = CT > 0 ? CT : CMAX;      // unrolled class count
+  float acc[kRowsPerCta][CU];
 #pragma unroll
   for (int r = 0; r < kRowsPerCta; ++r)
 #pragma unroll
-    for (int c = 0; c < CMAX; ++c) acc[r][c] = 0.f;
+    for (int c = 0; c < CU; ++c) acc[r][c] = 0.f;
   if (vec_ok) {
     for (int k = kw0 + lane * 4; k < kw1; k += 128) {
       float a[kRowsPerCta][4];
@@ -85,14 +89,26 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
         if (b0 + r < B) load4(Ag + (int64_t)(b0 + r) * K + k, a[r]);
         else a[r][0] = a[r][1] = a[r][2] = a[r][3] = 0.f;
       }
+      if (CT > 0) {
+        // every class's weights are requested before the first product
+        float w[CU][4];
 #pragma unroll
-      for (int c = 0; c < CMAX; ++c) {
-        if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
-        float w[4];
-        load4(Wg + (int64_t)c * K + k, w);
+        for (int c = 0; c < CU; ++c) load4(Wg + (int64_t)c * K + k, w[c]);
 #pragma unroll
-        for (int r = 0; r < kRowsPerCta; ++r)
-          acc[r][c] = fmaf(a[r][3], w[3], fmaf(a[r][2], w[2], fmaf(a[r][1], w[1], fmaf(a[r][0], w[0], acc[r][c]))));
+        for (int c = 0; c < CU; ++c)
+#pragma unroll
+          for (int r = 0; r < kRowsPerCta; ++r)
+            acc[r][c] = fmaf(a[r][3], w[c][3], fmaf(a[r][2], w[c][2], fmaf(a[r][1], w[c][1], fmaf(a[r][0], w[c][0], acc[r][c]))));
+      } else {
+#pragma unroll
+        for (int c = 0; c < CU; ++c) {
+          if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
+          float w[4];
+          load4(Wg + (int64_t)c * K + k, w);
+#pragma unroll
+          for (int r = 0; r < kRowsPerCta; ++r)
+            acc[r][c] = fmaf(a[r][3], w[3], fmaf(a[r][2], w[2], fmaf(a[r][1], w[1], fmaf(a[r][0], w[0], acc[r][c]))));
+        }
       }
     }
   } else {
@@ -101,7 +117,7 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 #pragma unroll
       for (int r = 0; r < kRowsPerCta; ++r) a[r] = (b0 + r < B) ? to_f(Ag[(int64_t)(b0 + r) * K + k]) : 0.f;
 #pragma unroll
-      for (int c = 0; c < CMAX; ++c)
+      for (int c = 0; c < CU; ++c)
         if (c < C) {
           const float w = Wg[(int64_t)c * K + k];
 #pragma unroll
@@ -112,7 +128,7 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 #pragma unroll
   for (int r = 0; r < kRowsPerCta; ++r)
 #pragma unroll
-    for (int c = 0; c < CMAX; ++c)
+    for (int c = 0; c < CU; ++c)
       if (c < C) {
         float v = acc[r][c];
 #pragma unroll
@@ -202,7 +218,7 @@ __device__ __forceinline__ void store_cols(__nv_bfloat16* p, const float (&r)[2]
 // it will update, the biases, the first rows of A) is requested before the first wait, so the kernel
 // costs about one memory round trip plus the arithmetic.  The CTA of column block 0 also adds the row
 // losses that head_fwd_kernel left behind (training steps) into the mini-batch mean.
-template <typename TA, int VEC>
+template <typename TA, int VEC, int CT>
 __global__ void __launch_bounds__(kThreads, 2)
 head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
                 float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb,
@@ -212,9 +228,11 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   constexpr int COLS = 32 * VEC;
   constexpr int kTrip = 16 / VEC;                   // rows per thread per trip
   constexpr int kUpd = (CMAX * COLS) / kThreads;    // elements of the C x COLS block per thread, at most
+  constexpr int CU = CT > 0 ? CT : CMAX;            // unrolled class count
+  const int CP = CT > 0 ? (CT + 3) / 4 * 4 : C;     // floats per row of dz in shared memory (16-byte rows when known)
   extern __shared__ float sm[];
-  float* dz = sm;                                   // [B][C]
-  float* part = sm + (size_t)B * C;                 // [8][CMAX][COLS]
+  float* dz = sm;                                   // [B][CP]
+  float* part = sm + (size_t)B * CP;                // [8][CMAX][COLS]
   grid_dep_wait();
   grid_dep_launch();
   const int g = blockIdx.y;
@@ -226,9 +244,9 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
 
   // ---- requests --------------------------------------------------------------------------------
-  float wreg[CMAX][VEC];
+  float wreg[CU][VEC];
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c)
+  for (int c = 0; c < CU; ++c)
 #pragma unroll
     for (int v = 0; v < VEC; ++v)
       wreg[c][v] = (c < C && in[v]) ? W[(int64_t)g * w_gstride + (int64_t)c * K + k + v] : 0.f;
@@ -276,13 +294,13 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
     if (cx == 0) loss_out[g] = p * (1.0f / (float)B);
   }
-  for (int i = threadIdx.x; i < B * C; i += kThreads) dz[i] = dZ[(int64_t)g * B * C + i];
+  for (int i = threadIdx.x; i < B * C; i += kThreads) dz[(i / C) * CP + i % C] = dZ[(int64_t)g * B * C + i];
   __syncthreads();
 
   // ---- both gradients in one pass over the rows ------------------------------------------------------
-  float gw[CMAX][VEC];
+  float gw[CU][VEC];
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c)
+  for (int c = 0; c < CU; ++c)
 #pragma unroll
     for (int v = 0; v < VEC; ++v) gw[c][v] = 0.f;
   float cs[VEC];      // column sums of dPrev over this thread's rows (bias gradient of the layer below)
@@ -308,14 +326,31 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
       float da[VEC];
 #pragma unroll
       for (int v = 0; v < VEC; ++v) da[v] = 0.f;
+      if (CT > 0) {
+        // the row of dZ in whole 16-byte pieces, then the products: no branch between the loads
+        float drow[(CU + 3) / 4 * 4];
 #pragma unroll
-      for (int c = 0; c < CMAX; ++c) {
-        if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
-        const float d = dz[b * C + c];
+        for (int i = 0; i < (CU + 3) / 4; ++i) {
+          const float4 d4 = *reinterpret_cast<const float4*>(dz + b * CP + 4 * i);
+          drow[4 * i] = d4.x; drow[4 * i + 1] = d4.y; drow[4 * i + 2] = d4.z; drow[4 * i + 3] = d4.w;
+        }
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) {
-          gw[c][v] = fmaf(d, av[u][v], gw[c][v]);
-          da[v] = fmaf(d, wreg[c][v], da[v]);
+        for (int c = 0; c < CU; ++c)
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) {
+            gw[c][v] = fmaf(drow[c], av[u][v], gw[c][v]);
+            da[v] = fmaf(drow[c], wreg[c][v], da[v]);
+          }
+      } else {
+#pragma unroll
+        for (int c = 0; c < CU; ++c) {
+          if (c >= C) break;          // uniform: the remaining classes are skipped, not predicated off
+          const float d = dz[b * CP + c];
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) {
+            gw[c][v] = fmaf(d, av[u][v], gw[c][v]);
+            da[v] = fmaf(d, wreg[c][v], da[v]);
+          }
         }
       }
       if (dPrev != nullptr && in[0]) {
@@ -332,7 +367,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     }
   }
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c)
+  for (int c = 0; c < CU; ++c)
 #pragma unroll
     for (int v = 0; v < VEC; ++v) part[(ry * CMAX + c) * COLS + cx * VEC + v] = gw[c][v];
   __syncthreads();
@@ -360,7 +395,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   if (own_bias) {
     const int c = threadIdx.x;
     float s = 0.f;
-    for (int b = 0; b < B; ++b) s += dz[b * C + c];
+    for (int b = 0; b < B; ++b) s += dz[b * CP + c];
     const int64_t at = (int64_t)g * w_gstride + c;
     float step = s;
     if (mu != 0.f) {
@@ -399,18 +434,29 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   dim3 grid((unsigned)((a.B + kRowsPerCta - 1) / kRowsPerCta), (unsigned)a.groups);
   const int vec_ok = (a.K % 4 == 0) && (reinterpret_cast<uintptr_t>(a.A) % 16 == 0) &&
                      (reinterpret_cast<uintptr_t>(a.W) % 16 == 0) && (a.w_gstride % 4 == 0);
-  if (a_bf16)
-    return launch_dep(head_fwd_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, st, 1,
-                      static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off,
-                      a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K, a.loss_kind, vec_ok, a.defer_loss);
-  return launch_dep(head_fwd_kernel<float>, grid, dim3(kThreads), 0, st, 1, static_cast<const float*>(a.A),
-                    a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters,
-                    a.B, a.C, a.K, a.loss_kind, vec_ok, a.defer_loss);
+  if (a_bf16) {
+    auto go = [&](auto kern) {
+      return launch_dep(kern, grid, dim3(kThreads), 0, st, 1, static_cast<const __nv_bfloat16*>(a.A), a.a_row_off, a.W,
+                        a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K,
+                        a.loss_kind, vec_ok, a.defer_loss);
+    };
+    if (a.C == 10) return go(head_fwd_kernel<__nv_bfloat16, 10>);
+    if (a.C == 1) return go(head_fwd_kernel<__nv_bfloat16, 1>);
+    return go(head_fwd_kernel<__nv_bfloat16, 0>);
+  }
+  auto go = [&](auto kern) {
+    return launch_dep(kern, grid, dim3(kThreads), 0, st, 1, static_cast<const float*>(a.A), a.a_row_off, a.W,
+                      a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters, a.B, a.C, a.K,
+                      a.loss_kind, vec_ok, a.defer_loss);
+  };
+  if (a.C == 10) return go(head_fwd_kernel<float, 10>);
+  if (a.C == 1) return go(head_fwd_kernel<float, 1>);
+  return go(head_fwd_kernel<float, 0>);
 }
 
-template <typename TA, int VEC>
-int launch_head_bwd_t(const HeadBwdArgs& a, cudaStream_t st) {
-  auto kern = head_bwd_kernel<TA, VEC>;
+template <typename TA, int VEC, int CT>
+int launch_head_bwd_c(const HeadBwdArgs& a, cudaStream_t st) {
+  auto kern = head_bwd_kernel<TA, VEC, CT>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -419,10 +465,17 @@ int launch_head_bwd_t(const HeadBwdArgs& a, cudaStream_t st) {
   }
   constexpr int COLS = 32 * VEC;
   dim3 grid((unsigned)((a.K + COLS - 1) / COLS), (unsigned)a.groups);
-  const size_t smem = ((size_t)a.B * a.C + 8 * CMAX * COLS) * sizeof(float);
+  const size_t smem = ((size_t)a.B * (CT > 0 ? (CT + 3) / 4 * 4 : a.C) + 8 * CMAX * COLS) * sizeof(float);
   return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const TA*>(a.A), a.a_row_off, a.dZ, a.W, a.V,
                     a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<TA*>(a.dPrev), a.dPrev ? a.pbias : nullptr,
                     a.pvbias, a.row_loss, a.loss_out, a.B, a.C, a.K, a.lr, a.mu);
+}
+
+template <typename TA, int VEC>
+int launch_head_bwd_t(const HeadBwdArgs& a, cudaStream_t st) {
+  if (a.C == 10) return launch_head_bwd_c<TA, VEC, 10>(a, st);
+  if (a.C == 1) return launch_head_bwd_c<TA, VEC, 1>(a, st);
+  return launch_head_bwd_c<TA, VEC, 0>(a, st);
 }
 
 int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
