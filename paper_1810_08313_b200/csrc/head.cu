@@ -193,6 +193,128 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   }
 }
 
+// The same layer for wide inputs (K in the thousands): one CTA = 16 mini-batch rows, warp w owns rows 2w and
+// 2w + 1 over all of K, so the C x K weights are read once per 16 rows instead of once per 4 and the CTAs
+// of the bf16 MLP's output layer (16 per replica) fit the GPU in one wave.  A lane takes 8 consecutive
+// elements of K per trip; every load of a trip is issued before its first product.
+constexpr int kWideRows = 16;
+
+__device__ __forceinline__ void load8(const float* p, float (&r)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  r[0] = a.x; r[1] = a.y; r[2] = a.z; r[3] = a.w; r[4] = b.x; r[5] = b.y; r[6] = b.z; r[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&r)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    r[2 * i] = __uint_as_float(w[i] << 16);               // a bf16 is the upper half of an fp32
+    r[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+template <typename TA, int CT>
+__global__ void __launch_bounds__(kThreads, 2)
+head_fwd_wide_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ W,
+                     int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
+                     const int64_t* __restrict__ y_row_off, float* __restrict__ dZ, float* __restrict__ row_loss,
+                     float* __restrict__ loss_out, unsigned int* __restrict__ counters, int B, int K, int kind,
+                     int defer_loss) {
+  __shared__ unsigned int is_last;
+  __shared__ float red[kThreads];
+  grid_dep_wait();
+  grid_dep_launch();
+  const int g = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b0 = blockIdx.x * kWideRows + 2 * warp;          // this warp's first row
+  const TA* Ag = A + ((a_row_off ? a_row_off[g] : (int64_t)g * B) + b0) * K;
+  const float* Wg = W + (int64_t)g * w_gstride;
+  const float bz = (bias != nullptr && lane < CT) ? bias[(int64_t)g * w_gstride + lane] : 0.f;
+  int label[2] = {0, 0};
+  float target[2] = {0.f, 0.f};
+  {
+    const int64_t y0 = y_row_off[g] + b0;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (kind == LS_LOSS_SOFTMAX_CE) label[r] = static_cast<const int32_t*>(y)[y0 + r];
+      else target[r] = static_cast<const float*>(y)[y0 + r];
+    }
+  }
+  float acc[2][CT];
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int c = 0; c < CT; ++c) acc[r][c] = 0.f;
+  for (int k = lane * 8; k < K; k += 256) {
+    float a[2][8], w[CT][8];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) load8(Ag + (int64_t)r * K + k, a[r]);
+#pragma unroll
+    for (int c = 0; c < CT; ++c) load8(Wg + (int64_t)c * K + k, w[c]);
+#pragma unroll
+    for (int c = 0; c < CT; ++c)
+#pragma unroll
+      for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[r][c] = fmaf(a[r][e], w[c][e], acc[r][c]);
+  }
+  // lane sums, then lane c keeps class c of both rows
+  float z[2] = {0.f, 0.f};
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int c = 0; c < CT; ++c) {
+      float v = acc[r][c];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == c) z[r] = v + bz;
+    }
+  const float invB = 1.0f / (float)B;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int b = b0 + r;
+    const float zz = (lane < CT) ? z[r] : -INFINITY;
+    float loss, d;
+    if (kind == LS_LOSS_SOFTMAX_CE) {
+      float mx = zz;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float e = (lane < CT) ? expf(zz - mx) : 0.f;
+      float sum = e;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const bool valid = label[r] >= 0 && label[r] < CT;
+      const float zy = __shfl_sync(0xffffffffu, zz, valid ? label[r] : 0);
+      loss = (mx + logf(sum)) - (valid ? zy : mx);
+      d = (e / sum - (lane == label[r] ? 1.f : 0.f)) * invB;
+    } else {
+      const float res = __shfl_sync(0xffffffffu, zz, 0) - target[r];
+      loss = 0.5f * res * res;
+      d = res * invB;
+    }
+    if (lane == 0) row_loss[(int64_t)g * B + b] = loss;
+    if (dZ != nullptr && lane < CT) dZ[((int64_t)g * B + b) * CT + lane] = d;
+  }
+  if (defer_loss) return;
+  // the last CTA of this replica adds the row losses in row order
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicInc(&counters[g], gridDim.x - 1) == gridDim.x - 1) ? 1u : 0u;
+  __syncthreads();
+  if (is_last && loss_out != nullptr) {
+    __threadfence();
+    float p = 0.f;
+    for (int b = threadIdx.x; b < B; b += kThreads) p += __ldcg(&row_loss[(int64_t)g * B + b]);
+    red[threadIdx.x] = p;
+    __syncthreads();
+    for (int s = kThreads / 2; s > 0; s >>= 1) {
+      if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) loss_out[g] = red[0] * invB;
+  }
+}
+
 __device__ __forceinline__ void load_cols(const float* p, float (&r)[1]) { r[0] = *p; }
 __device__ __forceinline__ void load_cols(const __nv_bfloat16* p, float (&r)[1]) { r[0] = __bfloat162float(*p); }
 __device__ __forceinline__ void load_cols(const float* p, float (&r)[2]) {
@@ -218,7 +340,10 @@ __device__ __forceinline__ void store_cols(__nv_bfloat16* p, const float (&r)[2]
 // it will update, the biases, the first rows of A) is requested before the first wait, so the kernel
 // costs about one memory round trip plus the arithmetic.  The CTA of column block 0 also adds the row
 // losses that head_fwd_kernel left behind (training steps) into the mini-batch mean.
-template <typename TA, int VEC, int CT>
+// SLAB: the CTA's columns of A (all B rows) are copied to shared memory with one batch of 16-byte
+// asynchronous copies at the start, so the layer input costs one memory round trip instead of one per
+// 8 * kTrip rows (needs whole column blocks, 16-byte aligned rows, and room in shared memory).
+template <typename TA, int VEC, int CT, bool SLAB>
 __global__ void __launch_bounds__(kThreads, 2)
 head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off, const float* __restrict__ dZ,
                 float* __restrict__ W, float* __restrict__ V, __nv_bfloat16* __restrict__ Wb,
@@ -233,6 +358,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
   extern __shared__ float sm[];
   float* dz = sm;                                   // [B][CP]
   float* part = sm + (size_t)B * CP;                // [8][CMAX][COLS]
+  TA* slab = reinterpret_cast<TA*>(part + 8 * CMAX * COLS);   // SLAB: [B][COLS]
   grid_dep_wait();
   grid_dep_launch();
   const int g = blockIdx.y;
@@ -242,6 +368,18 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 #pragma unroll
   for (int v = 0; v < VEC; ++v) in[v] = k + v < K;
   const TA* Ag = A + (a_row_off ? a_row_off[g] : (int64_t)g * B) * K;
+  if (SLAB) {
+    constexpr int kRowBytes = COLS * (int)sizeof(TA), kPieces = kRowBytes / 16;
+    const char* src = reinterpret_cast<const char*>(Ag + blockIdx.x * COLS);
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(slab));
+    for (int i = threadIdx.x; i < B * kPieces; i += kThreads) {
+      const int row = i / kPieces, pc = i % kPieces;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kRowBytes + pc * 16),
+                   "l"(src + (int64_t)row * K * (int)sizeof(TA) + pc * 16)
+                   : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
 
   // ---- requests --------------------------------------------------------------------------------
   float wreg[CU][VEC];
@@ -281,7 +419,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     const int b = ry + 8 * u;
 #pragma unroll
     for (int v = 0; v < VEC; ++v) av[u][v] = 0.f;
-    if (b < B && in[0]) {
+    if (!SLAB && b < B && in[0]) {
       if (VEC == 1 || in[VEC - 1]) load_cols(Ag + (int64_t)b * K + k, av[u]);
       else av[u][0] = to_f(Ag[(int64_t)b * K + k]);
     }
@@ -295,6 +433,7 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
     if (cx == 0) loss_out[g] = p * (1.0f / (float)B);
   }
   for (int i = threadIdx.x; i < B * C; i += kThreads) dz[(i / C) * CP + i % C] = dZ[(int64_t)g * B * C + i];
+  if (SLAB) asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
   // ---- both gradients in one pass over the rows ------------------------------------------------------
@@ -307,7 +446,15 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 #pragma unroll
   for (int v = 0; v < VEC; ++v) cs[v] = 0.f;
   for (int bb = 0; bb < B; bb += 8 * kTrip) {
-    if (bb > 0) {
+    if (SLAB) {
+#pragma unroll
+      for (int u = 0; u < kTrip; ++u) {
+        const int b = bb + ry + 8 * u;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) av[u][v] = 0.f;
+        if (b < B) load_cols(slab + b * COLS + cx * VEC, av[u]);
+      }
+    } else if (bb > 0) {
 #pragma unroll
       for (int u = 0; u < kTrip; ++u) {
         const int b = bb + ry + 8 * u;
@@ -429,8 +576,23 @@ head_bwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 
 bool head_shape_ok(int B, int C) { return C >= 1 && C <= CMAX && B >= 1 && (size_t)B * C * 4 <= 64 * 1024; }
 
+template <typename TA, int CT>
+int launch_head_fwd_wide(const HeadFwdArgs& a, cudaStream_t st) {
+  dim3 grid((unsigned)(a.B / kWideRows), (unsigned)a.groups);
+  return launch_dep(head_fwd_wide_kernel<TA, CT>, grid, dim3(kThreads), 0, st, 1, static_cast<const TA*>(a.A),
+                    a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters,
+                    a.B, a.K, a.loss_kind, a.defer_loss);
+}
+
 int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
+  // wide inputs with enough rows to fill the GPU 16 at a time: the kernel that reads W once per 16 rows
+  if ((a.C == 10 || a.C == 1) && a.K >= 1024 && a.K % 8 == 0 && a.B % kWideRows == 0 &&
+      (int64_t)(a.B / kWideRows) * a.groups >= 64 && reinterpret_cast<uintptr_t>(a.A) % 16 == 0 &&
+      reinterpret_cast<uintptr_t>(a.W) % 16 == 0 && a.w_gstride % 4 == 0) {
+    if (a_bf16) return a.C == 10 ? launch_head_fwd_wide<__nv_bfloat16, 10>(a, st) : launch_head_fwd_wide<__nv_bfloat16, 1>(a, st);
+    return a.C == 10 ? launch_head_fwd_wide<float, 10>(a, st) : launch_head_fwd_wide<float, 1>(a, st);
+  }
   dim3 grid((unsigned)((a.B + kRowsPerCta - 1) / kRowsPerCta), (unsigned)a.groups);
   const int vec_ok = (a.K % 4 == 0) && (reinterpret_cast<uintptr_t>(a.A) % 16 == 0) &&
                      (reinterpret_cast<uintptr_t>(a.W) % 16 == 0) && (a.w_gstride % 4 == 0);
@@ -454,21 +616,32 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
   return go(head_fwd_kernel<float, 0>);
 }
 
-template <typename TA, int VEC, int CT>
-int launch_head_bwd_c(const HeadBwdArgs& a, cudaStream_t st) {
-  auto kern = head_bwd_kernel<TA, VEC, CT>;
+template <typename TA, int VEC, int CT, bool SLAB>
+int launch_head_bwd_s(const HeadBwdArgs& a, size_t smem, cudaStream_t st) {
+  auto kern = head_bwd_kernel<TA, VEC, CT, SLAB>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   constexpr int COLS = 32 * VEC;
   dim3 grid((unsigned)((a.K + COLS - 1) / COLS), (unsigned)a.groups);
-  const size_t smem = ((size_t)a.B * (CT > 0 ? (CT + 3) / 4 * 4 : a.C) + 8 * CMAX * COLS) * sizeof(float);
   return launch_dep(kern, grid, dim3(kThreads), smem, st, 1, static_cast<const TA*>(a.A), a.a_row_off, a.dZ, a.W, a.V,
                     a.Wb, a.bias, a.vbias, a.w_gstride, static_cast<TA*>(a.dPrev), a.dPrev ? a.pbias : nullptr,
                     a.pvbias, a.row_loss, a.loss_out, a.B, a.C, a.K, a.lr, a.mu);
+}
+
+template <typename TA, int VEC, int CT>
+int launch_head_bwd_c(const HeadBwdArgs& a, cudaStream_t st) {
+  constexpr int COLS = 32 * VEC;
+  const size_t base = ((size_t)a.B * (CT > 0 ? (CT + 3) / 4 * 4 : a.C) + 8 * CMAX * COLS) * sizeof(float);
+  const size_t slab = (size_t)a.B * COLS * sizeof(TA);
+  // the slab variant: whole column blocks, rows that start on 16-byte boundaries, two CTAs per SM still fit
+  const bool ok = COLS * sizeof(TA) % 16 == 0 && a.K % COLS == 0 && ((size_t)a.K * sizeof(TA)) % 16 == 0 &&
+                  reinterpret_cast<uintptr_t>(a.A) % 16 == 0 && base % 16 == 0 && base + slab <= 100 * 1024;
+  if (ok) return launch_head_bwd_s<TA, VEC, CT, true>(a, base + slab, st);
+  return launch_head_bwd_s<TA, VEC, CT, false>(a, base, st);
 }
 
 template <typename TA, int VEC>
