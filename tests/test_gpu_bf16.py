@@ -70,6 +70,21 @@ def test_eval_loss_bf16():
     eng.close()
 
 
+def test_eval_loss_bf16_wide_layers():
+    """Forward-only pass through the CTA-pair kernels (512-wide layers, batch 256) with shared weights."""
+    from paper_1810_08313_b200.binding import LocalSGD
+    dims = (384, 512, 512, 10)
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 7, bf16=True)
+    xd, yd = to_device(X, y, bf16=True)
+    eng = LocalSGD(3, dims, gemm_dtype="bf16", lr=0.05, momentum=0.9, batch=256)
+    eng.bind_dataset(xd, yd); eng.set_params(x1)
+    for rows in (256, 768):
+        F = eng.eval_loss(2, 0, rows)
+        want = orc.batch_loss(spec, x1, X[:rows], y[:rows])
+        assert abs(F - want) / want <= BF16_LOSS_TOL, (rows, F, want)
+    eng.close()
+
+
 def _one_step_gradients(dims, m, B, seed=29):
     """Momentum buffers after one step from v = 0 (they equal the stochastic gradient) vs the oracle's gradient."""
     from paper_1810_08313_b200.binding import LocalSGD
