@@ -571,6 +571,36 @@ def run_ours(args, w: wl.Workload):
                 "speedup_model": {str(t): round((1 + alpha) / (1 + alpha / t), 4) for t in sweep},
                 "note": "model: (1 + alpha) / (1 + alpha / tau) with alpha = D / Y fitted at tau = 1 and 100"}
 
+        # ---- the workload's whole job in the native run loop (ls_run): K iterations, AdaComm where configured -------
+        if args.full_run:
+            runs = {}
+            Kfull = w.n_iters
+            fo = wl.batch_row_offsets(w.seed + 7, Kfull, m, w.n_rows, B)
+            schedules = [(w.adacomm_tau0, w.adacomm_interval)] if w.adacomm_tau0 else [(t, 0) for t in w.taus]
+            for tau0, interval in schedules:
+                eng.set_params(x1)
+                for i in range(m):
+                    eng.set_state(i, None, np.zeros_like(x1))
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                out = eng.run(Kfull, tau0, fo, interval=interval or 0, probe_rows=probe if interval else 0)
+                eng.sync()
+                dt = time.perf_counter() - t0
+                F_end = eng.eval_loss(0, 0, probe)
+                taus = out["taus"]
+                # run-length form of the period list: [[tau, how many periods in a row], ...]
+                rle = []
+                for t in taus:
+                    if rle and rle[-1][0] == t:
+                        rle[-1][1] += 1
+                    else:
+                        rle.append([int(t), 1])
+                runs[f"tau0_{tau0}" + ("_adacomm" if interval else "")] = {
+                    "iterations": Kfull, "seconds": round(dt, 4), "replica_steps_per_s": round(m * Kfull / dt, 1),
+                    "averaging_steps": len(taus), "periods_rle": rle[:40], "F_0": F_0, "F_end": F_end,
+                    "decisions": len(out["decision_k"])}
+            line["full_run"] = runs
+
         # ---- the CPU oracle on the host cores, bounded sample -----------------------------------
         if not args.no_cpu_baseline:
             v, iters, dt = oracle_replica_steps_per_s(w, X[:8192], y[:8192], x1, tau, budget_s=args.cpu_budget,
@@ -598,6 +628,9 @@ def main():
     ap.add_argument("--tau-sweep", action="store_true",
                     help="also time iterations at tau = 1, 2, 5, 20, 100 and compare with the speed-up model of Section 3.2")
     ap.add_argument("--avg-1b", action="store_true", help="add the 10^9-element point to the averaging sweep (128 GB)")
+    ap.add_argument("--full-run", action="store_true",
+                    help="also run the workload's whole job (its iteration count, tau or AdaComm schedule) in the native "
+                         "run loop and report its throughput, loss and the periods chosen")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, averaging sweep or CPU baseline")
     args = ap.parse_args()
