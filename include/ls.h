@@ -54,7 +54,7 @@ enum {
   LS_ERR_NO_DATASET = -4,        /* ls_bind_dataset() has not been called */
   LS_ERR_ROW_RANGE = -5,         /* a mini-batch would read past the bound dataset */
   LS_ERR_CUDA = -6,              /* a CUDA runtime call failed; ls_last_cuda_error() has its code */
-  LS_ERR_UNSUPPORTED = -7,       /* valid request that this build does not implement (e.g. weight decay) */
+  LS_ERR_UNSUPPORTED = -7,       /* valid request that the library does not implement (e.g. weight decay) */
   LS_ERR_OVERFLOW = -8,          /* a result does not fit its type */
   LS_ERR_DEVICE_TIMEOUT = -9,    /* a bounded wait inside a kernel ran out; results of that launch are invalid */
   LS_ERR_TOO_LARGE = -10         /* a size exceeds a fixed capacity of the entry point */

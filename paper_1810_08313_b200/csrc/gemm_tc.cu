@@ -676,14 +676,13 @@ struct SmemPair {
   static constexpr int kRingBytes = kPairStages * kStageBytes;
   static constexpr int kBoxBytes = 64 * KB_BYTES;               // epilogue: 64 rows x 64 bf16
   static constexpr int kOutBytes = 2 * kPairGroups * kBoxBytes; // the CTA's 128 x 512 outputs (and mask) as boxes
-  static constexpr int kTransBytes = 4 * 32 * 33 * 4;           // backward: per-warp transposes for the column sums
-  static constexpr int kColsumBytes = 4 * kPairN * 4;
-  static constexpr int kBars = 2 * kPairStages + 1 + kPairGroups;
+  static constexpr int kColsumBytes = 2 * kPairN * 4;           // backward: column sums of the CTA's two row halves
+  static constexpr int kBars = 2 * kPairStages + 1 + 2 * kPairGroups;
   static constexpr int kBarBytes = (kBars * 8 + 16 + 15) / 16 * 16;
   static constexpr int kBiasBytes = kPairN * 4;                 // forward: the bias of the tile's columns
   static constexpr int kTotal = 1024 + kRingBytes + kBarBytes + kBiasBytes;
   static_assert(kBarBytes % 16 == 0, "bias block alignment");
-  static_assert(kOutBytes + kTransBytes + kColsumBytes <= kRingBytes, "epilogue scratch");
+  static_assert(kOutBytes + kColsumBytes <= kRingBytes, "epilogue scratch");
   static_assert(kStageBytes % kBoxBytes == 0, "whole boxes per stage");
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
@@ -711,13 +710,13 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
-  float* staging = reinterpret_cast<float*>(smem + L::kOutBytes);           // [4][32 x 33]
-  float* colsum = reinterpret_cast<float*>(smem + L::kOutBytes + L::kTransBytes);   // [4][kPairN]
+  float* colsum = reinterpret_cast<float*>(smem + L::kOutBytes);            // [2][kPairN]
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kRingBytes);
   uint64_t* empty = full + STAGES;
   uint64_t* acc_full = empty + STAGES;
   uint64_t* mask_full = acc_full + 1;                           // [kPairGroups]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mask_full + kPairGroups);
+  uint64_t* box_done = mask_full + kPairGroups;                 // [kPairGroups] both row halves of a group written
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(box_done + kPairGroups);
   float* bias_s = reinterpret_cast<float*>(smem + L::kRingBytes + L::kBarBytes);   // [kPairN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -731,7 +730,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
-    for (int i = 0; i < kPairGroups; ++i) mbar_init(&mask_full[i], 1);
+    for (int i = 0; i < kPairGroups; ++i) { mbar_init(&mask_full[i], 1); mbar_init(&box_done[i], 2); }
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
@@ -898,18 +897,6 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           *reinterpret_cast<uint4*>(myrow + (((sub * 4 + i) ^ (rih & 7)) << 4)) = make_uint4(u[0], u[1], u[2], u[3]);
         }
-        if (EPI == EPI_DX && p.dbias != nullptr) {
-          // column sums over this warp's 32 rows, of the unrounded gradients like the single-CTA kernel
-          float* tile = staging + q * (32 * 33);
-          __syncwarp();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = o[i];
-          __syncwarp();
-          float cs = 0.f;
-#pragma unroll
-          for (int rr = 0; rr < 32; ++rr) cs += tile[rr * 33 + lane];
-          colsum[q * kPairN + c * 32 + lane] = cs;
-        }
         if (sub == 1) {
           // both warps of the half have written the box: hand it to the bulk-copy engine
           fence_proxy_async_smem();
@@ -918,6 +905,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if ((q & 1) == 0 && lane == 0) {
             tma_store_2d(&tmC, box, n0 + grp * 64, out_row0 + half * 64);
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            if (EPI == EPI_DX) mbar_arrive(&box_done[grp]);
           }
         }
       }
@@ -925,9 +913,32 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if ((q & 1) == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before_sync();
   }
+  if (EPI == EPI_DX && p.dbias != nullptr && warp < 2) {
+    // Column sums of the tile for the bias update of the layer below, by the two warps whose other work is over:
+    // thread (h, cp) adds columns 2 cp, 2 cp + 1 over the 64 rows of row half h, in row order, from each box as the
+    // epilogue warps finish it (the values as stored, i.e. rounded to bf16, like the stand-alone bias kernel).
+    __syncwarp();
+    const int h = warp, cp = lane;
+    bool ok2 = true;
+    for (int grp = 0; grp < kPairGroups; ++grp) {
+      if (ok2) ok2 = __all_sync(0xffffffffu, mbar_wait(&box_done[grp], 0));
+      const uint8_t* box = smem + (grp * 2 + h) * L::kBoxBytes;
+      float s0 = 0.f, s1 = 0.f;
+      if (ok2) {
+#pragma unroll 8
+        for (int r = 0; r < 64; ++r) {
+          const uint32_t u = *reinterpret_cast<const uint32_t*>(box + r * 128 + (((cp >> 2) ^ (r & 7)) << 4) + (cp & 3) * 4);
+          s0 += __uint_as_float(u << 16);
+          s1 += __uint_as_float(u & 0xFFFF0000u);
+        }
+      }
+      colsum[h * kPairN + grp * 64 + 2 * cp] = s0;
+      colsum[h * kPairN + grp * 64 + 2 * cp + 1] = s1;
+    }
+  }
   if (EPI == EPI_DX && p.dbias != nullptr) {
     // bias update of the layer below: column sums over the pair's 256 rows, added in row order (leader's
-    // warps 0-3, then the peer's) by the CTA that owns the column half
+    // two halves, then the peer's) by the CTA that owns the column half
     cluster_sync_all();
     if (warp >= 2) {
       const uint32_t mine = smem_u32(colsum);
@@ -937,9 +948,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int t = rank * 256 + (int)threadIdx.x - 64 + i2 * 128;
         float gsum = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) gsum += ld_cluster_f32(src0 + (uint32_t)((i * kPairN + t) * 4));
+        for (int i = 0; i < 2; ++i) gsum += ld_cluster_f32(src0 + (uint32_t)((i * kPairN + t) * 4));
 #pragma unroll
-        for (int i = 0; i < 4; ++i) gsum += ld_cluster_f32(src1 + (uint32_t)((i * kPairN + t) * 4));
+        for (int i = 0; i < 2; ++i) gsum += ld_cluster_f32(src1 + (uint32_t)((i * kPairN + t) * 4));
         const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
         float step = gsum;
         if (p.mu != 0.f) {
