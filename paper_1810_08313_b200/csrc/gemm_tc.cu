@@ -50,8 +50,8 @@ using namespace ptx;
 constexpr int BM = 128;            // rows of the output tile = TMEM lanes
 constexpr int KB_BYTES = 128;      // bytes of K per stage row (one swizzle row)
 constexpr int kThreadsBf16 = 192;  // warps 0-5
-constexpr int kThreadsFp32 = 256;  // + two splitter warps
-constexpr int kSplitWarps = 2;
+constexpr int kSplitWarps = 4;
+constexpr int kThreadsFp32 = 192 + 32 * kSplitWarps;  // + the splitter warps
 constexpr int kHeadMax = 16;       // outputs of a fused narrow output layer, at most
 constexpr int kStageLd = 36;       // floats per staged row (32 + 4 padding) in the update epilogue
 constexpr int kChunkStages = 4;    // fp32 forward/backward: stages per TMEM accumulation chunk (48 MMAs)
@@ -279,9 +279,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) atomicExch(p.err_flag, 5);
         break;
       }
-      static_assert(L::kStageBytes % (8 * 16 * kSplitWarps * 32) == 0, "whole batches of pieces");
-      split_lo_smem(smem_u32(stage_base + s * L::kStageBytes), smem_u32(lo_base + sl * L::kStageBytes),
-                    L::kStageBytes, tid, kSplitWarps * 32);
+      constexpr int kSplitDepth = (L::kStageBytes % (8 * 16 * kSplitWarps * 32) == 0) ? 8 : 4;
+      static_assert(L::kStageBytes % (kSplitDepth * 16 * kSplitWarps * 32) == 0, "whole batches of pieces");
+      split_lo_smem<kSplitDepth>(smem_u32(stage_base + s * L::kStageBytes), smem_u32(lo_base + sl * L::kStageBytes),
+                                 L::kStageBytes, tid, kSplitWarps * 32);
       fence_proxy_async_smem();     // the tensor core reads shared memory through the async proxy
       __syncwarp();
       if (lane == 0) mbar_arrive(&lo_full[sl]);

@@ -91,23 +91,24 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
 
 // ---- fp32 operands as tf32 pairs -----------------------------------------------
 // lo = x - tf32(x) for `bytes` bytes of shared memory at `src` (32-bit shared address), written to the
-// same offsets at `dst`; thread `tid` of `nthreads` takes every nthreads-th 16-byte piece, eight pieces
-// in flight at a time.  bytes must be a multiple of 8 * 16 * nthreads.
+// same offsets at `dst`; thread `tid` of `nthreads` takes every nthreads-th 16-byte piece, U pieces
+// in flight at a time.  bytes must be a multiple of U * 16 * nthreads.
+template <int U = 8>
 __device__ __forceinline__ void split_lo_smem(uint32_t src, uint32_t dst, int bytes, int tid, int nthreads) {
   const int step = nthreads * 16;
-  for (int c0 = tid * 16; c0 < bytes; c0 += 8 * step) {
-    float v[8][4];
+  for (int c0 = tid * 16; c0 < bytes; c0 += U * step) {
+    float v[U][4];
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < U; ++u)
       asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                    : "=f"(v[u][0]), "=f"(v[u][1]), "=f"(v[u][2]), "=f"(v[u][3])
                    : "r"(src + c0 + u * step));
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < U; ++u)
 #pragma unroll
       for (int e = 0; e < 4; ++e) v[u][e] = v[u][e] - __uint_as_float(__float_as_uint(v[u][e]) & 0xFFFFE000u);
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < U; ++u)
       asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(dst + c0 + u * step), "f"(v[u][0]), "f"(v[u][1]),
                    "f"(v[u][2]), "f"(v[u][3])
                    : "memory");
