@@ -66,6 +66,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return true;
 }
 
+// One arrival on a barrier that may live in another CTA of the cluster (`cluster_addr` from map_to_rank).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
 // ---- thread-block clusters: rank, barrier, distributed shared memory ----------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

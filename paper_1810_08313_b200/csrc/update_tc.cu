@@ -384,6 +384,261 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
   }
 }
 
+// ---- bf16 models whose layers are multiples of 256 wide: the same stream on CTA pairs ---------------------------
+// Two CTAs of a cluster share every tcgen05.mma (cta_group::2): the pair's unit is a 256 x 256 block of W, CTA r
+// owns rows 128 r .. of it.  A CTA stages its own 128 columns of dZ and HALF of the unit's 256 columns of the layer
+// input per 64-row stage, i.e. the same 32 KB as the one-CTA kernel, for twice the products: cycle traces of that
+// kernel show its update warps waiting for the products (one 32 KB operand stage, four loads in sequence per
+// tile), and shared memory has no room for a second stage beside the W / v ring.  Everything else (the per-warp
+// W / v rings, the update arithmetic, the left-over strips) is as in tc_update_kernel.
+//   full[s]        on the leader: both CTAs' operand bytes of a stage
+//   empty[s], tmem_full[b]   in each CTA, signalled by the leader's multicast commits
+//   tmem_empty[b]  on the leader: the 8 update warps of the pair have read accumulator b
+constexpr int PN = 256;                 // columns of a pair's unit
+struct PLayer {
+  int N, n_tiles, tiles_per_group, tile_begin;
+  const int64_t* b_row_off;
+  __nv_bfloat16* Wb;
+};
+struct PParams {
+  PLayer layer[kMaxLayers];
+  int n_layers;
+  int full_rounds;                     // whole units per pair; unit t of round n on pair b is b + n * pairs
+  int tail_units;                      // 128-column strips of the left-over units, strip u on pair u % pairs
+  int K, rows_per_group;
+  float lr, mu;
+  int64_t w_gstride;
+  int* err_flag;
+};
+struct PUnit { int layer, g, m0, n0, nc; };      // columns [n0, n0 + 32 nc) of rows [m0, m0 + 256)
+
+__device__ __forceinline__ PUnit decode_punit(const PParams& p, int n, int pb, int pairs) {
+  int t, c0 = 0, nc = PN / 32;
+  if (n < p.full_rounds) {
+    t = pb + n * pairs;
+  } else {
+    const int u = pb + (n - p.full_rounds) * pairs;
+    t = p.full_rounds * pairs + (u >> 1);
+    nc = PN / 64;
+    c0 = (u & 1) * nc;
+  }
+  int l = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxLayers; ++i)
+    if (i < p.n_layers && t >= p.layer[i].tile_begin) l = i;
+  const int r = t - p.layer[l].tile_begin;
+  const int tpg = p.layer[l].tiles_per_group, nt = p.layer[l].n_tiles;
+  const int g = r / tpg, rem = r % tpg;
+  return PUnit{l, g, (rem / nt) * 256, (rem % nt) * PN + c0 * 32, nc};
+}
+
+template <int R, int KS>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ PParams p) {
+  using L = USmem<false, 1, R, KS>;
+  constexpr int MMA_K = 16;
+  constexpr int CHUNK_BYTES = KS * KB_BYTES;
+  constexpr int kABytes = BM * KS * 2;               // this CTA's 128 columns of dZ, KS rows
+  constexpr uint32_t IDESC_FULL = make_idesc(1u, true, true, 256, PN);
+  constexpr uint32_t IDESC_STRIP = make_idesc(1u, true, true, 256, PN / 2);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage = smem;
+  uint8_t* ring_base = smem + L::kOperandBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(ring_base + L::kRingBytes);
+  uint64_t* empty = full + 1;
+  uint64_t* tmem_full = empty + 1;            // [2]
+  uint64_t* tmem_empty = tmem_full + 2;       // [2]
+  uint64_t* wv_full = tmem_empty + 2;         // [4][R]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wv_full + 4 * R);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int num_kb = p.K / KS;
+  const int pb = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+  const int my_strips = pb < p.tail_units ? (p.tail_units - 1 - pb) / pairs + 1 : 0;
+  const int my_units = p.full_rounds + my_strips;
+  const bool has_v = p.mu != 0.f;
+
+  if (threadIdx.x == 0) {
+    mbar_init(full, 1); mbar_init(empty, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
+    for (int i = 0; i < 4 * R; ++i) mbar_init(&wv_full[i], 1);
+    fence_mbar_init();
+    for (int l = 0; l < p.n_layers; ++l) {
+      prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
+    }
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, 2 * PN);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  cluster_sync_all();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
+
+  if (warp == 0) {
+    // ---- operand producer (each CTA loads its own parts; the leader's barrier counts both) -----------
+    if (elect_one()) {
+      const uint64_t pol = l2_policy(2);
+      const uint32_t full_leader = map_to_rank(smem_u32(full), 0);
+      int it = 0;
+      bool ok = true;
+      for (int n = 0; n < my_units && ok; ++n) {
+        const PUnit un = decode_punit(p, n, pb, pairs);
+        const int a_row = un.g * p.rows_per_group;
+        const int64_t* b_off = p.layer[un.layer].b_row_off;
+        const int b_row = b_off ? (int)b_off[un.g] : a_row;
+        const CUtensorMap* tmA = &maps.a[un.layer];
+        const CUtensorMap* tmB = &maps.b[un.layer];
+        const int bcols = un.nc * 16;                          // this CTA's half of the unit's columns
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          if (!mbar_wait(empty, (it & 1) ^ 1)) { atomicExch(p.err_flag, 31); ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full, 2 * (kABytes + bcols * KS * 2));
+          uint8_t* sa = stage;
+          uint8_t* sb = stage + kABytes;
+#pragma unroll
+          for (int c = 0; c < BM / 64; ++c)
+            tma_load_2d_pair(sa + c * CHUNK_BYTES, tmA, full_leader, un.m0 + rank * BM + c * 64, a_row + kb * KS, pol);
+          for (int c = 0; c < bcols / 64; ++c)
+            tma_load_2d_pair(sb + c * CHUNK_BYTES, tmB, full_leader, un.n0 + rank * bcols + c * 64, b_row + kb * KS, pol);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer (leader CTA) -----------------------------------------------------------------
+    if (rank == 0 && elect_one()) {
+      int it = 0;
+      bool ok = true;
+      for (int n = 0; n < my_units && ok; ++n) {
+        const int buf = n & 1;
+        const uint32_t idesc = n < p.full_rounds ? IDESC_FULL : IDESC_STRIP;
+        if (!mbar_wait(&tmem_empty[buf], ((n >> 1) & 1) ^ 1)) { atomicExch(p.err_flag, 32); break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * PN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          if (!mbar_wait(full, it & 1)) { atomicExch(p.err_flag, 33); ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(stage);
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < KS / MMA_K; ++k) {
+            const uint32_t adv = k * MMA_K * KB_BYTES;
+            const uint64_t da = make_smem_desc(a_addr + adv, CHUNK_BYTES, 1024, kSwizzle128B);
+            const uint64_t db = make_smem_desc(b_addr + adv, CHUNK_BYTES, 1024, kSwizzle128B);
+            mma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit_pair(empty);
+        }
+        if (ok) mma_commit_pair(&tmem_full[buf]);
+      }
+    }
+  } else if (warp >= 4) {
+    // ---- update warps: as in tc_update_kernel, on this CTA's 128 rows of the unit ----------------------
+    const int q = warp & 3;
+    uint8_t* my_ring = ring_base + q * R * kSlotBytes;
+    uint64_t* my_full = wv_full + q * R;
+    const int full_chunks = p.full_rounds * (PN / 32);
+    const int my_chunks = full_chunks + my_strips * (PN / 64);
+    const uint32_t tmem_empty_leader = map_to_rank(smem_u32(tmem_empty), 0);
+
+    auto load_chunk = [&](int j) {
+      if (j >= my_chunks) return;
+      const int n = j < full_chunks ? (j >> 3) : p.full_rounds + ((j - full_chunks) >> 2);
+      const PUnit un = decode_punit(p, n, pb, pairs);
+      const int c = j < full_chunks ? (j & 7) : ((j - full_chunks) & 3);
+      const int y = un.m0 + rank * BM + q * 32, x = un.n0 + c * 32;
+      uint8_t* slot = my_ring + (j % R) * kSlotBytes;
+      mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
+      tma_load_3d(slot, &maps.w[un.layer], &my_full[j % R], x, y, un.g);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.v[un.layer], &my_full[j % R], x, y, un.g);
+    };
+    if (lane == 0)
+      for (int j = 0; j < R; ++j) load_chunk(j);
+
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    bool ok = true;
+    int j = 0;
+    for (int n = 0; n < my_units && ok; ++n) {
+      const PUnit un = decode_punit(p, n, pb, pairs);
+      const int g = un.g, m0 = un.m0 + rank * BM, n0 = un.n0;
+      const int ldw = p.layer[un.layer].N;
+      __nv_bfloat16* Wb = p.layer[un.layer].Wb;
+      const int buf = n & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (n >> 1) & 1));
+      if (!ok) { if (lane == 0) atomicExch(p.err_flag, 34); break; }
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int ci = 0; ci < un.nc; ++ci, ++j) {
+        uint8_t* slot = my_ring + (j % R) * kSlotBytes;
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + buf * PN + ci * 32, r);
+        ok = __all_sync(0xffffffffu, mbar_wait(&my_full[j % R], (j / R) & 1));
+        tmem_ld_wait();
+        if (ci == un.nc - 1) {
+          // the accumulator has been read: tell the leader's MMA warp (8 arrivals free the buffer)
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + (uint32_t)(buf * 8));
+        }
+        if (!ok) { if (lane == 0) atomicExch(p.err_flag, 35); break; }
+        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * ldw + n0 + ci * 32;
+        uint32_t cp[8];
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+          float4 w = *reinterpret_cast<float4*>(slot + off);
+          float ws[4] = {w.x, w.y, w.z, w.w};
+          float vs[4] = {0.f, 0.f, 0.f, 0.f};
+          if (has_v) {
+            const float4 v = *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off);
+            vs[0] = v.x; vs[1] = v.y; vs[2] = v.z; vs[3] = v.w;
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float gr = __uint_as_float(r[jj * 4 + e]);
+            const float step = has_v ? fmaf(p.mu, vs[e], gr) : gr;
+            vs[e] = step;
+            ws[e] = fmaf(-p.lr, step, ws[e]);
+          }
+          *reinterpret_cast<float4*>(slot + off) = make_float4(ws[0], ws[1], ws[2], ws[3]);
+          if (has_v) *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) = make_float4(vs[0], vs[1], vs[2], vs[3]);
+          if (Wb != nullptr) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(ws[0], ws[1]);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(ws[2], ws[3]);
+            cp[(jj & 3) * 2] = *reinterpret_cast<uint32_t*>(&lo);
+            cp[(jj & 3) * 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
+            if ((jj & 3) == 3) st_global_v8(Wb + at + (jj - 3) * 4, cp);
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int y = m0 + q * 32, x = n0 + ci * 32;
+          tma_store_3d(&maps.w[un.layer], slot, x, y, g);
+          if (has_v) tma_store_3d(&maps.v[un.layer], slot + kSlotBytes / 2, x, y, g);
+          bulk_commit();
+          bulk_wait_read<1>();
+          if (j >= 1) load_chunk(j - 1 + R);
+        }
+        __syncwarp();
+      }
+    }
+    if (lane == 0) bulk_wait_all();
+    tc_fence_before_sync();
+  }
+  // neither CTA leaves while the other may still read its operands or signal its barriers
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, 2 * PN);
+  }
+}
+
 int num_sms() {
   static int sms = 0;
   if (sms == 0) {
@@ -435,6 +690,45 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   return launch_dep(kern, dim3(grid), dim3(kThreads), L::kTotal, st, 1, maps, p);
 }
 
+template <int R, int KS>
+int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
+  using L = USmem<false, 1, R, KS>;
+  auto kern = tc_update_pair_kernel<R, KS>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const TcUpdateArgs& a0 = layers[0];
+  PParams p{};
+  UMaps maps;
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const TcUpdateArgs& a = layers[i];
+    PLayer& l = p.layer[i];
+    l.N = a.N;
+    l.n_tiles = a.N / PN;
+    l.tiles_per_group = (a.M / 256) * (a.N / PN);
+    l.tile_begin = total;
+    l.b_row_off = a.row_off;
+    l.Wb = a.Wb;
+    total += l.tiles_per_group * a.groups;
+    maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
+  }
+  for (int i = n; i < kMaxLayers; ++i) {
+    maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
+  }
+  const int max_pairs = num_sms() / 2;
+  const int pairs = total < max_pairs ? total : max_pairs;
+  p.n_layers = n;
+  p.full_rounds = total / pairs;
+  p.tail_units = (total - p.full_rounds * pairs) * 2;
+  p.K = a0.B; p.rows_per_group = a0.B;
+  p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
+  return launch_dep(kern, dim3(2 * pairs), dim3(kThreads), L::kTotal, st, 2, maps, p);
+}
+
 }  // namespace
 
 bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
@@ -449,6 +743,10 @@ int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (layers[0].fp32) return launch_update<true, 5, 4, kRowsFp32>(layers, n, st);
+  // bf16 layers that are multiples of 256 in both directions: the CTA-pair kernel
+  bool pair = true;
+  for (int i = 0; i < n; ++i) pair = pair && layers[i].M % 256 == 0 && layers[i].N % PN == 0;
+  if (pair) return launch_update_pair<6, kRowsBf16>(layers, n, st);
   return launch_update<false, 1, 6, kRowsBf16>(layers, n, st);
 }
 

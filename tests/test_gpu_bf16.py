@@ -128,7 +128,9 @@ def test_tensor_core_update_kernel_tight():
 @pytest.mark.parametrize("dims,m,B", [((256, 256, 128, 10), 2, 128), ((384, 256, 256, 256, 10), 3, 256),
                                       ((256, 128, 128), 2, 128),
                                       ((384, 512, 1024, 10), 3, 256),      # CTA pairs, two and four column tiles
-                                      ((256, 512, 512, 10), 2, 512)])      # CTA pairs, two row tiles per replica
+                                      ((256, 512, 512, 10), 2, 512),       # CTA pairs, two row tiles per replica
+                                      ((512, 512, 256, 10), 3, 256),       # update on CTA pairs: fewer units than pairs
+                                      ((1024, 1024, 10), 5, 256)])         # update on CTA pairs: 80 units, left-over strips
 def test_single_step_gradients_through_relu(dims, m, B):
     """All three tensor-core kernels in one step.  bf16 rounding flips a few ReLU masks, which moves single
     entries by O(10 %) of the largest one; the direction of every tensor's gradient is what is checked."""
