@@ -44,6 +44,7 @@ CASES = [
     ((256, 256, 1), "mse_half", True, 2, 128, 0.9),              # fused output layer with one output and squared error
     ((256, 384, 10), "softmax_ce", True, 5, 256, 0.9),           # two row blocks per replica: no fused output layer / bias
     ((512, 256, 10), "softmax_ce", False, 2, 128, 0.0),          # fused output layer without biases or momentum
+    ((1024, 1024, 10), "softmax_ce", True, 5, 128, 0.9),         # update on CTA pairs: 80 units on 74 pairs, left-over strips
 ]
 
 
