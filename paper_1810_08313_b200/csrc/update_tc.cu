@@ -744,7 +744,9 @@ int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t
   if (launches) ++*launches;
   if (layers[0].fp32) return launch_update<true, 5, 4, kRowsFp32>(layers, n, st);
   // bf16 layers that are multiples of 256 in both directions: the CTA-pair kernel
-  bool pair = true;
+  // (LS_DISABLE_PAIR=1 in the environment: one-CTA kernel, a diagnostic switch)
+  const char* e = getenv("LS_DISABLE_PAIR");
+  bool pair = !(e && e[0] == '1');
   for (int i = 0; i < n; ++i) pair = pair && layers[i].M % 256 == 0 && layers[i].N % PN == 0;
   if (pair) return launch_update_pair<6, kRowsBf16>(layers, n, st);
   return launch_update<false, 1, 6, kRowsBf16>(layers, n, st);

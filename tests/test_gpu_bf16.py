@@ -136,3 +136,37 @@ def test_single_step_gradients_through_relu(dims, m, B):
     entries by O(10 %) of the largest one; the direction of every tensor's gradient is what is checked."""
     for i, name, err, cos in _one_step_gradients(dims, m, B):
         assert cos > 0.995 and err < 0.5, (i, name, err, cos)
+
+
+@pytest.mark.parametrize("dims,m,B", [((512, 512, 1024, 10), 3, 256), ((1024, 1024, 10), 5, 256)])
+def test_cta_pair_kernels_match_one_cta_kernels(dims, m, B, monkeypatch):
+    """The CTA-pair GEMM and update kernels against the one-CTA kernels they replace (LS_DISABLE_PAIR=1), one
+    step from the same state: the same products in the same order, so weights and their momentum must agree far
+    more tightly than either agrees with the fp64 oracle.  (The bias gradient of a hidden layer is summed from
+    the bf16-rounded dZ in the pair kernel and from the unrounded values in the one-CTA kernel: biases get a
+    looser bound.)"""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    from tests.helpers import tensor_slices
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 31, bf16=True)
+    offs = wl.batch_row_offsets(9, 1, m, 1024, B)
+    xd, yd = to_device(X, y, bf16=True)
+    out = {}
+    for tag, val in (("pair", "0"), ("one", "1")):
+        monkeypatch.setenv("LS_DISABLE_PAIR", val)
+        eng = LocalSGD(m, dims, gemm_dtype="bf16", lr=0.05, momentum=0.9, batch=B)
+        eng.bind_dataset(xd, yd); eng.set_params(x1)
+        ld = torch.zeros((1, m), device="cuda")
+        eng.local_steps(1, offs, ld)
+        eng.sync()
+        out[tag] = eng.get_all() + (ld.cpu().numpy(),)
+        eng.close()
+    (px, pv, pl), (ox, ov, ol) = out["pair"], out["one"]
+    assert np.max(np.abs(pl - ol) / np.abs(ol)) < 1e-5
+    for i in range(m):
+        for name, sl in tensor_slices(dims, True):
+            tol = 2e-2 if name.startswith("b") else 1e-5
+            for a, b in ((px[i][sl], ox[i][sl]), (pv[i][sl], ov[i][sl])):
+                err = np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-30)
+                assert err < tol, (i, name, err)
+
