@@ -395,8 +395,7 @@ def run_ours(args, w: wl.Workload):
     F_0 = eng.eval_loss(0, 0, probe)
 
     def period(p):
-        eng.local_steps(tau, offs[p * tau:(p + 1) * tau], loss_dev)
-        eng.average()
+        eng.local_steps(tau, offs[p * tau:(p + 1) * tau], loss_dev, average=True)    # the period and its averaging step
         F_t = eng.eval_loss(0, 0, probe)
         return F_t, adacomm_next_tau(F_t, F_0, tau)
 

@@ -155,6 +155,13 @@ int ls_bind_dataset(ls_handle* h, const void* x_dev, const void* y_dev, int64_t 
  * Errors: tau < 1, NULL offsets, a batch outside the dataset. */
 int ls_local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev);
 
+/* One whole communication period: the tau local steps of ls_local_steps followed by
+ * the averaging step of ls_average (Section 2, PASGD update rule: the update of
+ * iteration k is averaged when k mod tau = 0), in one call.  The state after the
+ * call is bit for bit the state after ls_local_steps(tau) then ls_average().
+ * Arguments and errors as ls_local_steps. */
+int ls_local_steps_avg(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev);
+
 /* Same steps, but the mini-batches come from host memory and the losses go
  * back to host memory: x_host is [tau][m][batch][dims[0]] (float or bf16 as
  * for ls_bind_dataset), y_host [tau][m][batch] (int32 or float), loss_host

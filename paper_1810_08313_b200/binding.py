@@ -85,6 +85,7 @@ def _lib():
         "ls_state_view": (C.c_int, [vp, P(vp), P(vp), P(i64)]),
         "ls_bind_dataset": (C.c_int, [vp, vp, vp, i64]),
         "ls_local_steps": (C.c_int, [vp, C.c_int, vp, vp]),
+        "ls_local_steps_avg": (C.c_int, [vp, C.c_int, vp, vp]),
         "ls_local_steps_host": (C.c_int, [vp, C.c_int, vp, vp, vp]),
         "ls_average": (C.c_int, [vp]),
         "ls_average_flat": (C.c_int, [vp, C.c_int, i64, i64, vp]),
@@ -377,7 +378,8 @@ class LocalSGD:
         _check(self.lib.ls_bind_dataset(self.h, x.data_ptr(), y.data_ptr(), int(x.shape[0])), "ls_bind_dataset")
 
     # -- hot path -----------------------------------------------------------
-    def local_steps(self, tau: int, row_offsets: np.ndarray, loss_out=None):
+    def local_steps(self, tau: int, row_offsets: np.ndarray, loss_out=None, average: bool = False):
+        """tau local steps; average=True: followed by the averaging step (one whole period, ls_local_steps_avg)."""
         offs = np.ascontiguousarray(row_offsets, dtype=np.int64)
         if offs.size != tau * self.m:
             raise ValueError("row_offsets must be [tau][m]")
@@ -388,7 +390,10 @@ class LocalSGD:
                     and loss_out.numel() >= tau * self.m):
                 raise ValueError("loss_out must be a contiguous float32 CUDA tensor [tau][m]")
             lp = loss_out.data_ptr()
-        _check(self.lib.ls_local_steps(self.h, int(tau), offs.ctypes.data, lp), "ls_local_steps")
+        if average:
+            _check(self.lib.ls_local_steps_avg(self.h, int(tau), offs.ctypes.data, lp), "ls_local_steps_avg")
+        else:
+            _check(self.lib.ls_local_steps(self.h, int(tau), offs.ctypes.data, lp), "ls_local_steps")
 
     def local_steps_host(self, tau: int, x_host, y_host, loss_host):
         """x_host [tau][m][batch][d_in], y_host [tau][m][batch], loss_host float32 [tau][m]: CPU torch

@@ -228,8 +228,12 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
 }
 
 // One local update of all m replicas (forward, backward, fused SGD-momentum).
+static int average(ls_handle* h);
+
+// avg_after: this is the last local step of a period; the replicas leave the call averaged (Section 2, PASGD
+// update rule, k mod tau = 0).
 static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
-                      float* loss_out) {
+                      float* loss_out, bool avg_after = false) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
   const TcMaps& mn = bf ? h->maps : h->maps_mn;     // descriptors for MN-major reads
@@ -362,6 +366,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
     ProfScope ps(h, LS_K_DW, upd[i].layer);
     LS_CUDA(h, launch_tc_update(upd + i, n, h->stream, &h->launches));
   }
+  if (avg_after) return average(h);
   return LS_OK;
 }
 
@@ -411,7 +416,7 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
   return LS_OK;
 }
 
-static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev) {
+static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev, bool avg_after = false) {
   const Layout& lay = h->lay;
   if (tau < 1 || row_offset_host == nullptr) return LS_ERR_INVALID_ARG;
   if (h->x_dev == nullptr) return LS_ERR_NO_DATASET;
@@ -425,7 +430,7 @@ static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, fl
     for (int s = 0; s < n; ++s) {
       const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
       int rc = local_step(h, h->x_dev, XMaps{&h->maps.x_data, &mnm.x_data, &h->maps_upd.x_data}, h->y_dev, off_dev + (int64_t)s * lay.m,
-                          loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr);
+                          loss_dev ? loss_dev + (int64_t)(s0 + s) * lay.m : nullptr, avg_after && s0 + s == tau - 1);
       if (rc != LS_OK) return rc;
     }
   }
@@ -710,6 +715,11 @@ int ls_local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, float*
   return local_steps(h, tau, row_offset_host, loss_dev);
 }
 
+int ls_local_steps_avg(ls_handle* h, int tau, const int64_t* row_offset_host, float* loss_dev) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  return local_steps(h, tau, row_offset_host, loss_dev, true);
+}
+
 int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y_host, float* loss_host) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   if (tau < 1 || x_host == nullptr || y_host == nullptr || loss_host == nullptr) return LS_ERR_INVALID_ARG;
@@ -851,11 +861,10 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
     const int steps = (int)((K - k < tau) ? K - k : tau);
     if (period_tau && np < max_periods) period_tau[np] = tau;
     ++np;
-    int rc = local_steps(h, steps, row_offset_host + k * lay.m, loss_dev ? loss_dev + k * lay.m : nullptr);
+    // the period's local steps and its averaging step (the last step's update launch forms the average where it can)
+    int rc = local_steps(h, steps, row_offset_host + k * lay.m, loss_dev ? loss_dev + k * lay.m : nullptr, true);
     if (rc != LS_OK) return rc;
     k += steps;
-    rc = average(h);
-    if (rc != LS_OK) return rc;
     bool decide = interval > 0 && k >= next_interval * (int64_t)interval;
     double elapsed_ms = 0.0;
     if (timed) {

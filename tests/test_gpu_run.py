@@ -323,3 +323,54 @@ def test_wall_clock_intervals():
         last = int(ms // T0)
     assert sum(min(t, K) for t in out["taus"]) >= K
     eng.close()
+
+
+@pytest.mark.parametrize("dims,dtype,m,B,mu", [
+    ((256, 128, 128, 10), "fp32", 3, 128, 0.9),        # fp32 tensor-core layers, one tile per layer and replica
+    ((384, 256, 256, 10), "fp32", 4, 128, 0.0),        # no momentum buffers
+    ((256, 256, 128, 10), "bf16", 5, 128, 0.9),        # bf16 with the operand copies
+    ((1024, 1024, 10), "bf16", 3, 256, 0.9),           # more tiles than SMs per replica set: several rounds, strips
+    ((2048, 1280, 10), "bf16", 2, 128, 0.9),           # 160 tiles on 148 CTAs: a whole round and left-over strips
+    ((1536, 1280, 10), "fp32", 2, 128, 0.9),           # the same with fp32 strips (120 tiles: fewer than CTAs ... one round)
+    ((100, 70, 10), "fp32", 3, 32, 0.9),               # no tensor-core layer: nothing to fuse, same call
+])
+def test_period_call_equals_steps_then_average(dims, dtype, m, B, mu):
+    """ls_local_steps_avg (one call per period) against ls_local_steps followed by ls_average, from the same
+    state and batches: every replica's parameters and momentum bit for bit, and all replicas equal (Section 2,
+    PASGD update rule for k mod tau = 0)."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    bf = dtype == "bf16"
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 41, bf16=bf)
+    tau = 3
+    offs = wl.batch_row_offsets(13, tau, m, 1024, B)
+    xd, yd = to_device(X, y, bf16=bf)
+    rng = np.random.default_rng(5)
+    xs = [x1 + 0.01 * rng.standard_normal(x1.size).astype(np.float32) for _ in range(m)]
+    vs = [0.01 * rng.standard_normal(x1.size).astype(np.float32) for _ in range(m)]
+    res = {}
+    for tag in ("fused", "separate"):
+        eng = LocalSGD(m, dims, gemm_dtype=dtype, lr=0.05, momentum=mu, batch=B)
+        eng.bind_dataset(xd, yd)
+        for i in range(m):
+            eng.set_state(i, xs[i], vs[i])
+        if tag == "separate":
+            eng.local_steps(tau, offs)
+            eng.average()
+        else:
+            eng.local_steps(tau, offs, average=True)
+        eng.sync()
+        px, pv = eng.get_all()
+        F = eng.eval_loss(m - 1, 0, 2 * B)          # reads the operand copies of the last replica (bf16 models)
+        res[tag] = (np.array(px), np.array(pv), F)
+        eng.close()
+    fx, fv, fF = res["fused"]
+    for tag in ("separate",):
+        ox, ov, oF = res[tag]
+        assert np.array_equal(fx.view(np.uint32), ox.view(np.uint32)), tag
+        assert np.array_equal(fv.view(np.uint32), ov.view(np.uint32)), tag
+        assert fF == oF, tag
+    assert all(np.array_equal(fx[0], fx[i]) for i in range(m))
+    if mu != 0.0:        # without momentum the buffers are neither used nor averaged
+        assert all(np.array_equal(fv[0], fv[i]) for i in range(m))
+
