@@ -195,23 +195,13 @@ head_fwd_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row_off,
 
 // The same layer for wide inputs (K in the thousands): one CTA = 16 mini-batch rows, warp w owns rows 2w and
 // 2w + 1 over all of K, so the C x K weights are read once per 16 rows instead of once per 4 and the CTAs
-// of the bf16 MLP's output layer (16 per replica) fit the GPU in one wave.  A lane takes 8 consecutive
-// elements of K per trip; every load of a trip is issued before its first product.
+// of the bf16 MLP's output layer (16 per replica) fit the GPU in one wave.  The weights of the replica are
+// copied to shared memory with one batch of asynchronous copies (when they fit), and a lane requests its
+// elements of eight 128-element slices of both rows before the first product: the kernel costs about two
+// memory round trips.  A lane takes elements [128 u + 4 lane, + 4) of slice u.
 constexpr int kWideRows = 16;
-
-__device__ __forceinline__ void load8(const float* p, float (&r)[8]) {
-  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
-  r[0] = a.x; r[1] = a.y; r[2] = a.z; r[3] = a.w; r[4] = b.x; r[5] = b.y; r[6] = b.z; r[7] = b.w;
-}
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&r)[8]) {
-  const uint4 u = *reinterpret_cast<const uint4*>(p);
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    r[2 * i] = __uint_as_float(w[i] << 16);               // a bf16 is the upper half of an fp32
-    r[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
+constexpr int kWideBatch = 8;             // slices of K requested together
+constexpr int kWideSmemMax = 100 * 1024;  // weights staged in shared memory up to this size (two CTAs per SM)
 
 template <typename TA, int CT>
 __global__ void __launch_bounds__(kThreads, 2)
@@ -219,7 +209,8 @@ head_fwd_wide_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row
                      int64_t w_gstride, const float* __restrict__ bias, const void* __restrict__ y,
                      const int64_t* __restrict__ y_row_off, float* __restrict__ dZ, float* __restrict__ row_loss,
                      float* __restrict__ loss_out, unsigned int* __restrict__ counters, int B, int K, int kind,
-                     int defer_loss) {
+                     int defer_loss, int stage_w) {
+  extern __shared__ float wsm[];           // [CT][K] when stage_w
   __shared__ unsigned int is_last;
   __shared__ float red[kThreads];
   grid_dep_wait();
@@ -229,6 +220,12 @@ head_fwd_wide_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row
   const int b0 = blockIdx.x * kWideRows + 2 * warp;          // this warp's first row
   const TA* Ag = A + ((a_row_off ? a_row_off[g] : (int64_t)g * B) + b0) * K;
   const float* Wg = W + (int64_t)g * w_gstride;
+  if (stage_w) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(wsm));
+    for (int i = threadIdx.x; i < CT * K / 4; i += kThreads)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * 16), "l"(Wg + i * 4) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
   const float bz = (bias != nullptr && lane < CT) ? bias[(int64_t)g * w_gstride + lane] : 0.f;
   int label[2] = {0, 0};
   float target[2] = {0.f, 0.f};
@@ -245,18 +242,34 @@ head_fwd_wide_kernel(const TA* __restrict__ A, const int64_t* __restrict__ a_row
   for (int r = 0; r < 2; ++r)
 #pragma unroll
     for (int c = 0; c < CT; ++c) acc[r][c] = 0.f;
-  for (int k = lane * 8; k < K; k += 256) {
-    float a[2][8], w[CT][8];
+  const int slices = K / 128;
+  for (int u0 = 0; u0 < slices; u0 += kWideBatch) {
+    float a[kWideBatch][2][4];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) load8(Ag + (int64_t)r * K + k, a[r]);
+    for (int u = 0; u < kWideBatch; ++u)
 #pragma unroll
-    for (int c = 0; c < CT; ++c) load8(Wg + (int64_t)c * K + k, w[c]);
+      for (int r = 0; r < 2; ++r) {
+        if (u0 + u < slices) load4(Ag + (int64_t)r * K + (u0 + u) * 128 + lane * 4, a[u][r]);
+        else a[u][r][0] = a[u][r][1] = a[u][r][2] = a[u][r][3] = 0.f;
+      }
+    if (u0 == 0 && stage_w) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+    }
 #pragma unroll
-    for (int c = 0; c < CT; ++c)
+    for (int u = 0; u < kWideBatch; ++u) {
+      if (u0 + u < slices) {
+        const int k = (u0 + u) * 128 + lane * 4;
 #pragma unroll
-      for (int r = 0; r < 2; ++r)
+        for (int c = 0; c < CT; ++c) {
+          float w[4];
+          load4((stage_w ? wsm : Wg) + (int64_t)c * K + k, w);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[r][c] = fmaf(a[r][e], w[c][e], acc[r][c]);
+          for (int r = 0; r < 2; ++r)
+            acc[r][c] = fmaf(a[u][r][3], w[3], fmaf(a[u][r][2], w[2], fmaf(a[u][r][1], w[1], fmaf(a[u][r][0], w[0], acc[r][c]))));
+        }
+      }
+    }
   }
   // lane sums, then lane c keeps class c of both rows
   float z[2] = {0.f, 0.f};
@@ -578,16 +591,25 @@ bool head_shape_ok(int B, int C) { return C >= 1 && C <= CMAX && B >= 1 && (size
 
 template <typename TA, int CT>
 int launch_head_fwd_wide(const HeadFwdArgs& a, cudaStream_t st) {
+  auto kern = head_fwd_wide_kernel<TA, CT>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideSmemMax);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const size_t wbytes = (size_t)CT * a.K * sizeof(float);
+  const int stage_w = wbytes <= (size_t)kWideSmemMax ? 1 : 0;
   dim3 grid((unsigned)(a.B / kWideRows), (unsigned)a.groups);
-  return launch_dep(head_fwd_wide_kernel<TA, CT>, grid, dim3(kThreads), 0, st, 1, static_cast<const TA*>(a.A),
+  return launch_dep(kern, grid, dim3(kThreads), stage_w ? wbytes : 0, st, 1, static_cast<const TA*>(a.A),
                     a.a_row_off, a.W, a.w_gstride, a.bias, a.y, a.y_row_off, a.dZ, a.row_loss, a.loss_out, a.counters,
-                    a.B, a.K, a.loss_kind, a.defer_loss);
+                    a.B, a.K, a.loss_kind, a.defer_loss, stage_w);
 }
 
 int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches) {
   if (launches) ++*launches;
   // wide inputs with enough rows to fill the GPU 16 at a time: the kernel that reads W once per 16 rows
-  if ((a.C == 10 || a.C == 1) && a.K >= 1024 && a.K % 8 == 0 && a.B % kWideRows == 0 &&
+  if ((a.C == 10 || a.C == 1) && a.K >= 1024 && a.K % 128 == 0 && a.B % kWideRows == 0 &&
       (int64_t)(a.B / kWideRows) * a.groups >= 64 && reinterpret_cast<uintptr_t>(a.A) % 16 == 0 &&
       reinterpret_cast<uintptr_t>(a.W) % 16 == 0 && a.w_gstride % 4 == 0) {
     if (a_bf16) return a.C == 10 ? launch_head_fwd_wide<__nv_bfloat16, 10>(a, st) : launch_head_fwd_wide<__nv_bfloat16, 1>(a, st);
