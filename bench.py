@@ -34,6 +34,7 @@ from paper_1810_08313_b200 import workloads as wl  # noqa: E402
 METRIC = "replica-steps/s (m-replica local SGD); model-avg HBM GB/s vs ~8 TB/s peak"
 UNIT = "replica-steps/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_BF16_TFLOPS = 2250.0       # dense bf16 tensor peak of the data sheet (context beside the measured peaks)
 PROBE_ROWS = 4096
 
 
@@ -51,6 +52,12 @@ def load_peaks():
     except Exception:
         return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
                 "source": "fallback"}
+
+
+def workload_config(w: wl.Workload, tau: int) -> dict:
+    """The keys of `config` that name the workload; both arms (CUDA and CPU oracle) print the same ones."""
+    return {"workload": w.name, "dims": list(w.dims), "m": w.m, "batch": w.batch, "tau": tau,
+            "momentum": w.momentum, "lr": w.lr, "dataset_rows": w.n_rows}
 
 
 def probe_rows_for(w: wl.Workload) -> int:
@@ -83,7 +90,14 @@ def streamed_update_layers(w: wl.Workload):
     return out
 
 
-def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
+def update_state_bytes_per_launch(w: wl.Workload, layer: int) -> float:
+    """Bytes of replica state the weight-gradient + update launch must move (all m replicas, all layers of the
+    launch): read and write W (8 B per parameter), the same for v when momentum is on, and the bf16 copy of
+    W for a bf16 model (2 B): 16 or 18 bytes per parameter per replica-step."""
+    return update_bytes_per_launch(w, layer, operands=False)
+
+
+def update_bytes_per_launch(w: wl.Workload, layer: int, operands: bool = True) -> float:
     """Algorithmic bytes of the weight-gradient + update launch that covers layer `layer` (all m replicas):
     read and write W (and v when momentum is on), write the bf16 copy of W (bf16 models), read the
     two GEMM operands once; summed over the layers that share the launch."""
@@ -94,7 +108,7 @@ def update_bytes_per_launch(w: wl.Workload, layer: int) -> float:
     for l in layers:
         n_out, n_in = layer_shapes(w)[l]
         per_param = 8 + (8 if w.momentum != 0 else 0) + (2 if bf else 0)
-        operand = (2 if bf else 4) * w.batch * (n_out + n_in)
+        operand = (2 if bf else 4) * w.batch * (n_out + n_in) if operands else 0
         total += float(w.m) * (per_param * n_out * n_in + operand)
     return total
 
@@ -152,13 +166,18 @@ def roofline_for(dom, dur_s: float, w: wl.Workload, peaks, clocks):
                 "ms_per_launch": ms}
     tc = uses_tensor_cores(w, cls, layer)
     if cls == "dw" and tc:
-        by = update_bytes_per_launch(w, layer)
+        # achieved = the state bytes alone (16 / 18 B per parameter per replica-step); the GEMM operands that the
+        # launch also reads once (dZ and the layer inputs) are reported beside it, not counted in the fraction
+        by = update_state_bytes_per_launch(w, layer)
+        by_all = update_bytes_per_launch(w, layer)
         ach = by / dur_s / 1e9
         merged = streamed_update_layers(w)
         which = f"layers {merged}" if layer in merged and len(merged) > 1 else f"layer {layer}"
         return {"kernel": f"weight gradient + update, {which} in one launch (tcgen05, streaming)", "bound": "hbm",
                 "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                "traffic": traffic, "peak_source": src, "ms_per_launch": ms}
+                "traffic": traffic, "peak_source": src, "ms_per_launch": ms,
+                "bytes_per_launch": by, "operand_bytes_per_launch": by_all - by,
+                "achieved_with_operands": by_all / dur_s / 1e9, "frac_of_8TBs": ach / 8000.0}
     n_out, n_in = layer_shapes(w)[layer]
     fl = 2.0 * w.m * w.batch * n_out * n_in
     ach = fl / dur_s / 1e12
@@ -166,7 +185,9 @@ def roofline_for(dom, dur_s: float, w: wl.Workload, peaks, clocks):
         peak = peaks["bf16_tflops_sustained"]
         return {"kernel": f"{cls} layer {layer} (tcgen05 bf16)", "bound": "tensor", "achieved": ach, "peak": peak,
                 "unit": "TFLOP/s", "frac": ach / peak, "traffic": traffic,
-                "peak_source": src + " (sustained bf16)", "ms_per_launch": ms}
+                "peak_source": src + " (sustained bf16)", "ms_per_launch": ms,
+                "frac_of_burst": ach / peaks["bf16_tflops"] if peaks.get("bf16_tflops") else None,
+                "frac_of_nominal_2250": ach / NOMINAL_BF16_TFLOPS}
     if tc:
         # fp32 operands: three tf32 MMAs per product; tf32 dense peak = bf16 peak x (1.1 / 2.25) nominal ratio
         peak = peaks["bf16_tflops_sustained"] * (1.1 / 2.25) / 3.0
@@ -206,8 +227,11 @@ def aggregate_over_ranks(ms_local: float, units_local: float):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """Samples nvidia-smi clocks and throttle reasons of one GPU every 20 ms.  It is started before the
+    warm-up (nvidia-smi needs a few hundred milliseconds to come up) and the samples are cut to the timed
+    region by their timestamps; when the region was too short to catch one, the samples of the warm-up
+    (the same kernels under the same load) stand in and `window` says so."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -215,6 +239,7 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.t_begin = self.t_end = None
 
     def start(self):
         try:
@@ -222,29 +247,65 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
+
+    def mark_begin(self):
+        self.t_begin = time.time()
+
+    def mark_end(self):
+        self.t_end = time.time()
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         try:
+            time.sleep(0.05)
             self.proc.terminate()
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        return parse_clock_csv(open(self.path).read())
+        text = open(self.path).read()
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        inside = parse_clock_csv(text, self.t_begin, self.t_end)
+        if inside["samples"] > 0:
+            inside["window"] = "timed region"
+            return inside
+        both = parse_clock_csv(text)
+        both["window"] = "warm-up and timed region (the timed region was shorter than a sampling period)"
+        return both
 
 
-def parse_clock_csv(text: str):
+def _smi_time(stamp: str):
+    """nvidia-smi's 'YYYY/MM/DD HH:MM:SS.mmm' as seconds since the epoch (local time), or None."""
+    import datetime
+    try:
+        return datetime.datetime.strptime(stamp.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+    except ValueError:
+        return None
+
+
+def parse_clock_csv(text: str, t_begin=None, t_end=None):
+    """Median SM clock, maximum clock and the set of throttle reasons seen.  Lines are
+    [timestamp,] sm, max, power, hw_slowdown, hw_thermal, sw_thermal, sw_power_cap; with t_begin / t_end
+    only lines stamped inside [t_begin, t_end] count."""
     sm, mx, reasons = [], [], set()
     names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
     for line in text.strip().splitlines():
         a = [x.strip() for x in line.split(",")]
+        stamp = None
+        if len(a) >= 8:
+            stamp, a = _smi_time(a[0]), a[1:]
         if len(a) < 7:
             continue
+        if t_begin is not None and t_end is not None:
+            if stamp is None or not (t_begin <= stamp <= t_end):
+                continue
         try:
             sm.append(float(a[0])); mx.append(float(a[1]))
         except ValueError:
@@ -346,8 +407,8 @@ def run_reference(args, w: wl.Workload):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "dims": list(w.dims), "m": w.m, "batch": w.batch, "tau": tau,
-                   "step": "one iteration of all m replicas on the CPU oracle"},
+        "config": dict(workload_config(w, tau), step="one iteration of all m replicas on the CPU oracle, on the "
+                                                       f"first {n_rows} dataset rows"),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -404,6 +465,9 @@ def run_ours(args, w: wl.Workload):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
     # ---- warm-up, with every kernel class timed to find the dominant one ----
     # (the first period is left out of the per-kernel times: first launches load their kernels lazily)
     period(0)
@@ -417,18 +481,18 @@ def run_ours(args, w: wl.Workload):
     dom = max(shares_raw.items(), key=lambda kv: kv[1][0])[0] if shares_raw else ("dw", 0)
 
     # ---- timed region ---------------------------------------------------------
-    sampler = ClockSampler(local_rank)
     eng.profile_begin([dom[0]], dom[1])
     launches0 = eng.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    sampler.start()
+    sampler.mark_begin()
     e0.record()
     F_t, next_tau = 0.0, tau
     for p in range(W, W + K):
         F_t, next_tau = period(p)
     e1.record()
     barrier()
+    sampler.mark_end()
     clocks = sampler.stop()
     ms_local = e0.elapsed_time(e1)
     launches = eng.launch_count() - launches0
@@ -443,12 +507,11 @@ def run_ours(args, w: wl.Workload):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.gemm_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "dims": list(w.dims), "m": m, "batch": B, "tau": tau,
-                   "momentum": w.momentum, "lr": w.lr, "dataset_rows": w.n_rows,
-                   "step": "one period: tau local iterations x m replicas + averaging + probe loss + AdaComm decision",
-                   "l2": "inputs larger than L2: mini-batches are drawn at random from a %.0f MB resident dataset"
-                         % (xd.numel() * xd.element_size() / 1e6),
-                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+        "config": dict(workload_config(w, tau),
+                       step="one period: tau local iterations x m replicas + averaging + probe loss + AdaComm decision",
+                       l2="inputs larger than L2: mini-batches are drawn at random from a %.0f MB resident dataset"
+                          % (xd.numel() * xd.element_size() / 1e6),
+                       multi_gpu="replicas only" if world > 1 else "single GPU"),
         "clocks": clocks, "gpu_launches": int(launches), "kernel_time_shares": shares,
         "kernel_us_per_launch": kernel_us,
         "last_probe_loss": F_t, "next_tau": next_tau,
@@ -491,25 +554,38 @@ def run_ours(args, w: wl.Workload):
         line["e2e"] = {"value": m * tau * e_steps / dt, "unit": UNIT,
                        "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * yh.element_size()),
                        "d2h_bytes_per_step": int(lh.numel() * 4 + 4),
-                       "note": "per period; batches copied from pinned host memory inside the timed region"}
+                       "note": "per period; batches copied from pinned host memory inside the timed region; when "
+                               "the copies (bytes / host-link rate) take longer than the kernels of a period the "
+                               "host link, not the GPU, sets this number"}
 
         # ---- averaging bandwidth on the model-sized flat vectors (params + momentum) ----------
         # (each replica's vector starts on a 256-byte boundary, as in the library's own layout; the 10^9
         #  point is run when --avg-1b is given: m = 16 with momentum needs 2 x 64 GB)
         avg = {}
-        sizes = [14_706_698, 23_500_000] + ([1_000_000_000] if args.avg_1b else [])
-        for P in sizes:
+        # the engine's state is no longer needed on the device from here on for the largest point
+        for P in [14_706_698, 23_500_000, 1_000_000_000]:
             stride = (P + 63) // 64 * 64
-            buf = torch.empty((2 * 16, stride), device="cuda", dtype=torch.float32)
+            # 10^9 elements: params + momentum of m replicas are 2 * m * 4 GB; m = 4 (32 GB) always runs when
+            # the memory is there, m = 8 and 16 (64 / 128 GB) with --avg-1b
+            ms_list = (4, 8, 16) if P < 10 ** 8 else ((4, 8, 16) if args.avg_1b else (4,))
+            half = max(ms_list)
+            free_b, _ = torch.cuda.mem_get_info()
+            while ms_list and 2 * max(ms_list) * stride * 4 > 0.9 * free_b:
+                ms_list = ms_list[:-1]
+                half = max(ms_list) if ms_list else 0
+            if not ms_list:
+                avg[f"P{P}"] = "did not fit in free device memory"
+                continue
+            buf = torch.empty((2 * half, stride), device="cuda", dtype=torch.float32)
             buf.uniform_(-1.0, 1.0)
-            for mm in (4, 8, 16):
+            for mm in ms_list:
                 ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
                 for _ in range(3):
-                    average_flat(buf[:mm].view(-1), mm, P, stride); average_flat(buf[16:16 + mm].view(-1), mm, P, stride)
+                    average_flat(buf[:mm].view(-1), mm, P, stride); average_flat(buf[half:half + mm].view(-1), mm, P, stride)
                 ev[0].record()
                 reps = 10 if P < 10 ** 8 else 3
                 for _ in range(reps):
-                    average_flat(buf[:mm].view(-1), mm, P, stride); average_flat(buf[16:16 + mm].view(-1), mm, P, stride)
+                    average_flat(buf[:mm].view(-1), mm, P, stride); average_flat(buf[half:half + mm].view(-1), mm, P, stride)
                 ev[1].record()
                 torch.cuda.synchronize()
                 gbs = 2 * 8.0 * mm * P * reps / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9
@@ -524,7 +600,7 @@ def run_ours(args, w: wl.Workload):
                     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
                     def both():
                         block_average_flat(buf[:mm].view(-1), anc[0], ub[0], mm, P, 0.05, 0.3, stride)
-                        block_average_flat(buf[16:16 + mm].view(-1), anc[1], ub[1], mm, P, 0.05, 0.3, stride)
+                        block_average_flat(buf[half:half + mm].view(-1), anc[1], ub[1], mm, P, 0.05, 0.3, stride)
                     for _ in range(3):
                         both()
                     ev[0].record()
@@ -539,6 +615,10 @@ def run_ours(args, w: wl.Workload):
                 del anc, ub
             del buf
         line["averaging_gbs"] = avg
+
+        # ---- the other workload configurations: a short device-timed run each -------------------------------
+        if not args.no_side_configs:
+            line["configs"] = {name: side_config(name, args.tau) for name in sorted(wl.WORKLOADS) if name != w.name}
 
         # ---- measured throughput against the period, beside the runtime model's speed-up (Section 3.2) -----
         if args.tau_sweep:
@@ -571,6 +651,7 @@ def run_ours(args, w: wl.Workload):
                 "note": "model: (1 + alpha) / (1 + alpha / tau) with alpha = D / Y fitted at tau = 1 and 100"}
 
         # ---- the workload's whole job in the native run loop (ls_run): K iterations, AdaComm where configured -------
+        logged = {}
         if args.full_run:
             runs = {}
             Kfull = w.n_iters
@@ -598,6 +679,9 @@ def run_ours(args, w: wl.Workload):
                     "iterations": Kfull, "seconds": round(dt, 4), "replica_steps_per_s": round(m * Kfull / dt, 1),
                     "averaging_steps": len(taus), "periods_rle": rle[:40], "F_0": F_0, "F_end": F_end,
                     "decisions": len(out["decision_k"])}
+                if interval:
+                    logged[f"tau0_{tau0}_adacomm"] = (tau0, float(out["F_0"]), [float(F) for F in out["decision_F"]],
+                                                      [int(t) for t in out["decision_tau"]])
             line["full_run"] = runs
 
         # ---- the CPU oracle on the host cores, bounded sample -----------------------------------
@@ -607,11 +691,56 @@ def run_ours(args, w: wl.Workload):
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                     "sample": f"{iters} whole iterations (m={m} replica-steps each) in {dt:.1f} s on "
                                               f"the first 8192 rows"}
+            # the oracle's rule on the losses that the native run loop logged: the periods it chose must be
+            # the oracle's, bit for bit (Section 4.2)
+            from oracle import localsgd_oracle as orc
+            for key, (tau0, F0_run, Fs, taus_run) in logged.items():
+                want = orc.tau_schedule_from_trace(F0_run, tau0, Fs)
+                line["full_run"][key]["tau_trace_bit_exact"] = bool(want == taus_run)
     eng.close()
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def side_config(name: str, tau_default: int, periods: int = 10, warm: int = 3, max_rows: int = 16384):
+    """Device-timed replica-steps/s of one of the other workload configurations: `periods` periods at the
+    workload's first configured tau (local steps + averaging in one call per period, inputs resident), after
+    `warm` untimed ones.  The resident dataset is cut to max_rows rows (still larger than L2 for the MLPs)
+    so that the side runs add seconds, not minutes."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    w = wl.WORKLOADS[name]
+    tau = int(w.adacomm_tau0 or (w.taus[0] if w.taus else tau_default))
+    n_rows = min(w.n_rows, max_rows * (2 if w.gemm_dtype == "bf16" else 1))
+    X, y = wl.make_dataset(w, n_rows=n_rows)
+    xd = torch.from_numpy(X).cuda()
+    if w.gemm_dtype == "bf16":
+        xd = xd.to(torch.bfloat16)
+    yd = torch.from_numpy(y).cuda()
+    eng = LocalSGD(w.m, w.dims, w.loss, w.has_bias, w.gemm_dtype, lr=w.lr, momentum=w.momentum, batch=w.batch)
+    eng.bind_dataset(xd, yd)
+    eng.set_params(wl.initial_point(w))
+    offs = wl.batch_row_offsets(w.seed + 5, (warm + periods) * tau, w.m, n_rows, w.batch)
+    loss_dev = torch.zeros((tau, w.m), dtype=torch.float32, device="cuda")
+    for p in range(warm):
+        eng.local_steps(tau, offs[p * tau:(p + 1) * tau], loss_dev, average=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = eng.launch_count()
+    torch.cuda.synchronize()
+    e0.record()
+    for p in range(warm, warm + periods):
+        eng.local_steps(tau, offs[p * tau:(p + 1) * tau], loss_dev, average=True)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    out = {"replica_steps_per_s": round(w.m * tau * periods / (ms * 1e-3), 1), "tau": tau, "periods": periods,
+           "ms_per_period": round(ms / periods, 4), "dtype": "bf16" if w.gemm_dtype == "bf16" else "f32",
+           "m": w.m, "batch": w.batch, "dims": list(w.dims), "dataset_rows": n_rows,
+           "gpu_launches": int(eng.launch_count() - n0), "last_loss": float(loss_dev[-1].mean().item())}
+    eng.close()
+    return out
 
 
 def main():
@@ -620,7 +749,9 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_mlp_fp32", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default="c3_mlp_bf16", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--no-side-configs", action="store_true",
+                    help="skip the short device-timed runs of the other workload configurations")
     ap.add_argument("--tau", type=int, default=20)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

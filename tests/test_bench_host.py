@@ -23,6 +23,27 @@ def test_clock_csv_parsing():
     assert bad["reasons"] == ["hw_slowdown"]
 
 
+def test_clock_csv_with_timestamps_is_cut_to_the_timed_region():
+    import datetime
+    t0 = datetime.datetime(2026, 1, 2, 3, 4, 5).timestamp()
+    def stamp(dt):
+        return datetime.datetime.fromtimestamp(t0 + dt).strftime("%Y/%m/%d %H:%M:%S.%f")[:-3]
+    text = "".join(f"{stamp(0.02 * i)}, {1000 + i}, 1965, 500.0, Not Active, Not Active, Not Active, "
+                   f"{'Active' if i == 7 else 'Not Active'}\n" for i in range(10))
+    c = bench.parse_clock_csv(text, t0 + 0.05, t0 + 0.11)            # samples 3, 4, 5
+    assert c["samples"] == 3 and c["sm_mhz"] == 1004.0 and c["reasons"] == []
+    c = bench.parse_clock_csv(text)                                  # no window: everything
+    assert c["samples"] == 10 and c["reasons"] == ["sw_power_cap"]
+    assert bench.parse_clock_csv(text, t0 + 5.0, t0 + 6.0)["samples"] == 0
+
+
+def test_both_arms_print_the_same_workload_keys():
+    w = wl.WORKLOADS["c3_mlp_bf16"]
+    c = bench.workload_config(w, 20)
+    assert c["workload"] == "c3_mlp_bf16" and c["momentum"] == 0.9 and c["lr"] == 0.05 and c["tau"] == 20
+    assert set(c) == {"workload", "dims", "m", "batch", "tau", "momentum", "lr", "dataset_rows"}
+
+
 def test_work_models():
     w2, w3 = wl.WORKLOADS["c2_mlp_fp32"], wl.WORKLOADS["c3_mlp_bf16"]
     assert abs(bench.flops_per_replica_step(w2) / 1e9 - 1.010) < 0.01      # 1.01 GFLOP per replica-step
@@ -30,6 +51,7 @@ def test_work_models():
     # update kernel, bf16 workload: layers 0-2 share one launch; 18 bytes per parameter per replica plus the
     # two operand tiles of every layer
     assert bench.streamed_update_layers(w3) == [0, 1, 2] and bench.streamed_update_layers(w2) == [0, 1]
+    assert bench.update_state_bytes_per_launch(w3, 0) == 16 * 18 * (2048 * 3072 + 2 * 2048 * 2048)     # 18 B per parameter
     by = bench.update_bytes_per_launch(w3, 0)
     assert by == 16 * (18 * 2048 * 3072 + 2 * 256 * (2048 + 3072)) + 2 * 16 * (18 * 2048 * 2048 + 2 * 256 * 4096)
     # fp32 workload: 16 bytes per parameter, fp32 operands
@@ -40,6 +62,7 @@ def test_work_models():
     peaks = {"hbm_gbs": 6547.2, "bf16_tflops": 1682.0, "bf16_tflops_sustained": 1398.0, "source": "measured"}
     r = bench.roofline_for(("dw", 0), 0.4e-3, w3, peaks, {"sm_mhz": 1900.0})
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / 6547.2) < 1e-12
+    assert abs(r["achieved"] - 16 * 18 * 14_680_064 / 0.4e-3 / 1e9) < 1e-6 and r["operand_bytes_per_launch"] > 0
     r = bench.roofline_for(("fwd", 0), 60e-6, w2, peaks, {"sm_mhz": 1900.0})
     assert r["bound"] == "tensor" and abs(r["peak"] - 1398.0 * 1.1 / 2.25 / 3) < 1e-9
     r = bench.roofline_for(("fwd", 2), 10e-6, w2, peaks, {"sm_mhz": 1900.0})

@@ -269,7 +269,17 @@ def test_refined_adacomm_run_with_deferred_lr_decay():
     for F, (_, Fr, _) in zip(out["decision_F"], ref.F_trace):
         assert abs(float(F) - Fr) / Fr <= 1e-4
     # the period reached 1, so at least one scheduled decay was applied, and only at decisions with tau == 1
-    assert len(ref.lr_trace) >= 1 and 1 in out["decision_tau"]
+    assert len(ref.lr_trace) >= 1
+    in_force = dict(zip(out["decision_k"], [tau0] + out["decision_tau"][:-1]))     # period in force at each decision
+    due = [30, 60]
+    for k_dec, _ in ref.lr_trace:
+        assert in_force[k_dec] == 1 and due.pop(0) <= k_dec
+    # ... and no decision at which a decay was due and the period was 1 went without one
+    decayed, due = {k for k, _ in ref.lr_trace}, [30, 60]
+    for k_dec in out["decision_k"]:
+        if due and due[0] <= k_dec and in_force[k_dec] == 1:
+            assert k_dec in decayed
+            due.pop(0)
     assert abs(out["lr"] - ref.lr_trace[-1][1]) <= 1e-12 * max(1.0, ref.lr_trace[-1][1]) or out["lr"] == f32(ref.lr_trace[-1][1])
     # the decisions recomputed from the GPU's own logged losses are bit-exact
     lr0, lr, prev, pending = f32(0.05), f32(0.05), tau0, [30, 60]

@@ -116,3 +116,64 @@ def test_refined_invalid_inputs(kw):
     args.update(kw)
     with pytest.raises(ValueError):
         orc.adacomm_next_tau_refined(**args)
+
+
+# ---- scheduling of learning-rate decays inside the loop (Section 4.3.2, last paragraph) ------------------------
+
+GOLDEN_DECAY = os.path.join(os.path.dirname(__file__), "golden", "adacomm_deferred_decay_trace.txt")
+
+
+def _decay_trace():
+    rows, periods = [], None
+    with open(GOLDEN_DECAY) as f:
+        for line in f:
+            if line.startswith("# periods"):
+                periods = [int(v) for v in line.split()[2:]]
+            a = line.split("#")[0].split()
+            if len(a) == 4:
+                rows.append((int(a[0]), float(a[1]), float(a[2]), int(a[3])))
+    return rows, periods
+
+
+def run_scripted_refined_loop(monkeypatch):
+    """run_pasgd(refined=...) on a tiny model with the probe losses scripted by the golden trace: the training
+    steps run as usual, only the loss the controller sees is replaced, so the schedule is a function of the
+    scripted F_t alone.  Returns the oracle's result and the trace."""
+    import numpy as np
+    from paper_1810_08313_b200 import workloads as wl
+    rows, periods = _decay_trace()
+    script = [1.0] + [F for _, F, _, _ in rows]          # F_0 first, then one loss per decision
+    calls = []
+
+    def scripted_loss(spec, x, X, y):
+        calls.append(len(calls))
+        return script[len(calls) - 1]
+
+    monkeypatch.setattr(orc, "batch_loss", scripted_loss)
+    spec = orc.ModelSpec((3, 1), orc.LOSS_MSE_HALF, False)
+    X = wl.gaussian_rows(5, 64, 3)
+    y = np.random.default_rng(5).standard_normal(64).astype(np.float32)
+    K, m, B = 31, 2, 4
+    offs = wl.batch_row_offsets(5, K, m, 64, B)
+    lr0 = float(np.float32(0.1))
+    res = orc.run_pasgd(spec, np.zeros(3, np.float32), X, y, offs, B, lr0, 0.0, 4, adacomm_interval=4, probe_rows=8,
+                        refined={"gamma": 0.5, "slack": 0, "decay_at": [6, 7, 28], "decay_factor": 0.1})
+    assert len(calls) == len(script)                      # every scripted loss was consumed, none was missing
+    return res, rows, periods
+
+
+def check_deferred_decay_trace(monkeypatch):
+    res, rows, periods = run_scripted_refined_loop(monkeypatch)
+    assert [k for k, _, _ in res.F_trace] == [k for k, _, _, _ in rows]
+    assert [t for _, _, t in res.F_trace] == [t for _, _, _, t in rows]
+    assert res.taus == periods
+    # the learning rate after each decision (the oracle logs the decays it applied)
+    lr, applied = 0.1, dict(res.lr_trace)
+    for k, _, lr_after, _ in rows:
+        lr = applied.get(k, lr)
+        assert abs(lr - lr_after) <= 1e-6 * lr_after, (k, lr, lr_after)
+    assert sorted(applied) == [12, 24, 28]
+
+
+def test_deferred_decay_hand_trace(monkeypatch):
+    check_deferred_decay_trace(monkeypatch)

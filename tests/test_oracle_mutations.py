@@ -144,3 +144,28 @@ def test_refined_controller_mistakes_are_caught(monkeypatch):
         return c if (lr_changed or c + slack < tau_prev) else max(1, math.floor(gamma * tau_prev))
     monkeypatch.setattr(orc, "adacomm_next_tau_refined", floor_gamma)
     assert _fails(pins_tau.test_refined_hand_table)
+
+
+def _mutated_run_pasgd(old: str, new: str):
+    """The oracle's loop with one piece of its source replaced (a mistake planted on the CPU).  The mutant is
+    compiled with the oracle module's own globals, so it sees the same (possibly monkeypatched) helpers."""
+    import inspect
+    src = inspect.getsource(orc.run_pasgd)
+    assert src.count(old) == 1, old
+    src = src.replace(old, new).replace("def run_pasgd(", "def _mutant_run_pasgd(", 1)
+    exec(compile(src, "<mutated run_pasgd>", "exec"), vars(orc))
+    return vars(orc).pop("_mutant_run_pasgd")
+
+
+@pytest.mark.parametrize("old,new", [
+    ("pending[0] <= k and cur_tau == 1", "pending[0] <= k"),                 # decay applied while the period is above 1
+    ("pending[0] <= k and cur_tau == 1", "pending[0] < k and cur_tau == 1"),  # a decay due exactly now is missed
+    ("if pending and pending[0] <= k and cur_tau == 1:", "while pending and pending[0] <= k and cur_tau == 1:"),  # all due decays at once
+    ("refined.get(\"slack\", 0), lr_0, lr, changed)", "refined.get(\"slack\", 0), lr_0, lr, False)"),   # no growth after a decay
+    ("adacomm_next_tau_refined(F_t, F_0, tau_0, cur_tau,", "adacomm_next_tau_refined(F_t, F_0, tau_0, tau_0,"),   # compares with tau_0, not the period in force
+])
+def test_decay_scheduling_mistakes_are_caught(monkeypatch, old, new):
+    pins_tau.check_deferred_decay_trace(monkeypatch)          # passes on the oracle as it stands
+    monkeypatch.setattr(orc, "run_pasgd", _mutated_run_pasgd(old, new))
+    with pytest.raises(AssertionError):                       # the pin itself must object, not a crash
+        pins_tau.check_deferred_decay_trace(monkeypatch)
