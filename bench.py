@@ -712,7 +712,7 @@ def side_config(name: str, tau_default: int, periods: int = 10, warm: int = 3, m
     import torch
     from paper_1810_08313_b200.binding import LocalSGD
     w = wl.WORKLOADS[name]
-    tau = int(w.adacomm_tau0 or (w.taus[0] if w.taus else tau_default))
+    tau = int(w.adacomm_tau0 or (tau_default if tau_default in w.taus else w.taus[0]))
     n_rows = min(w.n_rows, max_rows * (2 if w.gemm_dtype == "bf16" else 1))
     X, y = wl.make_dataset(w, n_rows=n_rows)
     xd = torch.from_numpy(X).cuda()
