@@ -96,8 +96,8 @@ const char* ls_strerror(int code);
 /* P, the number of parameters of one replica.  (x in R^d of Section 2.) */
 int ls_param_count(const ls_model_spec* spec, int64_t* P);
 
-/* Bytes of the caller-allocated state block for m replicas and mini-batches of
- * `batch` rows: parameters, momentum, bf16 weight copies (bf16 models),
+/* Housekeeping (no passage of the paper): bytes of the caller-allocated state block for m replicas and
+ * mini-batches of `batch` rows: parameters, momentum, bf16 weight copies (bf16 models),
  * activation / gradient workspace, staging for host batches. */
 int ls_state_bytes(int m, const ls_model_spec* spec, int batch, size_t* bytes);
 
@@ -114,8 +114,19 @@ int ls_state_bytes(int m, const ls_model_spec* spec, int batch, size_t* bytes);
 int ls_create(ls_handle** h, int m, const ls_model_spec* spec, float lr, float momentum, int batch,
               void* state_dev, size_t state_bytes, void* cuda_stream);
 int ls_destroy(ls_handle* h);
-/* Wait for everything enqueued so far; returns LS_ERR_CUDA if any of it failed. */
+/* Wait for everything enqueued so far; returns LS_ERR_CUDA if any of it failed.
+ * Every wait inside the kernels (on a barrier, on a copy) is bounded; one that runs out makes its kernel
+ * record a code in the state block and return.  ls_sync() and every call that waits for the stream itself
+ * (ls_eval_loss, ls_local_steps_host, the decision points of ls_run / ls_run_refined / ls_run_timed, the state
+ * accessors) then return LS_ERR_DEVICE_TIMEOUT once and clear the record: the results of the launches since the
+ * last successful wait are invalid (restore the replicas with ls_set_state), the handle itself stays usable. */
 int ls_sync(ls_handle* h);
+/* Housekeeping (no passage of the paper): exercises the report path above without touching any other kernel.
+ * Enqueues a one-thread kernel that waits, for at most limit_cycles SM clock ticks (1 .. 2e9), on a barrier on
+ * which nothing ever arrives, gives up, and records the failure like a training kernel would.  The next
+ * ls_sync() returns LS_ERR_DEVICE_TIMEOUT, the one after it LS_OK.  Nothing faults or hangs: the wait is the
+ * bounded one the library uses everywhere. */
+int ls_selftest_wait_timeout(ls_handle* h, int64_t limit_cycles);
 int ls_last_cuda_error(const ls_handle* h);
 int ls_set_lr(ls_handle* h, float lr);
 
@@ -134,7 +145,8 @@ int ls_state_view(ls_handle* h, float** params_dev, float** momentum_dev, int64_
 
 /* ---- data -------------------------------------------------------------- */
 
-/* Bind the training set resident in device memory: x_dev is [n_rows][dims[0]]
+/* Housekeeping (the paper's workers read their partition of the training set, Section 5.1; here it is one
+ * resident array).  Bind the training set resident in device memory: x_dev is [n_rows][dims[0]]
  * row-major, float for LS_GEMM_FP32 and bf16 for LS_GEMM_BF16 (16-byte aligned);
  * y_dev is int32[n_rows] class labels for LS_LOSS_SOFTMAX_CE (each in
  * [0, d_out)) or float[n_rows] targets for LS_LOSS_MSE_HALF.  Borrowed: must

@@ -309,7 +309,7 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
     row_offsets[k][i] is the first dataset row of the mini-batch replica i uses
     at iteration k (k = 0..K-1); the batch is rows [off, off + batch).
 
-    Readings taken where the paper is silent or the scope statement differs:
+    Readings taken where the paper is silent, or where this library departs from it (the momentum buffers):
       * the average is taken on the models *after* the tau-th update;
       * momentum buffers follow `momentum_mode`; the default averages them with
         the parameters (which is what makes tau = 1 equal to synchronous

@@ -77,6 +77,7 @@ def _lib():
         "ls_create": (C.c_int, [P(vp), C.c_int, P(ModelSpec), f32, f32, C.c_int, vp, C.c_size_t, vp]),
         "ls_destroy": (C.c_int, [vp]),
         "ls_sync": (C.c_int, [vp]),
+        "ls_selftest_wait_timeout": (C.c_int, [vp, i64]),
         "ls_last_cuda_error": (C.c_int, [vp]),
         "ls_set_lr": (C.c_int, [vp, f32]),
         "ls_set_params": (C.c_int, [vp, vp]),
@@ -308,6 +309,11 @@ class LocalSGD:
 
     def sync(self):
         _check(self.lib.ls_sync(self.h), "ls_sync")
+
+    def selftest_wait_timeout(self, limit_cycles: int = 2_000_000):
+        """Enqueue the kernel whose bounded wait runs out (ls_selftest_wait_timeout); the next call that waits
+        for the stream raises LsError(LS_ERR_DEVICE_TIMEOUT)."""
+        _check(self.lib.ls_selftest_wait_timeout(self.h, int(limit_cycles)), "ls_selftest_wait_timeout")
 
     def set_lr(self, lr: float):
         _check(self.lib.ls_set_lr(self.h, float(lr)), "ls_set_lr")

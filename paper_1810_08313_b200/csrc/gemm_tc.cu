@@ -993,11 +993,10 @@ template <bool TF32, int BN, bool A_MN, bool B_MN, int EPI, int STAGES, int SPLI
 int launch_one(const TcOperandMaps& mp, const Params& p, int groups, cudaStream_t st) {
   using L = Smem<TF32, BN, STAGES, MT>;
   auto kern = tc_gemm_kernel<TF32, BN, A_MN, B_MN, EPI, STAGES, SPLIT, MT>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(L::kTotal), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   dim3 grid((unsigned)(p.N / BN * SPLIT), (unsigned)(p.M / (BM * MT)), (unsigned)groups);
   return launch_dep(kern, grid, dim3(TF32 ? kThreadsFp32 : kThreadsBf16), L::kTotal, st, SPLIT, *mp.a, *mp.b, p);
@@ -1007,23 +1006,17 @@ template <bool B_MN, int EPI>
 int launch_pair(const TcOperandMaps& mp, const CUtensorMap* c_map, const CUtensorMap* mask_map, const Params& p,
                 int groups, cudaStream_t st) {
   auto kern = tc_gemm_pair_kernel<B_MN, EPI>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPair::kTotal);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(SmemPair::kTotal), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   dim3 grid((unsigned)(p.N / kPairN * 2), (unsigned)(p.M / 256), (unsigned)groups);
   return launch_dep(kern, grid, dim3(kThreadsBf16), SmemPair::kTotal, st, 2, *mp.a, *mp.b, *c_map,
                     mask_map ? *mask_map : *c_map, p);
 }
-// bf16 shapes that the pair kernel covers.  LS_DISABLE_PAIR=1 in the environment keeps every launch on the
-// one-CTA kernels (a diagnostic switch: the tests compare the two).
-bool pair_shape_ok(int M, int N, int K) {
-  const char* e = getenv("LS_DISABLE_PAIR");
-  if (e && e[0] == '1') return false;
-  return M % 256 == 0 && N % kPairN == 0 && K % 64 == 0;
-}
+// bf16 shapes that the pair kernel covers
+bool pair_shape_ok(int M, int N, int K) { return M % 256 == 0 && N % kPairN == 0 && K % 64 == 0; }
 
 // fp32 forward / backward: tile width and K split.  128-wide tiles when N allows; K is split over a
 // cluster while that keeps the grid within one wave of SMs and every slice keeps whole stages.
@@ -1125,7 +1118,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   if (p.head.W != nullptr && !tc_fwd_fuses_head(a.fp32, a.M, a.N, p.head.C)) return cudaErrorInvalidValue;
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, false, EPI_FWD>(a.maps, p, a.groups, st);
-  if (p.head.W == nullptr && a.c_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
+  if (a.allow_pair && p.head.W == nullptr && a.c_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
     return launch_pair<false, EPI_FWD>(a.maps, a.c_map, nullptr, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, false, EPI_FWD, 4>(a.maps, p, a.groups, st);
@@ -1143,7 +1136,7 @@ int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   }
   if (launches) ++*launches;
   if (a.fp32) return launch_fp32<false, true, EPI_DX>(a.maps, p, a.groups, st);
-  if (a.c_map != nullptr && a.act_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
+  if (a.allow_pair && a.c_map != nullptr && a.act_map != nullptr && pair_shape_ok(a.M, a.N, a.K))
     return launch_pair<true, EPI_DX>(a.maps, a.c_map, a.act_map, p, a.groups, st);
   if (a.N % 256 == 0 && a.M % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 3, 1, 2>(a.maps, p, a.groups, st);
   if (a.N % 256 == 0) return launch_one<false, 256, false, true, EPI_DX, 4>(a.maps, p, a.groups, st);

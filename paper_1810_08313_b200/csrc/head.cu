@@ -592,11 +592,10 @@ bool head_shape_ok(int B, int C) { return C >= 1 && C <= CMAX && B >= 1 && (size
 template <typename TA, int CT>
 int launch_head_fwd_wide(const HeadFwdArgs& a, cudaStream_t st) {
   auto kern = head_fwd_wide_kernel<TA, CT>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideSmemMax);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(kWideSmemMax), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   const size_t wbytes = (size_t)CT * a.K * sizeof(float);
   const int stage_w = wbytes <= (size_t)kWideSmemMax ? 1 : 0;
@@ -641,11 +640,10 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
 template <typename TA, int VEC, int CT, bool SLAB>
 int launch_head_bwd_s(const HeadBwdArgs& a, size_t smem, cudaStream_t st) {
   auto kern = head_bwd_kernel<TA, VEC, CT, SLAB>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(112 * 1024), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   constexpr int COLS = 32 * VEC;
   dim3 grid((unsigned)((a.K + COLS - 1) / COLS), (unsigned)a.groups);
@@ -705,6 +703,17 @@ static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScr
 // Device address of the scratch, looked up once per device (index = CUDA device ordinal).
 static StaticScratch* g_scratch_addr[64] = {nullptr};
 
+// What must be fresh at every call: the CTA counters start at zero and chunk c starts at row c * chunk_rows.
+// (Device code names the array directly.)  A kernel rather than host-to-device copies: the call enqueues
+// nothing that reads host memory later.
+__global__ void static_scratch_reset_kernel(int chunks, int chunk_rows) {
+  StaticScratch* sc = reinterpret_cast<StaticScratch*>(g_static_scratch);
+  for (int c = threadIdx.x; c < kStaticMaxChunks; c += blockDim.x) {
+    sc->counters[c] = 0u;
+    if (c < chunks) sc->row_off[c] = (long long)c * chunk_rows;
+  }
+}
+
 }  // namespace
 
 extern "C" int ls_linear_loss_static(const float* W_dev, const float* bias_dev, const float* x_dev, const void* y_dev,
@@ -730,11 +739,8 @@ extern "C" int ls_linear_loss_static(const float* W_dev, const float* bias_dev, 
   StaticScratch* sc = g_scratch_addr[dev];
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   // the counters must start at zero; the first row of every chunk is chunk * chunk_rows
-  if (cudaMemsetAsync(sc->counters, 0, sizeof(sc->counters), st) != cudaSuccess) return LS_ERR_CUDA;
-  long long offs[kStaticMaxChunks];
-  for (int64_t c = 0; c < chunks; ++c) offs[c] = c * (long long)chunk_rows;
-  if (cudaMemcpyAsync(sc->row_off, offs, (size_t)chunks * sizeof(long long), cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return LS_ERR_CUDA;
+  static_scratch_reset_kernel<<<1, 256, 0, st>>>((int)chunks, chunk_rows);
+  if (cudaGetLastError() != cudaSuccess) return LS_ERR_CUDA;
   HeadFwdArgs a;
   a.A = x_dev; a.a_row_off = reinterpret_cast<const int64_t*>(sc->row_off);
   a.W = W_dev; a.w_gstride = 0; a.bias = bias_dev;

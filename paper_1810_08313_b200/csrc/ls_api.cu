@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "ls_internal.h"
+#include "tc_ptx.cuh"
 
 using namespace ls;
 
@@ -141,6 +142,33 @@ static int refresh_shadow(ls_handle* h) {
 // (w_gstride == 0: every group uses the same replica).
 static inline int* err_flag_of(const ls_handle* h) { return reinterpret_cast<int*>(h->state + h->lay.err_off); }
 
+// The device-side error flag after the stream has drained: a bounded wait that ran out inside a kernel left a
+// code there.  Reports it once (LS_ERR_DEVICE_TIMEOUT) and clears it, so that the handle stays usable.
+static int take_device_flag(ls_handle* h, int flag) {
+  if (flag == 0) return LS_OK;
+  LS_CUDA(h, cudaMemsetAsync(err_flag_of(h), 0, sizeof(int), h->stream));
+  LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  return LS_ERR_DEVICE_TIMEOUT;
+}
+static int check_device_flag(ls_handle* h) {
+  int flag = 0;
+  LS_CUDA(h, cudaMemcpyAsync(&flag, err_flag_of(h), sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  return take_device_flag(h, flag);
+}
+
+// A kernel whose only job is to let a bounded wait run out: one thread waits, for at most `limit` clock ticks,
+// on a barrier on which nobody ever arrives, then records the failure in *err_flag and returns, exactly as the
+// tensor-core kernels do when one of their waits gives up.  No tensor memory, no bulk copies, nothing to drain.
+__global__ void wait_timeout_selftest_kernel(int* err_flag, long long limit) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+    if (!ptx::mbar_wait(&bar, 0, limit)) atomicExch(err_flag, 99);
+  }
+}
+
 // x maps: [0] for K-major reads, [1] for MN-major reads of the mini-batch rows
 struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; const CUtensorMap* upd; };
 
@@ -182,6 +210,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       t.c_map = (bf && lay.dims[l + 1] % 8 == 0) ? &h->maps.act[l + 1] : nullptr;
       t.M = lay.batch; t.N = lay.dims[l + 1]; t.K = lay.dims[l]; t.groups = groups; t.relu = 1;
       t.err_flag = err_flag_of(h);
+      t.allow_pair = h->allow_pair;
       t.head = TcHead{};
       const bool fuse_head = l == lay.L - 2 && lay.headpart_off != 0 && groups <= lay.m;
       if (fuse_head) {
@@ -287,6 +316,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
         bias_done[l - 1] = true;
       }
       t.err_flag = err_flag_of(h);
+      t.allow_pair = h->allow_pair;
       ProfScope ps(h, LS_K_DX, l);
       LS_CUDA(h, launch_tc_dx(t, h->stream, &h->launches));
     } else if (l > 0) {
@@ -314,6 +344,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.lr = h->lr; t.mu = h->mu;
       t.err_flag = err_flag_of(h);
       t.layer = l;
+      t.allow_pair = h->allow_pair;
     } else if (tc_shape_ok(!bf, lay.dims[l + 1], lay.dims[l], lay.batch)) {
       TcDwArgs t;
       t.fp32 = !bf;
@@ -409,7 +440,10 @@ static int eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_ro
     if (rc != LS_OK) return rc;
   }
   LS_CUDA(h, cudaMemcpyAsync(h->pinned, loss_dev, (size_t)chunks * 4, cudaMemcpyDeviceToHost, h->stream));
+  int* flag_host = reinterpret_cast<int*>(h->pinned + kEvalCap);
+  LS_CUDA(h, cudaMemcpyAsync(flag_host, err_flag_of(h), sizeof(int), cudaMemcpyDeviceToHost, h->stream));
   LS_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (int rc = take_device_flag(h, *flag_host)) return rc;      // a wait ran out: the losses are not valid
   double s = 0.0;
   for (int64_t c = 0; c < chunks; ++c) s += (double)h->pinned[c];
   *F_host = (float)(s / (double)chunks);
@@ -502,12 +536,13 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
   h->mu = momentum;
   h->state = static_cast<char*>(state_dev);
   h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->allow_pair = pair_kernels_enabled();
   int e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
   for (int s = 0; s < 2 && e == cudaSuccess; ++s) {
     e = cudaEventCreateWithFlags(&h->ev_copied[s], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_consumed[s], cudaEventDisableTiming);
   }
-  if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&h->pinned), (size_t)kEvalCap * 4);
+  if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&h->pinned), (size_t)(kEvalCap + 16) * 4);
   // parameters, momentum, workspace start at zero; the staging row offsets are g*batch
   if (e == cudaSuccess) e = cudaMemsetAsync(h->state, 0, lay.total, h->stream);
   if (e == cudaSuccess) {
@@ -588,10 +623,7 @@ int ls_sync(ls_handle* h) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   LS_CUDA(h, cudaStreamSynchronize(h->stream));
   LS_CUDA(h, cudaGetLastError());
-  int flag = 0;
-  LS_CUDA(h, cudaMemcpy(&flag, err_flag_of(h), sizeof(int), cudaMemcpyDeviceToHost));
-  if (flag != 0) return LS_ERR_DEVICE_TIMEOUT;
-  return LS_OK;
+  return check_device_flag(h);
 }
 
 int ls_last_cuda_error(const ls_handle* h) { return ok_handle(h) ? h->last_cuda : LS_ERR_BAD_HANDLE; }
@@ -759,7 +791,7 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
     }
     LS_CUDA(h, cudaMemcpyAsync(loss_host + (int64_t)s0 * lay.m, loss_stage, (size_t)n * lay.m * 4,
                                cudaMemcpyDeviceToHost, h->stream));
-    LS_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (int rc = check_device_flag(h)) return rc;        // waits for the stream; a wait that ran out ends the call
   }
   return LS_OK;
 }
@@ -861,7 +893,7 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
     const int steps = (int)((K - k < tau) ? K - k : tau);
     if (period_tau && np < max_periods) period_tau[np] = tau;
     ++np;
-    // the period's local steps and its averaging step (the last step's update launch forms the average where it can)
+    // the period's local steps, then its averaging step
     int rc = local_steps(h, steps, row_offset_host + k * lay.m, loss_dev ? loss_dev + k * lay.m : nullptr, true);
     if (rc != LS_OK) return rc;
     k += steps;
@@ -869,7 +901,7 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
     double elapsed_ms = 0.0;
     if (timed) {
       // wall-clock intervals (Section 4): the averaging step has to be over before the clock is read
-      LS_CUDA(h, cudaStreamSynchronize(h->stream));
+      if (int frc = check_device_flag(h)) return frc;      // waits for the stream
       elapsed_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_start).count();
       decide = t0_ms <= 0.0 || elapsed_ms >= (double)next_interval * t0_ms;
     }
@@ -910,6 +942,15 @@ static int run_loop(ls_handle* h, int64_t K, int tau_0, int interval, int64_t pr
 }
 
 extern "C" {
+
+int ls_selftest_wait_timeout(ls_handle* h, int64_t limit_cycles) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (limit_cycles < 1 || limit_cycles > 2000000000ll) return LS_ERR_INVALID_ARG;
+  wait_timeout_selftest_kernel<<<1, 32, 0, h->stream>>>(err_flag_of(h), (long long)limit_cycles);
+  ++h->launches;
+  LS_CUDA(h, cudaGetLastError());
+  return LS_OK;
+}
 
 int ls_get_lr(const ls_handle* h, float* lr) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;

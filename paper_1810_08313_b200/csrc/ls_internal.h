@@ -88,6 +88,7 @@ struct ls_handle {
   const void* y_dev;
   int64_t n_rows;
   int last_cuda;
+  bool allow_pair;        // CTA-pair kernels enabled (see pair_kernels_enabled)
   int64_t launches;
   float* pinned;          // small pinned host scratch (eval losses)
   // per-kernel timing (ls_profile_begin / ls_profile_end)
@@ -142,6 +143,27 @@ inline cudaError_t launch_dep(void (*kern)(P...), dim3 grid, dim3 block, size_t 
   return cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...);
 }
 #endif
+
+// LS_DISABLE_PAIR=1 in the environment keeps every launch of a handle on the one-CTA tensor-core kernels (a
+// diagnostic switch; read once, when the handle is created, and carried in the launch arguments).
+inline bool pair_kernels_enabled() {
+  const char* e = getenv("LS_DISABLE_PAIR");
+  return !(e && e[0] == '1');
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device attribute of a kernel: set it once per device
+// (`done` is a per-kernel bit mask over the device ordinals, kept by the caller in a function-local static).
+template <typename K>
+inline cudaError_t allow_dynamic_smem(K kern, int bytes, uint64_t* done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (*done & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) *done |= bit;
+  return e;
+}
 
 inline float* params_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.params_off); }
 inline float* mom_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.mom_off); }
@@ -286,6 +308,7 @@ struct TcFwdArgs {
   TcHead head;
   int M, N, K, groups, relu;
   int* err_flag;
+  bool allow_pair;           // CTA-pair kernels may be chosen
 };
 struct TcDxArgs {
   TcOperandMaps maps;        // a: dZ_l [groups*M][K]; b: weights
@@ -298,6 +321,7 @@ struct TcDxArgs {
   // from the column sums of C inside the kernel when tc_dx_fuses_bias(); else null
   float* bias; float* vbias; int64_t bias_gstride; float lr, mu;
   int* err_flag;
+  bool allow_pair;
 };
 // whether launch_tc_dx can also apply the bias update (every output tile holds all M rows)
 bool tc_dx_fuses_bias(bool fp32, int M, int N);
@@ -322,6 +346,7 @@ struct TcUpdateArgs {
   float lr, mu;
   int* err_flag;
   int layer;                 // which layer of the model this is (bookkeeping of the caller)
+  bool allow_pair;
 };
 bool tc_update_shape_ok(bool fp32, int M, int N, int B);
 int tc_update_max_layers();

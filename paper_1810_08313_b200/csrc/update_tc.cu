@@ -653,11 +653,10 @@ template <bool TF32, int STAGES, int R, int KS>
 int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   using L = USmem<TF32, STAGES, R, KS>;
   auto kern = tc_update_kernel<TF32, STAGES, R, KS>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(L::kTotal), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   const TcUpdateArgs& a0 = layers[0];
   UParams p{};
@@ -694,11 +693,10 @@ template <int R, int KS>
 int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   using L = USmem<false, 1, R, KS>;
   auto kern = tc_update_pair_kernel<R, KS>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+  static uint64_t configured = 0;        // one bit per device
+  {
+    cudaError_t e = allow_dynamic_smem(kern, (int)(L::kTotal), &configured);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   const TcUpdateArgs& a0 = layers[0];
   PParams p{};
@@ -744,9 +742,7 @@ int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t
   if (launches) ++*launches;
   if (layers[0].fp32) return launch_update<true, 5, 4, kRowsFp32>(layers, n, st);
   // bf16 layers that are multiples of 256 in both directions: the CTA-pair kernel
-  // (LS_DISABLE_PAIR=1 in the environment: one-CTA kernel, a diagnostic switch)
-  const char* e = getenv("LS_DISABLE_PAIR");
-  bool pair = !(e && e[0] == '1');
+  bool pair = layers[0].allow_pair;
   for (int i = 0; i < n; ++i) pair = pair && layers[i].M % 256 == 0 && layers[i].N % PN == 0;
   if (pair) return launch_update_pair<6, kRowsBf16>(layers, n, st);
   return launch_update<false, 1, 6, kRowsBf16>(layers, n, st);

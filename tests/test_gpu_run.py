@@ -384,3 +384,53 @@ def test_period_call_equals_steps_then_average(dims, dtype, m, B, mu):
     if mu != 0.0:        # without momentum the buffers are neither used nor averaged
         assert all(np.array_equal(fv[0], fv[i]) for i in range(m))
 
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_cleared():
+    """A kernel whose bounded wait gives up records the failure and returns; every call that waits for the
+    stream reports it once as LS_ERR_DEVICE_TIMEOUT, and the handle keeps working afterwards.  The wait that
+    runs out is the self-test kernel's (a barrier on which nothing arrives, limit of about a millisecond):
+    nothing faults or hangs."""
+    import torch
+    from paper_1810_08313_b200 import binding
+    from paper_1810_08313_b200.binding import LocalSGD, LsError
+    dims, m, B = (96, 64, 10), 3, 32
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 3)
+    xd, yd = to_device(X, y)
+    eng = LocalSGD(m, dims, lr=0.05, momentum=0.9, batch=B); eng.bind_dataset(xd, yd); eng.set_params(x1)
+    offs = wl.batch_row_offsets(2, 12, m, 1024, B)
+    # (1) ls_sync
+    eng.selftest_wait_timeout(2_000_000)
+    with pytest.raises(LsError) as e:
+        eng.sync()
+    assert e.value.code == binding.LS_ERR_DEVICE_TIMEOUT
+    eng.sync()                                           # reported once, then clear
+    # (2) a synchronous loss evaluation
+    eng.selftest_wait_timeout(2_000_000)
+    with pytest.raises(LsError) as e:
+        eng.eval_loss(0, 0, 2 * B)
+    assert e.value.code == binding.LS_ERR_DEVICE_TIMEOUT
+    F = eng.eval_loss(0, 0, 2 * B)
+    assert np.isfinite(F) and F > 0
+    # (3) the native run loop stops at its next decision point instead of feeding the controller
+    eng.selftest_wait_timeout(2_000_000)
+    with pytest.raises(LsError) as e:
+        eng.run(12, 4, offs, interval=4, probe_rows=2 * B)
+    assert e.value.code == binding.LS_ERR_DEVICE_TIMEOUT
+    # (4) host-fed steps
+    xh = torch.from_numpy(X[:2 * m * B].reshape(2, m, B, dims[0])).pin_memory()
+    yh = torch.from_numpy(y[:2 * m * B].reshape(2, m, B)).pin_memory()
+    lh = torch.zeros((2, m)).pin_memory()
+    eng.selftest_wait_timeout(2_000_000)
+    with pytest.raises(LsError) as e:
+        eng.local_steps_host(2, xh, yh, lh)
+    assert e.value.code == binding.LS_ERR_DEVICE_TIMEOUT
+    # the handle is as good as new: a run from a fresh start equals the oracle's
+    eng.set_params(x1)
+    eng.run(8, 4, offs[:8])
+    eng.sync()
+    ref = orc.run_pasgd(spec, x1, X, y, offs[:8], B, f32(0.05), f32(0.9), 4)
+    p, _ = eng.get_state(0)
+    assert max_rel_err_per_tensor(p, ref.params[0], dims, True) <= 1e-4
+    assert eng.lib.ls_selftest_wait_timeout(eng.h, 0) == binding.LS_ERR_INVALID_ARG
+    eng.close()
