@@ -196,6 +196,34 @@ def average_replicas(X: np.ndarray) -> None:
     X[:] = mean[None, :]
 
 
+def average_replicas_grouped(X: np.ndarray, groups: int) -> None:
+    """The same averaging step when the m replicas are spread over `groups` devices (Section 2: the workers'
+    models are averaged "by a fusion node or by performing an all-node broadcast"; here one partial sum per
+    device is exchanged).  Replicas are dealt out in index order, m / groups consecutive ones per device.
+    Specified to the bit, the grouped order:
+        partial_g = x^(g*q) + x^(g*q+1) + ... + x^(g*q+q-1)   sequentially in fp32, q = m / groups
+        total     = partial_0 + partial_1 + ... + partial_{groups-1}   sequentially in fp32 (device order)
+        mean      = total / m   (one fp32 division)
+    groups = 1 and groups = m are both the sequential order of average_replicas; anything between is a
+    different rounding order (and so a different, equally valid, fp32 mean).  In place.
+    """
+    if X.dtype != np.float32:
+        raise TypeError("average_replicas_grouped is specified on float32 state")
+    m = X.shape[0]
+    groups = int(groups)
+    if groups < 1 or m % groups != 0:
+        raise ValueError("the replicas must divide evenly over the groups")
+    q = m // groups
+    total = None
+    for g in range(groups):
+        part = X[g * q].copy()
+        for j in range(1, q):
+            part = part + X[g * q + j]
+        total = part if total is None else total + part
+    mean = total / np.float32(m)
+    X[:] = mean[None, :]
+
+
 def block_momentum_average(X: np.ndarray, anchor: np.ndarray, u: np.ndarray, lr: float, beta: float) -> None:
     """Averaging step with block momentum (Section 5.3):
         u_j = beta_glob * u_{j-1} + G_j ;   x_{(j+1)tau+1} = x_{j tau+1} - eta_j * u_j
@@ -301,7 +329,8 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
               batch: int, lr: float, mu: float, tau: int,
               momentum_mode: str = MOMENTUM_AVERAGE,
               adacomm_interval: Optional[int] = None, probe_rows: int = 0,
-              state_hook=None, refined: Optional[dict] = None, block_beta: float = 0.0) -> PasgdResult:
+              state_hook=None, refined: Optional[dict] = None, block_beta: float = 0.0,
+              avg_groups: int = 1) -> PasgdResult:
     """m workers start at the same x_1; each takes local mini-batch steps on its
     own batches; after every tau-th local step (counting from the start of the
     current period) the updated models are replaced by their mean.
@@ -324,6 +353,8 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
         same loss at x_1.  A period is never cut by an interval boundary.
       * momentum_mode "block" (Section 5.3): the averaging step is block_momentum_average with factor
         `block_beta` on the model the period started from, and the local buffers restart from zero.
+      * avg_groups = G > 1: the replicas live on G devices, m / G each, and the averaging step sums in the
+        grouped order of average_replicas_grouped (not available with block momentum).
       * refined = {"gamma", "slack", "decay_at": [iterations], "decay_factor"} switches the decision
         to adacomm_next_tau_refined (Section 4.3).  A learning-rate decay scheduled for iteration d
         is applied at the first decision point with k >= d at which the period in force is 1
@@ -364,10 +395,20 @@ def run_pasgd(spec: ModelSpec, x1: np.ndarray, X: np.ndarray, y: np.ndarray, row
             k += 1
             if state_hook is not None:
                 state_hook(k, xs, vs, False)
+        if momentum_mode == MOMENTUM_BLOCK and avg_groups > 1:
+            raise ValueError("block momentum is defined here on the sequential mean only")
         if momentum_mode == MOMENTUM_BLOCK:
             # Section 5.3: global momentum on the period's accumulated step, local buffers restart
             block_momentum_average(xs, anchor, u_glob, lr, block_beta)
             vs[:] = 0
+        elif avg_groups > 1:
+            average_replicas_grouped(xs, avg_groups)
+            if momentum_mode == MOMENTUM_AVERAGE:
+                average_replicas_grouped(vs, avg_groups)
+            elif momentum_mode == MOMENTUM_RESET:
+                vs[:] = 0
+            elif momentum_mode != MOMENTUM_KEEP:
+                raise ValueError(momentum_mode)
         else:
             average_replicas(xs)
             if momentum_mode == MOMENTUM_AVERAGE:

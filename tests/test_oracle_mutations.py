@@ -169,3 +169,25 @@ def test_decay_scheduling_mistakes_are_caught(monkeypatch, old, new):
     monkeypatch.setattr(orc, "run_pasgd", _mutated_run_pasgd(old, new))
     with pytest.raises(AssertionError):                       # the pin itself must object, not a crash
         pins_tau.check_deferred_decay_trace(monkeypatch)
+
+
+def test_grouped_averaging_mistakes_are_caught(monkeypatch):
+    real = orc.average_replicas_grouped
+
+    def device_order_reversed(X, groups):
+        q = X.shape[0] // groups
+        perm = np.concatenate([np.arange(g * q, (g + 1) * q) for g in range(groups - 1, -1, -1)])
+        Y = np.ascontiguousarray(X[perm]); real(Y, groups); X[:] = Y[0][None, :]
+    monkeypatch.setattr(orc, "average_replicas_grouped", device_order_reversed)
+    assert _fails(pins_avg.test_grouped_brute_force_scalar_fp32_chain, 16, 8)
+
+    def divides_by_group_size(X, groups):
+        real(X, groups); X *= np.float32(groups)
+    monkeypatch.setattr(orc, "average_replicas_grouped", divides_by_group_size)
+    assert _fails(pins_avg.test_grouped_brute_force_scalar_fp32_chain, 8, 2)
+    assert _fails(pins_avg.test_grouped_within_rounding_bound_of_exact_rational_mean, 8, 2)
+
+    def ignores_the_grouping(X, groups):
+        orc.average_replicas(X)
+    monkeypatch.setattr(orc, "average_replicas_grouped", ignores_the_grouping)
+    assert _fails(pins_avg.test_grouped_order_is_a_different_rounding_order)

@@ -252,3 +252,20 @@ def test_block_momentum_run_resets_local_buffers_and_synchronizes():
     plain = orc.run_pasgd(spec, x1, X, y, offs, B, 0.05, 0.9, tau, momentum_mode=orc.MOMENTUM_RESET)
     assert not np.array_equal(res.params[0], plain.params[0])       # the global momentum changes the trajectory
     assert np.any(res.block_u != 0)
+
+
+@pytest.mark.parametrize("groups", [2, 4])
+def test_grouped_averaging_tau1_is_still_synchronous_sgd(groups):
+    """Replicas spread over several devices (grouped summation order): tau = 1 remains fully synchronous
+    momentum SGD on the m-fold batch, and all replicas are bitwise equal after every averaging step."""
+    spec, X, y, x1 = _tiny_problem()
+    B, K, m = 8, 10, 4
+    offs = wl.batch_row_offsets(2, K, m, X.shape[0], B)
+    same = []
+    res = orc.run_pasgd(spec, x1, X, y, offs, B, lr=0.05, mu=0.9, tau=1, avg_groups=groups,
+                        state_hook=lambda k, xs, vs, avg: same.append(bool(avg) and bool((xs == xs[0]).all() and (vs == vs[0]).all())))
+    batches = [np.concatenate([np.arange(int(o), int(o) + B) for o in offs[k]]) for k in range(K)]
+    want = _torch_sgd(spec.dims, True, x1, X, y, batches, 0.05, 0.9)
+    for i in range(m):
+        assert np.max(np.abs(res.params[i] - want)) / np.max(np.abs(want)) < 1e-6
+    assert same[1::2] == [True] * K               # the hook runs after each step and after each average
