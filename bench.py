@@ -445,13 +445,25 @@ def run_ours(args, w: wl.Workload):
     if w.gemm_dtype == "bf16":
         xd = xd.to(torch.bfloat16)
     yd = torch.from_numpy(y).cuda()
-    eng = LocalSGD(m, w.dims, w.loss, w.has_bias, w.gemm_dtype, lr=w.lr, momentum=w.momentum, batch=B,
-                   device=f"cuda:{local_rank}")
+    total_periods = W + K
+    if args.shard:
+        # ONE job of w.m replicas dealt out over the ranks (m / N each): local steps need no communication, every
+        # averaging step is one all-gather of partial sums over NCCL plus the rank-ordered combining kernel
+        from paper_1810_08313_b200.sharded import ShardedLocalSGD
+        sh = ShardedLocalSGD(w.m, w.dims, w.loss, w.has_bias, w.gemm_dtype, lr=w.lr, momentum=w.momentum, batch=B,
+                             device=f"cuda:{local_rank}")
+        eng, m = sh.eng, sh.m
+        offs = wl.batch_row_offsets(w.seed + 100, total_periods * tau, w.m, w.n_rows, B)
+        offs = np.ascontiguousarray(offs[:, sh.first:sh.first + sh.m])
+    else:
+        eng = LocalSGD(m, w.dims, w.loss, w.has_bias, w.gemm_dtype, lr=w.lr, momentum=w.momentum, batch=B,
+                       device=f"cuda:{local_rank}")
+        offs = wl.batch_row_offsets(w.seed + 100 + rank, total_periods * tau, m, w.n_rows, B)
+    import dataclasses
+    w_r = dataclasses.replace(w, m=m)          # this rank's share, for the per-launch byte and flop counts
     eng.bind_dataset(xd, yd)
     eng.set_params(x1)
     probe = probe_rows_for(w)
-    total_periods = W + K
-    offs = wl.batch_row_offsets(w.seed + 100 + rank, total_periods * tau, m, w.n_rows, B)
     loss_dev = torch.zeros((tau, m), dtype=torch.float32, device="cuda")
     F_0 = eng.eval_loss(0, 0, probe)
 
@@ -501,17 +513,20 @@ def run_ours(args, w: wl.Workload):
     value = units / (ms * 1e-3)
 
     # ---- roofline of the dominant kernel ---------------------------------------
-    roofline = roofline_for(dom, dom_ms * 1e-3 / dom_n, w, peaks, clocks) if dom_n else None
+    roofline = roofline_for(dom, dom_ms * 1e-3 / dom_n, w_r, peaks, clocks) if dom_n else None
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong" if args.shard else "weak",
+        "vs_baseline": None,
         "dtype": "bf16" if w.gemm_dtype == "bf16" else "f32", "data": "synthetic",
         "config": dict(workload_config(w, tau),
                        step="one period: tau local iterations x m replicas + averaging + probe loss + AdaComm decision",
                        l2="inputs larger than L2: mini-batches are drawn at random from a %.0f MB resident dataset"
                           % (xd.numel() * xd.element_size() / 1e6),
-                       multi_gpu="replicas only" if world > 1 else "single GPU"),
+                       multi_gpu=("one job sharded by replica, one all-gather of partial sums per period" if args.shard
+                                  else "replicas only: independent jobs, no data-path collective") if world > 1
+                       else "single GPU"),
         "clocks": clocks, "gpu_launches": int(launches), "kernel_time_shares": shares,
         "kernel_us_per_launch": kernel_us,
         "last_probe_loss": F_t, "next_tau": next_tau,
@@ -522,7 +537,7 @@ def run_ours(args, w: wl.Workload):
     gemm = {}
     for (c, l), v in shares_raw.items():
         if c in ("fwd", "dx") and v[1] and uses_tensor_cores(w, c, l):
-            r = roofline_for((c, l), v[0] * 1e-3 / v[1], w, peaks, clocks)
+            r = roofline_for((c, l), v[0] * 1e-3 / v[1], w_r, peaks, clocks)
             gemm[f"{c}{l}"] = {"TFLOP/s": round(r["achieved"], 1), "frac": round(r["frac"], 4),
                                "us_per_launch": round(v[0] / v[1] * 1e3, 2)}
     if gemm:
@@ -750,6 +765,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_mlp_bf16", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--shard", action="store_true",
+                    help="with --gpus N: one job whose m replicas are dealt out over the N ranks (m / N each) with one "
+                         "NCCL all-gather of partial sums per averaging step, instead of N independent jobs")
     ap.add_argument("--no-side-configs", action="store_true",
                     help="skip the short device-timed runs of the other workload configurations")
     ap.add_argument("--tau", type=int, default=20)

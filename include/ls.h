@@ -57,7 +57,8 @@ enum {
   LS_ERR_UNSUPPORTED = -7,       /* valid request that the library does not implement (e.g. weight decay) */
   LS_ERR_OVERFLOW = -8,          /* a result does not fit its type */
   LS_ERR_DEVICE_TIMEOUT = -9,    /* a bounded wait inside a kernel ran out; results of that launch are invalid */
-  LS_ERR_TOO_LARGE = -10         /* a size exceeds a fixed capacity of the entry point */
+  LS_ERR_TOO_LARGE = -10,        /* a size exceeds a fixed capacity of the entry point */
+  LS_ERR_EXCHANGE = -11          /* the exchange callback of ls_set_shard() reported a failure */
 };
 
 enum { LS_LOSS_SOFTMAX_CE = 0, LS_LOSS_MSE_HALF = 1 };
@@ -194,6 +195,58 @@ int ls_local_steps_host(ls_handle* h, int tau, const void* x_host, const void* y
  * x' replaces every replica's parameters and a, u' replaces u, the local
  * momentum buffers are cleared.  lr is the rate in force when ls_average runs. */
 int ls_average(ls_handle* h);
+
+/* ---- one job on several GPUs --------------------------------------------------
+ * The paper's own layout (Section 2: m workers, models averaged "by a fusion node or by performing an
+ * all-node broadcast"; its experiments ran one worker per GPU): the m_total replicas of a job are dealt out in
+ * index order over n_gpus GPUs, one process and one handle per GPU, m = m_total / n_gpus replicas in each
+ * handle.  Local steps need no communication.  The averaging step becomes
+ *     p_g   = x^(0) + x^(1) + ... + x^(m-1)            on GPU g, over its own replicas in index order, fp32
+ *     total = p_0 + p_1 + ... + p_{n_gpus-1}           in rank order, fp32, after ONE exchange that brings every
+ *                                                      GPU's partial sum into this GPU's own memory
+ *     mean  = total / (float)m_total                   written to every local replica
+ * (the same for the momentum buffers in LS_MOMENTUM_AVERAGE).  This GROUPED order replaces the sequential
+ * order of ls_average() on such a handle: it rounds differently for 1 < n_gpus < m_total, is identical for
+ * n_gpus = 1, is fixed, and gives every GPU the same bits, so all m_total replicas end bitwise equal.
+ * LS_MOMENTUM_BLOCK is not available on several GPUs (LS_ERR_UNSUPPORTED).
+ *
+ * The library links no communication library and never reads another GPU's memory: the exchange is the
+ * caller's (an all-gather, e.g. NCCL through torch.distributed), handed over as a callback. */
+
+/* exchange(ctx, partial_dev, gathered_dev, bytes, n_gpus): gathered_dev[g*bytes .. (g+1)*bytes) must receive
+ * rank g's `bytes` bytes at partial_dev, for every g (this rank's own included).  The copy must be ordered
+ * after the work already enqueued on the handle's stream and before anything enqueued on it afterwards
+ * (enqueue the collective on that stream, or make the stream wait for it).  Returns 0 on success. */
+typedef int (*ls_exchange_fn)(void* ctx, const float* partial_dev, float* gathered_dev, size_t bytes, int n_gpus);
+
+/* Floats that partial_dev of ls_set_shard() must hold (two padded replica vectors: parameters and momentum);
+ * gathered_dev holds n_gpus times as many. */
+int ls_shard_buffer_floats(const ls_handle* h, int64_t* floats);
+
+/* Declare that this handle's m replicas are rank-local shares of a job of m_total = n_gpus * m replicas.  From
+ * then on every averaging step of the handle (ls_average, ls_local_steps_avg, the run loops) is the grouped
+ * average above, with one call of `exchange` per averaging step.  partial_dev / gathered_dev: caller-allocated
+ * device buffers (256-byte aligned, sizes above), borrowed until ls_destroy() or ls_set_shard(h, 0, ...).
+ * n_gpus = 1 needs no callback (and equals ls_average() bit for bit); n_gpus = 0 switches back.
+ * All ranks must call the hot-path functions in the same order (the exchange is collective); the controller
+ * needs no exchange of its own: every rank evaluates the same synchronized model on the same probe rows and
+ * reaches the same decision. */
+int ls_set_shard(ls_handle* h, int n_gpus, int m_total, float* partial_dev, float* gathered_dev, ls_exchange_fn exchange,
+                 void* ctx);
+
+/* The two halves of the grouped average for callers that run the exchange themselves: the partial sums of this
+ * handle's replicas into partial_dev, and, given all ranks' partial sums in rank order, the mean into every
+ * local replica (momentum buffers as in ls_average). */
+int ls_shard_partial_sum(ls_handle* h, float* partial_dev);
+int ls_shard_average(ls_handle* h, const float* gathered_dev, int n_gpus, int m_total);
+
+/* The same two kernels on raw buffers (32-byte aligned, strides multiples of 8 floats):
+ * out_dev[0..P) = sum of the m vectors at buf_dev + j*stride in index order;
+ * every one of the m_local vectors at dst_dev + j*dst_stride = (sum of the G vectors at
+ * partials_dev + g*part_stride, in that order) / (float)m_total. */
+int ls_partial_sum_flat(const float* buf_dev, int m, int64_t P, int64_t stride, float* out_dev, void* cuda_stream);
+int ls_combine_partials_flat(const float* partials_dev, int G, int64_t part_stride, int m_total, int64_t P,
+                             float* dst_dev, int m_local, int64_t dst_stride, void* cuda_stream);
 
 /* Block-momentum state of a LS_MOMENTUM_BLOCK handle in the flat interface layout
  * (P floats each): the period-start model and the global buffer.  Either pointer

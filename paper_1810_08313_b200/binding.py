@@ -28,6 +28,7 @@ LS_ERR_UNSUPPORTED = -7
 LS_ERR_OVERFLOW = -8
 LS_ERR_DEVICE_TIMEOUT = -9
 LS_ERR_TOO_LARGE = -10
+LS_ERR_EXCHANGE = -11
 
 LOSS = {"softmax_ce": 0, "mse_half": 1}
 GEMM = {"fp32": 0, "bf16": 1}
@@ -51,6 +52,10 @@ class ModelSpec(C.Structure):
         ("weight_decay", C.c_float),
         ("block_momentum", C.c_float),
     ]
+
+
+# int exchange(void* ctx, const float* partial_dev, float* gathered_dev, size_t bytes, int n_gpus)
+EXCHANGE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int)
 
 
 class LsError(RuntimeError):
@@ -111,6 +116,12 @@ def _lib():
                                      vp, i64, P(i64), P(f32)]),
         "ls_get_lr": (C.c_int, [vp, P(f32)]),
         "ls_linear_loss_static": (C.c_int, [vp, vp, vp, vp, i64, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]),
+        "ls_shard_buffer_floats": (C.c_int, [vp, P(i64)]),
+        "ls_set_shard": (C.c_int, [vp, C.c_int, C.c_int, vp, vp, EXCHANGE_FN, vp]),
+        "ls_shard_partial_sum": (C.c_int, [vp, vp]),
+        "ls_shard_average": (C.c_int, [vp, vp, C.c_int, C.c_int]),
+        "ls_partial_sum_flat": (C.c_int, [vp, C.c_int, i64, i64, vp, vp]),
+        "ls_combine_partials_flat": (C.c_int, [vp, C.c_int, i64, C.c_int, i64, vp, C.c_int, i64, vp]),
         "ls_profile_begin": (C.c_int, [vp, C.c_uint32, C.c_int]),
         "ls_profile_end": (C.c_int, [vp, P(C.c_double), P(i64)]),
     }
@@ -193,6 +204,23 @@ def average_flat(buf, m: int, P: int, stride: Optional[int] = None, stream=None)
     if buf.numel() < (m - 1) * stride + P:
         raise ValueError("buf too small")
     _check(_lib().ls_average_flat(buf.data_ptr(), int(m), int(P), stride, _stream_ptr(stream)), "ls_average_flat")
+
+
+def partial_sum_flat(buf, m: int, P: int, out, stride: Optional[int] = None, stream=None) -> None:
+    """out[0..P) = sum of the m vectors of buf (vector j at j*stride) in index order, fp32 (ls_partial_sum_flat)."""
+    stride = int(P if stride is None else stride)
+    _check(_lib().ls_partial_sum_flat(buf.data_ptr(), int(m), int(P), stride, out.data_ptr(), _stream_ptr(stream)),
+           "ls_partial_sum_flat")
+
+
+def combine_partials_flat(partials, G: int, part_stride: int, m_total: int, P: int, dst, m_local: int,
+                          dst_stride: Optional[int] = None, stream=None) -> None:
+    """Every one of the m_local vectors of dst = (partials[0] + ... + partials[G-1], in that order) / m_total
+    (ls_combine_partials_flat)."""
+    dst_stride = int(P if dst_stride is None else dst_stride)
+    _check(_lib().ls_combine_partials_flat(partials.data_ptr(), int(G), int(part_stride), int(m_total), int(P),
+                                           dst.data_ptr(), int(m_local), dst_stride, _stream_ptr(stream)),
+           "ls_combine_partials_flat")
 
 
 def block_average_flat(buf, anchor, u, m: int, P: int, lr: float, beta: float, stride: Optional[int] = None,
@@ -500,6 +528,31 @@ class LocalSGD:
         n_p, n_d = n_p.value, n_d.value
         return {"taus": period_tau[:n_p].tolist(), "decision_k": dk[:n_d].tolist(), "decision_F": dF[:n_d].copy(),
                 "decision_tau": dt[:n_d].tolist(), "F_0": float(F0.value), "lr": float(lr.value)}
+
+    # -- one job on several GPUs ----------------------------------------------
+    def shard_buffer_floats(self) -> int:
+        n = C.c_int64()
+        _check(self.lib.ls_shard_buffer_floats(self.h, C.byref(n)), "ls_shard_buffer_floats")
+        return n.value
+
+    def set_shard(self, n_gpus: int, m_total: int, partial=None, gathered=None, exchange=None):
+        """ls_set_shard: this handle's replicas are one rank's share of a job of m_total replicas.  `exchange` is
+        a Python callable (partial_ptr, gathered_ptr, nbytes, n_gpus) -> 0 on success; the buffers and the
+        callback object are kept alive by this wrapper."""
+        if n_gpus == 0:
+            _check(self.lib.ls_set_shard(self.h, 0, 0, None, None, EXCHANGE_FN(0), None), "ls_set_shard")
+            self._shard = None
+            return
+        cb = EXCHANGE_FN(0) if exchange is None else EXCHANGE_FN(lambda ctx, p, g, nbytes, n: int(exchange(p, g, nbytes, n)))
+        _check(self.lib.ls_set_shard(self.h, int(n_gpus), int(m_total), partial.data_ptr(),
+                                     None if gathered is None else gathered.data_ptr(), cb, None), "ls_set_shard")
+        self._shard = (partial, gathered, cb)
+
+    def shard_partial_sum(self, partial):
+        _check(self.lib.ls_shard_partial_sum(self.h, partial.data_ptr()), "ls_shard_partial_sum")
+
+    def shard_average(self, gathered, n_gpus: int, m_total: int):
+        _check(self.lib.ls_shard_average(self.h, gathered.data_ptr(), int(n_gpus), int(m_total)), "ls_shard_average")
 
     def launch_count(self) -> int:
         n = C.c_int64()

@@ -406,6 +406,27 @@ static int average(ls_handle* h) {
   const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
   const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
   const bool block = h->spec.momentum_mode == LS_MOMENTUM_BLOCK;
+  if (h->shard_G >= 1) {
+    // Replicas spread over G GPUs: local partial sums, one exchange, then the sum over the ranks in rank
+    // order and one division by the job's replica count (see shard_average.cu).
+    const int n_buf = both ? 2 : 1;
+    ProfScope ps(h, LS_K_AVG, 0);
+    LS_CUDA(h, launch_partial_sum(params_of(h), n_buf, buf_stride, lay.m, lay.stride, lay.stride, h->shard_partial,
+                                  lay.stride, h->stream, &h->launches));
+    const float* parts = h->shard_partial;
+    if (h->shard_fn != nullptr) {
+      const int rc = h->shard_fn(h->shard_ctx, h->shard_partial, h->shard_gathered, (size_t)n_buf * lay.stride * 4,
+                                 h->shard_G);
+      if (rc != 0) return LS_ERR_EXCHANGE;
+      parts = h->shard_gathered;
+    }
+    LS_CUDA(h, launch_combine(parts, h->shard_fn ? h->shard_G : 1, (int64_t)n_buf * lay.stride, lay.stride,
+                              h->shard_m_total, lay.stride, params_of(h), n_buf, buf_stride, lay.m, lay.stride,
+                              shadow_of(h), h->stream, &h->launches));
+    if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
+      LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+    return LS_OK;
+  }
   {
     ProfScope ps(h, LS_K_AVG, 0);
     BlockMomentum bm{anchor_of(h), blocku_of(h), h->lr, h->spec.block_momentum};
@@ -492,6 +513,7 @@ const char* ls_strerror(int code) {
     case LS_ERR_OVERFLOW: return "result does not fit";
     case LS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case LS_ERR_TOO_LARGE: return "size beyond the fixed capacity of this entry point";
+    case LS_ERR_EXCHANGE: return "the caller's exchange of partial sums failed";
     default: return "unknown error";
   }
 }
@@ -804,6 +826,58 @@ int ls_average(ls_handle* h) {
 int ls_eval_loss(ls_handle* h, int replica, int64_t row_offset, int64_t n_rows, float* F_host) {
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   return eval_loss(h, replica, row_offset, n_rows, F_host);
+}
+
+int ls_shard_buffer_floats(const ls_handle* h, int64_t* floats) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (floats == nullptr) return LS_ERR_INVALID_ARG;
+  *floats = 2 * h->lay.stride;
+  return LS_OK;
+}
+
+int ls_set_shard(ls_handle* h, int n_gpus, int m_total, float* partial_dev, float* gathered_dev, ls_exchange_fn exchange,
+                 void* ctx) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (n_gpus == 0) {                       // back to a job that lives on this GPU alone
+    h->shard_G = 0; h->shard_fn = nullptr; h->shard_ctx = nullptr;
+    return LS_OK;
+  }
+  if (h->spec.momentum_mode == LS_MOMENTUM_BLOCK) return LS_ERR_UNSUPPORTED;
+  if (n_gpus < 1 || m_total != n_gpus * h->lay.m || partial_dev == nullptr) return LS_ERR_INVALID_ARG;
+  if (n_gpus > 1 && (exchange == nullptr || gathered_dev == nullptr)) return LS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(partial_dev) % 256 != 0 || reinterpret_cast<uintptr_t>(gathered_dev) % 256 != 0)
+    return LS_ERR_INVALID_ARG;
+  h->shard_G = n_gpus; h->shard_m_total = m_total;
+  h->shard_partial = partial_dev; h->shard_gathered = gathered_dev;
+  h->shard_fn = n_gpus > 1 ? exchange : nullptr; h->shard_ctx = ctx;
+  return LS_OK;
+}
+
+int ls_shard_partial_sum(ls_handle* h, float* partial_dev) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (partial_dev == nullptr || reinterpret_cast<uintptr_t>(partial_dev) % 256 != 0) return LS_ERR_INVALID_ARG;
+  const Layout& lay = h->lay;
+  const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
+  LS_CUDA(h, launch_partial_sum(params_of(h), both ? 2 : 1, (int64_t)((lay.mom_off - lay.params_off) / 4), lay.m,
+                                lay.stride, lay.stride, partial_dev, lay.stride, h->stream, &h->launches));
+  return LS_OK;
+}
+
+int ls_shard_average(ls_handle* h, const float* gathered_dev, int n_gpus, int m_total) {
+  if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
+  if (h->spec.momentum_mode == LS_MOMENTUM_BLOCK) return LS_ERR_UNSUPPORTED;
+  if (gathered_dev == nullptr || reinterpret_cast<uintptr_t>(gathered_dev) % 256 != 0 || n_gpus < 1 ||
+      m_total != n_gpus * h->lay.m)
+    return LS_ERR_INVALID_ARG;
+  const Layout& lay = h->lay;
+  const bool both = h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_AVERAGE;
+  const int n_buf = both ? 2 : 1;
+  LS_CUDA(h, launch_combine(gathered_dev, n_gpus, (int64_t)n_buf * lay.stride, lay.stride, m_total, lay.stride,
+                            params_of(h), n_buf, (int64_t)((lay.mom_off - lay.params_off) / 4), lay.m, lay.stride,
+                            shadow_of(h), h->stream, &h->launches));
+  if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
+    LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  return LS_OK;
 }
 
 int adacomm_next_tau(double F_t, double F_0, int tau_0) {

@@ -89,6 +89,12 @@ struct ls_handle {
   int64_t n_rows;
   int last_cuda;
   bool allow_pair;        // CTA-pair kernels enabled (see pair_kernels_enabled)
+  // replicas spread over several GPUs (ls_set_shard): this handle holds m of m_total replicas
+  int shard_G, shard_m_total;
+  float* shard_partial;   // [n_buf][stride] this GPU's partial sums
+  float* shard_gathered;  // [G][n_buf][stride] every GPU's partial sums, in rank order
+  ls_exchange_fn shard_fn;
+  void* shard_ctx;
   int64_t launches;
   float* pinned;          // small pinned host scratch (eval losses)
   // per-kernel timing (ls_profile_begin / ls_profile_end)
@@ -186,6 +192,16 @@ struct BlockMomentum {
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
                    __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
                    const BlockMomentum* bm = nullptr);
+
+// ---- averaging over several GPUs (shard_average.cu) -------------------------
+// out[b] = sum over the m vectors of buffer b in index order; then, with the G partial sums of every GPU
+// gathered in rank order (vector g of buffer b at parts + g*part_stride + b*part_buf_stride), the mean
+// (p_0 + ... + p_{G-1}) / m_total written to the m_local replicas of every buffer (and the bf16 copy of buffer 0).
+int launch_partial_sum(const float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride, float* out,
+                       int64_t out_stride, cudaStream_t st, int64_t* launches);
+int launch_combine(const float* parts, int G, int64_t part_stride, int64_t part_buf_stride, int m_total, int64_t n,
+                   float* base, int n_buf, int64_t buf_stride, int m_local, int64_t stride, __nv_bfloat16* shadow,
+                   cudaStream_t st, int64_t* launches);
 
 // ---- fp32-accumulate CUDA-core grouped GEMMs (gemm_simt.cu) ---------------
 struct FwdArgs {           // Z = A W^T + b, optional ReLU

@@ -14,6 +14,7 @@ def _declared_functions():
             continue
         src = open(os.path.join(ROOT, "include", fn)).read()
         src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        src = re.sub(r"typedef\s+\w+\s*\(\s*\*[^;]*;", "", src)          # function-pointer types are not functions
         for m in re.finditer(r"^\s*(?:const\s+)?[A-Za-z_][\w\s\*]*?\b(\w+)\s*\([^;{]*\)\s*;", src, flags=re.M):
             names.add(m.group(1))
     return names
