@@ -90,6 +90,7 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   }
   lay.stage_loss_off = take((size_t)kRowOffCap * m * 4);
   lay.err_off = take(256);
+  lay.sync_off = take((size_t)2 * lay.stride * 4);
   if (spec->momentum_mode == LS_MOMENTUM_BLOCK) {
     lay.anchor_off = take((size_t)lay.stride * 4);
     lay.blocku_off = take((size_t)lay.stride * 4);
@@ -337,6 +338,10 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.maps.b = (l == 0) ? xmap.upd : &h->maps_upd.act[l];
       t.mapW = &h->maps.wf[l];
       t.mapV = &h->maps.vf[l];
+      // every replica still holds the synchronized model (first local step after an averaging step): the old
+      // W and v are read once, from the synchronized copy, instead of once per replica
+      t.mapWsync = h->sync_valid ? &h->maps.wsync[l] : nullptr;
+      t.mapVsync = h->sync_valid ? &h->maps.vsync[l] : nullptr;
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
       t.w_gstride = lay.stride;
@@ -392,11 +397,43 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   std::sort(upd, upd + n_upd, [](const TcUpdateArgs& x, const TcUpdateArgs& y) {
     return (int64_t)x.M * x.N > (int64_t)y.M * y.N;
   });
+  // A step that starts from synchronized replicas and ends in an averaging step (communication period 1): the
+  // streamed layers' update and their average are one launch that never writes the per-replica values; the
+  // small tensors (biases, a narrow output layer), updated per replica above, are averaged by the plain kernel.
+  bool fused = avg_after && h->sync_valid && n_upd > 0 && bf && h->shard_G == 0 &&
+               (h->mu == 0.f ? h->spec.momentum_mode != LS_MOMENTUM_BLOCK : h->spec.momentum_mode == LS_MOMENTUM_AVERAGE);
+  for (int i = 0; i < n_upd && fused; ++i) fused = tc_sync_step_shape_ok(false, upd[i].M, upd[i].N, upd[i].B);
+  if (fused) {
+    for (int i = 0; i < n_upd; i += tc_update_max_layers()) {
+      const int n = std::min(n_upd - i, tc_update_max_layers());
+      ProfScope ps(h, LS_K_DW, upd[i].layer);
+      LS_CUDA(h, launch_tc_sync_step(upd + i, n, h->stream, &h->launches));
+    }
+    // what is left of a replica vector: the gaps between the streamed weight matrices, in layout order
+    std::sort(upd, upd + n_upd, [&](const TcUpdateArgs& x, const TcUpdateArgs& y) {
+      return lay.w_off[x.layer] < lay.w_off[y.layer];
+    });
+    const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
+    const int n_buf = h->mu != 0.f ? 2 : 1;
+    int64_t pos = 0;
+    for (int i = 0; i <= n_upd; ++i) {
+      const int64_t end = i < n_upd ? lay.w_off[upd[i].layer] : lay.stride;
+      if (end > pos) {
+        ProfScope ps(h, LS_K_AVG, 0);
+        LS_CUDA(h, launch_average(params_of(h) + pos, n_buf, buf_stride, lay.m, end - pos, lay.stride, shadow_of(h) + pos,
+                                  h->stream, &h->launches, nullptr, sync_of(h) + pos, lay.stride));
+      }
+      if (i < n_upd) pos = round_up(lay.w_off[upd[i].layer] + (int64_t)upd[i].M * upd[i].N, kAlignFloats);
+    }
+    h->sync_valid = true;
+    return LS_OK;
+  }
   for (int i = 0; i < n_upd; i += tc_update_max_layers()) {
     const int n = std::min(n_upd - i, tc_update_max_layers());
     ProfScope ps(h, LS_K_DW, upd[i].layer);
     LS_CUDA(h, launch_tc_update(upd + i, n, h->stream, &h->launches));
   }
+  h->sync_valid = false;           // the replicas have moved apart
   if (avg_after) return average(h);
   return LS_OK;
 }
@@ -425,16 +462,22 @@ static int average(ls_handle* h) {
                               shadow_of(h), h->stream, &h->launches));
     if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
       LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+    h->sync_valid = false;         // the combining kernel keeps no synchronized copy
     return LS_OK;
   }
   {
     ProfScope ps(h, LS_K_AVG, 0);
     BlockMomentum bm{anchor_of(h), blocku_of(h), h->lr, h->spec.block_momentum};
     LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                              shadow_of(h), h->stream, &h->launches, block ? &bm : nullptr));
+                              shadow_of(h), h->stream, &h->launches, block ? &bm : nullptr, sync_of(h)));
   }
-  if (h->mu != 0.f && (h->spec.momentum_mode == LS_MOMENTUM_RESET || block))
+  if (h->mu != 0.f && (h->spec.momentum_mode == LS_MOMENTUM_RESET || block)) {
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+    LS_CUDA(h, cudaMemsetAsync(sync_of(h) + lay.stride, 0, (size_t)lay.stride * 4, h->stream));
+  }
+  // the synchronized copy now equals every replica: parameters always; momentum when it was averaged or
+  // cleared (or is not used at all)
+  h->sync_valid = h->mu == 0.f || h->spec.momentum_mode != LS_MOMENTUM_KEEP;
   return LS_OK;
 }
 
@@ -594,6 +637,9 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
           if (lay.dims[l] % 4 == 0) {
             ok(tc_make_block_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
             ok(tc_make_block_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
+            ok(tc_make_block_map_3d(&mp.wsync[l], sync_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], 1, lay.stride));
+            ok(tc_make_block_map_3d(&mp.vsync[l], sync_of(h) + lay.stride + lay.w_off[l], lay.dims[l + 1], lay.dims[l], 1,
+                                    lay.stride));
           }
       }
       if (lay.dims[0] % q == 0) {
@@ -685,6 +731,9 @@ int ls_set_params(ls_handle* h, const float* x1_host) {
     LS_CUDA(h, cudaMemcpyAsync(params_of(h) + (int64_t)i * lay.stride, params_of(h), (size_t)lay.stride * 4,
                                cudaMemcpyDeviceToDevice, h->stream));
   LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  LS_CUDA(h, cudaMemcpyAsync(sync_of(h), params_of(h), (size_t)lay.stride * 4, cudaMemcpyDeviceToDevice, h->stream));
+  LS_CUDA(h, cudaMemsetAsync(sync_of(h) + lay.stride, 0, (size_t)lay.stride * 4, h->stream));
+  h->sync_valid = true;
   if (h->spec.momentum_mode == LS_MOMENTUM_BLOCK) {
     LS_CUDA(h, cudaMemcpyAsync(anchor_of(h), params_of(h), (size_t)lay.stride * 4, cudaMemcpyDeviceToDevice,
                                h->stream));
@@ -719,6 +768,7 @@ int ls_set_state(ls_handle* h, int replica, const float* params_host, const floa
   if (!ok_handle(h)) return LS_ERR_BAD_HANDLE;
   if (replica < 0 || replica >= h->lay.m) return LS_ERR_INVALID_ARG;
   int rc = LS_OK;
+  h->sync_valid = false;
   if (params_host)
     rc = copy_replica(h, params_of(h) + (int64_t)replica * h->lay.stride, const_cast<float*>(params_host), true);
   if (rc == LS_OK && momentum_host)
@@ -877,6 +927,7 @@ int ls_shard_average(ls_handle* h, const float* gathered_dev, int n_gpus, int m_
                             shadow_of(h), h->stream, &h->launches));
   if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
+  h->sync_valid = false;
   return LS_OK;
 }
 

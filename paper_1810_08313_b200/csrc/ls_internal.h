@@ -55,6 +55,8 @@ struct Layout {
   size_t stage_loss_off = 0;                 // float [kRowOffCap][m]
   size_t err_off = 0;                        // int: device-side error flag (bounded waits that ran out)
   size_t anchor_off = 0, blocku_off = 0;     // block momentum: period-start model and global buffer, [stride] each
+  size_t sync_off = 0;                       // synchronized copy: [2][stride] parameters and momentum as every replica
+                                             // held them right after the last averaging step
   size_t total = 0;
 };
 
@@ -70,6 +72,7 @@ struct alignas(64) TcMaps {
   CUtensorMap x_data;                                     // bound dataset, 2-D [n_rows][dims[0]]
   CUtensorMap x_stage[2];                                 // staging buffers of host batches
   CUtensorMap wf[LS_MAX_LAYERS], vf[LS_MAX_LAYERS];       // fp32 master weights / momentum, 32 x 32 blocks
+  CUtensorMap wsync[LS_MAX_LAYERS], vsync[LS_MAX_LAYERS]; // the same blocks of the synchronized copy (one vector each)
 };
 
 struct ls_handle {
@@ -89,6 +92,7 @@ struct ls_handle {
   int64_t n_rows;
   int last_cuda;
   bool allow_pair;        // CTA-pair kernels enabled (see pair_kernels_enabled)
+  bool sync_valid;        // every replica's parameters and momentum equal the synchronized copy, bit for bit
   // replicas spread over several GPUs (ls_set_shard): this handle holds m of m_total replicas
   int shard_G, shard_m_total;
   float* shard_partial;   // [n_buf][stride] this GPU's partial sums
@@ -178,6 +182,7 @@ inline __nv_bfloat16* shadow_of(const ls_handle* h) {
 }
 inline float* anchor_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.anchor_off); }
 inline float* blocku_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.blocku_off); }
+inline float* sync_of(const ls_handle* h) { return reinterpret_cast<float*>(h->state + h->lay.sync_off); }
 
 // ---- averaging (average.cu) ---------------------------------------------
 // n_buf buffers of m vectors each; buffer b starts at base + b*buf_stride floats,
@@ -189,9 +194,11 @@ struct BlockMomentum {
   float* u;
   float lr, beta;
 };
+// sync_out (optional): the mean of buffer b is also written to sync_out + b*sync_stride (the synchronized copy;
+// sync_stride 0 means n).
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
                    __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
-                   const BlockMomentum* bm = nullptr);
+                   const BlockMomentum* bm = nullptr, float* sync_out = nullptr, int64_t sync_stride = 0);
 
 // ---- averaging over several GPUs (shard_average.cu) -------------------------
 // out[b] = sum over the m vectors of buffer b in index order; then, with the G partial sums of every GPU
@@ -355,6 +362,9 @@ struct TcUpdateArgs {
   TcOperandMaps maps;        // a: dZ_l [groups*B][M]; b: layer input [rows][N]   (MN-major reads)
   const CUtensorMap* mapW;   // fp32 master weights [replica][M][N], 32 x 32 blocks
   const CUtensorMap* mapV;   // momentum, same shape
+  // when every replica enters the step with the same W and v: descriptors of the synchronized copy (one
+  // vector, [1][M][N]) that the old values are read from instead; null otherwise
+  const CUtensorMap* mapWsync; const CUtensorMap* mapVsync;
   bool fp32;
   const int64_t* row_off;
   __nv_bfloat16* Wb; int64_t w_gstride;
@@ -369,6 +379,11 @@ int tc_update_max_layers();
 int tc_update_box_rows(bool fp32);     // rows of the TMA boxes its operand maps (dZ, layer input) must have
 // one launch for the updates of layers[0..n) (n <= tc_update_max_layers(); same batch, replicas, rates, type)
 int launch_tc_update(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches);
+// One local step of all replicas from a synchronized start, fused with the averaging step that follows it
+// (communication period 1): the layers' W and v leave the launch averaged, in every replica and in the
+// synchronized copy.  Same argument records; mapWsync / mapVsync are required.
+bool tc_sync_step_shape_ok(bool fp32, int M, int N, int B);
+int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches);
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches);
 int launch_tc_dw(const TcDwArgs& a, cudaStream_t st, int64_t* launches);

@@ -57,14 +57,18 @@ struct UParams {
   int full_rounds;                     // whole tiles per CTA; tile t of round n on CTA b is b + n * gridDim.x
   int tail_units;                      // column strips of the left-over tiles, strip u on CTA u % gridDim.x
   int K, groups;                       // batch, replicas
+  int shared_state;                    // 1: all replicas enter with the same W, v: read the synchronized copy (maps.wl / vl,
+                                       //    one vector) instead of each replica's own, and walk the list replica-minor
   int rows_per_group;                  // = batch
   float lr, mu;
   int64_t w_gstride;                   // elements between replicas
   int* err_flag;
 };
 // dZ_l (a), layer input (b), weights and momentum (w, v) of every layer of the launch
+// (w, v: where the new values are stored; wl, vl: where the old ones are loaded from -- the same tensors, or the
+// synchronized copy when every replica holds the same values)
 struct alignas(64) UMaps {
-  CUtensorMap a[kMaxLayers], b[kMaxLayers], w[kMaxLayers], v[kMaxLayers];
+  CUtensorMap a[kMaxLayers], b[kMaxLayers], w[kMaxLayers], v[kMaxLayers], wl[kMaxLayers], vl[kMaxLayers];
 };
 
 struct Tile { int layer, g, m0, n0; };
@@ -77,7 +81,8 @@ __device__ __forceinline__ Tile decode_tile(const UParams& p, int t) {
     if (i < p.n_layers && t >= p.layer[i].tile_begin) l = i;
   const int r = t - p.layer[l].tile_begin;
   const int tpg = p.layer[l].tiles_per_group, nt = p.layer[l].n_tiles;
-  const int g = r / tpg, rem = r % tpg;
+  // replica-minor when the replicas share their old state: the CTAs that read one tile of it run side by side
+  const int g = p.shared_state ? r % p.groups : r / tpg, rem = p.shared_state ? r / p.groups : r % tpg;
   return Tile{l, g, (rem / nt) * BM, (rem % nt) * BN};
 }
 
@@ -177,6 +182,7 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
     fence_mbar_init();
     for (int l = 0; l < p.n_layers; ++l) {
       prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
+      prefetch_tmap(&maps.wl[l]); prefetch_tmap(&maps.vl[l]);
     }
   }
   if (warp == 1) {
@@ -293,8 +299,9 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
       const int y = tl.m0 + q * 32, x = tl.n0 + c * 32;
       uint8_t* slot = my_ring + (j % R) * kSlotBytes;
       mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
-      tma_load_3d(slot, &maps.w[tl.layer], &my_full[j % R], x, y, tl.g);
-      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.v[tl.layer], &my_full[j % R], x, y, tl.g);
+      const int z = p.shared_state ? 0 : tl.g;
+      tma_load_3d(slot, &maps.wl[tl.layer], &my_full[j % R], x, y, z);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.vl[tl.layer], &my_full[j % R], x, y, z);
     };
     if (lane == 0)
       for (int j = 0; j < R; ++j) load_chunk(j);
@@ -406,6 +413,7 @@ struct PParams {
   int full_rounds;                     // whole units per pair; unit t of round n on pair b is b + n * pairs
   int tail_units;                      // 128-column strips of the left-over units, strip u on pair u % pairs
   int K, rows_per_group;
+  int groups, shared_state;            // as in UParams
   float lr, mu;
   int64_t w_gstride;
   int* err_flag;
@@ -428,12 +436,13 @@ __device__ __forceinline__ PUnit decode_punit(const PParams& p, int n, int pb, i
     if (i < p.n_layers && t >= p.layer[i].tile_begin) l = i;
   const int r = t - p.layer[l].tile_begin;
   const int tpg = p.layer[l].tiles_per_group, nt = p.layer[l].n_tiles;
-  const int g = r / tpg, rem = r % tpg;
+  const int g = p.shared_state ? r % p.groups : r / tpg, rem = p.shared_state ? r / p.groups : r % tpg;
   return PUnit{l, g, (rem / nt) * 256, (rem % nt) * PN + c0 * 32, nc};
 }
 
+constexpr int kPairThreads = 384;      // producer, MMA issuer, two idle warps, eight update warps
 template <int R, int KS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kPairThreads, 1)
 tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ PParams p) {
   using L = USmem<false, 1, R, KS>;
   constexpr int MMA_K = 16;
@@ -463,11 +472,12 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
 
   if (threadIdx.x == 0) {
     mbar_init(full, 1); mbar_init(empty, 1);
-    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 16); }
     for (int i = 0; i < 4 * R; ++i) mbar_init(&wv_full[i], 1);
     fence_mbar_init();
     for (int l = 0; l < p.n_layers; ++l) {
       prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
+      prefetch_tmap(&maps.wl[l]); prefetch_tmap(&maps.vl[l]);
     }
   }
   if (warp == 1) {
@@ -539,26 +549,39 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
     }
   } else if (warp >= 4) {
     // ---- update warps: as in tc_update_kernel, on this CTA's 128 rows of the unit ----------------------
-    const int q = warp & 3;
-    uint8_t* my_ring = ring_base + q * R * kSlotBytes;
-    uint64_t* my_full = wv_full + q * R;
-    const int full_chunks = p.full_rounds * (PN / 32);
-    const int my_chunks = full_chunks + my_strips * (PN / 64);
+    // Eight of them: a warp can only read the 32 tensor-memory lanes of its quarter (warp index mod 4), so
+    // two warps share every quarter and take the even / the odd 32-column blocks of a unit, each with its
+    // own ring of R / 2 slots.  One warp per quarter spent most of its time in its own issue latencies
+    // (shared-memory round trips, copy issue) with the data already waiting; two per scheduler hide them.
+    static_assert(R % 2 == 0, "the ring is split between two warps");
+    constexpr int R2 = R / 2;
+    const int q = warp & 3, half = (warp - 4) >> 2;
+    uint8_t* my_ring = ring_base + (half * 4 + q) * R2 * kSlotBytes;
+    uint64_t* my_full = wv_full + (half * 4 + q) * R2;
+    // this warp's chunks: every second 32-column block of every unit, in order
+    const int my_chunks = p.full_rounds * (PN / 64) + my_strips * (PN / 128);
     const uint32_t tmem_empty_leader = map_to_rank(smem_u32(tmem_empty), 0);
 
-    auto load_chunk = [&](int j) {
-      if (j >= my_chunks) return;
-      const int n = j < full_chunks ? (j >> 3) : p.full_rounds + ((j - full_chunks) >> 2);
-      const PUnit un = decode_punit(p, n, pb, pairs);
-      const int c = j < full_chunks ? (j & 7) : ((j - full_chunks) & 3);
-      const int y = un.m0 + rank * BM + q * 32, x = un.n0 + c * 32;
-      uint8_t* slot = my_ring + (j % R) * kSlotBytes;
-      mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
-      tma_load_3d(slot, &maps.w[un.layer], &my_full[j % R], x, y, un.g);
-      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.v[un.layer], &my_full[j % R], x, y, un.g);
+    // the loader walks the unit list on its own, one decode per unit
+    int ld_j = 0, ld_n = 0, ld_c = half;
+    PUnit ld_un = decode_punit(p, 0, pb, pairs);
+    auto load_next = [&]() {
+      if (ld_j >= my_chunks) return;
+      const int y = ld_un.m0 + rank * BM + q * 32, x = ld_un.n0 + ld_c * 32;
+      uint8_t* slot = my_ring + (ld_j % R2) * kSlotBytes;
+      mbar_expect_tx(&my_full[ld_j % R2], has_v ? kSlotBytes : kSlotBytes / 2);
+      const int z = p.shared_state ? 0 : ld_un.g;
+      tma_load_3d(slot, &maps.wl[ld_un.layer], &my_full[ld_j % R2], x, y, z);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.vl[ld_un.layer], &my_full[ld_j % R2], x, y, z);
+      ++ld_j;
+      ld_c += 2;
+      if (ld_c >= ld_un.nc) {
+        ld_c = half;
+        if (++ld_n < my_units) ld_un = decode_punit(p, ld_n, pb, pairs);
+      }
     };
     if (lane == 0)
-      for (int j = 0; j < R; ++j) load_chunk(j);
+      for (int j = 0; j < R2; ++j) load_next();
 
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     bool ok = true;
@@ -573,14 +596,15 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
       if (!ok) { if (lane == 0) atomicExch(p.err_flag, 34); break; }
       tc_fence_after_sync();
 #pragma unroll 1
-      for (int ci = 0; ci < un.nc; ++ci, ++j) {
-        uint8_t* slot = my_ring + (j % R) * kSlotBytes;
+      for (int ci = half; ci < un.nc; ci += 2, ++j) {
+        uint8_t* slot = my_ring + (j % R2) * kSlotBytes;
         uint32_t r[32];
         tmem_ld_32x32(taddr + buf * PN + ci * 32, r);
-        ok = __all_sync(0xffffffffu, mbar_wait(&my_full[j % R], (j / R) & 1));
+        ok = __all_sync(0xffffffffu, mbar_wait(&my_full[j % R2], (j / R2) & 1));
         tmem_ld_wait();
-        if (ci == un.nc - 1) {
-          // the accumulator has been read: tell the leader's MMA warp (8 arrivals free the buffer)
+        if (ci + 2 >= un.nc) {
+          // this warp's part of the accumulator has been read: tell the leader's MMA warp (16 arrivals, the
+          // eight update warps of both CTAs, free the buffer)
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + (uint32_t)(buf * 8));
@@ -623,7 +647,7 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
           if (has_v) tma_store_3d(&maps.v[un.layer], slot + kSlotBytes / 2, x, y, g);
           bulk_commit();
           bulk_wait_read<1>();
-          if (j >= 1) load_chunk(j - 1 + R);
+          if (j >= 1) load_next();
         }
         __syncwarp();
       }
@@ -636,6 +660,274 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc_pair(tmem_base, 2 * PN);
+  }
+}
+
+// ---- one local step of every replica AND the averaging step, from a synchronized start ------------------------
+// With a communication period of 1 (where AdaComm ends up for most of a long run, Section 4.2) every local step
+// starts with all m replicas holding the same W and v, and ends with the average of the m updated replicas
+// (Section 2, PASGD update rule, k mod tau = 0).  Done as update-then-average, that is: read W, v of m replicas,
+// write them, read them again, write the mean m times.  Here a CTA owns a 128 x 64 block of W for ALL replicas:
+//   * the old block (W, v) comes in once, from the synchronized copy, and stays in shared memory;
+//   * for g = 0 .. m-1 the tensor core forms G_g = dZ_g^T A_g for the block (two accumulators in tensor memory, so
+//     the products of replica g+1 overlap the arithmetic of replica g), and the update warps form
+//     v_g = mu v + G_g, w_g = w - lr v_g exactly as the update kernel would and add them, in replica order, to
+//     running sums kept in registers (one thread: one row, 32 columns, both sums);
+//   * after the last replica the sums are divided by (float)m and the mean goes out to all m replicas, their bf16
+//     copies and the synchronized copy.
+// The arithmetic per element is that of tc_update_kernel followed by average_kernel (same fused multiply-adds,
+// same order of the m additions, one division), so the state is the same bit for bit; the per-replica values are
+// never written.  Traffic: 8 m + 2 m + 16 bytes per parameter instead of 2 * (16 m + 2 m).
+// Eight update warps: warp w reads tensor-memory lanes 32 (w mod 4).., the two warps of a quarter take the
+// left / right 32 columns.
+constexpr int SN = 64;                  // columns of a unit
+constexpr int kSyncThreads = 384;
+constexpr int kSyncStages = 3;
+struct SLayer {
+  int N, n_tiles, tile_begin;           // row length of W, units per row block, first unit of the layer
+  const int64_t* b_row_off;
+  __nv_bfloat16* Wb;
+};
+struct SParams {
+  SLayer layer[kMaxLayers];
+  int n_layers, total_units;
+  int K, groups, rows_per_group;
+  float lr, mu;
+  int64_t w_gstride;
+  int* err_flag;
+};
+struct SSmem {
+  static constexpr int kStageBytes = (BM + SN) * kRowsBf16 * 2;        // dZ tile + layer-input tile, 64 rows
+  static constexpr int kOperandBytes = kSyncStages * kStageBytes;
+  static constexpr int kBaseBytes = 8 * kSlotBytes;                    // 8 blocks of 32 x 32 (W and v) = the unit
+  static constexpr int kBars = 2 * kSyncStages + 4 + 2 * 8;
+  static constexpr int kTotal = 1024 + kOperandBytes + 2 * kBaseBytes + kBars * 8 + 16;
+  static_assert(kTotal <= 227 * 1024, "shared memory budget");
+};
+struct SUnit { int layer, m0, n0; };
+__device__ __forceinline__ SUnit decode_sunit(const SParams& p, int u) {
+  int l = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxLayers; ++i)
+    if (i < p.n_layers && u >= p.layer[i].tile_begin) l = i;
+  const int r = u - p.layer[l].tile_begin, nt = p.layer[l].n_tiles;
+  return SUnit{l, (r / nt) * BM, (r % nt) * SN};
+}
+
+__global__ void __launch_bounds__(kSyncThreads, 1)
+tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ SParams p) {
+  using L = SSmem;
+  constexpr int KS = kRowsBf16, MMA_K = 16, STAGES = kSyncStages;
+  constexpr int CHUNK_BYTES = KS * KB_BYTES;
+  constexpr int kABytes = BM * KS * 2;
+  constexpr uint32_t IDESC = make_idesc(1u, true, true, BM, SN);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem;
+  uint8_t* base_buf = smem + L::kOperandBytes;                 // [2][8 blocks][W 4 KB | v 4 KB]
+  uint64_t* full = reinterpret_cast<uint64_t*>(base_buf + 2 * L::kBaseBytes);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;       // [2]
+  uint64_t* tmem_empty = tmem_full + 2;       // [2]
+  uint64_t* base_full = tmem_empty + 2;       // [2][8]: the old block of update warp i of buffer b has arrived
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_full + 16);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = p.K / KS;
+  const int bx = blockIdx.x, grid = gridDim.x;
+  const int my_units = bx < p.total_units ? (p.total_units - 1 - bx) / grid + 1 : 0;
+  const int m = p.groups;
+  const bool has_v = p.mu != 0.f;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
+    for (int i = 0; i < 16; ++i) mbar_init(&base_full[i], 1);
+    fence_mbar_init();
+    for (int l = 0; l < p.n_layers; ++l) {
+      prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
+      prefetch_tmap(&maps.wl[l]); prefetch_tmap(&maps.vl[l]);
+    }
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 2 * SN);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
+
+  if (warp == 0) {
+    // ---- operand producer: for every unit, the tiles of replica 0, 1, ... in turn ----------------------------
+    if (elect_one()) {
+      const uint64_t pol = l2_policy(2);
+      int it = 0;
+      bool ok = true;
+      for (int n = 0; n < my_units && ok; ++n) {
+        const SUnit un = decode_sunit(p, bx + n * grid);
+        const CUtensorMap* tmA = &maps.a[un.layer];
+        const CUtensorMap* tmB = &maps.b[un.layer];
+        const int64_t* b_off = p.layer[un.layer].b_row_off;
+        for (int g = 0; g < m && ok; ++g) {
+          const int a_row = g * p.rows_per_group;
+          const int b_row = b_off ? (int)b_off[g] : a_row;
+          for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            const int s = it % STAGES;
+            if (!mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1)) { atomicExch(p.err_flag, 51); ok = false; break; }
+            mbar_expect_tx(&full[s], L::kStageBytes);
+            uint8_t* sa = stage_base + s * L::kStageBytes;
+            issue_mn_tile<64, KS>(sa, tmA, &full[s], un.m0, BM, a_row + kb * KS, pol);
+            issue_mn_tile<64, KS>(sa + kABytes, tmB, &full[s], un.n0, SN, b_row + kb * KS, pol);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ----------------------------------------------------------------------------------------
+    if (elect_one()) {
+      int it = 0;
+      bool ok = true;
+      const int total_acc = my_units * m;
+      for (int a = 0; a < total_acc && ok; ++a) {
+        const int buf = a & 1;
+        if (!mbar_wait(&tmem_empty[buf], ((a >> 1) & 1) ^ 1)) { atomicExch(p.err_flag, 52); break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * SN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&full[s], (it / STAGES) & 1)) { atomicExch(p.err_flag, 53); ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(stage_base + s * L::kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < KS / MMA_K; ++k) {
+            const uint32_t adv = k * MMA_K * KB_BYTES;
+            const uint64_t da = make_smem_desc(a_addr + adv, CHUNK_BYTES, 1024, kSwizzle128B);
+            const uint64_t db = make_smem_desc(b_addr + adv, CHUNK_BYTES, 1024, kSwizzle128B);
+            mma_bf16(d_tmem, da, db, IDESC, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(&empty[s]);
+        }
+        if (ok) mma_commit(&tmem_full[buf]);
+      }
+    }
+  } else if (warp >= 4) {
+    // ---- update warps ------------------------------------------------------------------------------------------
+    const int q = warp & 3, half = (warp - 4) >> 2, wi = half * 4 + q;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 32);
+    const float mf = (float)m;
+    auto load_base = [&](int n) {            // lane 0: this warp's 32 x 32 block of the old W and v of unit n
+      const SUnit un = decode_sunit(p, bx + n * grid);
+      uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
+      uint64_t* bar = &base_full[(n & 1) * 8 + wi];
+      mbar_expect_tx(bar, has_v ? kSlotBytes : kSlotBytes / 2);
+      tma_load_3d(slot, &maps.wl[un.layer], bar, un.n0 + half * 32, un.m0 + q * 32, 0);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.vl[un.layer], bar, un.n0 + half * 32, un.m0 + q * 32, 0);
+    };
+    if (lane == 0 && my_units > 0) load_base(0);
+    bool ok = true;
+    int a = 0;                                // accumulators consumed so far
+    for (int n = 0; n < my_units && ok; ++n) {
+      const SUnit un = decode_sunit(p, bx + n * grid);
+      uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
+      const int ldw = p.layer[un.layer].N;
+      __nv_bfloat16* Wb = p.layer[un.layer].Wb;
+      float sw[32], sv[32];
+      ok = __all_sync(0xffffffffu, mbar_wait(&base_full[(n & 1) * 8 + wi], (n >> 1) & 1));
+      if (!ok) { if (lane == 0) atomicExch(p.err_flag, 54); break; }
+#pragma unroll 1
+      for (int g = 0; g < m; ++g, ++a) {
+        const int buf = a & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (a >> 1) & 1));
+        if (!ok) { if (lane == 0) atomicExch(p.err_flag, 55); break; }
+        tc_fence_after_sync();
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + buf * SN, r);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+        // halfway through a unit the stores of the unit before have long left shared memory: its buffer takes
+        // the old block of the next unit
+        if (g == m / 2 && lane == 0 && n + 1 < my_units) {
+          bulk_wait_read<0>();
+          load_base(n + 1);
+        }
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+          const float4 w = *reinterpret_cast<const float4*>(slot + off);
+          const float ws[4] = {w.x, w.y, w.z, w.w};
+          float vs[4] = {0.f, 0.f, 0.f, 0.f};
+          if (has_v) {
+            const float4 v = *reinterpret_cast<const float4*>(slot + kSlotBytes / 2 + off);
+            vs[0] = v.x; vs[1] = v.y; vs[2] = v.z; vs[3] = v.w;
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float gr = __uint_as_float(r[jj * 4 + e]);
+            const float step = has_v ? fmaf(p.mu, vs[e], gr) : gr;          // v_g
+            const float wn = fmaf(-p.lr, step, ws[e]);                     // w_g
+            // the mean's sum, in replica order: s = x^(0); s = s + x^(g)
+            sw[jj * 4 + e] = g == 0 ? wn : __fadd_rn(sw[jj * 4 + e], wn);
+            sv[jj * 4 + e] = g == 0 ? step : __fadd_rn(sv[jj * 4 + e], step);
+          }
+        }
+      }
+      if (!ok) break;
+      // the mean, into the block's place in shared memory, and from there to every replica and the synchronized copy
+#pragma unroll
+      for (int e = 0; e < 32; ++e) { sw[e] = __fdiv_rn(sw[e], mf); sv[e] = __fdiv_rn(sv[e], mf); }
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+        *reinterpret_cast<float4*>(slot + off) = make_float4(sw[jj * 4], sw[jj * 4 + 1], sw[jj * 4 + 2], sw[jj * 4 + 3]);
+        if (has_v)
+          *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) =
+              make_float4(sv[jj * 4], sv[jj * 4 + 1], sv[jj * 4 + 2], sv[jj * 4 + 3]);
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      const int y = un.m0 + q * 32, x = un.n0 + half * 32;
+      if (lane == 0) {
+        for (int g = 0; g < m; ++g) {
+          tma_store_3d(&maps.w[un.layer], slot, x, y, g);
+          if (has_v) tma_store_3d(&maps.v[un.layer], slot + kSlotBytes / 2, x, y, g);
+        }
+        tma_store_3d(&maps.wl[un.layer], slot, x, y, 0);
+        if (has_v) tma_store_3d(&maps.vl[un.layer], slot + kSlotBytes / 2, x, y, 0);
+        bulk_commit();
+      }
+      if (Wb != nullptr) {
+        uint32_t cp[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          __nv_bfloat162 t = __floats2bfloat162_rn(sw[2 * k], sw[2 * k + 1]);
+          cp[k] = *reinterpret_cast<uint32_t*>(&t);
+        }
+        uint32_t lo[8], hi[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { lo[k] = cp[k]; hi[k] = cp[8 + k]; }
+        __nv_bfloat16* dst = Wb + (int64_t)(y + lane) * ldw + x;
+        for (int g = 0; g < m; ++g) {
+          st_global_v8(dst + (int64_t)g * p.w_gstride, lo);
+          st_global_v8(dst + (int64_t)g * p.w_gstride + 16, hi);
+        }
+      }
+      __syncwarp();
+    }
+    if (lane == 0) bulk_wait_all();
+    tc_fence_before_sync();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 2 * SN);
   }
 }
 
@@ -662,6 +954,8 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   UParams p{};
   UMaps maps;
   int total = 0;
+  bool shared = true;
+  for (int i = 0; i < n; ++i) shared = shared && layers[i].mapWsync != nullptr && layers[i].mapVsync != nullptr;
   for (int i = 0; i < n; ++i) {
     const TcUpdateArgs& a = layers[i];
     ULayer& l = p.layer[i];
@@ -673,9 +967,11 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.Wb = a.Wb;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
+    maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
   }
   for (int i = n; i < kMaxLayers; ++i) {     // unused slots hold valid descriptors
     maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
+    maps.wl[i] = maps.wl[0]; maps.vl[i] = maps.vl[0];
   }
   p.n_layers = n; p.total_tiles = total;
   {
@@ -683,7 +979,7 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     p.full_rounds = total / ctas;
     p.tail_units = (total - p.full_rounds * ctas) * (TF32 ? 4 : 2);
   }
-  p.K = a0.B; p.groups = a0.groups; p.rows_per_group = a0.B;
+  p.K = a0.B; p.groups = a0.groups; p.rows_per_group = a0.B; p.shared_state = shared ? 1 : 0;
   p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
   const int grid = total < num_sms() ? total : num_sms();
   return launch_dep(kern, dim3(grid), dim3(kThreads), L::kTotal, st, 1, maps, p);
@@ -702,6 +998,8 @@ int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
   PParams p{};
   UMaps maps;
   int total = 0;
+  bool shared = true;
+  for (int i = 0; i < n; ++i) shared = shared && layers[i].mapWsync != nullptr && layers[i].mapVsync != nullptr;
   for (int i = 0; i < n; ++i) {
     const TcUpdateArgs& a = layers[i];
     PLayer& l = p.layer[i];
@@ -713,24 +1011,64 @@ int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.Wb = a.Wb;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
+    maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
   }
   for (int i = n; i < kMaxLayers; ++i) {
     maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
+    maps.wl[i] = maps.wl[0]; maps.vl[i] = maps.vl[0];
   }
   const int max_pairs = num_sms() / 2;
   const int pairs = total < max_pairs ? total : max_pairs;
   p.n_layers = n;
   p.full_rounds = total / pairs;
   p.tail_units = (total - p.full_rounds * pairs) * 2;
-  p.K = a0.B; p.rows_per_group = a0.B;
+  p.K = a0.B; p.rows_per_group = a0.B; p.groups = a0.groups; p.shared_state = shared ? 1 : 0;
   p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
-  return launch_dep(kern, dim3(2 * pairs), dim3(kThreads), L::kTotal, st, 2, maps, p);
+  return launch_dep(kern, dim3(2 * pairs), dim3(kPairThreads), L::kTotal, st, 2, maps, p);
 }
 
 }  // namespace
 
 bool tc_update_shape_ok(bool fp32, int M, int N, int B) {
   return M > 0 && N > 0 && B > 0 && M % BM == 0 && N % BN == 0 && B % (fp32 ? 32 : 64) == 0;
+}
+
+bool tc_sync_step_shape_ok(bool fp32, int M, int N, int B) {
+  return !fp32 && M > 0 && N > 0 && B > 0 && M % BM == 0 && N % SN == 0 && B % kRowsBf16 == 0;
+}
+
+// layers[0..n): every layer needs its synchronized-copy descriptors (mapWsync / mapVsync)
+int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
+  if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
+  for (int i = 0; i < n; ++i)
+    if (layers[i].fp32 || layers[i].mapWsync == nullptr || layers[i].mapVsync == nullptr) return cudaErrorInvalidValue;
+  static uint64_t configured = 0;
+  {
+    cudaError_t e = allow_dynamic_smem(tc_sync_step_kernel, (int)SSmem::kTotal, &configured);
+    if (e != cudaSuccess) return e;
+  }
+  const TcUpdateArgs& a0 = layers[0];
+  SParams p{};
+  UMaps maps;
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const TcUpdateArgs& a = layers[i];
+    SLayer& l = p.layer[i];
+    l.N = a.N; l.n_tiles = a.N / SN; l.tile_begin = total; l.b_row_off = a.row_off; l.Wb = a.Wb;
+    total += (a.M / BM) * (a.N / SN);
+    maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
+    maps.wl[i] = *a.mapWsync; maps.vl[i] = *a.mapVsync;
+  }
+  for (int i = n; i < kMaxLayers; ++i) {
+    maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
+    maps.wl[i] = maps.wl[0]; maps.vl[i] = maps.vl[0];
+  }
+  p.n_layers = n; p.total_units = total;
+  p.K = a0.B; p.groups = a0.groups; p.rows_per_group = a0.B;
+  p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
+  if (launches) ++*launches;
+  const int grid = total < num_sms() ? total : num_sms();
+  return launch_dep(tc_sync_step_kernel, dim3(grid), dim3(kSyncThreads), SSmem::kTotal, st, 1, maps, p);
 }
 
 int tc_update_max_layers() { return kMaxLayers; }

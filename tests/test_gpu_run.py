@@ -434,3 +434,59 @@ def test_bounded_wait_that_runs_out_is_reported_and_cleared():
     assert max_rel_err_per_tensor(p, ref.params[0], dims, True) <= 1e-4
     assert eng.lib.ls_selftest_wait_timeout(eng.h, 0) == binding.LS_ERR_INVALID_ARG
     eng.close()
+
+
+@pytest.mark.parametrize("dims,dtype,m,B,mu", [
+    ((256, 256, 128, 10), "bf16", 5, 128, 0.9),        # strips of 64 columns over three layers
+    ((1024, 1024, 10), "bf16", 16, 256, 0.9),          # 128 units on 148 SMs, sixteen replicas
+    ((2048, 1280, 10), "bf16", 2, 128, 0.0),           # no momentum buffers; more units than SMs
+    ((3072, 512, 512, 10), "fp32", 4, 128, 0.9),       # fp32 model: only the shared reads apply
+])
+def test_period_of_one_from_a_synchronized_start(dims, dtype, m, B, mu):
+    """Communication period 1 (Section 4.2: where AdaComm ends up).  Every step starts with all replicas equal, and
+    the library uses that: the update reads the old W, v once (from its synchronized copy), and for bf16 models
+    the step and its averaging are one launch that never writes the per-replica values.  Both must leave the
+    state of ls_local_steps + ls_average bit for bit: compared with a handle that is forced onto the general
+    path (its replicas are injected one by one with identical values, so the library cannot assume equality)."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    bf = dtype == "bf16"
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 43, bf16=bf)
+    K = 4
+    offs = wl.batch_row_offsets(17, K, m, 1024, B)
+    xd, yd = to_device(X, y, bf16=bf)
+    out = {}
+    for tag in ("fused", "shared_reads", "general"):
+        eng = LocalSGD(m, dims, gemm_dtype=dtype, lr=0.05, momentum=mu, batch=B)
+        eng.bind_dataset(xd, yd)
+        eng.set_params(x1)
+        losses = torch.zeros((K, m), device="cuda")
+        for k in range(K):
+            if tag == "fused":
+                eng.local_steps(1, offs[k:k + 1], losses[k:k + 1], average=True)
+            elif tag == "shared_reads":
+                eng.local_steps(1, offs[k:k + 1], losses[k:k + 1])
+                eng.average()
+            else:
+                eng.sync()
+                px, pv = eng.get_all()
+                for i in range(m):
+                    eng.set_state(i, px[i], pv[i])          # same values, but now "unknown" to the library
+                eng.local_steps(1, offs[k:k + 1], losses[k:k + 1])
+                eng.average()
+        eng.sync()
+        px, pv = eng.get_all()
+        F = eng.eval_loss(m - 1, 0, 2 * B)                  # reads the bf16 copies of the last replica
+        p_dev, v_dev = eng.state_view()
+        assert bool((p_dev[0:1] == p_dev).all())
+        out[tag] = (px, pv, F, losses.cpu().numpy())
+        eng.close()
+    for tag in ("shared_reads", "general"):
+        assert np.array_equal(out["fused"][0].view(np.uint32), out[tag][0].view(np.uint32)), tag
+        assert np.array_equal(out["fused"][1].view(np.uint32), out[tag][1].view(np.uint32)), tag
+        assert out["fused"][2] == out[tag][2], tag
+        assert np.array_equal(out["fused"][3], out[tag][3]), tag
+    # and it is still the method: against the oracle over the four periods
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(mu), 1)
+    lerr = np.max(np.abs(out["fused"][3] - ref.loss) / ref.loss)
+    assert lerr <= (2e-2 if bf else 1e-4)
