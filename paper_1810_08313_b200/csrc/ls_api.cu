@@ -342,6 +342,8 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       // W and v are read once, from the synchronized copy, instead of once per replica
       t.mapWsync = h->sync_valid ? &h->maps.wsync[l] : nullptr;
       t.mapVsync = h->sync_valid ? &h->maps.vsync[l] : nullptr;
+      t.W = params_of(h) + lay.w_off[l]; t.V = mom_of(h) + lay.w_off[l];
+      t.Wsync = sync_of(h) + lay.w_off[l]; t.Vsync = sync_of(h) + lay.stride + lay.w_off[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
       t.w_gstride = lay.stride;

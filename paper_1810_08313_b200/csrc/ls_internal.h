@@ -365,6 +365,9 @@ struct TcUpdateArgs {
   // when every replica enters the step with the same W and v: descriptors of the synchronized copy (one
   // vector, [1][M][N]) that the old values are read from instead; null otherwise
   const CUtensorMap* mapWsync; const CUtensorMap* mapVsync;
+  // the same four tensors as plain pointers (replica 0; replica stride w_gstride): the fused step + average
+  // kernel stores through them
+  float* W; float* V; float* Wsync; float* Vsync;
   bool fp32;
   const int64_t* row_off;
   __nv_bfloat16* Wb; int64_t w_gstride;

@@ -687,6 +687,8 @@ struct SLayer {
   int N, n_tiles, tile_begin;           // row length of W, units per row block, first unit of the layer
   const int64_t* b_row_off;
   __nv_bfloat16* Wb;
+  float *W, *V;                         // master weights / momentum of replica 0 (replica stride w_gstride)
+  float *Ws, *Vs;                       // the same tensors in the synchronized copy
 };
 struct SParams {
   SLayer layer[kMaxLayers];
@@ -700,7 +702,7 @@ struct SSmem {
   static constexpr int kStageBytes = (BM + SN) * kRowsBf16 * 2;        // dZ tile + layer-input tile, 64 rows
   static constexpr int kOperandBytes = kSyncStages * kStageBytes;
   static constexpr int kBaseBytes = 8 * kSlotBytes;                    // 8 blocks of 32 x 32 (W and v) = the unit
-  static constexpr int kBars = 2 * kSyncStages + 4 + 2 * 8;
+  static constexpr int kBars = 2 * kSyncStages + 4 + 3 * 2 * 8;
   static constexpr int kTotal = 1024 + kOperandBytes + 2 * kBaseBytes + kBars * 8 + 16;
   static_assert(kTotal <= 227 * 1024, "shared memory budget");
 };
@@ -731,7 +733,9 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
   uint64_t* tmem_full = empty + STAGES;       // [2]
   uint64_t* tmem_empty = tmem_full + 2;       // [2]
   uint64_t* base_full = tmem_empty + 2;       // [2][8]: the old block of update warp i of buffer b has arrived
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_full + 16);
+  uint64_t* mean_ready = base_full + 16;      // [2][8]: update warp i has left the mean of its block in buffer b
+  uint64_t* mean_gone = mean_ready + 16;      // [2][8]: the stores of that block have read shared memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mean_gone + 16);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = p.K / KS;
@@ -743,7 +747,7 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 8); }
-    for (int i = 0; i < 16; ++i) mbar_init(&base_full[i], 1);
+    for (int i = 0; i < 48; ++i) mbar_init(&base_full[i], 1);        // base_full, mean_ready, mean_gone
     fence_mbar_init();
     for (int l = 0; l < p.n_layers; ++l) {
       prefetch_tmap(&maps.a[l]); prefetch_tmap(&maps.b[l]); prefetch_tmap(&maps.w[l]); prefetch_tmap(&maps.v[l]);
@@ -815,6 +819,61 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
         if (ok) mma_commit(&tmem_full[buf]);
       }
     }
+  } else if (warp == 2 || warp == 3) {
+    // ---- store warps: one per column half.  The mean of a block goes out to every replica, to the bf16 copies
+    // and to the synchronized copy with plain 16-byte stores, eight lanes to a 128-byte row, from registers: the
+    // block is read from shared memory once and its buffer is free at once.  These warps wait for memory, not
+    // for arithmetic, so they run beside the update warps, which are already working on the next unit; and the
+    // bulk-copy engine stays free for the operand tiles (with the mean leaving through it as well, the products
+    // waited behind the queued stores: 5.6 k cycles per replica against 2 k).
+    const int half = warp - 2;
+    const int row0 = lane >> 3, piece = lane & 7;
+    bool ok = true;
+    for (int n = 0; n < my_units && ok; ++n) {
+      const SUnit un = decode_sunit(p, bx + n * grid);
+      const SLayer& ly = p.layer[un.layer];
+      const int64_t ldw = ly.N;
+      for (int q = 0; q < 4 && ok; ++q) {
+        const int wi = half * 4 + q;
+        const uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
+        ok = __all_sync(0xffffffffu, mbar_wait(&mean_ready[(n & 1) * 8 + wi], (n >> 1) & 1));
+        if (!ok) { if (lane == 0) atomicExch(p.err_flag, 57); break; }
+        float4 w4[8], v4[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int row = i * 4 + row0;
+          w4[i] = *reinterpret_cast<const float4*>(slot + row * 128 + ((piece ^ (row & 7)) << 4));
+          if (has_v) v4[i] = *reinterpret_cast<const float4*>(slot + kSlotBytes / 2 + row * 128 + ((piece ^ (row & 7)) << 4));
+        }
+        // the block is in registers: release its buffer (the arrival orders the reads above before it)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&mean_gone[(n & 1) * 8 + wi]);
+        uint2 cp[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(w4[i].x, w4[i].y);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(w4[i].z, w4[i].w);
+          cp[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+        }
+        const int64_t at = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
+        for (int g = 0; g <= m; ++g) {
+          // g = m: the synchronized copy
+          float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + at;
+          float* Vd = (g < m ? ly.V + (int64_t)g * p.w_gstride : ly.Vs) + at;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Wd + (int64_t)i * 4 * ldw) = w4[i];
+          if (has_v) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Vd + (int64_t)i * 4 * ldw) = v4[i];
+          }
+          if (ly.Wb != nullptr && g < m) {
+            __nv_bfloat16* Bd = ly.Wb + (int64_t)g * p.w_gstride + at;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(Bd + (int64_t)i * 4 * ldw) = cp[i];
+          }
+        }
+      }
+    }
   } else if (warp >= 4) {
     // ---- update warps ------------------------------------------------------------------------------------------
     const int q = warp & 3, half = (warp - 4) >> 2, wi = half * 4 + q;
@@ -851,11 +910,14 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tmem_empty[buf]);
-        // halfway through a unit the stores of the unit before have long left shared memory: its buffer takes
-        // the old block of the next unit
-        if (g == m / 2 && lane == 0 && n + 1 < my_units) {
-          bulk_wait_read<0>();
-          load_base(n + 1);
+        // halfway through a unit the stores of the unit before have normally left shared memory: its buffer
+        // takes the old block of the next unit
+        if (g == m / 2 && n + 1 < my_units) {
+          if (n >= 1) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&mean_gone[((n + 1) & 1) * 8 + wi], (((n + 1) >> 1) - 1) & 1));
+            if (!ok) { if (lane == 0) atomicExch(p.err_flag, 56); break; }
+          }
+          if (lane == 0) load_base(n + 1);
         }
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
@@ -890,37 +952,11 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
           *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) =
               make_float4(sv[jj * 4], sv[jj * 4 + 1], sv[jj * 4 + 2], sv[jj * 4 + 3]);
       }
+      // hand the block to the store warp of this column half and go on with the next unit
       fence_proxy_async_smem();
       __syncwarp();
-      const int y = un.m0 + q * 32, x = un.n0 + half * 32;
-      if (lane == 0) {
-        for (int g = 0; g < m; ++g) {
-          tma_store_3d(&maps.w[un.layer], slot, x, y, g);
-          if (has_v) tma_store_3d(&maps.v[un.layer], slot + kSlotBytes / 2, x, y, g);
-        }
-        tma_store_3d(&maps.wl[un.layer], slot, x, y, 0);
-        if (has_v) tma_store_3d(&maps.vl[un.layer], slot + kSlotBytes / 2, x, y, 0);
-        bulk_commit();
-      }
-      if (Wb != nullptr) {
-        uint32_t cp[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          __nv_bfloat162 t = __floats2bfloat162_rn(sw[2 * k], sw[2 * k + 1]);
-          cp[k] = *reinterpret_cast<uint32_t*>(&t);
-        }
-        uint32_t lo[8], hi[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { lo[k] = cp[k]; hi[k] = cp[8 + k]; }
-        __nv_bfloat16* dst = Wb + (int64_t)(y + lane) * ldw + x;
-        for (int g = 0; g < m; ++g) {
-          st_global_v8(dst + (int64_t)g * p.w_gstride, lo);
-          st_global_v8(dst + (int64_t)g * p.w_gstride + 16, hi);
-        }
-      }
-      __syncwarp();
+      if (lane == 0) mbar_arrive(&mean_ready[(n & 1) * 8 + wi]);
     }
-    if (lane == 0) bulk_wait_all();
     tc_fence_before_sync();
   }
   __syncthreads();
@@ -1041,7 +1077,9 @@ bool tc_sync_step_shape_ok(bool fp32, int M, int N, int B) {
 int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
   for (int i = 0; i < n; ++i)
-    if (layers[i].fp32 || layers[i].mapWsync == nullptr || layers[i].mapVsync == nullptr) return cudaErrorInvalidValue;
+    if (layers[i].fp32 || layers[i].mapWsync == nullptr || layers[i].mapVsync == nullptr || layers[i].W == nullptr ||
+        layers[i].V == nullptr || layers[i].Wsync == nullptr || layers[i].Vsync == nullptr)
+      return cudaErrorInvalidValue;
   static uint64_t configured = 0;
   {
     cudaError_t e = allow_dynamic_smem(tc_sync_step_kernel, (int)SSmem::kTotal, &configured);
@@ -1055,6 +1093,7 @@ int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int6
     const TcUpdateArgs& a = layers[i];
     SLayer& l = p.layer[i];
     l.N = a.N; l.n_tiles = a.N / SN; l.tile_begin = total; l.b_row_off = a.row_off; l.Wb = a.Wb;
+    l.W = a.W; l.V = a.V; l.Ws = a.Wsync; l.Vs = a.Vsync;
     total += (a.M / BM) * (a.N / SN);
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = *a.mapWsync; maps.vl[i] = *a.mapVsync;
