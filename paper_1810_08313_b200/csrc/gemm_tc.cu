@@ -1128,7 +1128,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
   p.a = Operand{nullptr, a.M, 0, 0, 0};
-  p.b = Operand{nullptr, 0, 0, 1, 1};
+  p.b = Operand{nullptr, 0, 0, a.w_zstep, 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.C = a.C; p.act = a.act; p.err_flag = a.err_flag;
   if (a.bias != nullptr && tc_dx_fuses_bias(a.fp32, a.M, a.N)) {

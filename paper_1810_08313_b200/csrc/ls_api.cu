@@ -173,8 +173,11 @@ __global__ void wait_timeout_selftest_kernel(int* err_flag, long long limit) {
 // x maps: [0] for K-major reads, [1] for MN-major reads of the mini-batch rows
 struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; const CUtensorMap* upd; };
 
+// shared_w: the groups are different replicas whose weights are known to be bitwise equal (first step after an
+// averaging step): the tensor-core layers all read replica 0's operand copy, which then stays in L2.
 static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
-                   int groups, int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out) {
+                   int groups, int64_t replica0, int64_t w_gstride, bool want_dz, float* loss_out,
+                   bool shared_w = false) {
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
   const float* P = params_of(h) + replica0 * lay.stride;
@@ -204,7 +207,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       t.maps.a = (l == 0) ? xmap.k : &h->maps.act[l];
       t.maps.b = &h->maps.w[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
-      t.w_z0 = (int)replica0; t.w_zstep = w_gstride != 0 ? 1 : 0;
+      t.w_z0 = (int)replica0; t.w_zstep = (w_gstride != 0 && !shared_w) ? 1 : 0;
       t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
       t.bias_gstride = w_gstride;
       t.C = h->state + lay.act_off[l + 1];
@@ -267,7 +270,8 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   const Layout& lay = h->lay;
   const bool bf = lay.bf16;
   const TcMaps& mn = bf ? h->maps : h->maps_mn;     // descriptors for MN-major reads
-  int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out);
+  const bool shared_w = h->sync_valid;
+  int rc = forward(h, x, xmap, y, row_off_dev, lay.m, 0, lay.stride, true, loss_out, shared_w);
   if (rc != LS_OK) return rc;
   bool bias_done[LS_MAX_LAYERS] = {false};     // bias l already updated by the kernel that produced dZ_l
   // Weight updates that run on the streaming tensor-core kernel are collected and launched together after
@@ -310,6 +314,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.c_map = (bf && lay.dims[l] % 8 == 0) ? &h->maps.dz[l - 1] : nullptr;
       t.act_map = (bf && lay.dims[l] % 8 == 0) ? &h->maps.act[l] : nullptr;
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
+      t.w_zstep = shared_w ? 0 : 1;
       t.bias = nullptr; t.vbias = nullptr; t.bias_gstride = lay.stride; t.lr = h->lr; t.mu = h->mu;
       if (lay.has_bias && tc_dx_fuses_bias(!bf, t.M, t.N)) {
         t.bias = params_of(h) + lay.b_off[l - 1];

@@ -339,6 +339,7 @@ struct TcDxArgs {
   const void* act; void* C;
   const CUtensorMap* c_map;   // bf16: C and act as 2-D tensors [groups*M][N], boxes of 64 x 64, or null
   const CUtensorMap* act_map;
+  int w_zstep;               // replica whose weights group g reads = g * w_zstep (0: every group reads replica 0's)
   int M, N, K, groups;
   // bias / its momentum of the layer that produced `act` (group 0; replica stride bias_gstride): updated
   // from the column sums of C inside the kernel when tc_dx_fuses_bias(); else null
