@@ -781,6 +781,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3_mlp_bf16", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--replicas", type=int, default=0,
+                    help="run the workload with this many replicas instead of its own count (a smaller footprint for "
+                         "profiler captures; the line's workload name then ends in @mN)")
     ap.add_argument("--shard", action="store_true",
                     help="with --gpus N: one job whose m replicas are dealt out over the N ranks (m / N each) with one "
                          "NCCL all-gather of partial sums per averaging step, instead of N independent jobs")
@@ -803,6 +806,9 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = wl.WORKLOADS[args.workload]
+    if args.replicas:
+        import dataclasses
+        w = dataclasses.replace(w, m=int(args.replicas), name=f"{w.name}@m{int(args.replicas)}")
     if args.impl == "reference":
         run_reference(args, w)
     else:

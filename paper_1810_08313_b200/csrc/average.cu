@@ -71,7 +71,8 @@ __device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&v)[W]
 template <int M, int W, bool BM>
 __global__ void __launch_bounds__(kThreads)
 average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n_vec, int64_t stride,
-               __nv_bfloat16* __restrict__ shadow, BlockMomentum bm, float* __restrict__ sync_out, int64_t sync_stride) {
+               __nv_bfloat16* __restrict__ shadow, BlockMomentum bm, float* __restrict__ sync_out, int64_t sync_stride,
+               TileMap tiles) {
   grid_dep_wait();
   grid_dep_launch();
   const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -125,8 +126,10 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
   for (int j = 0; j < m; ++j) s.store(p + (int64_t)j * stride);
   // the synchronized copy: what every replica holds now (read by the next local step while they are still equal)
   if (sync_out != nullptr) s.store(sync_out + (int64_t)blockIdx.y * sync_stride + i * W);
-  if (blockIdx.y == 0 && shadow != nullptr)
-    for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + i * W, s.v);
+  if (blockIdx.y == 0 && shadow != nullptr) {
+    const int64_t at = rowmajor_index(tiles, i * W);      // the bf16 copies are row-major
+    for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + at, s.v);
+  }
 }
 
 // Scalar path: the ragged tail (n mod W elements) and buffers that are not
@@ -134,7 +137,7 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
 __global__ void __launch_bounds__(kThreads)
 average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64_t first, int64_t n, int64_t stride,
                       __nv_bfloat16* __restrict__ shadow, BlockMomentum bm, float* __restrict__ sync_out,
-                      int64_t sync_stride) {
+                      int64_t sync_stride, TileMap tiles) {
   grid_dep_wait();
   grid_dep_launch();
   float* buf = base + (int64_t)blockIdx.y * buf_stride;
@@ -154,14 +157,16 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
   }
   for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
   if (sync_out != nullptr) sync_out[(int64_t)blockIdx.y * sync_stride + i] = mean;
-  if (blockIdx.y == 0 && shadow != nullptr)
-    for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + i] = __float2bfloat16_rn(mean);
+  if (blockIdx.y == 0 && shadow != nullptr) {
+    const int64_t at = rowmajor_index(tiles, i);
+    for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + at] = __float2bfloat16_rn(mean);
+  }
 }
 
 template <int W, bool BM>
 void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
-                __nv_bfloat16* shadow, const BlockMomentum& bm, float* sync_out, int64_t sync_stride) {
-#define LS_AVG(M) launch_dep(average_kernel<M, W, BM>, grid, dim3(kThreads), 0, st, 1, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride)
+                __nv_bfloat16* shadow, const BlockMomentum& bm, float* sync_out, int64_t sync_stride, const TileMap& tiles) {
+#define LS_AVG(M) launch_dep(average_kernel<M, W, BM>, grid, dim3(kThreads), 0, st, 1, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride, tiles)
   switch (m) {
     case 2: LS_AVG(2); break;
     case 4: LS_AVG(4); break;
@@ -178,8 +183,9 @@ inline bool aligned_to(const void* p, size_t a) { return p == nullptr || reinter
 
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
                    __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches, const BlockMomentum* bmp, float* sync_out,
-                   int64_t sync_stride) {
+                   int64_t sync_stride, const TileMap* tilesp) {
   if (sync_stride <= 0) sync_stride = n;
+  const TileMap tiles = tilesp ? *tilesp : TileMap{};
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
   BlockMomentum bm{nullptr, nullptr, 0.f, 0.f};
   if (bmp != nullptr) {
@@ -201,11 +207,11 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
     if (W == 8) {
-      if (BM) launch_vec<8, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride);
-      else launch_vec<8, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride);
+      if (BM) launch_vec<8, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride, tiles);
+      else launch_vec<8, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride, tiles);
     } else {
-      if (BM) launch_vec<4, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride);
-      else launch_vec<4, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride);
+      if (BM) launch_vec<4, true>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride, tiles);
+      else launch_vec<4, false>(grid, st, base, buf_stride, m, n_vec, stride, shadow, bm, sync_out, sync_stride, tiles);
     }
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
@@ -217,7 +223,7 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     if (gx > 2147483647LL) return cudaErrorInvalidValue;
     dim3 grid((unsigned)gx, (unsigned)n_buf);
     launch_dep(average_scalar_kernel, grid, dim3(kThreads), 0, st, 1, base, buf_stride, m, first, n, stride, shadow, bm,
-               sync_out, sync_stride);
+               sync_out, sync_stride, tiles);
     if (launches) ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -231,7 +237,7 @@ extern "C" int ls_average_flat(float* buf_dev, int m, int64_t P, int64_t stride,
   if (buf_dev == nullptr || m < 1 || P < 0 || stride < P) return LS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(buf_dev) % 4 != 0) return LS_ERR_INVALID_ARG;
   int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr,
-                             nullptr, nullptr, 0);
+                             nullptr, nullptr, 0, nullptr);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
@@ -245,6 +251,6 @@ extern "C" int ls_block_average_flat(float* buf_dev, float* anchor_dev, float* u
     return LS_ERR_INVALID_ARG;
   ls::BlockMomentum bm{anchor_dev, u_dev, lr, beta};
   int e = ls::launch_average(buf_dev, 1, 0, m, P, stride, nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr,
-                             &bm, nullptr, 0);
+                             &bm, nullptr, 0, nullptr);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

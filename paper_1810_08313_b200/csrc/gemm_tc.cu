@@ -1077,8 +1077,11 @@ int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int
   return make_map(out, base, fp32, mn32, false, 3, rows, cols, groups, gstride);
 }
 // 3-D map over fp32 matrices read and written in 32 x 32 blocks (128-byte swizzle, 16-byte units).
+// blocked: the matrix is stored as 32 x 32 blocks (TileMap): block b is rows [32 b, 32 b + 32) of a
+// [rows * cols / 32][32] matrix, i.e. box coordinates (0, 32 b).
 int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups,
-                         int64_t gstride) {
+                         int64_t gstride, bool blocked) {
+  if (blocked) return make_map(out, base, true, false, true, 3, rows * cols / 32, 32, groups, gstride);
   return make_map(out, base, true, false, true, 3, rows, cols, groups, gstride);
 }
 

@@ -102,9 +102,26 @@ bias_kernel(const TD* __restrict__ dZ, float* __restrict__ bias, float* __restri
 }
 
 __global__ void __launch_bounds__(kThreads)
-to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t n) {
+to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int64_t n, TileMap tiles) {
   const int64_t step = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) dst[i] = __float2bfloat16_rn(src[i]);
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) {
+    const int64_t rep = i / stride, e = i - rep * stride;
+    dst[rep * stride + rowmajor_index(tiles, e)] = __float2bfloat16_rn(src[i]);
+  }
+}
+
+// one CTA per 32 x 32 block; a warp moves one 128-byte row at a time on both sides
+__global__ void __launch_bounds__(kThreads)
+retile_kernel(float* __restrict__ dst, const float* __restrict__ src, int rows, int cols, int to_blocked) {
+  const int nb = cols >> 5;
+  const int64_t blk = blockIdx.x;
+  const int rb = (int)(blk / nb), cb = (int)(blk % nb);
+  const int c = threadIdx.x & 31, r0 = threadIdx.x >> 5;
+  for (int r = r0; r < 32; r += kThreads / 32) {
+    const int64_t rm = (int64_t)(rb * 32 + r) * cols + cb * 32 + c, bl = blk * 1024 + r * 32 + c;
+    if (to_blocked) dst[bl] = src[rm];
+    else dst[rm] = src[bl];
+  }
 }
 
 }  // namespace
@@ -128,12 +145,21 @@ int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches
                     a.vbias, a.gstride, a.B, a.N, a.lr, a.mu);
 }
 
-int launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st, int64_t* launches) {
+int launch_to_bf16(const float* src, __nv_bfloat16* dst, int m, int64_t stride, const TileMap* tiles, cudaStream_t st,
+                   int64_t* launches) {
+  const int64_t n = (int64_t)m * stride;
   if (n <= 0) return cudaSuccess;
   if (launches) ++*launches;
   int64_t gx = (n + kThreads - 1) / kThreads;
   if (gx > 148 * 16) gx = 148 * 16;
-  to_bf16_kernel<<<(unsigned)gx, kThreads, 0, st>>>(src, dst, n);
+  to_bf16_kernel<<<(unsigned)gx, kThreads, 0, st>>>(src, dst, stride, n, tiles ? *tiles : TileMap{});
+  return cudaGetLastError();
+}
+
+int launch_retile(float* dst, const float* src, int rows, int cols, bool to_blocked, cudaStream_t st, int64_t* launches) {
+  if (rows <= 0 || cols <= 0 || rows % 32 != 0 || cols % 32 != 0) return cudaErrorInvalidValue;
+  if (launches) ++*launches;
+  retile_kernel<<<(unsigned)((int64_t)rows * cols / 1024), kThreads, 0, st>>>(dst, src, rows, cols, to_blocked ? 1 : 0);
   return cudaGetLastError();
 }
 

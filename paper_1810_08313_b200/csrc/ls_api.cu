@@ -91,6 +91,14 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   lay.stage_loss_off = take((size_t)kRowOffCap * m * 4);
   lay.err_off = take(256);
   lay.sync_off = take((size_t)2 * lay.stride * 4);
+  // bf16 models: the master copy of every matrix that the streaming update kernels own is stored in 32 x 32
+  // blocks (see TileMap); fp32 models keep row-major matrices, because their GEMMs read the master copy itself
+  size_t retile = 0;
+  for (int l = 0; l < lay.L; ++l) {
+    lay.tiled[l] = lay.bf16 && tc_update_shape_ok(false, lay.dims[l + 1], lay.dims[l], batch) ? 1 : 0;
+    if (lay.tiled[l]) retile = std::max(retile, (size_t)lay.dims[l + 1] * lay.dims[l] * 4);
+  }
+  if (retile) lay.retile_off = take(retile);
   if (spec->momentum_mode == LS_MOMENTUM_BLOCK) {
     lay.anchor_off = take((size_t)lay.stride * 4);
     lay.blocku_off = take((size_t)lay.stride * 4);
@@ -134,7 +142,9 @@ struct ProfScope {
 // Refresh the bf16 operand copies of the weights (bf16 models).
 static int refresh_shadow(ls_handle* h) {
   const int64_t n = (int64_t)h->lay.m * h->lay.stride;
-  if (h->lay.bf16) LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), n, h->stream, &h->launches));
+  (void)n;
+  if (h->lay.bf16)
+    LS_CUDA(h, launch_to_bf16(params_of(h), shadow_of(h), h->lay.m, h->lay.stride, &h->tiles, h->stream, &h->launches));
   return LS_OK;
 }
 
@@ -349,6 +359,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.mapVsync = h->sync_valid ? &h->maps.vsync[l] : nullptr;
       t.W = params_of(h) + lay.w_off[l]; t.V = mom_of(h) + lay.w_off[l];
       t.Wsync = sync_of(h) + lay.w_off[l]; t.Vsync = sync_of(h) + lay.stride + lay.w_off[l];
+      t.blocked = lay.tiled[l] != 0;
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
       t.w_gstride = lay.stride;
@@ -466,7 +477,7 @@ static int average(ls_handle* h) {
     }
     LS_CUDA(h, launch_combine(parts, h->shard_fn ? h->shard_G : 1, (int64_t)n_buf * lay.stride, lay.stride,
                               h->shard_m_total, lay.stride, params_of(h), n_buf, buf_stride, lay.m, lay.stride,
-                              shadow_of(h), h->stream, &h->launches));
+                              shadow_of(h), h->stream, &h->launches, &h->tiles));
     if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
       LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
     h->sync_valid = false;         // the combining kernel keeps no synchronized copy
@@ -476,7 +487,7 @@ static int average(ls_handle* h) {
     ProfScope ps(h, LS_K_AVG, 0);
     BlockMomentum bm{anchor_of(h), blocku_of(h), h->lr, h->spec.block_momentum};
     LS_CUDA(h, launch_average(params_of(h), both ? 2 : 1, buf_stride, lay.m, lay.stride, lay.stride,
-                              shadow_of(h), h->stream, &h->launches, block ? &bm : nullptr, sync_of(h)));
+                              shadow_of(h), h->stream, &h->launches, block ? &bm : nullptr, sync_of(h), 0, &h->tiles));
   }
   if (h->mu != 0.f && (h->spec.momentum_mode == LS_MOMENTUM_RESET || block)) {
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
@@ -609,6 +620,12 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
   h->state = static_cast<char*>(state_dev);
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->allow_pair = pair_kernels_enabled();
+  for (int l = 0; l < lay.L; ++l)
+    if (lay.tiled[l]) {
+      TileMap& tm = h->tiles;
+      tm.begin[tm.n] = lay.w_off[l]; tm.size[tm.n] = (int64_t)lay.dims[l + 1] * lay.dims[l]; tm.cols[tm.n] = lay.dims[l];
+      ++tm.n;
+    }
   int e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
   for (int s = 0; s < 2 && e == cudaSuccess; ++s) {
     e = cudaEventCreateWithFlags(&h->ev_copied[s], cudaEventDisableTiming);
@@ -642,11 +659,13 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
       if (!mn) {
         for (int l = 0; l < lay.L; ++l)
           if (lay.dims[l] % 4 == 0) {
-            ok(tc_make_block_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
-            ok(tc_make_block_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride));
-            ok(tc_make_block_map_3d(&mp.wsync[l], sync_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], 1, lay.stride));
+            const bool blk = lay.tiled[l] != 0;
+            ok(tc_make_block_map_3d(&mp.wf[l], params_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride, blk));
+            ok(tc_make_block_map_3d(&mp.vf[l], mom_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], m, lay.stride, blk));
+            ok(tc_make_block_map_3d(&mp.wsync[l], sync_of(h) + lay.w_off[l], lay.dims[l + 1], lay.dims[l], 1, lay.stride,
+                                    blk));
             ok(tc_make_block_map_3d(&mp.vsync[l], sync_of(h) + lay.stride + lay.w_off[l], lay.dims[l + 1], lay.dims[l], 1,
-                                    lay.stride));
+                                    lay.stride, blk));
           }
       }
       if (lay.dims[0] % q == 0) {
@@ -713,8 +732,26 @@ int ls_set_lr(ls_handle* h, float lr) {
 // copy one replica between the flat interface layout (host) and the padded device layout
 static int copy_replica(ls_handle* h, float* dev_base, float* host, bool to_dev) {
   const Layout& lay = h->lay;
+  float* stage = reinterpret_cast<float*>(h->state + lay.retile_off);
   for (int l = 0; l < lay.L; ++l) {
     const size_t wn = (size_t)lay.dims[l + 1] * lay.dims[l] * 4, bn = (size_t)lay.dims[l + 1] * 4;
+    if (lay.tiled[l]) {
+      // the interface is row-major, the device keeps this matrix in 32 x 32 blocks: through the staging buffer
+      if (to_dev) {
+        LS_CUDA(h, cudaMemcpyAsync(stage, host + lay.w_flat[l], wn, cudaMemcpyHostToDevice, h->stream));
+        LS_CUDA(h, launch_retile(dev_base + lay.w_off[l], stage, lay.dims[l + 1], lay.dims[l], true, h->stream, &h->launches));
+      } else {
+        LS_CUDA(h, launch_retile(stage, dev_base + lay.w_off[l], lay.dims[l + 1], lay.dims[l], false, h->stream, &h->launches));
+        LS_CUDA(h, cudaMemcpyAsync(host + lay.w_flat[l], stage, wn, cudaMemcpyDeviceToHost, h->stream));
+      }
+      if (lay.has_bias) {
+        if (to_dev)
+          LS_CUDA(h, cudaMemcpyAsync(dev_base + lay.b_off[l], host + lay.b_flat[l], bn, cudaMemcpyHostToDevice, h->stream));
+        else
+          LS_CUDA(h, cudaMemcpyAsync(host + lay.b_flat[l], dev_base + lay.b_off[l], bn, cudaMemcpyDeviceToHost, h->stream));
+      }
+      continue;
+    }
     if (to_dev) {
       LS_CUDA(h, cudaMemcpyAsync(dev_base + lay.w_off[l], host + lay.w_flat[l], wn, cudaMemcpyHostToDevice, h->stream));
       if (lay.has_bias)
@@ -931,7 +968,7 @@ int ls_shard_average(ls_handle* h, const float* gathered_dev, int n_gpus, int m_
   const int n_buf = both ? 2 : 1;
   LS_CUDA(h, launch_combine(gathered_dev, n_gpus, (int64_t)n_buf * lay.stride, lay.stride, m_total, lay.stride,
                             params_of(h), n_buf, (int64_t)((lay.mom_off - lay.params_off) / 4), lay.m, lay.stride,
-                            shadow_of(h), h->stream, &h->launches));
+                            shadow_of(h), h->stream, &h->launches, &h->tiles));
   if (h->mu != 0.f && h->spec.momentum_mode == LS_MOMENTUM_RESET)
     LS_CUDA(h, cudaMemsetAsync(mom_of(h), 0, (size_t)lay.m * lay.stride * 4, h->stream));
   h->sync_valid = false;

@@ -78,7 +78,7 @@ partial_sum_kernel(const float* __restrict__ base, int64_t buf_stride, int m, in
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(const float* __restrict__ parts, int G, int64_t part_stride, int64_t part_buf_stride, float m_total,
                int64_t n, float* __restrict__ base, int64_t buf_stride, int m_local, int64_t stride,
-               __nv_bfloat16* __restrict__ shadow) {
+               __nv_bfloat16* __restrict__ shadow, TileMap tiles) {
   grid_dep_wait();
   grid_dep_launch();
   const int64_t n_vec = n / 8;
@@ -97,16 +97,19 @@ combine_kernel(const float* __restrict__ parts, int G, int64_t part_stride, int6
         __nv_bfloat162 t = __floats2bfloat162_rn(s.v[2 * e], s.v[2 * e + 1]);
         u[e] = *reinterpret_cast<uint32_t*>(&t);
       }
+      const int64_t at = rowmajor_index(tiles, i * 8);      // the bf16 copies are row-major
       for (int j = 0; j < m_local; ++j)
-        *reinterpret_cast<uint4*>(shadow + (int64_t)j * stride + i * 8) = make_uint4(u[0], u[1], u[2], u[3]);
+        *reinterpret_cast<uint4*>(shadow + (int64_t)j * stride + at) = make_uint4(u[0], u[1], u[2], u[3]);
     }
   } else {
     const int64_t e = n_vec * 8 + (i - n_vec);
     if (e < n) {
       const float mean = __fdiv_rn(ordered_sum_scalar(src + e, G, part_stride), m_total);
       for (int j = 0; j < m_local; ++j) dst[(int64_t)j * stride + e] = mean;
-      if (blockIdx.y == 0 && shadow != nullptr)
-        for (int j = 0; j < m_local; ++j) shadow[(int64_t)j * stride + e] = __float2bfloat16_rn(mean);
+      if (blockIdx.y == 0 && shadow != nullptr) {
+        const int64_t at = rowmajor_index(tiles, e);
+        for (int j = 0; j < m_local; ++j) shadow[(int64_t)j * stride + at] = __float2bfloat16_rn(mean);
+      }
     }
   }
 }
@@ -129,7 +132,7 @@ int launch_partial_sum(const float* base, int n_buf, int64_t buf_stride, int m, 
 
 int launch_combine(const float* parts, int G, int64_t part_stride, int64_t part_buf_stride, int m_total, int64_t n,
                    float* base, int n_buf, int64_t buf_stride, int m_local, int64_t stride, __nv_bfloat16* shadow,
-                   cudaStream_t st, int64_t* launches) {
+                   cudaStream_t st, int64_t* launches, const TileMap* tiles) {
   if (n <= 0 || n_buf <= 0) return cudaSuccess;
   if (!aligned32(parts) || !aligned32(base) || stride % 8 != 0 || buf_stride % 8 != 0 || part_stride % 8 != 0 ||
       part_buf_stride % 8 != 0 || reinterpret_cast<uintptr_t>(shadow) % 16 != 0 ||
@@ -137,7 +140,8 @@ int launch_combine(const float* parts, int G, int64_t part_stride, int64_t part_
     return cudaErrorInvalidValue;
   if (launches) ++*launches;
   return launch_dep(combine_kernel, dim3(grid_x(n), (unsigned)n_buf), dim3(kThreads), 0, st, 1, parts, G, part_stride,
-                    part_buf_stride, (float)m_total, n, base, buf_stride, m_local, stride, shadow);
+                    part_buf_stride, (float)m_total, n, base, buf_stride, m_local, stride, shadow,
+                    tiles ? *tiles : TileMap{});
 }
 
 }  // namespace ls
@@ -160,6 +164,6 @@ extern "C" int ls_combine_partials_flat(const float* partials_dev, int G, int64_
       part_stride % 8 != 0 || dst_stride % 8 != 0)
     return LS_ERR_INVALID_ARG;
   int e = ls::launch_combine(partials_dev, G, part_stride, 0, m_total, P, dst_dev, 1, 0, m_local, dst_stride, nullptr,
-                             static_cast<cudaStream_t>(cuda_stream), nullptr);
+                             static_cast<cudaStream_t>(cuda_stream), nullptr, nullptr);
   return e == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

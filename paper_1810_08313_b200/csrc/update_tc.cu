@@ -50,6 +50,7 @@ struct ULayer {
   int tile_begin;                      // first tile of this layer in the launch's list
   const int64_t* b_row_off;            // layer input = dataset rows: first row of replica g, else null
   __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
+  int blocked;                         // W, v stored as 32 x 32 blocks (TileMap): box coordinates differ
 };
 struct UParams {
   ULayer layer[kMaxLayers];
@@ -104,6 +105,14 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* s
                    reinterpret_cast<uint64_t>(m)),
                "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
                : "memory");
+}
+// Box coordinates of the 32 x 32 block at row y, column x of a matrix with rows of ldw elements: (x, y) in a
+// row-major matrix; in blocked storage block b is rows 32 b .. of a [.][32] matrix.
+__device__ __forceinline__ void block_coords(int blocked, int ldw, int& x, int& y) {
+  if (blocked) {
+    y = ((y >> 5) * (ldw >> 5) + (x >> 5)) << 5;
+    x = 0;
+  }
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
@@ -296,7 +305,8 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
       const Unit un = decode_unit<SUB>(p, n, bx, grid);
       const Tile tl = un.tl;
       const int c = j < full_chunks ? (j & 3) : un.c0 + (j - full_chunks) % NCS;
-      const int y = tl.m0 + q * 32, x = tl.n0 + c * 32;
+      int y = tl.m0 + q * 32, x = tl.n0 + c * 32;
+      block_coords(p.layer[tl.layer].blocked, p.layer[tl.layer].N, x, y);
       uint8_t* slot = my_ring + (j % R) * kSlotBytes;
       mbar_expect_tx(&my_full[j % R], has_v ? kSlotBytes : kSlotBytes / 2);
       const int z = p.shared_state ? 0 : tl.g;
@@ -369,7 +379,8 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          const int y = m0 + q * 32, x = n0 + c * 32;
+          int y = m0 + q * 32, x = n0 + c * 32;
+          block_coords(p.layer[tl.layer].blocked, ldw, x, y);
           tma_store_3d(&maps.w[tl.layer], slot, x, y, g);
           if (has_v) tma_store_3d(&maps.v[tl.layer], slot + kSlotBytes / 2, x, y, g);
           bulk_commit();
@@ -406,6 +417,7 @@ struct PLayer {
   int N, n_tiles, tiles_per_group, tile_begin;
   const int64_t* b_row_off;
   __nv_bfloat16* Wb;
+  int blocked;
 };
 struct PParams {
   PLayer layer[kMaxLayers];
@@ -567,7 +579,8 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
     PUnit ld_un = decode_punit(p, 0, pb, pairs);
     auto load_next = [&]() {
       if (ld_j >= my_chunks) return;
-      const int y = ld_un.m0 + rank * BM + q * 32, x = ld_un.n0 + ld_c * 32;
+      int y = ld_un.m0 + rank * BM + q * 32, x = ld_un.n0 + ld_c * 32;
+      block_coords(p.layer[ld_un.layer].blocked, p.layer[ld_un.layer].N, x, y);
       uint8_t* slot = my_ring + (ld_j % R2) * kSlotBytes;
       mbar_expect_tx(&my_full[ld_j % R2], has_v ? kSlotBytes : kSlotBytes / 2);
       const int z = p.shared_state ? 0 : ld_un.g;
@@ -642,7 +655,8 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          const int y = m0 + q * 32, x = n0 + ci * 32;
+          int y = m0 + q * 32, x = n0 + ci * 32;
+          block_coords(p.layer[un.layer].blocked, ldw, x, y);
           tma_store_3d(&maps.w[un.layer], slot, x, y, g);
           if (has_v) tma_store_3d(&maps.v[un.layer], slot + kSlotBytes / 2, x, y, g);
           bulk_commit();
@@ -689,6 +703,7 @@ struct SLayer {
   __nv_bfloat16* Wb;
   float *W, *V;                         // master weights / momentum of replica 0 (replica stride w_gstride)
   float *Ws, *Vs;                       // the same tensors in the synchronized copy
+  int blocked;
 };
 struct SParams {
   SLayer layer[kMaxLayers];
@@ -855,16 +870,22 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
           __nv_bfloat162 hi = __floats2bfloat162_rn(w4[i].z, w4[i].w);
           cp[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
         }
+        // where this lane's first row piece goes, and the distance to its next one (four rows down): row-major,
+        // or inside the block's own 4 KB when the master copy is blocked (the bf16 copy is always row-major)
         const int64_t at = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
+        const int64_t mat = ly.blocked ? ((int64_t)((un.m0 >> 5) + q) * (ldw >> 5) + (un.n0 >> 5) + half) * 1024 +
+                                             row0 * 32 + piece * 4
+                                       : at;
+        const int64_t mstep = ly.blocked ? 4 * 32 : 4 * ldw;
         for (int g = 0; g <= m; ++g) {
           // g = m: the synchronized copy
-          float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + at;
-          float* Vd = (g < m ? ly.V + (int64_t)g * p.w_gstride : ly.Vs) + at;
+          float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + mat;
+          float* Vd = (g < m ? ly.V + (int64_t)g * p.w_gstride : ly.Vs) + mat;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Wd + (int64_t)i * 4 * ldw) = w4[i];
+          for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Wd + i * mstep) = w4[i];
           if (has_v) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Vd + (int64_t)i * 4 * ldw) = v4[i];
+            for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Vd + i * mstep) = v4[i];
           }
           if (ly.Wb != nullptr && g < m) {
             __nv_bfloat16* Bd = ly.Wb + (int64_t)g * p.w_gstride + at;
@@ -884,8 +905,10 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
       uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
       uint64_t* bar = &base_full[(n & 1) * 8 + wi];
       mbar_expect_tx(bar, has_v ? kSlotBytes : kSlotBytes / 2);
-      tma_load_3d(slot, &maps.wl[un.layer], bar, un.n0 + half * 32, un.m0 + q * 32, 0);
-      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.vl[un.layer], bar, un.n0 + half * 32, un.m0 + q * 32, 0);
+      int x = un.n0 + half * 32, y = un.m0 + q * 32;
+      block_coords(p.layer[un.layer].blocked, p.layer[un.layer].N, x, y);
+      tma_load_3d(slot, &maps.wl[un.layer], bar, x, y, 0);
+      if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.vl[un.layer], bar, x, y, 0);
     };
     if (lane == 0 && my_units > 0) load_base(0);
     bool ok = true;
@@ -1001,6 +1024,7 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.tile_begin = total;
     l.b_row_off = a.row_off;
     l.Wb = a.Wb;
+    l.blocked = a.blocked ? 1 : 0;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
@@ -1045,6 +1069,7 @@ int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.tile_begin = total;
     l.b_row_off = a.row_off;
     l.Wb = a.Wb;
+    l.blocked = a.blocked ? 1 : 0;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
@@ -1093,7 +1118,7 @@ int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int6
     const TcUpdateArgs& a = layers[i];
     SLayer& l = p.layer[i];
     l.N = a.N; l.n_tiles = a.N / SN; l.tile_begin = total; l.b_row_off = a.row_off; l.Wb = a.Wb;
-    l.W = a.W; l.V = a.V; l.Ws = a.Wsync; l.Vs = a.Vsync;
+    l.W = a.W; l.V = a.V; l.Ws = a.Wsync; l.Vs = a.Vsync; l.blocked = a.blocked ? 1 : 0;
     total += (a.M / BM) * (a.N / SN);
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = *a.mapWsync; maps.vl[i] = *a.mapVsync;
