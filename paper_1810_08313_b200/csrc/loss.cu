@@ -101,12 +101,19 @@ bias_kernel(const TD* __restrict__ dZ, float* __restrict__ bias, float* __restri
   bias[at] = fmaf(-lr, step, bias[at]);
 }
 
+// eight consecutive elements per thread (replica vectors are padded to multiples of 64): one index translation
+// and one 16-byte store for each
 __global__ void __launch_bounds__(kThreads)
 to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int64_t n, TileMap tiles) {
   const int64_t step = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += step) {
-    const int64_t rep = i / stride, e = i - rep * stride;
-    dst[rep * stride + rowmajor_index(tiles, e)] = __float2bfloat16_rn(src[i]);
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n / 8; i += step) {
+    const int64_t e0 = i * 8, rep = e0 / stride, e = e0 - rep * stride;
+    const float4 a = *reinterpret_cast<const float4*>(src + e0), b = *reinterpret_cast<const float4*>(src + e0 + 4);
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
+    __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y), p3 = __floats2bfloat162_rn(b.z, b.w);
+    *reinterpret_cast<uint4*>(dst + rep * stride + rowmajor_index(tiles, e)) =
+        make_uint4(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1), *reinterpret_cast<uint32_t*>(&p2),
+                   *reinterpret_cast<uint32_t*>(&p3));
   }
 }
 
@@ -150,7 +157,9 @@ int launch_to_bf16(const float* src, __nv_bfloat16* dst, int m, int64_t stride, 
   const int64_t n = (int64_t)m * stride;
   if (n <= 0) return cudaSuccess;
   if (launches) ++*launches;
-  int64_t gx = (n + kThreads - 1) / kThreads;
+  if (stride % 8 != 0 || reinterpret_cast<uintptr_t>(src) % 16 != 0 || reinterpret_cast<uintptr_t>(dst) % 16 != 0)
+    return cudaErrorInvalidValue;
+  int64_t gx = (n / 8 + kThreads - 1) / kThreads;
   if (gx > 148 * 16) gx = 148 * 16;
   to_bf16_kernel<<<(unsigned)gx, kThreads, 0, st>>>(src, dst, stride, n, tiles ? *tiles : TileMap{});
   return cudaGetLastError();
