@@ -539,10 +539,32 @@ static int local_steps(ls_handle* h, int tau, const int64_t* row_offset_host, fl
   for (int64_t i = 0; i < (int64_t)tau * lay.m; ++i)
     if (row_offset_host[i] < 0 || row_offset_host[i] + lay.batch > h->n_rows) return LS_ERR_ROW_RANGE;
   int64_t* off_dev = reinterpret_cast<int64_t*>(h->state + lay.rowoff_off);
+  // a one-layer fp32 model that fits a CTA's shared memory: all steps of the call in one launch per chunk of
+  // offsets, one CTA per replica (the per-step launches of such a model are launch-latency bound)
+  const bool one_launch = lay.L == 1 && !lay.bf16 && lay.dims[0] % 4 == 0 &&
+                          linear_period_ok(lay.batch, lay.dims[0], lay.dims[1], h->mu != 0.f) &&
+                          reinterpret_cast<uintptr_t>(h->x_dev) % 16 == 0;
   for (int s0 = 0; s0 < tau; s0 += kRowOffCap) {
     const int n = (tau - s0 < kRowOffCap) ? tau - s0 : kRowOffCap;
     LS_CUDA(h, cudaMemcpyAsync(off_dev, row_offset_host + (int64_t)s0 * lay.m, (size_t)n * lay.m * 8,
                                cudaMemcpyHostToDevice, h->stream));
+    if (one_launch) {
+      {
+        ProfScope ps(h, LS_K_DW, 0);
+        LS_CUDA(h, launch_linear_period(static_cast<const float*>(h->x_dev), h->y_dev, off_dev,
+                                        params_of(h) + lay.w_off[0], mom_of(h) + lay.w_off[0],
+                                        lay.has_bias ? params_of(h) + lay.b_off[0] : nullptr, mom_of(h) + lay.b_off[0],
+                                        lay.stride, loss_dev ? loss_dev + (int64_t)s0 * lay.m : nullptr, n, lay.m,
+                                        lay.batch, lay.dims[0], lay.dims[1], h->spec.loss, h->lr, h->mu, h->stream,
+                                        &h->launches));
+      }
+      h->sync_valid = false;
+      if (avg_after && s0 + n == tau) {
+        int rc = average(h);
+        if (rc != LS_OK) return rc;
+      }
+      continue;
+    }
     for (int s = 0; s < n; ++s) {
       const TcMaps& mnm = lay.bf16 ? h->maps : h->maps_mn;
       int rc = local_step(h, h->x_dev, XMaps{&h->maps.x_data, &mnm.x_data, &h->maps_upd.x_data}, h->y_dev, off_dev + (int64_t)s * lay.m,

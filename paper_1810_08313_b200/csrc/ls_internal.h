@@ -302,6 +302,12 @@ struct BiasArgs {          // gb = colsum(dZ); v = mu v + gb; b -= lr v
 };
 int launch_bias(const BiasArgs& a, bool bf16, cudaStream_t st, int64_t* launches);
 
+// ---- small linear models: all local steps of a call in one launch (period_linear.cu) -------------------
+bool linear_period_ok(int B, int K, int C, bool has_v);
+int launch_linear_period(const float* X, const void* y, const int64_t* row_off, float* W, float* V, float* bias,
+                         float* vbias, int64_t gstride, float* loss_out, int tau, int m, int B, int K, int C, int kind,
+                         float lr, float mu, cudaStream_t st, int64_t* launches);
+
 // ---- narrow output layer (head.cu) ---------------------------------------------
 struct HeadFwdArgs {
   const void* A; const int64_t* a_row_off;   // layer input [groups][B][K] (or dataset rows)

@@ -37,6 +37,10 @@ CASES = [
     ((3072, 512, 512, 10), "softmax_ce", True, 2, 128, 0.9),     # the fp32 MLP's layer shapes
     ((130, 65, 10), "softmax_ce", False, 5, 64, 0.5),            # no bias
     ((4096, 1), "mse_half", False, 4, 64, 0.0),                  # least squares
+    # small linear models: all steps of a call in one launch, one CTA per replica
+    ((100, 10), "softmax_ce", True, 3, 48, 0.9),                 # momentum, a batch that is no multiple of 32
+    ((64, 1), "mse_half", True, 2, 20, 0.5),                     # one output, squared error, bias
+    ((256, 10), "softmax_ce", False, 5, 70, 0.0),                # no bias, three passes of 32 samples
     ((50, 33, 1), "mse_half", True, 2, 16, 0.9),
     # kernel-selection corners of the tensor-core path
     ((256, 128, 128, 128, 128, 128, 10), "softmax_ce", True, 3, 128, 0.9),  # 5 tensor-core layers: two update launches; few tiles: strips
