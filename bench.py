@@ -543,8 +543,9 @@ def run_ours(args, w: wl.Workload):
     if gemm:
         line["gemm_tensor"] = gemm
 
-    if rank == 0 and world == 1 and not args.kernel_only:
-        # ---- end to end: mini-batches from pinned host memory, losses back to the host -------
+    if not args.kernel_only:
+        # ---- end to end: mini-batches from pinned host memory, losses back to the host (every rank; the
+        # time is the maximum over ranks, the units add up) -------
         e_steps = max(1, min(K, 3))
         xh = torch.empty((tau, m, B, w.dims[0]), dtype=xd.dtype).pin_memory()
         yh = torch.empty((tau, m, B), dtype=yd.dtype).pin_memory()
@@ -560,19 +561,21 @@ def run_ours(args, w: wl.Workload):
             F = eng.eval_loss(0, 0, probe)
             return adacomm_next_tau(F, F_0, tau)
         e2e_period()
-        torch.cuda.synchronize()
+        barrier()
         t0 = time.perf_counter()
         for _ in range(e_steps):
             e2e_period()
-        torch.cuda.synchronize()
+        barrier()
         dt = time.perf_counter() - t0
-        line["e2e"] = {"value": m * tau * e_steps / dt, "unit": UNIT,
+        e_ms, e_units = aggregate_over_ranks(dt * 1e3, float(m * tau * e_steps))
+        line["e2e"] = {"value": e_units / (e_ms * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * yh.element_size()),
                        "d2h_bytes_per_step": int(lh.numel() * 4 + 4),
                        "note": "per period; batches copied from pinned host memory inside the timed region; when "
                                "the copies (bytes / host-link rate) take longer than the kernels of a period the "
                                "host link, not the GPU, sets this number"}
 
+    if rank == 0 and world == 1 and not args.kernel_only:
         # ---- averaging bandwidth on the model-sized flat vectors (params + momentum) ----------
         # (each replica's vector starts on a 256-byte boundary, as in the library's own layout; the 10^9
         #  point is run when --avg-1b is given: m = 16 with momentum needs 2 x 64 GB)
