@@ -127,7 +127,7 @@ average_kernel(float* __restrict__ base, int64_t buf_stride, int m_rt, int64_t n
   // the synchronized copy: what every replica holds now (read by the next local step while they are still equal)
   if (sync_out != nullptr) s.store(sync_out + (int64_t)blockIdx.y * sync_stride + i * W);
   if (blockIdx.y == 0 && shadow != nullptr) {
-    const int64_t at = rowmajor_index(tiles, i * W);      // the bf16 copies are row-major
+    const int64_t at = shadow_index(tiles, i * W);
     for (int j = 0; j < m; ++j) store_bf16<W>(shadow + (int64_t)j * stride + at, s.v);
   }
 }
@@ -158,7 +158,7 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
   for (int j = 0; j < m; ++j) buf[(int64_t)j * stride + i] = mean;
   if (sync_out != nullptr) sync_out[(int64_t)blockIdx.y * sync_stride + i] = mean;
   if (blockIdx.y == 0 && shadow != nullptr) {
-    const int64_t at = rowmajor_index(tiles, i);
+    const int64_t at = shadow_index(tiles, i);
     for (int j = 0; j < m; ++j) shadow[(int64_t)j * stride + at] = __float2bfloat16_rn(mean);
   }
 }

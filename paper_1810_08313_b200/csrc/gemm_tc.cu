@@ -62,7 +62,7 @@ struct Operand {
   const int64_t* row_off;    // first row of group g (dataset rows), or null
   int64_t rows_per_group;    // else group g starts at row g*rows_per_group (2-D maps)
   int z0, z_step;            // 3-D maps: z = z0 + g*z_step
-  int rank3;
+  int rank3;                 // 0: 2-D map; 1: 3-D map [group][row][column]; 2: panel map [group][column / 64][row][64]
 };
 
 struct Params {
@@ -118,7 +118,8 @@ __device__ __forceinline__ void issue_tile(void* dst, const CUtensorMap* tm, uin
     char* d = static_cast<char*>(dst) + c * kChunkBytes;
     const int x = mn_major ? tile0 + c * ELEMS : k0;
     const int y = mn_major ? k0 : tile0 + c * 64;
-    if (op.rank3) tma_load_3d_hint(d, tm, bar, x, y, z, pol);
+    if (op.rank3 == 2) tma_load_4d_hint(d, tm, bar, 0, y, x >> 6, z, pol);     // x is a multiple of 64
+    else if (op.rank3) tma_load_3d_hint(d, tm, bar, x, y, z, pol);
     else tma_load_2d_hint(d, tm, bar, x, row_base + y, pol);
   }
 }
@@ -755,6 +756,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint64_t pol_a = l2_policy(2), pol_b = l2_policy(1);
       const int a_base = operand_row_base(p.a, g);
       const int zb = p.b.z0 + g * p.b.z_step;
+      const bool b_panel = p.b.rank3 == 2;
       const uint32_t full_leader = map_to_rank(smem_u32(&full[0]), 0);
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
@@ -774,8 +776,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             uint8_t* d = sb + j * L::kBBlockBytes + c * CHUNK_BYTES;
-            if (B_MN) tma_load_3d_pair(d, &tmB, bar, nb + c * 64, k0, zb, pol_b);
-            else tma_load_3d_pair(d, &tmB, bar, k0, nb + c * 64, zb, pol_b);
+            const int x = B_MN ? nb + c * 64 : k0, y = B_MN ? k0 : nb + c * 64;
+            if (b_panel) tma_load_4d_pair(d, &tmB, bar, 0, y, x >> 6, zb, pol_b);    // x is a multiple of 64
+            else tma_load_3d_pair(d, &tmB, bar, x, y, zb, pol_b);
           }
         }
       }
@@ -1084,6 +1087,20 @@ int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64
   if (blocked) return make_map(out, base, true, false, true, 3, rows * cols / 32, 32, groups, gstride);
   return make_map(out, base, true, false, true, 3, rows, cols, groups, gstride);
 }
+int tc_make_panel_map(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups, int64_t gstride) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
+  if (rows < 1 || cols < 64 || cols % 64 != 0 || groups < 1 || gstride < rows * cols || gstride % 8 != 0)
+    return cudaErrorInvalidValue;
+  cuuint64_t dims[4] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64), (cuuint64_t)groups};
+  cuuint64_t strides[3] = {128, (cuuint64_t)rows * 128, (cuuint64_t)gstride * 2};
+  cuuint32_t box[4] = {64, 64, 1, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
 
 // The forward kernel can also evaluate a narrow output layer that follows when one CTA holds every row of
 // its columns and the layer fits kHeadMax outputs.  Used for one row block (M = 128): with the 256-row
@@ -1113,7 +1130,7 @@ bool tc_shape_ok(bool fp32, int M, int N, int K) {
 int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
   p.a = Operand{a.row_off, a.M, 0, 0, 0};
-  p.b = Operand{nullptr, 0, a.w_z0, a.w_zstep, 1};
+  p.b = Operand{nullptr, 0, a.w_z0, a.w_zstep, a.w_panel ? 2 : 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.bias = a.bias; p.bias_gstride = a.bias_gstride; p.relu = a.relu;
   p.C = a.C; p.err_flag = a.err_flag;
@@ -1131,7 +1148,7 @@ int launch_tc_fwd(const TcFwdArgs& a, cudaStream_t st, int64_t* launches) {
 int launch_tc_dx(const TcDxArgs& a, cudaStream_t st, int64_t* launches) {
   Params p{};
   p.a = Operand{nullptr, a.M, 0, 0, 0};
-  p.b = Operand{nullptr, 0, 0, a.w_zstep, 1};
+  p.b = Operand{nullptr, 0, 0, a.w_zstep, a.w_panel ? 2 : 1};
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.C = a.C; p.act = a.act; p.err_flag = a.err_flag;
   if (a.bias != nullptr && tc_dx_fuses_bias(a.fp32, a.M, a.N)) {

@@ -111,7 +111,7 @@ to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, i
     const float4 a = *reinterpret_cast<const float4*>(src + e0), b = *reinterpret_cast<const float4*>(src + e0 + 4);
     __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
     __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y), p3 = __floats2bfloat162_rn(b.z, b.w);
-    *reinterpret_cast<uint4*>(dst + rep * stride + rowmajor_index(tiles, e)) =
+    *reinterpret_cast<uint4*>(dst + rep * stride + shadow_index(tiles, e)) =
         make_uint4(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1), *reinterpret_cast<uint32_t*>(&p2),
                    *reinterpret_cast<uint32_t*>(&p3));
   }

@@ -96,6 +96,10 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   size_t retile = 0;
   for (int l = 0; l < lay.L; ++l) {
     lay.tiled[l] = lay.bf16 && tc_update_shape_ok(false, lay.dims[l + 1], lay.dims[l], batch) ? 1 : 0;
+    // the bf16 copy goes into panels when every GEMM that reads it is a tensor-core one (forward; data gradient)
+    lay.panel[l] = lay.tiled[l] && l < lay.L - 1 && tc_shape_ok(false, batch, lay.dims[l + 1], lay.dims[l]) &&
+                           (l == 0 || tc_shape_ok(false, batch, lay.dims[l], lay.dims[l + 1]))
+                       ? 1 : 0;
     if (lay.tiled[l]) retile = std::max(retile, (size_t)lay.dims[l + 1] * lay.dims[l] * 4);
   }
   if (retile) lay.retile_off = take(retile);
@@ -218,6 +222,7 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
       t.maps.b = &h->maps.w[l];
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.w_z0 = (int)replica0; t.w_zstep = (w_gstride != 0 && !shared_w) ? 1 : 0;
+      t.w_panel = lay.panel[l] != 0;
       t.bias = lay.has_bias ? P + lay.b_off[l] : nullptr;
       t.bias_gstride = w_gstride;
       t.C = h->state + lay.act_off[l + 1];
@@ -325,6 +330,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.act_map = (bf && lay.dims[l] % 8 == 0) ? &h->maps.act[l] : nullptr;
       t.M = lay.batch; t.N = lay.dims[l]; t.K = lay.dims[l + 1]; t.groups = lay.m;
       t.w_zstep = shared_w ? 0 : 1;
+      t.w_panel = lay.panel[l] != 0;
       t.bias = nullptr; t.vbias = nullptr; t.bias_gstride = lay.stride; t.lr = h->lr; t.mu = h->mu;
       if (lay.has_bias && tc_dx_fuses_bias(!bf, t.M, t.N)) {
         t.bias = params_of(h) + lay.b_off[l - 1];
@@ -360,6 +366,7 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
       t.W = params_of(h) + lay.w_off[l]; t.V = mom_of(h) + lay.w_off[l];
       t.Wsync = sync_of(h) + lay.w_off[l]; t.Vsync = sync_of(h) + lay.stride + lay.w_off[l];
       t.blocked = lay.tiled[l] != 0;
+      t.panel = lay.panel[l] != 0;
       t.row_off = (l == 0) ? row_off_dev : nullptr;
       t.Wb = bf ? shadow_of(h) + lay.w_off[l] : nullptr;
       t.w_gstride = lay.stride;
@@ -646,6 +653,7 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
     if (lay.tiled[l]) {
       TileMap& tm = h->tiles;
       tm.begin[tm.n] = lay.w_off[l]; tm.size[tm.n] = (int64_t)lay.dims[l + 1] * lay.dims[l]; tm.cols[tm.n] = lay.dims[l];
+      tm.panel[tm.n] = lay.panel[l];
       ++tm.n;
     }
   int e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
@@ -669,7 +677,8 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
       for (int l = 0; l < lay.L; ++l) {
         if (lay.dims[l] % q == 0) {
           const void* wsrc = f ? (const void*)(params_of(h) + lay.w_off[l]) : (const void*)(shadow_of(h) + lay.w_off[l]);
-          ok(tc_make_map_3d(&mp.w[l], wsrc, f, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+          if (lay.panel[l]) ok(tc_make_panel_map(&mp.w[l], wsrc, lay.dims[l + 1], lay.dims[l], m, lay.stride));
+          else ok(tc_make_map_3d(&mp.w[l], wsrc, f, mn, lay.dims[l + 1], lay.dims[l], m, lay.stride));
           if (l >= 1) {
             ok(tc_make_map_2d(&mp.act[l], h->state + lay.act_off[l], f, mn, rows, lay.dims[l]));
           }

@@ -56,6 +56,7 @@ struct Layout {
   size_t err_off = 0;                        // int: device-side error flag (bounded waits that ran out)
   size_t anchor_off = 0, blocku_off = 0;     // block momentum: period-start model and global buffer, [stride] each
   int tiled[LS_MAX_LAYERS] = {0};            // W_l (and v_l) stored as 32 x 32 blocks, see TileMap
+  int panel[LS_MAX_LAYERS] = {0};            // the bf16 copy of W_l stored as 64-column panels, see TileMap
   size_t retile_off = 0;                     // staging for one matrix in row-major order (host <-> tiled layout)
   size_t sync_off = 0;                       // synchronized copy: [2][stride] parameters and momentum as every replica
                                              // held them right after the last averaging step
@@ -71,25 +72,39 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out);
 // The update kernels move exactly such blocks, so every bulk copy of theirs is one contiguous 4 KB run instead of
 // 32 pieces of 128 bytes a row pitch apart, which DRAM serves markedly better (measured on the update of the
 // bf16 workload: 785 -> 734 us).  Everything element-wise (averaging, partial sums, the synchronized copy, block
-// momentum) is indifferent to the order; the bf16 operand copies that the GEMMs read stay row-major, so whoever
-// writes them from the blocked master translates the index with rowmajor_index().  The host interface
-// (ls_set_params, ls_get_state, ...) is row-major: copy_replica retiles.
+// momentum) is indifferent to the order.  The host interface (ls_set_params, ls_get_state, ...) is row-major:
+// copy_replica retiles.
+//
+// The bf16 operand copy of such a matrix, which only the tensor-core GEMMs read, is kept in panels of 64
+// columns (128 bytes, the width of one operand box): panel p holds columns [64 p, 64 p + 64) of all rows, row after
+// row, so element (r, c) sits at
+//     (c / 64) * M * 64 + r * 64 + c % 64 .
+// An operand box (64 columns x 64 rows) is then 8 KB of consecutive memory for both GEMMs, and what an update warp
+// writes for a 32 x 32 block (32 rows x 64 bytes) stays inside 4 KB instead of being spread over 32 rows of the
+// matrix.  The GEMMs address it as a 4-D tensor [replica][panel][row][64] (tc_make_panel_map).  Matrices that a
+// CUDA-core GEMM may read keep a row-major copy (panel = 0).  Whoever writes the copy from the master's element
+// order finds the place with shadow_index().
 struct TileMap {
   int n = 0;
   int64_t begin[LS_MAX_LAYERS] = {0};   // first element of the matrix inside a replica vector
   int64_t size[LS_MAX_LAYERS] = {0};    // rows * cols
   int cols[LS_MAX_LAYERS] = {0};
+  int panel[LS_MAX_LAYERS] = {0};       // bf16 copy in 64-column panels (else row-major)
 };
-// Index, in the row-major arrangement of a replica vector, of element e of the blocked arrangement (identity
-// outside the blocked matrices).  Eight consecutive e starting at a multiple of 8 stay consecutive.
-__host__ __device__ inline int64_t rowmajor_index(const TileMap& t, int64_t e) {
+// Index, in the bf16 operand copy of a replica vector, of element e of the master's arrangement: the panel
+// arrangement for matrices kept that way, row-major otherwise.  Eight consecutive e starting at a multiple of 8
+// stay consecutive.
+__host__ __device__ inline int64_t shadow_index(const TileMap& t, int64_t e) {
   for (int j = 0; j < t.n; ++j) {
     const int64_t local = e - t.begin[j];
     if (local >= 0 && local < t.size[j]) {
       const int64_t blk = local >> 10;
       const int r = (int)(local >> 5) & 31, c = (int)local & 31, nb = t.cols[j] >> 5;
       const int64_t rb = blk / nb, cb = blk - rb * nb;
-      return t.begin[j] + (rb * 32 + r) * t.cols[j] + cb * 32 + c;
+      const int64_t row = rb * 32 + r, col = cb * 32 + c;
+      if (!t.panel[j]) return t.begin[j] + row * t.cols[j] + col;
+      const int64_t rows = t.size[j] / t.cols[j];
+      return t.begin[j] + (col >> 6) * rows * 64 + row * 64 + (col & 63);
     }
   }
   return e;
@@ -233,7 +248,7 @@ struct BlockMomentum {
 int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n, int64_t stride,
                    __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
                    const BlockMomentum* bm = nullptr, float* sync_out = nullptr, int64_t sync_stride = 0,
-                   const TileMap* tiles = nullptr);    // tiles: `base` is blocked, `shadow` row-major
+                   const TileMap* tiles = nullptr);    // tiles: the blocked matrices of `base` (`shadow`: shadow_index)
 
 // ---- averaging over several GPUs (shard_average.cu) -------------------------
 // out[b] = sum over the m vectors of buffer b in index order; then, with the G partial sums of every GPU
@@ -334,7 +349,7 @@ int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t*
 int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches);
 
 // fp32 -> bf16 copy of n elements (refresh of the weight copies)
-// m vectors of `stride` elements each; tiles: src is blocked, dst row-major
+// m vectors of `stride` elements each; tiles: the matrices that src holds blocked (dst: shadow_index)
 int launch_to_bf16(const float* src, __nv_bfloat16* dst, int m, int64_t stride, const TileMap* tiles, cudaStream_t st,
                    int64_t* launches);
 // one matrix between row-major and blocked order (to_blocked: dst blocked <- src row-major, else the reverse)
@@ -348,6 +363,9 @@ int tc_make_map_3d(CUtensorMap* out, const void* base, bool fp32, bool mn32, int
                    int64_t groups, int64_t gstride);
 int tc_make_block_map_3d(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups,
                          int64_t gstride, bool blocked = false);
+// 4-D map over the bf16 copies of `groups` matrices [rows][cols] kept in 64-column panels (see TileMap):
+// dimensions (64, rows, cols / 64, groups); a box is 64 columns x 64 rows, read at (0, row, column / 64, group)
+int tc_make_panel_map(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t groups, int64_t gstride);
 bool tc_shape_ok(bool fp32, int M, int N, int K);   // output rows, output columns, contraction length
 struct TcOperandMaps {
   const CUtensorMap *a, *b;
@@ -370,6 +388,7 @@ struct TcFwdArgs {
   bool fp32;
   const int64_t* row_off;
   int w_z0, w_zstep;         // replica used by group g = w_z0 + g*w_zstep
+  bool w_panel = false;      // maps.b is a panel map (tc_make_panel_map)
   const float* bias; int64_t bias_gstride;
   void* C;                   // [groups][M][N] bf16 or fp32
   const CUtensorMap* c_map;  // bf16: C as a 2-D tensor [groups*M][N], boxes of 64 x 64 (pair kernel's stores), or null
@@ -385,6 +404,7 @@ struct TcDxArgs {
   const CUtensorMap* c_map;   // bf16: C and act as 2-D tensors [groups*M][N], boxes of 64 x 64, or null
   const CUtensorMap* act_map;
   int w_zstep;               // replica whose weights group g reads = g * w_zstep (0: every group reads replica 0's)
+  bool w_panel = false;      // maps.b is a panel map (tc_make_panel_map)
   int M, N, K, groups;
   // bias / its momentum of the layer that produced `act` (group 0; replica stride bias_gstride): updated
   // from the column sums of C inside the kernel when tc_dx_fuses_bias(); else null
@@ -414,7 +434,8 @@ struct TcUpdateArgs {
   // the same four tensors as plain pointers (replica 0; replica stride w_gstride): the fused step + average
   // kernel stores through them
   float* W; float* V; float* Wsync; float* Vsync;
-  bool blocked;              // W, v (and their synchronized copy) are stored as 32 x 32 blocks (TileMap); Wb is row-major
+  bool blocked;              // W, v (and their synchronized copy) are stored as 32 x 32 blocks (TileMap)
+  bool panel = false;        // Wb is kept in 64-column panels (TileMap), else row-major
   bool fp32;
   const int64_t* row_off;
   __nv_bfloat16* Wb; int64_t w_gstride;

@@ -97,7 +97,7 @@ combine_kernel(const float* __restrict__ parts, int G, int64_t part_stride, int6
         __nv_bfloat162 t = __floats2bfloat162_rn(s.v[2 * e], s.v[2 * e + 1]);
         u[e] = *reinterpret_cast<uint32_t*>(&t);
       }
-      const int64_t at = rowmajor_index(tiles, i * 8);      // the bf16 copies are row-major
+      const int64_t at = shadow_index(tiles, i * 8);
       for (int j = 0; j < m_local; ++j)
         *reinterpret_cast<uint4*>(shadow + (int64_t)j * stride + at) = make_uint4(u[0], u[1], u[2], u[3]);
     }
@@ -107,7 +107,7 @@ combine_kernel(const float* __restrict__ parts, int G, int64_t part_stride, int6
       const float mean = __fdiv_rn(ordered_sum_scalar(src + e, G, part_stride), m_total);
       for (int j = 0; j < m_local; ++j) dst[(int64_t)j * stride + e] = mean;
       if (blockIdx.y == 0 && shadow != nullptr) {
-        const int64_t at = rowmajor_index(tiles, e);
+        const int64_t at = shadow_index(tiles, e);
         for (int j = 0; j < m_local; ++j) shadow[(int64_t)j * stride + at] = __float2bfloat16_rn(mean);
       }
     }

@@ -51,6 +51,7 @@ struct ULayer {
   const int64_t* b_row_off;            // layer input = dataset rows: first row of replica g, else null
   __nv_bfloat16* Wb;                   // bf16 copy of W (bf16 models) or null
   int blocked;                         // W, v stored as 32 x 32 blocks (TileMap): box coordinates differ
+  int pM;                              // rows of W when Wb is kept in 64-column panels (TileMap), else 0: row-major
 };
 struct UParams {
   ULayer layer[kMaxLayers];
@@ -113,6 +114,11 @@ __device__ __forceinline__ void block_coords(int blocked, int ldw, int& x, int& 
     y = ((y >> 5) * (ldw >> 5) + (x >> 5)) << 5;
     x = 0;
   }
+}
+// Where, inside a replica's bf16 copy of W, the piece of row `row` that starts at column `col` begins (a piece
+// never crosses a multiple of 64 columns).
+__device__ __forceinline__ int64_t copy_index(int pM, int ldw, int row, int col) {
+  return pM ? ((int64_t)(col >> 6) * pM + row) * 64 + (col & 63) : (int64_t)row * ldw + col;
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
@@ -345,7 +351,7 @@ tc_update_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ UPa
         }
         if (!ok) { if (lane == 0) atomicExch(p.err_flag, 15); break; }
         // this thread's row of the 32 x 32 block; 16-byte pieces are XOR-swizzled by the row (128-byte swizzle)
-        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * ldw + n0 + c * 32;
+        const int64_t at = (int64_t)g * p.w_gstride + copy_index(p.layer[tl.layer].pM, ldw, m0 + q * 32 + lane, n0 + c * 32);
         uint32_t cp[8];
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
@@ -418,6 +424,7 @@ struct PLayer {
   const int64_t* b_row_off;
   __nv_bfloat16* Wb;
   int blocked;
+  int pM;                               // as in ULayer
 };
 struct PParams {
   PLayer layer[kMaxLayers];
@@ -623,7 +630,7 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
           if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + (uint32_t)(buf * 8));
         }
         if (!ok) { if (lane == 0) atomicExch(p.err_flag, 35); break; }
-        const int64_t at = (int64_t)g * p.w_gstride + (int64_t)(m0 + q * 32 + lane) * ldw + n0 + ci * 32;
+        const int64_t at = (int64_t)g * p.w_gstride + copy_index(p.layer[un.layer].pM, ldw, m0 + q * 32 + lane, n0 + ci * 32);
         uint32_t cp[8];
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
@@ -704,6 +711,7 @@ struct SLayer {
   float *W, *V;                         // master weights / momentum of replica 0 (replica stride w_gstride)
   float *Ws, *Vs;                       // the same tensors in the synchronized copy
   int blocked;
+  int pM;                               // as in ULayer
 };
 struct SParams {
   SLayer layer[kMaxLayers];
@@ -871,12 +879,14 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
           cp[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
         }
         // where this lane's first row piece goes, and the distance to its next one (four rows down): row-major,
-        // or inside the block's own 4 KB when the master copy is blocked (the bf16 copy is always row-major)
-        const int64_t at = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
+        // or inside the block's own 4 KB when the master copy is blocked; the bf16 copy row-major or in panels
+        const int64_t rm = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
         const int64_t mat = ly.blocked ? ((int64_t)((un.m0 >> 5) + q) * (ldw >> 5) + (un.n0 >> 5) + half) * 1024 +
                                              row0 * 32 + piece * 4
-                                       : at;
+                                       : rm;
         const int64_t mstep = ly.blocked ? 4 * 32 : 4 * ldw;
+        const int64_t at = copy_index(ly.pM, ldw, un.m0 + q * 32 + row0, un.n0 + half * 32 + piece * 4);
+        const int64_t bstep = ly.pM ? 4 * 64 : 4 * ldw;
         for (int g = 0; g <= m; ++g) {
           // g = m: the synchronized copy
           float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + mat;
@@ -890,7 +900,7 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
           if (ly.Wb != nullptr && g < m) {
             __nv_bfloat16* Bd = ly.Wb + (int64_t)g * p.w_gstride + at;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(Bd + (int64_t)i * 4 * ldw) = cp[i];
+            for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(Bd + i * bstep) = cp[i];
           }
         }
       }
@@ -1025,6 +1035,7 @@ int launch_update(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.b_row_off = a.row_off;
     l.Wb = a.Wb;
     l.blocked = a.blocked ? 1 : 0;
+    l.pM = a.panel ? a.M : 0;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
@@ -1070,6 +1081,7 @@ int launch_update_pair(const TcUpdateArgs* layers, int n, cudaStream_t st) {
     l.b_row_off = a.row_off;
     l.Wb = a.Wb;
     l.blocked = a.blocked ? 1 : 0;
+    l.pM = a.panel ? a.M : 0;
     total += l.tiles_per_group * a.groups;
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
@@ -1119,6 +1131,7 @@ int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int6
     SLayer& l = p.layer[i];
     l.N = a.N; l.n_tiles = a.N / SN; l.tile_begin = total; l.b_row_off = a.row_off; l.Wb = a.Wb;
     l.W = a.W; l.V = a.V; l.Ws = a.Wsync; l.Vs = a.Vsync; l.blocked = a.blocked ? 1 : 0;
+    l.pM = a.panel ? a.M : 0;
     total += (a.M / BM) * (a.N / SN);
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
     maps.wl[i] = *a.mapWsync; maps.vl[i] = *a.mapVsync;
