@@ -81,6 +81,10 @@ int make_layout(int m, const ls_model_spec* spec, int batch, Layout* out) {
   if (lay.L >= 2 && head_shape_ok(batch, lay.dims[lay.L]) &&
       tc_fwd_fuses_head(!lay.bf16, batch, lay.dims[lay.L - 1], lay.dims[lay.L]))
     lay.headpart_off = take((size_t)m * tc_fwd_head_parts(lay.dims[lay.L - 1]) * batch * 16 * 4);
+  if (lay.bf16 && lay.L >= 2 && lay.headpart_off == 0 && head_shape_ok(batch, lay.dims[lay.L])) {
+    lay.hstep_off = take(head_step_scratch_bytes(m, lay.dims[lay.L], lay.dims[lay.L - 1]));
+    lay.hstep_cnt_off = take(head_step_counter_bytes(m));
+  }
   lay.rowoff_off = take((size_t)kRowOffCap * m * 8);
   lay.evaloff_off = take((size_t)kEvalCap * 8);
   lay.evalloss_off = take((size_t)kEvalCap * 4);
@@ -187,6 +191,29 @@ __global__ void wait_timeout_selftest_kernel(int* err_flag, long long limit) {
 // x maps: [0] for K-major reads, [1] for MN-major reads of the mini-batch rows
 struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; const CUtensorMap* upd; };
 
+// The output layer of a training step as ONE launch (head_step.cu) when its shape allows: fills `a`.  False: the
+// forward kernel (stand-alone or riding on the GEMM before it) and head_bwd_kernel run instead.
+static bool head_step_args(ls_handle* h, const void* y, const int64_t* row_off_dev, float* loss_out, HeadStepArgs& a) {
+  const Layout& lay = h->lay;
+  const int l = lay.L - 1;
+  if (!lay.bf16 || l < 1 || lay.hstep_off == 0 || !head_shape_ok(lay.batch, lay.dims[lay.L])) return false;
+  a.A = h->state + lay.act_off[l];
+  a.y = y; a.y_row_off = row_off_dev;
+  a.W = params_of(h) + lay.w_off[l]; a.V = mom_of(h) + lay.w_off[l]; a.Wb = shadow_of(h) + lay.w_off[l];
+  a.bias = lay.has_bias ? params_of(h) + lay.b_off[l] : nullptr;
+  a.vbias = mom_of(h) + lay.b_off[l];
+  a.w_gstride = lay.stride;
+  a.dPrev = h->state + lay.dz_off[l - 1];
+  a.pbias = lay.has_bias ? params_of(h) + lay.b_off[l - 1] : nullptr;
+  a.pvbias = mom_of(h) + lay.b_off[l - 1];
+  a.loss_out = loss_out;
+  a.scratch = reinterpret_cast<float*>(h->state + lay.hstep_off);
+  a.counters = reinterpret_cast<unsigned int*>(h->state + lay.hstep_cnt_off);
+  a.B = lay.batch; a.C = lay.dims[lay.L]; a.K = lay.dims[l]; a.groups = lay.m; a.loss_kind = h->spec.loss;
+  a.lr = h->lr; a.mu = h->mu;
+  return head_step_ok(a);
+}
+
 // shared_w: the groups are different replicas whose weights are known to be bitwise equal (first step after an
 // averaging step): the tensor-core layers all read replica 0's operand copy, which then stays in L2.
 static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const int64_t* row_off_dev,
@@ -198,6 +225,11 @@ static int forward(ls_handle* h, const void* x, XMaps xmap, const void* y, const
   const __nv_bfloat16* S = bf ? shadow_of(h) + replica0 * lay.stride : nullptr;
   for (int l = 0; l < lay.L; ++l) {
     if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
+      if (want_dz && groups == lay.m && replica0 == 0 && w_gstride == lay.stride) {
+        // a training step: the kernel that local_step launches for this layer's backward pass does the forward too
+        HeadStepArgs s;
+        if (head_step_args(h, y, row_off_dev, loss_out, s)) return LS_OK;
+      }
       // narrow output layer: product, loss and dZ in one kernel
       HeadFwdArgs a;
       a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);
@@ -296,6 +328,14 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   for (int l = lay.L - 1; l >= 0; --l) {
     void* dZ = h->state + lay.dz_off[l];
     if (l == lay.L - 1 && head_shape_ok(lay.batch, lay.dims[lay.L])) {
+      HeadStepArgs s;
+      if (head_step_args(h, y, row_off_dev, loss_out, s)) {
+        // forward, loss, both gradients, update and the bias of the layer below in one launch
+        if (s.pbias != nullptr) bias_done[l - 1] = true;
+        ProfScope ps(h, LS_K_DW, l);
+        LS_CUDA(h, launch_head_step(s, h->stream, &h->launches));
+        continue;
+      }
       // narrow output layer: both gradients, the update and the bias in one pass over its input
       HeadBwdArgs a;
       a.A = (l == 0) ? x : (const void*)(h->state + lay.act_off[l]);

@@ -58,6 +58,7 @@ struct Layout {
   int tiled[LS_MAX_LAYERS] = {0};            // W_l (and v_l) stored as 32 x 32 blocks, see TileMap
   int panel[LS_MAX_LAYERS] = {0};            // the bf16 copy of W_l stored as 64-column panels, see TileMap
   size_t retile_off = 0;                     // staging for one matrix in row-major order (host <-> tiled layout)
+  size_t hstep_off = 0, hstep_cnt_off = 0;   // scratch and counters of the one-launch output layer (head_step.cu)
   size_t sync_off = 0;                       // synchronized copy: [2][stride] parameters and momentum as every replica
                                              // held them right after the last averaging step
   size_t total = 0;
@@ -344,6 +345,24 @@ struct HeadBwdArgs {
   int B, C, K, groups;
   float lr, mu;
 };
+// The output layer of a training step in one launch (head_step.cu): what launch_head_fwd (want dZ) followed by
+// launch_head_bwd compute, for bf16 layer inputs [groups][B][K] of a 10-class softmax layer.
+struct HeadStepArgs {
+  const void* A;                             // layer input, bf16, group g at row g*B
+  const void* y; const int64_t* y_row_off;   // int32 labels; first row of group g
+  float* W; float* V; __nv_bfloat16* Wb; float* bias; float* vbias; int64_t w_gstride;
+  void* dPrev;                               // dZ of the layer below [groups][B][K], bf16
+  float* pbias; float* pvbias;               // bias / its momentum of the layer below, or null
+  float* loss_out;                           // [groups] mini-batch mean loss, or null
+  float* scratch;                            // head_step_scratch_bytes(groups, C, K) bytes, contents irrelevant
+  unsigned int* counters;                    // head_step_counter_bytes(groups) bytes, zero before the first launch
+  int B, C, K, groups, loss_kind;
+  float lr, mu;
+};
+size_t head_step_scratch_bytes(int m, int C, int K);
+size_t head_step_counter_bytes(int m);
+bool head_step_ok(const HeadStepArgs& a);
+int launch_head_step(const HeadStepArgs& a, cudaStream_t st, int64_t* launches);
 bool head_shape_ok(int B, int C);
 int launch_head_fwd(const HeadFwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches);
 int launch_head_bwd(const HeadBwdArgs& a, bool a_bf16, cudaStream_t st, int64_t* launches);
