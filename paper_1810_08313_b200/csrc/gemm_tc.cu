@@ -671,6 +671,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 constexpr int kPairStages = 4;
 constexpr int kPairN = 512;          // columns of the pair's tile: two MMA blocks of 256
 constexpr int kPairGroups = kPairN / 64;      // 64-column groups of the epilogue (one 128-byte box row each)
+constexpr int kThreadsPair = 320;    // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue (two per TMEM lane quarter)
 struct SmemPair {
   static constexpr int kABytes = BM * KB_BYTES;                 // this CTA's 128 rows
   static constexpr int kBBlockBytes = 128 * KB_BYTES;           // this CTA's half of one 256-column block
@@ -699,7 +700,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* s
 // tmC: the output [groups*M][N] as boxes of 64 rows x 64 bf16 (128-byte swizzle); tmMask (backward): the
 // activations of the layer, same shape and boxes.
 template <bool B_MN, int EPI>
-__global__ void __launch_bounds__(kThreadsBf16, 1)
+__global__ void __launch_bounds__(kThreadsPair, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmMask, const Params p) {
   using L = SmemPair;
@@ -750,7 +751,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   grid_dep_wait();
   grid_dep_launch();
 
-  float dx_pb[2] = {0.f, 0.f}, dx_pvb[2] = {0.f, 0.f};   // backward: bias / momentum elements this thread updates
+  float dx_pb = 0.f, dx_pvb = 0.f;      // backward: the bias / momentum element this thread updates
   if (warp == 0) {
     if (elect_one()) {
       const uint64_t pol_a = l2_policy(2), pol_b = l2_policy(1);
@@ -822,26 +823,26 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (ok) mma_commit_pair(acc_full);
     }
   } else {
-    // ---- epilogue of this CTA's 128 rows x 512 columns ------------------------------------------
+    // ---- epilogue of this CTA's 128 rows x 512 columns: warps 2-5 take columns 0..255, warps 6-9 the rest ----
     const int q = warp & 3;                  // TMEM lanes 32 q .. 32 q + 31
+    const int cs = (warp - 2) >> 2;          // column half of the tile
     const int half = q >> 1;                 // rows 64 half .. of the CTA: one TMA box with the other warp of the half
     const int rih = (q & 1) * 32 + lane;     // this thread's row inside the box
-    const int et = (int)threadIdx.x - 64;    // 0..127 among the epilogue threads
+    const int et = (int)threadIdx.x - 64;    // 0..255 among the epilogue threads
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     // while the products run: the bias of the tile's columns goes to shared memory (forward), and the bias
     // elements that this thread will update are requested (backward)
     if (EPI == EPI_FWD) {
-      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + (int64_t)g * p.bias_gstride + n0) + et);
-      reinterpret_cast<float4*>(bias_s)[et] = bv;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-    } else if (p.dbias != nullptr) {
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const int64_t at = (int64_t)g * p.dbias_gstride + n0 + rank * 256 + et + i * 128;
-        dx_pb[i] = p.dbias[at];
-        if (p.mu != 0.f) dx_pvb[i] = p.dvbias[at];
+      if (et < kPairN / 4) {
+        float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.bias) bv = __ldg(reinterpret_cast<const float4*>(p.bias + (int64_t)g * p.bias_gstride + n0) + et);
+        reinterpret_cast<float4*>(bias_s)[et] = bv;
       }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    } else if (p.dbias != nullptr) {
+      const int64_t at = (int64_t)g * p.dbias_gstride + n0 + rank * 256 + et;
+      dx_pb = p.dbias[at];
+      if (p.mu != 0.f) dx_pvb = p.dvbias[at];
     }
     bool ok = mbar_wait(acc_full, 0);
     ok = __all_sync(0xffffffffu, ok);
@@ -849,15 +850,18 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (!ok && lane == 0) atomicExch(p.err_flag, 23);
     if (ok) {
       // the accumulator is read one 32-column block ahead of the arithmetic
+      constexpr int kBlocks = kPairN / 64;           // 32-column blocks per warp
+      const int c_begin = cs * kBlocks;
       uint32_t r[2][32];
-      tmem_ld_32x32(taddr, r[0]);
+      tmem_ld_32x32(taddr + c_begin * 32, r[0]);
 #pragma unroll
-      for (int c = 0; c < kPairN / 32; ++c) {
+      for (int ci = 0; ci < kBlocks; ++ci) {
+        const int c = c_begin + ci;
         const int grp = c >> 1, sub = c & 1;
         uint8_t* box = smem + (grp * 2 + half) * L::kBoxBytes;
         uint8_t* myrow = box + rih * 128;
         tmem_ld_wait();
-        if (c + 1 < kPairN / 32) tmem_ld_32x32(taddr + (c + 1) * 32, r[(c + 1) & 1]);
+        if (ci + 1 < kBlocks) tmem_ld_32x32(taddr + (c + 1) * 32, r[(ci + 1) & 1]);
         if (EPI == EPI_DX && sub == 0 && ok) {
           // (after a failed wait the loop goes on without the mask, so that every barrier below is still met)
           ok = __all_sync(0xffffffffu, mbar_wait(&mask_full[grp], 0));
@@ -872,7 +876,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const float b4[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float v = __uint_as_float(r[c & 1][4 * i + e]) + b4[e];
+              const float v = __uint_as_float(r[ci & 1][4 * i + e]) + b4[e];
               o[4 * i + e] = (p.relu && !(v > 0.f)) ? 0.f : v;
             }
           }
@@ -885,8 +889,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int j = 0; j < 4; ++j) {
               // a bf16 is positive iff it is non-zero with the sign bit clear
               const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
-              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[c & 1][i * 8 + j * 2]) : 0.f;
-              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[c & 1][i * 8 + j * 2 + 1]) : 0.f;
+              o[i * 8 + j * 2] = (lo != 0 && lo < 0x8000u) ? __uint_as_float(r[ci & 1][i * 8 + j * 2]) : 0.f;
+              o[i * 8 + j * 2 + 1] = (hi != 0 && hi < 0x8000u) ? __uint_as_float(r[ci & 1][i * 8 + j * 2 + 1]) : 0.f;
             }
           }
         }
@@ -904,8 +908,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (sub == 1) {
           // both warps of the half have written the box: hand it to the bulk-copy engine
           fence_proxy_async_smem();
-          if (half == 0) asm volatile("bar.sync 2, 64;" ::: "memory");
-          else asm volatile("bar.sync 3, 64;" ::: "memory");
+          asm volatile("bar.sync %0, 64;" ::"r"(2 + half + 2 * cs) : "memory");
           if ((q & 1) == 0 && lane == 0) {
             tma_store_2d(&tmC, box, n0 + grp * 64, out_row0 + half * 64);
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -947,9 +950,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp >= 2) {
       const uint32_t mine = smem_u32(colsum);
       const uint32_t src0 = map_to_rank(mine, 0), src1 = map_to_rank(mine, 1);
-#pragma unroll
-      for (int i2 = 0; i2 < 2; ++i2) {
-        const int t = rank * 256 + (int)threadIdx.x - 64 + i2 * 128;
+      {
+        const int t = rank * 256 + (int)threadIdx.x - 64;
         float gsum = 0.f;
 #pragma unroll
         for (int i = 0; i < 2; ++i) gsum += ld_cluster_f32(src0 + (uint32_t)((i * kPairN + t) * 4));
@@ -958,10 +960,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int64_t at = (int64_t)g * p.dbias_gstride + n0 + t;
         float step = gsum;
         if (p.mu != 0.f) {
-          step = fmaf(p.mu, dx_pvb[i2], gsum);
+          step = fmaf(p.mu, dx_pvb, gsum);
           p.dvbias[at] = step;
         }
-        p.dbias[at] = fmaf(-p.lr, step, dx_pb[i2]);
+        p.dbias[at] = fmaf(-p.lr, step, dx_pb);
       }
     }
   }
@@ -1015,7 +1017,7 @@ int launch_pair(const TcOperandMaps& mp, const CUtensorMap* c_map, const CUtenso
     if (e != cudaSuccess) return e;
   }
   dim3 grid((unsigned)(p.N / kPairN * 2), (unsigned)(p.M / 256), (unsigned)groups);
-  return launch_dep(kern, grid, dim3(kThreadsBf16), SmemPair::kTotal, st, 2, *mp.a, *mp.b, *c_map,
+  return launch_dep(kern, grid, dim3(kThreadsPair), SmemPair::kTotal, st, 2, *mp.a, *mp.b, *c_map,
                     mask_map ? *mask_map : *c_map, p);
 }
 // bf16 shapes that the pair kernel covers

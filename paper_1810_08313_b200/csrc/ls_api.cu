@@ -196,7 +196,8 @@ struct XMaps { const CUtensorMap* k; const CUtensorMap* mn; const CUtensorMap* u
 static bool head_step_args(ls_handle* h, const void* y, const int64_t* row_off_dev, float* loss_out, HeadStepArgs& a) {
   const Layout& lay = h->lay;
   const int l = lay.L - 1;
-  if (!lay.bf16 || l < 1 || lay.hstep_off == 0 || !head_shape_ok(lay.batch, lay.dims[lay.L])) return false;
+  if (!h->allow_head_step || !lay.bf16 || l < 1 || lay.hstep_off == 0 || !head_shape_ok(lay.batch, lay.dims[lay.L]))
+    return false;
   a.A = h->state + lay.act_off[l];
   a.y = y; a.y_row_off = row_off_dev;
   a.W = params_of(h) + lay.w_off[l]; a.V = mom_of(h) + lay.w_off[l]; a.Wb = shadow_of(h) + lay.w_off[l];
@@ -689,6 +690,7 @@ int ls_create(ls_handle** out, int m, const ls_model_spec* spec, float lr, float
   h->state = static_cast<char*>(state_dev);
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->allow_pair = pair_kernels_enabled();
+  h->allow_head_step = head_step_enabled();
   for (int l = 0; l < lay.L; ++l)
     if (lay.tiled[l]) {
       TileMap& tm = h->tiles;

@@ -141,6 +141,7 @@ struct ls_handle {
   int64_t n_rows;
   int last_cuda;
   bool allow_pair;        // CTA-pair kernels enabled (see pair_kernels_enabled)
+  bool allow_head_step;   // one-launch output layer enabled (see head_step_enabled)
   ls::TileMap tiles;      // the blocked matrices of a replica vector
   bool sync_valid;        // every replica's parameters and momentum equal the synchronized copy, bit for bit
   // replicas spread over several GPUs (ls_set_shard): this handle holds m of m_total replicas
@@ -206,6 +207,13 @@ inline cudaError_t launch_dep(void (*kern)(P...), dim3 grid, dim3 block, size_t 
 
 // LS_DISABLE_PAIR=1 in the environment keeps every launch of a handle on the one-CTA tensor-core kernels (a
 // diagnostic switch; read once, when the handle is created, and carried in the launch arguments).
+// LS_DISABLE_HEAD_STEP=1 in the environment at ls_create time: the output layer of a training step runs as the
+// forward kernel followed by head_bwd_kernel instead of the one-launch kernel (a diagnostic switch; the tests
+// compare the two).
+inline bool head_step_enabled() {
+  const char* e = getenv("LS_DISABLE_HEAD_STEP");
+  return !(e && e[0] == '1');
+}
 inline bool pair_kernels_enabled() {
   const char* e = getenv("LS_DISABLE_PAIR");
   return !(e && e[0] == '1');

@@ -170,3 +170,44 @@ def test_cta_pair_kernels_match_one_cta_kernels(dims, m, B, monkeypatch):
                 err = np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-30)
                 assert err < tol, (i, name, err)
 
+
+
+@pytest.mark.parametrize("dims,m,B", [((512, 512, 1024, 10), 3, 256), ((256, 384, 10), 5, 64), ((384, 2048, 10), 2, 32),
+                                      ((256, 128, 10), 17, 256)])
+def test_one_launch_output_layer_matches_two_kernels(dims, m, B, monkeypatch):
+    """The output layer of a training step as one launch (clusters of four CTAs, two per replica) against the
+    forward + backward kernels it replaces (LS_DISABLE_HEAD_STEP=1), three steps from the same state.  Both
+    compute the same fp32 products; only the order of the sums differs, so the output layer's weights, both
+    biases and the first loss agree to fp32 rounding; dZ of the layer below is stored in bf16, where a different
+    last bit of a sum can flip a rounding, so the layers below (and, from the second step on, everything) get the
+    bound of one bf16 step on a few elements.
+    Shapes: 32, 8 and 4 rows per CTA, one and several column groups per thread, more replicas than fit one round."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    from tests.helpers import tensor_slices
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 37, bf16=True)
+    steps = 3
+    offs = wl.batch_row_offsets(11, steps, m, 1024, B)
+    xd, yd = to_device(X, y, bf16=True)
+    out = {}
+    for tag, val in (("one", "0"), ("two", "1")):
+        monkeypatch.setenv("LS_DISABLE_HEAD_STEP", val)
+        eng = LocalSGD(m, dims, gemm_dtype="bf16", lr=0.05, momentum=0.9, batch=B)
+        eng.bind_dataset(xd, yd); eng.set_params(x1)
+        ld = torch.zeros((steps, m), device="cuda")
+        n0 = eng.launch_count()
+        eng.local_steps(steps, offs, ld)
+        eng.sync()
+        out[tag] = eng.get_all() + (ld.cpu().numpy(), eng.launch_count() - n0)
+        eng.close()
+    (px, pv, pl, pn), (ox, ov, ol, on) = out["one"], out["two"]
+    assert pn < on, (pn, on)                      # the one-launch path really ran: fewer launches per step
+    assert np.max(np.abs(pl[0] - ol[0]) / np.abs(ol[0])) < 1e-5     # first step: the same inputs, fp32 sums
+    assert np.max(np.abs(pl - ol) / np.abs(ol)) < 2e-3
+    L = len(dims) - 1
+    for i in range(m):
+        for name, sl in tensor_slices(dims, True):
+            tol = 2e-3 if name in (f"W{L}", f"b{L}") else 2e-2
+            for a, b in ((px[i][sl], ox[i][sl]), (pv[i][sl], ov[i][sl])):
+                err = np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-30)
+                assert err < tol, (i, name, err)
