@@ -152,12 +152,26 @@ def stored_traffic(w: wl.Workload, cls: str, layer: int):
     return None
 
 
-def roofline_for(dom, dur_s: float, w: wl.Workload, peaks, clocks):
+def roofline_for(dom, dur_s: float, w: wl.Workload, peaks, clocks, tau: int = 0):
     """Roofline object of the dominant kernel (class, layer) given its mean launch duration."""
     cls, layer = dom
     ms = dur_s * 1e3
     src = f"of {peaks['source']}"
     traffic = stored_traffic(w, cls, layer)
+    if cls == "avg" and layer == 1:
+        # last update of a period + averaging in one launch: per streamed parameter, write W, v and the bf16 copy
+        # of m replicas (10 m B) and the synchronized copy (8 B); read the old state once (8 B, period of 1) or
+        # every replica's own (8 m B)
+        merged = streamed_update_layers(w)
+        shapes = layer_shapes(w)
+        n = float(sum(shapes[l][0] * shapes[l][1] for l in merged))
+        sb = 8.0 if w.momentum != 0 else 4.0          # W and v, or W alone
+        by = n * ((sb + 2.0) * w.m + sb + (sb if tau == 1 else sb * w.m))
+        ach = by / dur_s / 1e9
+        return {"kernel": f"weight gradient + update + averaging, layers {merged} in one launch (tcgen05, streaming)",
+                "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": src, "ms_per_launch": ms,
+                "bytes_per_launch": by, "frac_of_8TBs": ach / 8000.0}
     if cls == "avg":
         by = 8.0 * w.m * wl.n_params(w.dims, w.has_bias) * (2 if w.momentum != 0 else 1)
         ach = by / dur_s / 1e9
@@ -513,7 +527,7 @@ def run_ours(args, w: wl.Workload):
     value = units / (ms * 1e-3)
 
     # ---- roofline of the dominant kernel ---------------------------------------
-    roofline = roofline_for(dom, dom_ms * 1e-3 / dom_n, w_r, peaks, clocks) if dom_n else None
+    roofline = roofline_for(dom, dom_ms * 1e-3 / dom_n, w_r, peaks, clocks, tau) if dom_n else None
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,

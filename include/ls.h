@@ -402,8 +402,10 @@ int ls_linear_loss_static(const float* W_dev, const float* bias_dev, const float
  * ls_profile_end() waits for the stream and adds up, per class and layer, the
  * elapsed milliseconds and the number of launches into
  * ms[LS_K_CLASSES * LS_MAX_LAYERS] and launches[...] (index class*LS_MAX_LAYERS
- * + layer; LS_K_LOSS and LS_K_AVG use layer 0).  At most 16384 launches are
- * recorded per profile; later ones are run but not timed. */
+ * + layer; LS_K_LOSS uses layer 0; LS_K_AVG uses layer 0 for the averaging
+ * kernel and layer 1 for the launch that does the last weight update of a
+ * period and its averaging step together, both whatever `layer` says).  At most
+ * 16384 launches are recorded per profile; later ones are run but not timed. */
 enum { LS_K_FWD = 0, LS_K_LOSS = 1, LS_K_DX = 2, LS_K_DW = 3, LS_K_BIAS = 4, LS_K_AVG = 5, LS_K_CLASSES = 6 };
 int ls_profile_begin(ls_handle* h, uint32_t class_mask, int layer);
 int ls_profile_end(ls_handle* h, double* ms, int64_t* launches);

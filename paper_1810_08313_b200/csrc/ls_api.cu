@@ -463,16 +463,17 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
   std::sort(upd, upd + n_upd, [](const TcUpdateArgs& x, const TcUpdateArgs& y) {
     return (int64_t)x.M * x.N > (int64_t)y.M * y.N;
   });
-  // A step that starts from synchronized replicas and ends in an averaging step (communication period 1): the
-  // streamed layers' update and their average are one launch that never writes the per-replica values; the
-  // small tensors (biases, a narrow output layer), updated per replica above, are averaged by the plain kernel.
-  bool fused = avg_after && h->sync_valid && n_upd > 0 && bf && h->shard_G == 0 &&
+  // A step that ends in an averaging step (the last of a communication period): the streamed layers' update and
+  // their average are one launch that never writes the per-replica values (and, at a period of 1, reads the old
+  // state once, from the synchronized copy: upd[].mapWsync is set then); the small tensors (biases, a narrow
+  // output layer), updated per replica above, are averaged by the plain kernel.
+  bool fused = avg_after && n_upd > 0 && bf && h->shard_G == 0 &&
                (h->mu == 0.f ? h->spec.momentum_mode != LS_MOMENTUM_BLOCK : h->spec.momentum_mode == LS_MOMENTUM_AVERAGE);
   for (int i = 0; i < n_upd && fused; ++i) fused = tc_sync_step_shape_ok(false, upd[i].M, upd[i].N, upd[i].B);
   if (fused) {
     for (int i = 0; i < n_upd; i += tc_update_max_layers()) {
       const int n = std::min(n_upd - i, tc_update_max_layers());
-      ProfScope ps(h, LS_K_DW, upd[i].layer);
+      ProfScope ps(h, LS_K_AVG, 1);
       LS_CUDA(h, launch_tc_sync_step(upd + i, n, h->stream, &h->launches));
     }
     // what is left of a replica vector: the gaps between the streamed weight matrices, in layout order

@@ -739,6 +739,60 @@ __device__ __forceinline__ SUnit decode_sunit(const SParams& p, int u) {
   return SUnit{l, (r / nt) * BM, (r % nt) * SN};
 }
 
+// The mean of one 32 x 32 block (W at `slot`, v 4 KB behind it, 128-byte rows with XOR-swizzled 16-byte pieces) goes
+// out to every replica, to the bf16 copies and to the synchronized copy with plain 16-byte stores, eight lanes to a
+// 128-byte row.  The block is read from shared memory once; after_read() runs when it is in registers.
+template <typename F>
+__device__ __forceinline__ void store_mean_block(const SParams& p, const SLayer& ly, const SUnit& un, int q, int half,
+                                                 const uint8_t* slot, int m, bool has_v, int lane, F after_read) {
+  const int row0 = lane >> 3, piece = lane & 7;
+  const int64_t ldw = ly.N;
+  float4 w4[8], v4[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = i * 4 + row0;
+    w4[i] = *reinterpret_cast<const float4*>(slot + row * 128 + ((piece ^ (row & 7)) << 4));
+    if (has_v) v4[i] = *reinterpret_cast<const float4*>(slot + kSlotBytes / 2 + row * 128 + ((piece ^ (row & 7)) << 4));
+  }
+  after_read();
+  uint2 cp[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(w4[i].x, w4[i].y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(w4[i].z, w4[i].w);
+    cp[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  }
+  // where this lane's first row piece goes, and the distance to its next one (four rows down): row-major,
+  // or inside the block's own 4 KB when the master copy is blocked; the bf16 copy row-major or in panels
+  const int64_t rm = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
+  const int64_t mat = ly.blocked ? ((int64_t)((un.m0 >> 5) + q) * (ldw >> 5) + (un.n0 >> 5) + half) * 1024 +
+                                       row0 * 32 + piece * 4
+                                 : rm;
+  const int64_t mstep = ly.blocked ? 4 * 32 : 4 * ldw;
+  const int64_t at = copy_index(ly.pM, (int)ldw, un.m0 + q * 32 + row0, un.n0 + half * 32 + piece * 4);
+  const int64_t bstep = ly.pM ? 4 * 64 : 4 * ldw;
+  for (int g = 0; g <= m; ++g) {
+    // g = m: the synchronized copy
+    float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + mat;
+    float* Vd = (g < m ? ly.V + (int64_t)g * p.w_gstride : ly.Vs) + mat;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Wd + i * mstep) = w4[i];
+    if (has_v) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Vd + i * mstep) = v4[i];
+    }
+    if (ly.Wb != nullptr && g < m) {
+      __nv_bfloat16* Bd = ly.Wb + (int64_t)g * p.w_gstride + at;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(Bd + i * bstep) = cp[i];
+    }
+  }
+}
+
+// SHARED: every replica enters with the synchronized W and v (a period of 1).  Otherwise (the last step of a longer
+// period) replica g's own block comes in for every g, through the two buffers of each update warp in turn, and the
+// update warps send the mean out themselves: the buffers have no room for a block that waits for a store warp.
+template <bool SHARED>
 __global__ void __launch_bounds__(kSyncThreads, 1)
 tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ SParams p) {
   using L = SSmem;
@@ -850,59 +904,20 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
     // bulk-copy engine stays free for the operand tiles (with the mean leaving through it as well, the products
     // waited behind the queued stores: 5.6 k cycles per replica against 2 k).
     const int half = warp - 2;
-    const int row0 = lane >> 3, piece = lane & 7;
     bool ok = true;
-    for (int n = 0; n < my_units && ok; ++n) {
+    for (int n = 0; SHARED && n < my_units && ok; ++n) {
       const SUnit un = decode_sunit(p, bx + n * grid);
       const SLayer& ly = p.layer[un.layer];
-      const int64_t ldw = ly.N;
       for (int q = 0; q < 4 && ok; ++q) {
         const int wi = half * 4 + q;
         const uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
         ok = __all_sync(0xffffffffu, mbar_wait(&mean_ready[(n & 1) * 8 + wi], (n >> 1) & 1));
         if (!ok) { if (lane == 0) atomicExch(p.err_flag, 57); break; }
-        float4 w4[8], v4[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int row = i * 4 + row0;
-          w4[i] = *reinterpret_cast<const float4*>(slot + row * 128 + ((piece ^ (row & 7)) << 4));
-          if (has_v) v4[i] = *reinterpret_cast<const float4*>(slot + kSlotBytes / 2 + row * 128 + ((piece ^ (row & 7)) << 4));
-        }
-        // the block is in registers: release its buffer (the arrival orders the reads above before it)
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&mean_gone[(n & 1) * 8 + wi]);
-        uint2 cp[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(w4[i].x, w4[i].y);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(w4[i].z, w4[i].w);
-          cp[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-        }
-        // where this lane's first row piece goes, and the distance to its next one (four rows down): row-major,
-        // or inside the block's own 4 KB when the master copy is blocked; the bf16 copy row-major or in panels
-        const int64_t rm = (int64_t)(un.m0 + q * 32 + row0) * ldw + un.n0 + half * 32 + piece * 4;
-        const int64_t mat = ly.blocked ? ((int64_t)((un.m0 >> 5) + q) * (ldw >> 5) + (un.n0 >> 5) + half) * 1024 +
-                                             row0 * 32 + piece * 4
-                                       : rm;
-        const int64_t mstep = ly.blocked ? 4 * 32 : 4 * ldw;
-        const int64_t at = copy_index(ly.pM, ldw, un.m0 + q * 32 + row0, un.n0 + half * 32 + piece * 4);
-        const int64_t bstep = ly.pM ? 4 * 64 : 4 * ldw;
-        for (int g = 0; g <= m; ++g) {
-          // g = m: the synchronized copy
-          float* Wd = (g < m ? ly.W + (int64_t)g * p.w_gstride : ly.Ws) + mat;
-          float* Vd = (g < m ? ly.V + (int64_t)g * p.w_gstride : ly.Vs) + mat;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Wd + i * mstep) = w4[i];
-          if (has_v) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(Vd + i * mstep) = v4[i];
-          }
-          if (ly.Wb != nullptr && g < m) {
-            __nv_bfloat16* Bd = ly.Wb + (int64_t)g * p.w_gstride + at;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(Bd + i * bstep) = cp[i];
-          }
-        }
+        // once the block is in registers its buffer is released (the arrival orders the reads before it)
+        store_mean_block(p, ly, un, q, half, slot, m, has_v, lane, [&] {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&mean_gone[(n & 1) * 8 + wi]);
+        });
       }
     }
   } else if (warp >= 4) {
@@ -910,6 +925,85 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
     const int q = warp & 3, half = (warp - 4) >> 2, wi = half * 4 + q;
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 32);
     const float mf = (float)m;
+    if (!SHARED) {
+      // ---- every replica's own W, v: block of accumulator a = n m + g in buffer a & 1 ---------------------------
+      const int total = my_units * m;
+      auto load_rep = [&](int a) {           // lane 0
+        const int n = a / m, g = a - n * m;
+        const SUnit un = decode_sunit(p, bx + n * grid);
+        uint8_t* slot = base_buf + (a & 1) * L::kBaseBytes + wi * kSlotBytes;
+        uint64_t* bar = &base_full[(a & 1) * 8 + wi];
+        mbar_expect_tx(bar, has_v ? kSlotBytes : kSlotBytes / 2);
+        int x = un.n0 + half * 32, y = un.m0 + q * 32;
+        block_coords(p.layer[un.layer].blocked, p.layer[un.layer].N, x, y);
+        tma_load_3d(slot, &maps.w[un.layer], bar, x, y, g);
+        if (has_v) tma_load_3d(slot + kSlotBytes / 2, &maps.v[un.layer], bar, x, y, g);
+      };
+      if (lane == 0 && total > 0) load_rep(0);
+      bool ok = true;
+      int a = 0;
+      for (int n = 0; n < my_units && ok; ++n) {
+        const SUnit un = decode_sunit(p, bx + n * grid);
+        float sw[32], sv[32];
+#pragma unroll 1
+        for (int g = 0; g < m; ++g, ++a) {
+          const int buf = a & 1;
+          uint8_t* slot = base_buf + buf * L::kBaseBytes + wi * kSlotBytes;
+          // the other buffer was last read by this warp (replica a - 1, or the mean of the unit before): refill it
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && a + 1 < total) load_rep(a + 1);
+          ok = __all_sync(0xffffffffu, mbar_wait(&base_full[buf * 8 + wi], (a >> 1) & 1));
+          if (!ok) { if (lane == 0) atomicExch(p.err_flag, 58); break; }
+          ok = __all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (a >> 1) & 1));
+          if (!ok) { if (lane == 0) atomicExch(p.err_flag, 55); break; }
+          tc_fence_after_sync();
+          uint32_t r[32];
+          tmem_ld_32x32(taddr + buf * SN, r);
+          tmem_ld_wait();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) {
+            const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+            const float4 w = *reinterpret_cast<const float4*>(slot + off);
+            const float ws[4] = {w.x, w.y, w.z, w.w};
+            float vs[4] = {0.f, 0.f, 0.f, 0.f};
+            if (has_v) {
+              const float4 v = *reinterpret_cast<const float4*>(slot + kSlotBytes / 2 + off);
+              vs[0] = v.x; vs[1] = v.y; vs[2] = v.z; vs[3] = v.w;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float gr = __uint_as_float(r[jj * 4 + e]);
+              const float step = has_v ? fmaf(p.mu, vs[e], gr) : gr;          // v_g
+              const float wn = fmaf(-p.lr, step, ws[e]);                     // w_g
+              sw[jj * 4 + e] = g == 0 ? wn : __fadd_rn(sw[jj * 4 + e], wn);
+              sv[jj * 4 + e] = g == 0 ? step : __fadd_rn(sv[jj * 4 + e], step);
+            }
+          }
+        }
+        if (!ok) break;
+        // the mean takes the place of the last replica's block (its buffer is not refilled before the next
+        // iteration), and this warp sends it out
+        uint8_t* slot = base_buf + ((a - 1) & 1) * L::kBaseBytes + wi * kSlotBytes;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) { sw[e] = __fdiv_rn(sw[e], mf); sv[e] = __fdiv_rn(sv[e], mf); }
+        __syncwarp();
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const int off = lane * 128 + ((jj ^ (lane & 7)) << 4);
+          *reinterpret_cast<float4*>(slot + off) = make_float4(sw[jj * 4], sw[jj * 4 + 1], sw[jj * 4 + 2], sw[jj * 4 + 3]);
+          if (has_v)
+            *reinterpret_cast<float4*>(slot + kSlotBytes / 2 + off) =
+                make_float4(sv[jj * 4], sv[jj * 4 + 1], sv[jj * 4 + 2], sv[jj * 4 + 3]);
+        }
+        __syncwarp();
+        store_mean_block(p, p.layer[un.layer], un, q, half, slot, m, has_v, lane, [] {});
+      }
+      tc_fence_before_sync();
+    } else {
     auto load_base = [&](int n) {            // lane 0: this warp's 32 x 32 block of the old W and v of unit n
       const SUnit un = decode_sunit(p, bx + n * grid);
       uint8_t* slot = base_buf + (n & 1) * L::kBaseBytes + wi * kSlotBytes;
@@ -991,6 +1085,7 @@ tc_sync_step_kernel(const __grid_constant__ UMaps maps, const __grid_constant__ 
       if (lane == 0) mbar_arrive(&mean_ready[(n & 1) * 8 + wi]);
     }
     tc_fence_before_sync();
+    }
   }
   __syncthreads();
   if (warp == 1) {
@@ -1110,16 +1205,21 @@ bool tc_sync_step_shape_ok(bool fp32, int M, int N, int B) {
   return !fp32 && M > 0 && N > 0 && B > 0 && M % BM == 0 && N % SN == 0 && B % kRowsBf16 == 0;
 }
 
-// layers[0..n): every layer needs its synchronized-copy descriptors (mapWsync / mapVsync)
+// layers[0..n): with the synchronized-copy descriptors (mapWsync / mapVsync) on every layer the replicas are taken to
+// enter synchronized and the old state is read from that copy; without them every replica's own state is read
 int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int64_t* launches) {
   if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
-  for (int i = 0; i < n; ++i)
-    if (layers[i].fp32 || layers[i].mapWsync == nullptr || layers[i].mapVsync == nullptr || layers[i].W == nullptr ||
-        layers[i].V == nullptr || layers[i].Wsync == nullptr || layers[i].Vsync == nullptr)
+  bool shared = true;
+  for (int i = 0; i < n; ++i) {
+    if (layers[i].fp32 || layers[i].W == nullptr || layers[i].V == nullptr || layers[i].Wsync == nullptr ||
+        layers[i].Vsync == nullptr)
       return cudaErrorInvalidValue;
-  static uint64_t configured = 0;
+    shared = shared && layers[i].mapWsync != nullptr && layers[i].mapVsync != nullptr;
+  }
+  static uint64_t configured[2] = {0, 0};
   {
-    cudaError_t e = allow_dynamic_smem(tc_sync_step_kernel, (int)SSmem::kTotal, &configured);
+    cudaError_t e = shared ? allow_dynamic_smem(tc_sync_step_kernel<true>, (int)SSmem::kTotal, &configured[0])
+                           : allow_dynamic_smem(tc_sync_step_kernel<false>, (int)SSmem::kTotal, &configured[1]);
     if (e != cudaSuccess) return e;
   }
   const TcUpdateArgs& a0 = layers[0];
@@ -1134,7 +1234,7 @@ int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int6
     l.pM = a.panel ? a.M : 0;
     total += (a.M / BM) * (a.N / SN);
     maps.a[i] = *a.maps.a; maps.b[i] = *a.maps.b; maps.w[i] = *a.mapW; maps.v[i] = *a.mapV;
-    maps.wl[i] = *a.mapWsync; maps.vl[i] = *a.mapVsync;
+    maps.wl[i] = shared ? *a.mapWsync : *a.mapW; maps.vl[i] = shared ? *a.mapVsync : *a.mapV;
   }
   for (int i = n; i < kMaxLayers; ++i) {
     maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.w[i] = maps.w[0]; maps.v[i] = maps.v[0];
@@ -1145,7 +1245,8 @@ int launch_tc_sync_step(const TcUpdateArgs* layers, int n, cudaStream_t st, int6
   p.lr = a0.lr; p.mu = a0.mu; p.w_gstride = a0.w_gstride; p.err_flag = a0.err_flag;
   if (launches) ++*launches;
   const int grid = total < num_sms() ? total : num_sms();
-  return launch_dep(tc_sync_step_kernel, dim3(grid), dim3(kSyncThreads), SSmem::kTotal, st, 1, maps, p);
+  if (shared) return launch_dep(tc_sync_step_kernel<true>, dim3(grid), dim3(kSyncThreads), SSmem::kTotal, st, 1, maps, p);
+  return launch_dep(tc_sync_step_kernel<false>, dim3(grid), dim3(kSyncThreads), SSmem::kTotal, st, 1, maps, p);
 }
 
 int tc_update_max_layers() { return kMaxLayers; }

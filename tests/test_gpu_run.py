@@ -490,3 +490,50 @@ def test_period_of_one_from_a_synchronized_start(dims, dtype, m, B, mu):
     ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(mu), 1)
     lerr = np.max(np.abs(out["fused"][3] - ref.loss) / ref.loss)
     assert lerr <= (2e-2 if bf else 1e-4)
+
+
+@pytest.mark.parametrize("dims,m,B,mu,tau", [
+    ((256, 256, 128, 10), 5, 128, 0.9, 3),             # odd replica count: the mean lands in the first buffer
+    ((1024, 1024, 10), 16, 256, 0.9, 2),               # sixteen replicas, CTA-pair GEMMs
+    ((2048, 1280, 10), 2, 128, 0.0, 4),                # no momentum buffers; more units than SMs
+])
+def test_last_step_of_a_period_fused_with_the_average(dims, m, B, mu, tau):
+    """Communication periods longer than 1: the last local step of a period and the averaging step are one launch for
+    the streamed layers of a bf16 model (every replica's own W, v read once, the per-replica results never
+    written).  It must leave the state of ls_local_steps followed by ls_average bit for bit, period after period."""
+    import torch
+    from paper_1810_08313_b200.binding import LocalSGD
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 47, bf16=True)
+    periods = 3
+    offs = wl.batch_row_offsets(19, periods * tau, m, 1024, B)
+    xd, yd = to_device(X, y, bf16=True)
+    out = {}
+    for tag in ("fused", "separate"):
+        eng = LocalSGD(m, dims, gemm_dtype="bf16", lr=0.05, momentum=mu, batch=B)
+        eng.bind_dataset(xd, yd)
+        eng.set_params(x1)
+        losses = torch.zeros((periods * tau, m), device="cuda")
+        n0 = eng.launch_count()
+        for j in range(periods):
+            sl = slice(j * tau, (j + 1) * tau)
+            if tag == "fused":
+                eng.local_steps(tau, offs[sl], losses[sl], average=True)
+            else:
+                eng.local_steps(tau, offs[sl], losses[sl])
+                eng.average()
+        eng.sync()
+        px, pv = eng.get_all()
+        F = eng.eval_loss(m - 1, 0, 2 * B)                  # reads the bf16 copies of the last replica
+        p_dev, _ = eng.state_view()
+        assert bool((p_dev[0:1] == p_dev).all())
+        out[tag] = (px, pv, F, losses.cpu().numpy(), eng.launch_count() - n0)
+        eng.close()
+    a, b = out["fused"], out["separate"]
+    assert np.array_equal(a[0].view(np.uint32), b[0].view(np.uint32))
+    assert np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+    assert a[2] == b[2]
+    assert np.array_equal(a[3], b[3])
+    if len(dims) > 3:            # (with one streamed matrix both sequences happen to have the same length)
+        assert a[4] != b[4]      # the two really took different launch sequences
+    ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(mu), tau)
+    assert np.max(np.abs(a[3] - ref.loss) / ref.loss) <= 2e-2
