@@ -25,6 +25,7 @@ namespace ls {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kMaxPieces = LS_MAX_LAYERS + 1;
 
 template <int W> struct Vec;
 template <> struct Vec<4> {
@@ -163,6 +164,51 @@ average_scalar_kernel(float* __restrict__ base, int64_t buf_stride, int m, int64
   }
 }
 
+// The same pass over several short pieces of the replica vectors in ONE launch (the biases and narrow layers
+// between the matrices that the step + averaging kernel owns): piece r covers elements [begin[r], begin[r] + 8 len[r])
+// and thread i of the launch takes 8-float slice i - first[r] of the piece with first[r] <= i < first[r + 1].
+// Arithmetic and order are those of average_kernel<0, 8, false>.
+struct Pieces {
+  int n;
+  int64_t begin[kMaxPieces];
+  int64_t first[kMaxPieces + 1];
+};
+__global__ void __launch_bounds__(kThreads)
+average_pieces_kernel(float* __restrict__ base, int64_t buf_stride, int m, Pieces pc, int64_t stride,
+                      __nv_bfloat16* __restrict__ shadow, float* __restrict__ sync_out, int64_t sync_stride) {
+  grid_dep_wait();
+  grid_dep_launch();
+  const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (i >= pc.first[pc.n]) return;
+  int r = 0;
+#pragma unroll
+  for (int k = 1; k < kMaxPieces; ++k)
+    if (k < pc.n && i >= pc.first[k]) r = k;
+  const int64_t at = pc.begin[r] + (i - pc.first[r]) * 8;
+  float* p = base + (int64_t)blockIdx.y * buf_stride + at;
+  const float mf = (float)m;
+  Vec<8> s;
+  s.load(p);
+  for (int j0 = 1; j0 < m; j0 += 8) {
+    Vec<8> v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j0 + j < m) v[j].load(p + (int64_t)(j0 + j) * stride);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j0 + j < m)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s.v[e] = __fadd_rn(s.v[e], v[j].v[e]);
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) s.v[e] = __fdiv_rn(s.v[e], mf);
+#pragma unroll 4
+  for (int j = 0; j < m; ++j) s.store(p + (int64_t)j * stride);
+  if (sync_out != nullptr) s.store(sync_out + (int64_t)blockIdx.y * sync_stride + at);
+  if (blockIdx.y == 0 && shadow != nullptr)
+    for (int j = 0; j < m; ++j) store_bf16<8>(shadow + (int64_t)j * stride + at, s.v);
+}
+
 template <int W, bool BM>
 void launch_vec(dim3 grid, cudaStream_t st, float* base, int64_t buf_stride, int m, int64_t n_vec, int64_t stride,
                 __nv_bfloat16* shadow, const BlockMomentum& bm, float* sync_out, int64_t sync_stride, const TileMap& tiles) {
@@ -229,6 +275,35 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+// pieces outside every blocked matrix (the bf16 copy has the master's element order there)
+int launch_average_pieces(float* base, int n_buf, int64_t buf_stride, int m, const int64_t* begin, const int64_t* len,
+                          int n_pieces, int64_t stride, __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
+                          float* sync_out, int64_t sync_stride) {
+  if (n_pieces <= 0 || n_buf <= 0) return cudaSuccess;
+  bool one = n_pieces <= kMaxPieces && aligned_to(base, 32) && stride % 8 == 0 && buf_stride % 8 == 0 &&
+             aligned_to(shadow, 16) && aligned_to(sync_out, 32) && sync_stride % 8 == 0;
+  for (int r = 0; r < n_pieces && one; ++r) one = begin[r] % 8 == 0 && len[r] % 8 == 0 && len[r] > 0;
+  if (!one) {
+    for (int r = 0; r < n_pieces; ++r) {
+      int e = launch_average(base + begin[r], n_buf, buf_stride, m, len[r], stride, shadow ? shadow + begin[r] : nullptr, st,
+                             launches, nullptr, sync_out ? sync_out + begin[r] : nullptr, sync_stride);
+      if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  }
+  Pieces pc{};
+  pc.n = n_pieces;
+  for (int r = 0; r < n_pieces; ++r) {
+    pc.begin[r] = begin[r];
+    pc.first[r + 1] = pc.first[r] + len[r] / 8;
+  }
+  const int64_t gx = (pc.first[n_pieces] + kThreads - 1) / kThreads;
+  if (gx > 2147483647LL) return cudaErrorInvalidValue;
+  if (launches) ++*launches;
+  return launch_dep(average_pieces_kernel, dim3((unsigned)gx, (unsigned)n_buf), dim3(kThreads), 0, st, 1, base, buf_stride, m,
+                    pc, stride, shadow, sync_out, sync_stride);
 }
 
 }  // namespace ls

@@ -482,15 +482,17 @@ static int local_step(ls_handle* h, const void* x, XMaps xmap, const void* y, co
     });
     const int64_t buf_stride = (int64_t)((lay.mom_off - lay.params_off) / 4);
     const int n_buf = h->mu != 0.f ? 2 : 1;
-    int64_t pos = 0;
+    int64_t pos = 0, begin[LS_MAX_LAYERS + 1], len[LS_MAX_LAYERS + 1];
+    int n_pieces = 0;
     for (int i = 0; i <= n_upd; ++i) {
       const int64_t end = i < n_upd ? lay.w_off[upd[i].layer] : lay.stride;
-      if (end > pos) {
-        ProfScope ps(h, LS_K_AVG, 0);
-        LS_CUDA(h, launch_average(params_of(h) + pos, n_buf, buf_stride, lay.m, end - pos, lay.stride, shadow_of(h) + pos,
-                                  h->stream, &h->launches, nullptr, sync_of(h) + pos, lay.stride));
-      }
+      if (end > pos) { begin[n_pieces] = pos; len[n_pieces] = end - pos; ++n_pieces; }
       if (i < n_upd) pos = round_up(lay.w_off[upd[i].layer] + (int64_t)upd[i].M * upd[i].N, kAlignFloats);
+    }
+    {
+      ProfScope ps(h, LS_K_AVG, 0);
+      LS_CUDA(h, launch_average_pieces(params_of(h), n_buf, buf_stride, lay.m, begin, len, n_pieces, lay.stride, shadow_of(h),
+                                       h->stream, &h->launches, sync_of(h), lay.stride));
     }
     h->sync_valid = true;
     return LS_OK;

@@ -259,6 +259,12 @@ int launch_average(float* base, int n_buf, int64_t buf_stride, int m, int64_t n,
                    const BlockMomentum* bm = nullptr, float* sync_out = nullptr, int64_t sync_stride = 0,
                    const TileMap* tiles = nullptr);    // tiles: the blocked matrices of `base` (`shadow`: shadow_index)
 
+// The same for n_pieces short pieces [begin[r], begin[r] + len[r]) of the replica vectors that lie outside every
+// blocked matrix, in one launch when their ends fall on multiples of 8 floats (else one launch each).
+int launch_average_pieces(float* base, int n_buf, int64_t buf_stride, int m, const int64_t* begin, const int64_t* len,
+                          int n_pieces, int64_t stride, __nv_bfloat16* shadow, cudaStream_t st, int64_t* launches,
+                          float* sync_out, int64_t sync_stride);
+
 // ---- averaging over several GPUs (shard_average.cu) -------------------------
 // out[b] = sum over the m vectors of buffer b in index order; then, with the G partial sums of every GPU
 // gathered in rank order (vector g of buffer b at parts + g*part_stride + b*part_buf_stride), the mean

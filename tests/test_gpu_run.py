@@ -513,7 +513,7 @@ def test_last_step_of_a_period_fused_with_the_average(dims, m, B, mu, tau):
         eng.bind_dataset(xd, yd)
         eng.set_params(x1)
         losses = torch.zeros((periods * tau, m), device="cuda")
-        n0 = eng.launch_count()
+        eng.profile_begin()
         for j in range(periods):
             sl = slice(j * tau, (j + 1) * tau)
             if tag == "fused":
@@ -526,14 +526,16 @@ def test_last_step_of_a_period_fused_with_the_average(dims, m, B, mu, tau):
         F = eng.eval_loss(m - 1, 0, 2 * B)                  # reads the bf16 copies of the last replica
         p_dev, _ = eng.state_view()
         assert bool((p_dev[0:1] == p_dev).all())
-        out[tag] = (px, pv, F, losses.cpu().numpy(), eng.launch_count() - n0)
+        prof = eng.profile_end()
+        eng.sync()
+        out[tag] = (px, pv, F, losses.cpu().numpy(), prof)
         eng.close()
     a, b = out["fused"], out["separate"]
     assert np.array_equal(a[0].view(np.uint32), b[0].view(np.uint32))
     assert np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
     assert a[2] == b[2]
     assert np.array_equal(a[3], b[3])
-    if len(dims) > 3:            # (with one streamed matrix both sequences happen to have the same length)
-        assert a[4] != b[4]      # the two really took different launch sequences
+    # the two really took different launch sequences: ("avg", 1) is the step + averaging launch
+    assert a[4][("avg", 1)][1] == periods and ("avg", 1) not in b[4]
     ref = orc.run_pasgd(spec, x1, X, y, offs, B, f32(0.05), f32(mu), tau)
     assert np.max(np.abs(a[3] - ref.loss) / ref.loss) <= 2e-2
