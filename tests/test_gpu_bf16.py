@@ -172,9 +172,13 @@ def test_cta_pair_kernels_match_one_cta_kernels(dims, m, B, monkeypatch):
 
 
 
-@pytest.mark.parametrize("dims,m,B", [((512, 512, 1024, 10), 3, 256), ((256, 384, 10), 5, 64), ((384, 2048, 10), 2, 32),
-                                      ((256, 128, 10), 17, 256)])
-def test_one_launch_output_layer_matches_two_kernels(dims, m, B, monkeypatch):
+@pytest.mark.parametrize("dims,m,B,has_bias,mu", [
+    ((512, 512, 1024, 10), 3, 256, True, 0.9), ((256, 384, 10), 5, 64, True, 0.9), ((384, 2048, 10), 2, 32, True, 0.9),
+    ((256, 128, 10), 17, 256, True, 0.9),
+    ((256, 512, 10), 3, 256, False, 0.9),         # no biases: nothing to finish for them
+    ((256, 512, 10), 3, 128 + 64, True, 0.0),     # no momentum buffers; 24 rows per CTA
+])
+def test_one_launch_output_layer_matches_two_kernels(dims, m, B, has_bias, mu, monkeypatch):
     """The output layer of a training step as one launch (clusters of four CTAs, two per replica) against the
     forward + backward kernels it replaces (LS_DISABLE_HEAD_STEP=1), three steps from the same state.  Both
     compute the same fp32 products; only the order of the sums differs, so the output layer's weights, both
@@ -185,14 +189,14 @@ def test_one_launch_output_layer_matches_two_kernels(dims, m, B, monkeypatch):
     import torch
     from paper_1810_08313_b200.binding import LocalSGD
     from tests.helpers import tensor_slices
-    spec, X, y, x1 = small_problem(dims, "softmax_ce", True, 1024, 37, bf16=True)
+    spec, X, y, x1 = small_problem(dims, "softmax_ce", has_bias, 1024, 37, bf16=True)
     steps = 3
     offs = wl.batch_row_offsets(11, steps, m, 1024, B)
     xd, yd = to_device(X, y, bf16=True)
     out = {}
     for tag, val in (("one", "0"), ("two", "1")):
         monkeypatch.setenv("LS_DISABLE_HEAD_STEP", val)
-        eng = LocalSGD(m, dims, gemm_dtype="bf16", lr=0.05, momentum=0.9, batch=B)
+        eng = LocalSGD(m, dims, has_bias=has_bias, gemm_dtype="bf16", lr=0.05, momentum=mu, batch=B)
         eng.bind_dataset(xd, yd); eng.set_params(x1)
         ld = torch.zeros((steps, m), device="cuda")
         n0 = eng.launch_count()
@@ -206,7 +210,7 @@ def test_one_launch_output_layer_matches_two_kernels(dims, m, B, monkeypatch):
     assert np.max(np.abs(pl - ol) / np.abs(ol)) < 2e-3
     L = len(dims) - 1
     for i in range(m):
-        for name, sl in tensor_slices(dims, True):
+        for name, sl in tensor_slices(dims, has_bias):
             tol = 2e-3 if name in (f"W{L}", f"b{L}") else 2e-2
             for a, b in ((px[i][sl], ox[i][sl]), (pv[i][sl], ov[i][sl])):
                 err = np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-30)
