@@ -720,6 +720,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* mask_full = acc_full + 1;                           // [kPairGroups]
   uint64_t* box_done = mask_full + kPairGroups;                 // [kPairGroups] both row halves of a group written
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(box_done + kPairGroups);
+  int* next_box = reinterpret_cast<int*>(tmem_slot + 1);        // backward: boxes whose column sums have been taken
   float* bias_s = reinterpret_cast<float*>(smem + L::kRingBytes + L::kBarBytes);   // [kPairN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -734,6 +735,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
     for (int i = 0; i < kPairGroups; ++i) { mbar_init(&mask_full[i], 1); mbar_init(&box_done[i], 2); }
+    *next_box = 0;
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
@@ -920,24 +922,27 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if ((q & 1) == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before_sync();
   }
-  if (EPI == EPI_DX && p.dbias != nullptr && warp < 2) {
-    // Column sums of the tile for the bias update of the layer below, by the two warps whose other work is over:
-    // thread (h, cp) adds columns 2 cp, 2 cp + 1 over the 64 rows of row half h, in row order, from each box as the
-    // epilogue warps finish it (the values as stored, i.e. rounded to bf16, like the stand-alone bias kernel).
+  if (EPI == EPI_DX && p.dbias != nullptr) {
+    // Column sums of the tile for the bias update of the layer below (the values as stored, i.e. rounded to bf16,
+    // like the stand-alone bias kernel).  A box is 64 rows x 64 columns; whichever warp is free takes the next one
+    // (producer and MMA warps at once, the epilogue warps as they finish), in the order in which the two sets of
+    // epilogue warps complete them; lane cp adds columns 2 cp, 2 cp + 1 of the box in row order.
     __syncwarp();
-    const int h = warp, cp = lane;
-    bool ok2 = true;
-    for (int grp = 0; grp < kPairGroups; ++grp) {
-      if (ok2) ok2 = __all_sync(0xffffffffu, mbar_wait(&box_done[grp], 0));
+    const int cp = lane;
+    for (;;) {
+      int k = 0;
+      if (lane == 0) k = atomicAdd(next_box, 1);
+      k = __shfl_sync(0xffffffffu, k, 0);
+      if (k >= 2 * kPairGroups) break;
+      const int grp = ((k >> 1) & 1) * (kPairGroups / 2) + (k >> 2), h = k & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&box_done[grp], 0))) break;     // (the epilogue has reported the failure)
       const uint8_t* box = smem + (grp * 2 + h) * L::kBoxBytes;
       float s0 = 0.f, s1 = 0.f;
-      if (ok2) {
 #pragma unroll 8
-        for (int r = 0; r < 64; ++r) {
-          const uint32_t u = *reinterpret_cast<const uint32_t*>(box + r * 128 + (((cp >> 2) ^ (r & 7)) << 4) + (cp & 3) * 4);
-          s0 += __uint_as_float(u << 16);
-          s1 += __uint_as_float(u & 0xFFFF0000u);
-        }
+      for (int r = 0; r < 64; ++r) {
+        const uint32_t u = *reinterpret_cast<const uint32_t*>(box + r * 128 + (((cp >> 2) ^ (r & 7)) << 4) + (cp & 3) * 4);
+        s0 += __uint_as_float(u << 16);
+        s1 += __uint_as_float(u & 0xFFFF0000u);
       }
       colsum[h * kPairN + grp * 64 + 2 * cp] = s0;
       colsum[h * kPairN + grp * 64 + 2 * cp + 1] = s1;
