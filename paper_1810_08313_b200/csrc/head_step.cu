@@ -34,9 +34,15 @@ constexpr int kStepThreads = 512;
 constexpr int kStepCluster = 4;         // CTAs per cluster
 constexpr int kStepBlocks = 8;          // row blocks per replica = 2 clusters
 constexpr int kStepMaxRows = 32;        // rows per CTA
-constexpr int kStepOwn = 10;            // elements of the owned C x K/4 block per thread, at most
+constexpr int kStepOwn4 = 3;            // 4-column groups of the owned C x K/4 block per thread, at most
 constexpr int kDzLd = 12;               // floats per row of dZ / logits in shared memory (16-byte rows)
 
+__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void bf16x4_to_f(uint2 u, float (&r)[4]) {
   r[0] = __uint_as_float(u.x << 16); r[1] = __uint_as_float(u.x & 0xFFFF0000u);
   r[2] = __uint_as_float(u.y << 16); r[3] = __uint_as_float(u.y & 0xFFFF0000u);
@@ -255,24 +261,27 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
   }
 
   // ---- 4. exchange ---------------------------------------------------------------------------------------------
+  // Everything below moves in groups of four consecutive columns (16 bytes).  Group e = tid + i * 512 of the
+  // CT x KO block this CTA owns: class e / (KO / 4), columns r KO + 4 (e mod (KO / 4)) ...
   // (the old values are requested before the barrier, so their round trip overlaps the wait)
-  // the elements of W / v whose update this thread may finish: element e = tid + i * 512 of the CT x KO block
-  float wu[kStepOwn], vu[kStepOwn];
+  const int KO4 = KO / 4;
+  float4 wu[kStepOwn4], vu[kStepOwn4];
 #pragma unroll
-  for (int i = 0; i < kStepOwn; ++i) {
+  for (int i = 0; i < kStepOwn4; ++i) {
     const int e = tid + i * kStepThreads;
-    wu[i] = vu[i] = 0.f;
-    if (e < CT * KO) {
-      const int64_t at = (int64_t)(e / KO) * K + r * KO + e % KO;
-      wu[i] = Wg[at];
-      if (mu != 0.f) vu[i] = Vg[at];
+    wu[i] = vu[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e < CT * KO4) {
+      const int64_t at = (int64_t)(e / KO4) * K + r * KO + (e % KO4) * 4;
+      wu[i] = *reinterpret_cast<const float4*>(Wg + at);
+      if (mu != 0.f) vu[i] = *reinterpret_cast<const float4*>(Vg + at);
     }
   }
-  float b_prev = 0.f, vb_prev = 0.f, b_own = 0.f, vb_own = 0.f;
-  const bool prev_bias = pbias != nullptr && tid < KO;
+  float4 b_prev = make_float4(0.f, 0.f, 0.f, 0.f), vb_prev = b_prev;
+  float b_own = 0.f, vb_own = 0.f;
+  const bool prev_bias = pbias != nullptr && tid < KO4;
   if (prev_bias) {
-    b_prev = pbias[(int64_t)g * w_gstride + r * KO + tid];
-    if (mu != 0.f) vb_prev = pvbias[(int64_t)g * w_gstride + r * KO + tid];
+    b_prev = *reinterpret_cast<const float4*>(pbias + (int64_t)g * w_gstride + r * KO + tid * 4);
+    if (mu != 0.f) vb_prev = *reinterpret_cast<const float4*>(pvbias + (int64_t)g * w_gstride + r * KO + tid * 4);
   }
   if (r == 0 && bias != nullptr && tid >= 1 && tid <= CT) {       // thread 1 + c: this layer's bias c
     b_own = bias[(int64_t)g * w_gstride + tid - 1];
@@ -280,7 +289,8 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
   }
   cluster_sync_all();
   // 4a. inside the cluster: the owner of a column adds the 4 partial sums in rank order (distributed shared memory)
-  float sw[kStepOwn], sc = 0.f, ss = 0.f;
+  float4 sw[kStepOwn4], sc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float ss = 0.f;
   {
     const uint32_t wbase = smem_u32(wbuf), cbase = smem_u32(cs), sbase = smem_u32(small);
     uint32_t peer_w[kStepCluster], peer_c[kStepCluster];
@@ -290,26 +300,26 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
       peer_c[j] = map_to_rank(cbase, (uint32_t)j);
     }
 #pragma unroll
-    for (int i = 0; i < kStepOwn; ++i) {
+    for (int i = 0; i < kStepOwn4; ++i) {
       const int e = tid + i * kStepThreads;
-      sw[i] = 0.f;
-      if (e < CT * KO) {
-        const uint32_t at = (uint32_t)((e / KO) * K + r * KO + e % KO);
-        float p[kStepCluster];
+      sw[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < CT * KO4) {
+        const uint32_t at = (uint32_t)((e / KO4) * K + r * KO + (e % KO4) * 4);
+        float4 p[kStepCluster];
 #pragma unroll
-        for (int j = 0; j < kStepCluster; ++j) p[j] = ld_cluster_f32(peer_w[j] + at * 4);
+        for (int j = 0; j < kStepCluster; ++j) p[j] = ld_cluster_f32x4(peer_w[j] + at * 4);
         sw[i] = p[0];
 #pragma unroll
-        for (int j = 1; j < kStepCluster; ++j) sw[i] += p[j];
+        for (int j = 1; j < kStepCluster; ++j) sw[i] = add4(sw[i], p[j]);
       }
     }
-    if (tid < KO) {
-      float p[kStepCluster];
+    if (tid < KO4) {
+      float4 p[kStepCluster];
 #pragma unroll
-      for (int j = 0; j < kStepCluster; ++j) p[j] = ld_cluster_f32(peer_c[j] + (uint32_t)((r * KO + tid) * 4));
+      for (int j = 0; j < kStepCluster; ++j) p[j] = ld_cluster_f32x4(peer_c[j] + (uint32_t)((r * KO + tid * 4) * 4));
       sc = p[0];
 #pragma unroll
-      for (int j = 1; j < kStepCluster; ++j) sc += p[j];
+      for (int j = 1; j < kStepCluster; ++j) sc = add4(sc, p[j]);
     }
     if (r == 0 && tid <= CT) {
       // slot 0: the loss sum; slot 1 + c: column sum of dZ (this layer's bias gradient)
@@ -329,11 +339,11 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
   float* mine = scratch + ((int64_t)g * 2 + half) * scratch_stride;
   const float* other = scratch + ((int64_t)g * 2 + (half ^ 1)) * scratch_stride;
 #pragma unroll
-  for (int i = 0; i < kStepOwn; ++i) {
+  for (int i = 0; i < kStepOwn4; ++i) {
     const int e = tid + i * kStepThreads;
-    if (e < CT * KO) __stcg(mine + (e / KO) * K + r * KO + e % KO, sw[i]);
+    if (e < CT * KO4) __stcg(reinterpret_cast<float4*>(mine + (e / KO4) * K + r * KO + (e % KO4) * 4), sw[i]);
   }
-  if (tid < KO) __stcg(mine + CT * K + r * KO + tid, sc);
+  if (tid < KO4) __stcg(reinterpret_cast<float4*>(mine + CT * K + r * KO + tid * 4), sc);
   if (r == 0 && tid <= CT) __stcg(mine + (CT + 1) * K + tid, ss);
   __threadfence();
   __syncthreads();
@@ -341,32 +351,39 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
   __syncthreads();
   if (!is_last) return;
   __threadfence();
+  auto finish = [&](float s, float vold, float wold, float& vnew) {      // v <- mu v + G; returns W - eta v
+    float step = s;
+    if (mu != 0.f) step = fmaf(mu, vold, s);
+    vnew = step;
+    return fmaf(-lr, step, wold);
+  };
 #pragma unroll
-  for (int i = 0; i < kStepOwn; ++i) {
+  for (int i = 0; i < kStepOwn4; ++i) {
     const int e = tid + i * kStepThreads;
-    if (e < CT * KO) {
-      const int64_t at = (int64_t)(e / KO) * K + r * KO + e % KO;
-      const float s = sw[i] + __ldcg(other + at);
-      float step = s;
-      if (mu != 0.f) {
-        step = fmaf(mu, vu[i], s);
-        Vg[at] = step;
+    if (e < CT * KO4) {
+      const int64_t at = (int64_t)(e / KO4) * K + r * KO + (e % KO4) * 4;
+      const float4 s = add4(sw[i], __ldcg(reinterpret_cast<const float4*>(other + at)));
+      float4 vn, wn;
+      wn.x = finish(s.x, vu[i].x, wu[i].x, vn.x); wn.y = finish(s.y, vu[i].y, wu[i].y, vn.y);
+      wn.z = finish(s.z, vu[i].z, wu[i].z, vn.z); wn.w = finish(s.w, vu[i].w, wu[i].w, vn.w);
+      if (mu != 0.f) *reinterpret_cast<float4*>(Vg + at) = vn;
+      *reinterpret_cast<float4*>(Wg + at) = wn;
+      if (Wb != nullptr) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(wn.x, wn.y), hi = __floats2bfloat162_rn(wn.z, wn.w);
+        *reinterpret_cast<uint2*>(Wb + (int64_t)g * w_gstride + at) =
+            make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
       }
-      const float wn = fmaf(-lr, step, wu[i]);
-      Wg[at] = wn;
-      if (Wb != nullptr) Wb[(int64_t)g * w_gstride + at] = __float2bfloat16_rn(wn);
     }
   }
   if (prev_bias) {
-    const int k = r * KO + tid;
-    const float s = sc + __ldcg(other + CT * K + k);
+    const int k = r * KO + tid * 4;
+    const float4 s = add4(sc, __ldcg(reinterpret_cast<const float4*>(other + CT * K + k)));
     const int64_t at = (int64_t)g * w_gstride + k;
-    float step = s;
-    if (mu != 0.f) {
-      step = fmaf(mu, vb_prev, s);
-      pvbias[at] = step;
-    }
-    pbias[at] = fmaf(-lr, step, b_prev);
+    float4 vn, bn;
+    bn.x = finish(s.x, vb_prev.x, b_prev.x, vn.x); bn.y = finish(s.y, vb_prev.y, b_prev.y, vn.y);
+    bn.z = finish(s.z, vb_prev.z, b_prev.z, vn.z); bn.w = finish(s.w, vb_prev.w, b_prev.w, vn.w);
+    if (mu != 0.f) *reinterpret_cast<float4*>(pvbias + at) = vn;
+    *reinterpret_cast<float4*>(pbias + at) = bn;
   }
   if (r == 0 && tid <= CT) {
     const float s = ss + __ldcg(other + (CT + 1) * K + tid);
@@ -374,12 +391,10 @@ head_step_kernel(const __nv_bfloat16* __restrict__ A, const int32_t* __restrict_
       if (loss_out != nullptr) loss_out[g] = s * invB;
     } else if (bias != nullptr) {
       const int64_t at = (int64_t)g * w_gstride + tid - 1;
-      float step = s;
-      if (mu != 0.f) {
-        step = fmaf(mu, vb_own, s);
-        vbias[at] = step;
-      }
-      bias[at] = fmaf(-lr, step, b_own);
+      float vn;
+      const float bn = finish(s, vb_own, b_own, vn);
+      if (mu != 0.f) vbias[at] = vn;
+      bias[at] = bn;
     }
   }
 }
@@ -397,7 +412,7 @@ bool head_step_ok(const HeadStepArgs& a) {
       a.counters == nullptr)
     return false;
   if (a.B % (kStepBlocks * 4) != 0 || a.B / kStepBlocks > kStepMaxRows) return false;
-  if (a.K < 128 || a.K % 128 != 0 || a.C * (a.K / kStepCluster) > kStepOwn * kStepThreads || a.K / kStepCluster > kStepThreads)
+  if (a.K < 128 || a.K % 128 != 0 || a.C * (a.K / kStepCluster) > kStepOwn4 * 4 * kStepThreads)
     return false;
   if (reinterpret_cast<uintptr_t>(a.A) % 16 != 0 || reinterpret_cast<uintptr_t>(a.W) % 16 != 0 || a.w_gstride % 4 != 0 ||
       reinterpret_cast<uintptr_t>(a.dPrev) % 8 != 0)
