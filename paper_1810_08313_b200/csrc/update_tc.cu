@@ -703,7 +703,8 @@ tc_update_pair_kernel(const __grid_constant__ UMaps maps, const __grid_constant_
 // left / right 32 columns.
 constexpr int SN = 64;                  // columns of a unit
 constexpr int kSyncThreads = 384;
-constexpr int kSyncStages = 3;
+constexpr int kSyncStages = 4;          // operand stages of 64 mini-batch rows: one replica's products ahead (the
+                                        // tensor core waited for operands 70 % of the time with three)
 struct SLayer {
   int N, n_tiles, tile_begin;           // row length of W, units per row block, first unit of the layer
   const int64_t* b_row_off;
